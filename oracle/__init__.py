@@ -1,0 +1,198 @@
+"""ctypes front end of the CPU oracle (oracle/squat_oracle.c)  --  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package.  It marshals numpy arrays into the C functions and adds nothing to their
+arithmetic.  It never imports the CUDA package.
+"""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "squat_oracle.c")
+_LIB = os.path.join(_HERE, "libsquat_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (strict IEEE: no contraction, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fno-fast-math", "-frounding-math",
+               "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.sqo_kv_cache_bytes.restype = ctypes.c_longlong
+        _lib.sqo_kv_cache_bytes.argtypes = [ctypes.c_longlong] * 6
+    return _lib
+
+
+def _p(a, ty):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ty))
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+_D, _F, _U8, _I16 = ctypes.c_double, ctypes.c_float, ctypes.c_uint8, ctypes.c_int16
+
+
+def gram(Qc):
+    Qc = np.ascontiguousarray(Qc, dtype=np.float64)
+    N, d = Qc.shape
+    M = np.empty((d, d), dtype=np.float64)
+    _check(_load().sqo_gram(_p(Qc, _D), ctypes.c_long(N), d, _p(M, _D)), "gram")
+    return M
+
+
+def jacobi_eig(A):
+    """Eigenvalues (descending) and eigenvectors (rows) of a symmetric matrix."""
+    A = np.array(A, dtype=np.float64, order="C", copy=True)
+    d = A.shape[0]
+    mu = np.empty(d, dtype=np.float64)
+    V = np.empty((d, d), dtype=np.float64)
+    _check(_load().sqo_jacobi_eig(_p(A, _D), d, _p(mu, _D), _p(V, _D)), "jacobi_eig")
+    return mu, V
+
+
+def query_subspace(Qc, r):
+    """Returns (Qhat [r, d], mu [d], V [d, d] rows = eigenvectors of Qc^T Qc)."""
+    Qc = np.ascontiguousarray(Qc, dtype=np.float64)
+    N, d = Qc.shape
+    Qhat = np.zeros((r, d), dtype=np.float64)
+    mu = np.empty(d, dtype=np.float64)
+    V = np.empty((d, d), dtype=np.float64)
+    _check(_load().sqo_query_subspace(_p(Qc, _D), ctypes.c_long(N), d, r, _p(Qhat, _D), _p(mu, _D), _p(V, _D)),
+           "query_subspace")
+    return Qhat, mu, V
+
+
+def update_matrices(Qhat, d, lam, g=1, want_chain=False):
+    """Returns dict with W, P, P_inv and (optionally) the list Ainv[1..T]."""
+    Qhat = np.ascontiguousarray(Qhat, dtype=np.float64).reshape(-1, d)
+    r = Qhat.shape[0]
+    W = np.empty((d, d), dtype=np.float64)
+    P = np.empty((d, d), dtype=np.float64)
+    Pinv = np.empty((d, d), dtype=np.float64)
+    T = d // g
+    chain = None
+    if want_chain:
+        chain = np.empty(sum((t * g) ** 2 for t in range(1, T + 1)), dtype=np.float64)
+    _check(_load().sqo_update_matrices(_p(Qhat, _D) if r else None, r, d, ctypes.c_double(lam), g,
+                                       _p(W, _D), _p(P, _D), _p(Pinv, _D), _p(chain, _D)), "update_matrices")
+    out = {"W": W, "P": P, "P_inv": Pinv}
+    if want_chain:
+        mats, off = {}, 0
+        for t in range(1, T + 1):
+            m = t * g
+            mats[t] = chain[off:off + m * m].reshape(m, m).copy()
+            off += m * m
+        out["Ainv"] = mats
+    return out
+
+
+def quant_keys(K, G, bits, W=None, force=None, want_tval=False):
+    """Algorithm 1 Quant on [n, d] keys. Returns dict(codes, scale, zero, Khat[, tval])."""
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    n, d = K.shape
+    codes = np.empty((n, d), dtype=np.uint8)
+    scale = np.empty((n // G, d), dtype=np.float32)
+    zero = np.empty((n // G, d), dtype=np.float32)
+    Khat = np.empty((n, d), dtype=np.float64)
+    tval = np.empty((n, d), dtype=np.float64) if want_tval else None
+    if W is not None:
+        W = np.ascontiguousarray(W, dtype=np.float64)
+        assert W.shape == (d, d)
+    if force is not None:
+        force = np.ascontiguousarray(force, dtype=np.int16)
+        assert force.shape == (n, d)
+    _check(_load().sqo_quant_keys(_p(K, _D), ctypes.c_long(n), d, G, bits, _p(W, _D), _p(codes, _U8),
+                                  _p(scale, _F), _p(zero, _F), _p(Khat, _D), _p(tval, _D), _p(force, _I16)),
+           "quant_keys")
+    out = {"codes": codes, "scale": scale, "zero": zero, "Khat": Khat}
+    if want_tval:
+        out["tval"] = tval
+    return out
+
+
+def quant_values_f32(V, G, bits):
+    V = np.ascontiguousarray(V, dtype=np.float32)
+    n, d = V.shape
+    codes = np.empty((n, d), dtype=np.uint8)
+    scale = np.empty((n, d // G), dtype=np.float32)
+    zero = np.empty((n, d // G), dtype=np.float32)
+    _check(_load().sqo_quant_values_f32(_p(V, _F), ctypes.c_long(n), d, G, bits, _p(codes, _U8), _p(scale, _F),
+                                        _p(zero, _F)), "quant_values_f32")
+    return {"codes": codes, "scale": scale, "zero": zero}
+
+
+def quant_values_f64(V, G, bits):
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    n, d = V.shape
+    codes = np.empty((n, d), dtype=np.uint8)
+    scale = np.empty((n, d // G), dtype=np.float32)
+    zero = np.empty((n, d // G), dtype=np.float32)
+    _check(_load().sqo_quant_values_f64(_p(V, _D), ctypes.c_long(n), d, G, bits, _p(codes, _U8), _p(scale, _F),
+                                        _p(zero, _F)), "quant_values_f64")
+    return {"codes": codes, "scale": scale, "zero": zero}
+
+
+def dequant_keys(codes, scale, zero, G):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    n, d = codes.shape
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    zero = np.ascontiguousarray(zero, dtype=np.float32)
+    out = np.empty((n, d), dtype=np.float64)
+    _check(_load().sqo_dequant_keys(_p(codes, _U8), _p(scale, _F), _p(zero, _F), ctypes.c_long(n), d, G, _p(out, _D)),
+           "dequant_keys")
+    return out
+
+
+def dequant_values(codes, scale, zero, G):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    n, d = codes.shape
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    zero = np.ascontiguousarray(zero, dtype=np.float32)
+    out = np.empty((n, d), dtype=np.float64)
+    _check(_load().sqo_dequant_values(_p(codes, _U8), _p(scale, _F), _p(zero, _F), ctypes.c_long(n), d, G,
+                                      _p(out, _D)), "dequant_values")
+    return out
+
+
+def pack(codes, bits):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    n, d = codes.shape
+    packed = np.empty((n, d * bits // 8), dtype=np.uint8)
+    _check(_load().sqo_pack(_p(codes, _U8), ctypes.c_long(n), d, bits, _p(packed, _U8)), "pack")
+    return packed
+
+
+def unpack(packed, d, bits):
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    n = packed.shape[0]
+    codes = np.empty((n, d), dtype=np.uint8)
+    _check(_load().sqo_unpack(_p(packed, _U8), ctypes.c_long(n), d, bits, _p(codes, _U8)), "unpack")
+    return codes
+
+
+def kv_cache_bytes(batch, seq_len, layers, heads, head_dim, bytes_per_param):
+    return int(_load().sqo_kv_cache_bytes(batch, seq_len, layers, heads, head_dim, bytes_per_param))
+
+
+def build_W(Qc, r, lam, g=1):
+    """Convenience: stacked queries -> assembled update matrix W (steps O1 + O2)."""
+    d = Qc.shape[1]
+    Qhat, mu, V = query_subspace(Qc, r)
+    mats = update_matrices(Qhat, d, lam, g)
+    mats.update({"Qhat": Qhat, "mu": mu, "V": V})
+    return mats
