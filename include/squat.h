@@ -1,0 +1,165 @@
+/*
+ * libsquat -- the KV-cache write path of SQuat (arXiv 2503.24358) on one NVIDIA B200 (sm_100a).
+ *
+ * Plain C ABI.  No exceptions, no C++ or framework types cross it.  Unless a parameter says
+ * "host", every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned, valid
+ * until the stream work enqueued by the call has finished.  Calls enqueue kernels on the given
+ * CUDA stream (a cudaStream_t passed as void*, NULL = default stream) and return without
+ * synchronising, except where stated.  Arguments are validated on the host before anything
+ * is launched; a rejected call launches nothing.  Kernels never trap or assert: numerical
+ * trouble (non-finite input, a group whose values are all equal) sets bits in a device status
+ * word, see squat_get_device_status.  There is no CPU fallback.
+ *
+ * Notation (the paper's): d = head dimension, r = subspace rank, lambda = regulariser of
+ * Eq. (2), g = elements quantized per iteration (Appendix A "Block-Wise Quantization"),
+ * G = quantization group size, b = bits, L = 2^b - 1.
+ *
+ * Cache layout written by the quantizers (the paper prescribes none):
+ *   codes  token-major; token i of (batch, head) owns d*b/8 consecutive bytes; channel j's code
+ *          sits at bit (j*b) mod 8 of byte floor(j*b/8), low bits first.
+ *   keys   scale, zero: float32 [batch, head, token/G, d]   (one grid per channel per G tokens)
+ *   values scale, zero: float32 [batch, head, token, d/G]   (one grid per G channels per token)
+ *   deq(c) = zero + scale * c      (Section 2, "Quantization").
+ */
+#ifndef SQUAT_H
+#define SQUAT_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SQUAT_OK = 0,
+    SQUAT_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, negative size, bad enum            */
+    SQUAT_ERR_SHAPE = 2,         /* sizes that do not divide as the method requires               */
+    SQUAT_ERR_UNSUPPORTED = 3,   /* valid in the paper, not built here (e.g. head_dim != 128)     */
+    SQUAT_ERR_ALLOC = 4,         /* device allocation failed                                      */
+    SQUAT_ERR_CUDA = 5,          /* a CUDA runtime call failed; see squat_last_cuda_error         */
+    SQUAT_ERR_NUMERIC = 6        /* the eigensolver did not converge                              */
+} squat_status;
+
+typedef enum { SQUAT_F32 = 0, SQUAT_BF16 = 1 } squat_dtype;
+typedef enum { SQUAT_KEYS = 0, SQUAT_VALUES = 1 } squat_kind;
+
+/* bits of the device status word */
+#define SQUAT_FLAG_NONFINITE   1u   /* a scale came out NaN/Inf: non-finite input                  */
+#define SQUAT_FLAG_ZERO_RANGE  2u   /* some group had max == min (scale 0, all codes 0)            */
+#define SQUAT_FLAG_NO_CONVERGE 4u   /* eigensolver hit its sweep limit for some head               */
+
+/* Opaque per-layer state: the update matrices of every KV head (shared by all samples of a
+ * batch, Appendix C) plus the scratch the subspace build needs.  Owns device memory. */
+typedef struct squat_subspace squat_subspace;
+
+/* Allocates the state for n_kv_heads heads of dimension head_dim (only 128 is built) on the
+ * current device.  Synchronous (cudaMalloc).  *out receives the handle; free it with
+ * squat_subspace_destroy.  The update matrices start as zero (= plain round-to-nearest). */
+int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out);
+int squat_subspace_destroy(squat_subspace *s);
+
+/*
+ * Step 1 -- query subspace and update matrices  (Section 3.2; Algorithm 1 lines 5-9;
+ * Prop. 1, Prop. 2, Lemma 3, Lemma 4; GQA and batch rules of Appendix C).
+ *
+ * q         prompt queries of ONE sample (the first of the batch), [n_q_heads, n_tokens, d],
+ *           d contiguous, element strides stride_h (between query heads) and stride_t (between
+ *           tokens).  Query heads h*(n_q/n_kv) .. (h+1)*(n_q/n_kv)-1 feed KV head h.
+ * rank_r    top singular directions kept, 0 <= r <= d (r = 0 gives plain round-to-nearest).
+ * lambda    >= 0, finite.          block_g   g, divides d; 1 = element by element (Prop. 1).
+ *
+ * Per KV head: Gram matrix of the stacked queries in fp64, its eigen-decomposition in fp64
+ * (sigma_i^2 and v_i of the SVD of Alg. 1 line 5), P = I + lambda Qhat^T Qhat with
+ * Qhat = diag(sigma[:r]) V[:r], and the update matrices B_t H_t of Lemma 3 for t = 1..d/g-1,
+ * assembled as one block-strictly-lower-triangular W (float32):  quantizing channel j with
+ * error e moves every later channel j' by e * W[j'][j].
+ * Enqueues on `stream`; the handle may be used by later calls on the same stream at once.
+ */
+int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
+                         long long stride_h, long long stride_t, int rank_r, double lambda,
+                         int block_g, void *stream);
+
+/* Test / checkpoint hooks.  Both synchronise `stream`.  Host pointers; any may be NULL.
+ *   W_host      [n_kv_heads, d, d] float32, row j' column j, block strictly lower triangular.
+ *   gram_host   [n_kv_heads, d, d] float64 Gram matrices of the last build.
+ *   eigval_host [n_kv_heads, d]    float64 eigenvalues, descending (sigma_i^2).
+ *   eigvec_host [n_kv_heads, d, d] float64, row i = unit eigenvector of eigval i. */
+int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,
+                          double *eigval_host, double *eigvec_host);
+int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream);
+
+/*
+ * Step 2 -- key quantization with error feedback  (Algorithm 1, function Quant; Eq. (3) and
+ * Eq. (update_block); quantizer of Section 2).
+ *
+ * k         [batch, n_kv_heads, n_tokens, d], d contiguous, element strides given.
+ * n_tokens  multiple of group_size (the tail stays in the caller's residual buffer,
+ *           Alg. 1 lines 10-11); groups are G consecutive tokens from the first one passed.
+ * codes     [batch, n_kv_heads, *, d*bits/8] bytes; scales, zeros [batch, n_kv_heads, *, d].
+ *           out_stride_b / out_stride_h are in TOKENS (a batch/head step moves the code pointer
+ *           by stride*d*bits/8 bytes and the scale/zero pointers by (stride/G)*d floats), so a
+ *           decode window can be written into a larger cache.  Must be multiples of G.
+ * For every group and channel j in order: grid from min/max over the G tokens of the current
+ * (corrected) values, round half to even, push each token's error on its later channels
+ * through W.  Splitting n_tokens at multiples of G over several calls gives identical bytes.
+ * bits in {2, 4}; group_size in {32, 64, 128}; d = 128; n_kv_heads must match the handle.
+ */
+int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
+                        int n_tokens, int head_dim, long long stride_b, long long stride_h,
+                        long long stride_t, int bits, int group_size, unsigned char *codes,
+                        float *scales, float *zeros, long long out_stride_b, long long out_stride_h,
+                        void *stream);
+
+/*
+ * Step 3 -- per-token value quantization  (Section 2 "Quantization"; Appendix C: each token's d
+ * channels in d/G groups of G).  Every operation is IEEE binary32 in the order
+ *   Delta = (M - m) / L;  t = (x - m) / Delta;  c = clamp(rint(t), 0, L).
+ * v [batch, n_kv_heads, n_tokens, d]; codes as for keys; scales, zeros
+ * [batch, n_kv_heads, *, d/G] with out strides in tokens.  d % G == 0, d*bits % 64 == 0.
+ */
+int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
+                          int head_dim, long long stride_b, long long stride_h, long long stride_t,
+                          int bits, int group_size, unsigned char *codes, float *scales, float *zeros,
+                          long long out_stride_b, long long out_stride_h, void *stream);
+
+/*
+ * Step 4 -- dequantize  (Section 2: deq(c) = c * Delta + m), for either layout kind.
+ * in strides in tokens as above; out is contiguous [batch, n_kv_heads, n_tokens, d] of out_dtype
+ * (float32: fma(c, scale, zero) rounded once; bf16: that value rounded to nearest even).
+ */
+int squat_dequantize(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+                     int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                     long long in_stride_b, long long in_stride_h, void *out, int out_dtype,
+                     void *stream);
+
+/*
+ * The whole write path from HOST buffers (prefill of one layer): copies q (sample 0,
+ * [n_q_heads, n_tokens, d]), k and v ([batch, n_kv_heads, n_tokens, d]), all contiguous, to the
+ * device workspace, runs steps 1-3, copies codes / scales / zeros back and synchronises the
+ * stream.  Host buffers should be pinned for full copy speed.  `workspace` is caller-owned device
+ * memory of at least squat_write_path_workspace_bytes(...) bytes, 256-byte aligned.
+ */
+size_t squat_write_path_workspace_bytes(int dtype, int batch, int n_q_heads, int n_kv_heads,
+                                        int n_tokens, int head_dim, int bits, int group_size);
+int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
+                          int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
+                          int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
+                          unsigned char *k_codes_host, float *k_scales_host, float *k_zeros_host,
+                          unsigned char *v_codes_host, float *v_scales_host, float *v_zeros_host,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/* Reads (and clears when `clear` != 0) the device status word of the current device.
+ * Synchronises `stream`.  flags is a host pointer. */
+int squat_get_device_status(void *stream, unsigned *flags, int clear);
+
+/* Number of kernels this library has launched in this process (all devices). */
+unsigned long long squat_kernel_launch_count(void);
+
+const char *squat_status_string(int status);
+/* Text of the last CUDA runtime error seen by the calling thread inside this library. */
+const char *squat_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQUAT_H */

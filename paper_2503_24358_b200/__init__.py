@@ -1,0 +1,12 @@
+"""SQuat KV-cache write path for NVIDIA B200 (sm_100a).
+
+The product is the C-ABI shared library `libsquat.so` (declared in include/squat.h, built from
+csrc/ by build.py).  This package is its thin Python binding: same names, argument marshalling
+only, torch used for device memory and streams.
+"""
+from .binding import (  # noqa: F401
+    EXPORTED_SYMBOLS, FLAG_NO_CONVERGE, FLAG_NONFINITE, FLAG_ZERO_RANGE, LIB_PATH, SQUAT_BF16, SQUAT_F32,
+    SQUAT_KEYS, SQUAT_VALUES, SquatError, Subspace, squat_build_subspace, squat_dequantize,
+    squat_get_device_status, squat_kernel_launch_count, squat_quantize_keys, squat_quantize_values,
+    squat_subspace_export, squat_subspace_import, squat_write_path_host, squat_write_path_workspace_bytes,
+)

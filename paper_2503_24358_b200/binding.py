@@ -1,0 +1,228 @@
+"""Thin ctypes binding of libsquat.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/squat.h) and takes
+torch tensors where the C function takes device pointers.  Nothing here computes: all
+steps of the write path run in the library's CUDA kernels.  If the shared library is
+missing or does not load, every call raises -- there is no fallback.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsquat.so")
+
+SQUAT_F32, SQUAT_BF16 = 0, 1
+SQUAT_KEYS, SQUAT_VALUES = 0, 1
+FLAG_NONFINITE, FLAG_ZERO_RANGE, FLAG_NO_CONVERGE = 1, 2, 4
+
+EXPORTED_SYMBOLS = (
+    "squat_subspace_create", "squat_subspace_destroy", "squat_build_subspace", "squat_subspace_export",
+    "squat_subspace_import", "squat_quantize_keys", "squat_quantize_values", "squat_dequantize",
+    "squat_write_path_workspace_bytes", "squat_write_path_host", "squat_get_device_status",
+    "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error",
+)
+
+_lib = None
+
+
+class SquatError(RuntimeError):
+    def __init__(self, status, where):
+        lib = _load()
+        msg = lib.squat_status_string(status).decode()
+        if status == 5:
+            msg += " (" + lib.squat_last_cuda_error().decode() + ")"
+        super().__init__(f"{where}: {msg} [status {status}]")
+        self.status = status
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_24358_b200.build` "
+                               "(there is no CPU fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        vp, i, ll, dbl = c.c_void_p, c.c_int, c.c_longlong, c.c_double
+        lib.squat_subspace_create.argtypes = [i, i, c.POINTER(vp)]
+        lib.squat_subspace_destroy.argtypes = [vp]
+        lib.squat_build_subspace.argtypes = [vp, vp, i, i, i, ll, ll, i, dbl, i, vp]
+        lib.squat_subspace_export.argtypes = [vp, vp, vp, vp, vp, vp]
+        lib.squat_subspace_import.argtypes = [vp, vp, vp]
+        lib.squat_quantize_keys.argtypes = [vp, vp, i, i, i, i, i, ll, ll, ll, i, i, vp, vp, vp, ll, ll, vp]
+        lib.squat_quantize_values.argtypes = [vp, i, i, i, i, i, ll, ll, ll, i, i, vp, vp, vp, ll, ll, vp]
+        lib.squat_dequantize.argtypes = [i, vp, vp, vp, i, i, i, i, i, i, ll, ll, vp, i, vp]
+        lib.squat_write_path_workspace_bytes.argtypes = [i] * 8
+        lib.squat_write_path_workspace_bytes.restype = c.c_size_t
+        lib.squat_write_path_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, dbl, i, i, i,
+                                              vp, vp, vp, vp, vp, vp, vp, c.c_size_t, vp]
+        lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
+        lib.squat_kernel_launch_count.restype = c.c_ulonglong
+        lib.squat_status_string.argtypes = [i]
+        lib.squat_status_string.restype = c.c_char_p
+        lib.squat_last_cuda_error.restype = c.c_char_p
+        _lib = lib
+    return _lib
+
+
+def _check(status, where):
+    if status != 0:
+        raise SquatError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SQUAT_F32
+    if t.dtype == torch.bfloat16:
+        return SQUAT_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dev(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+class Subspace:
+    """Owner of a squat_subspace handle (the per-layer update matrices of every KV head)."""
+
+    def __init__(self, n_kv_heads: int, head_dim: int = 128):
+        self._h = ctypes.c_void_p()
+        self.n_kv_heads, self.head_dim = n_kv_heads, head_dim
+        _check(_load().squat_subspace_create(n_kv_heads, head_dim, ctypes.byref(self._h)), "squat_subspace_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            _load().squat_subspace_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+
+def squat_build_subspace(s: Subspace, q: torch.Tensor, rank_r: int, lam: float, block_g: int = 1, stream=None):
+    """q: [n_q_heads, n_tokens, d] prompt queries of the first sample (last dim contiguous)."""
+    if q.dim() != 3 or q.stride(2) != 1 or q.shape[2] != s.head_dim:
+        raise ValueError("q must be [n_q_heads, n_tokens, head_dim] with contiguous last dim")
+    _check(_load().squat_build_subspace(s.handle, _dev(q, "q"), _dtype_code(q), q.shape[0], q.shape[1],
+                                        q.stride(0), q.stride(1), rank_r, float(lam), block_g, _stream(stream)),
+           "squat_build_subspace")
+
+
+def squat_subspace_export(s: Subspace, want=("W",), stream=None):
+    """Returns a dict of numpy arrays: W [H,d,d] f32, gram [H,d,d] f64, eigval [H,d], eigvec [H,d,d]."""
+    import numpy as np
+    H, d = s.n_kv_heads, s.head_dim
+    bufs = {
+        "W": np.empty((H, d, d), np.float32) if "W" in want else None,
+        "gram": np.empty((H, d, d), np.float64) if "gram" in want else None,
+        "eigval": np.empty((H, d), np.float64) if "eigval" in want else None,
+        "eigvec": np.empty((H, d, d), np.float64) if "eigvec" in want else None,
+    }
+    ptr = lambda a: None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+    _check(_load().squat_subspace_export(s.handle, _stream(stream), ptr(bufs["W"]), ptr(bufs["gram"]),
+                                         ptr(bufs["eigval"]), ptr(bufs["eigvec"])), "squat_subspace_export")
+    return {k: v for k, v in bufs.items() if v is not None}
+
+
+def squat_subspace_import(s: Subspace, W, stream=None):
+    """W: numpy [H, d, d] float32, row j' column j (block strictly lower triangular)."""
+    import numpy as np
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    if W.shape != (s.n_kv_heads, s.head_dim, s.head_dim):
+        raise ValueError("W must be [n_kv_heads, d, d]")
+    _check(_load().squat_subspace_import(s.handle, W.ctypes.data_as(ctypes.c_void_p), _stream(stream)),
+           "squat_subspace_import")
+
+
+def _check_bhtd(x, name):
+    if x.dim() != 4 or x.stride(3) != 1:
+        raise ValueError(f"{name} must be [batch, heads, tokens, head_dim] with contiguous last dim")
+
+
+def squat_quantize_keys(s: Subspace, k: torch.Tensor, bits: int, group_size: int, codes: torch.Tensor,
+                        scales: torch.Tensor, zeros: torch.Tensor, out_stride_b: int = None,
+                        out_stride_h: int = None, stream=None):
+    """k [B,H,T,d] -> codes (uint8), scales, zeros (float32), written in place.
+
+    out strides are in tokens; by default the outputs are dense [B,H,T,...]."""
+    _check_bhtd(k, "k")
+    B, H, T, d = k.shape
+    osh = T if out_stride_h is None else out_stride_h
+    osb = H * osh if out_stride_b is None else out_stride_b
+    _check(_load().squat_quantize_keys(s.handle, _dev(k, "k"), _dtype_code(k), B, H, T, d, k.stride(0), k.stride(1),
+                                       k.stride(2), bits, group_size, _dev(codes, "codes"), _dev(scales, "scales"),
+                                       _dev(zeros, "zeros"), osb, osh, _stream(stream)), "squat_quantize_keys")
+
+
+def squat_quantize_values(v: torch.Tensor, bits: int, group_size: int, codes: torch.Tensor, scales: torch.Tensor,
+                          zeros: torch.Tensor, out_stride_b: int = None, out_stride_h: int = None, stream=None):
+    _check_bhtd(v, "v")
+    B, H, T, d = v.shape
+    osh = T if out_stride_h is None else out_stride_h
+    osb = H * osh if out_stride_b is None else out_stride_b
+    _check(_load().squat_quantize_values(_dev(v, "v"), _dtype_code(v), B, H, T, d, v.stride(0), v.stride(1),
+                                         v.stride(2), bits, group_size, _dev(codes, "codes"), _dev(scales, "scales"),
+                                         _dev(zeros, "zeros"), osb, osh, _stream(stream)), "squat_quantize_values")
+
+
+def squat_dequantize(kind: int, codes: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor, batch: int,
+                     n_kv_heads: int, n_tokens: int, head_dim: int, bits: int, group_size: int, out: torch.Tensor,
+                     in_stride_b: int = None, in_stride_h: int = None, stream=None):
+    ish = n_tokens if in_stride_h is None else in_stride_h
+    isb = n_kv_heads * ish if in_stride_b is None else in_stride_b
+    if not out.is_contiguous():
+        raise ValueError("out must be contiguous")
+    _check(_load().squat_dequantize(kind, _dev(codes, "codes"), _dev(scales, "scales"), _dev(zeros, "zeros"), batch,
+                                    n_kv_heads, n_tokens, head_dim, bits, group_size, isb, ish, _dev(out, "out"),
+                                    _dtype_code(out), _stream(stream)), "squat_dequantize")
+
+
+def squat_write_path_workspace_bytes(dtype: torch.dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, bits,
+                                     group_size) -> int:
+    code = SQUAT_F32 if dtype == torch.float32 else SQUAT_BF16
+    return int(_load().squat_write_path_workspace_bytes(code, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, bits,
+                                                        group_size))
+
+
+def squat_write_path_host(s: Subspace, q, k, v, rank_r, lam, block_g, bits, group_size, k_codes, k_scales, k_zeros,
+                          v_codes, v_scales, v_zeros, workspace: torch.Tensor, stream=None):
+    """q, k, v and the six outputs are HOST tensors (pinned for speed); workspace is a CUDA uint8 tensor."""
+    for name, t in (("q", q), ("k", k), ("v", v), ("k_codes", k_codes), ("k_scales", k_scales), ("k_zeros", k_zeros),
+                    ("v_codes", v_codes), ("v_scales", v_scales), ("v_zeros", v_zeros)):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous host tensor")
+    B, H, T, d = k.shape
+    hp = lambda t: ctypes.c_void_p(t.data_ptr())
+    _check(_load().squat_write_path_host(s.handle, hp(q), hp(k), hp(v), _dtype_code(k), B, q.shape[0], H, T, d, rank_r,
+                                         float(lam), block_g, bits, group_size, hp(k_codes), hp(k_scales), hp(k_zeros),
+                                         hp(v_codes), hp(v_scales), hp(v_zeros), _dev(workspace, "workspace"),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)),
+           "squat_write_path_host")
+
+
+def squat_get_device_status(clear: bool = True, stream=None) -> int:
+    flags = ctypes.c_uint(0)
+    _check(_load().squat_get_device_status(_stream(stream), ctypes.byref(flags), 1 if clear else 0),
+           "squat_get_device_status")
+    return flags.value
+
+
+def squat_kernel_launch_count() -> int:
+    return int(_load().squat_kernel_launch_count())

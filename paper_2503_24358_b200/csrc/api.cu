@@ -1,0 +1,340 @@
+// extern "C" entry points of libsquat: argument validation, handle management and the
+// stream-ordered launch sequences.  All arithmetic of the method lives in the kernels.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "squat_internal.cuh"
+
+namespace {
+
+constexpr int D = SQUAT_D;
+constexpr int MAX_DEVICES = 64;
+
+thread_local char g_cuda_error[256] = "";
+std::atomic<unsigned long long> g_launches{0};
+
+__device__ unsigned g_status_word = 0;
+unsigned *g_status_ptr[MAX_DEVICES] = {nullptr};
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool valid_dtype(int dt) { return dt == SQUAT_F32 || dt == SQUAT_BF16; }
+size_t elem_size(int dt) { return dt == SQUAT_BF16 ? 2 : 4; }
+
+// Shared checks of the two quantizers.  Strides are in elements (input) / tokens (output).
+int check_quant_args(const void *x, int dtype, int batch, int H, int T, int d, long long sb, long long sh,
+                     long long st, int bits, int G, const void *codes, const void *scales, const void *zeros,
+                     long long osb, long long osh)
+{
+    if (!x || !codes || !scales || !zeros || !valid_dtype(dtype)) return SQUAT_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(codes) || !aligned16(scales) || !aligned16(zeros)) return SQUAT_ERR_INVALID_ARG;
+    if (batch < 0 || H <= 0 || T < 0 || d <= 0) return SQUAT_ERR_INVALID_ARG;
+    if (bits != 2 && bits != 4) return SQUAT_ERR_UNSUPPORTED;
+    if (G != 32 && G != 64 && G != 128) return SQUAT_ERR_UNSUPPORTED;
+    if (sb < 0 || sh < 0 || st < d || osb < 0 || osh < 0) return SQUAT_ERR_INVALID_ARG;
+    const long long vec = 16 / (long long)elem_size(dtype);       // 128-bit loads
+    if (sb % vec || sh % vec || st % vec) return SQUAT_ERR_INVALID_ARG;
+    return SQUAT_OK;
+}
+
+}  // namespace
+
+int squat_cuda_fail(cudaError_t e)
+{
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return SQUAT_ERR_CUDA;
+}
+
+void squat_count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+unsigned *squat_status_word()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    if (!g_status_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        g_status_ptr[dev] = static_cast<unsigned *>(p);
+    }
+    return g_status_ptr[dev];
+}
+
+extern "C" {
+
+const char *squat_status_string(int status)
+{
+    switch (status) {
+        case SQUAT_OK: return "ok";
+        case SQUAT_ERR_INVALID_ARG: return "invalid argument";
+        case SQUAT_ERR_SHAPE: return "shape does not divide as required";
+        case SQUAT_ERR_UNSUPPORTED: return "configuration not built";
+        case SQUAT_ERR_ALLOC: return "device allocation failed";
+        case SQUAT_ERR_CUDA: return "CUDA runtime error";
+        case SQUAT_ERR_NUMERIC: return "numerical failure";
+        default: return "unknown status";
+    }
+}
+
+const char *squat_last_cuda_error(void) { return g_cuda_error; }
+
+unsigned long long squat_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
+{
+    if (!out) return SQUAT_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n_kv_heads <= 0 || n_kv_heads > 65535 || head_dim <= 0) return SQUAT_ERR_INVALID_ARG;
+    if (head_dim != D) return SQUAT_ERR_UNSUPPORTED;
+    squat_subspace *s = new (std::nothrow) squat_subspace();
+    if (!s) return SQUAT_ERR_ALLOC;
+    memset(s, 0, sizeof(*s));
+    s->n_kv_heads = n_kv_heads;
+    s->head_dim = head_dim;
+    int sms = 148;
+    if (cudaGetDevice(&s->device) != cudaSuccess) { delete s; return SQUAT_ERR_CUDA; }
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, s->device);
+    s->gram_chunks_cap = (2 * sms + n_kv_heads - 1) / n_kv_heads;
+    if (s->gram_chunks_cap < 1) s->gram_chunks_cap = 1;
+    const size_t hdd = (size_t)n_kv_heads * D * D;
+    // one allocation, carved up (256-byte aligned pieces)
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
+    const size_t o_wt = carve(hdd * sizeof(float));
+    const size_t o_gram = carve(hdd * sizeof(double));
+    const size_t o_part = carve(hdd * sizeof(double) * s->gram_chunks_cap);
+    const size_t o_val = carve((size_t)n_kv_heads * D * sizeof(double));
+    const size_t o_vec = carve(hdd * sizeof(double));
+    char *base = nullptr;
+    if (cudaMalloc(&base, off) != cudaSuccess) { cudaGetLastError(); delete s; return SQUAT_ERR_ALLOC; }
+    if (cudaMemset(base, 0, off) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
+    s->Wt = reinterpret_cast<float *>(base + o_wt);
+    s->gram = reinterpret_cast<double *>(base + o_gram);
+    s->gram_partial = reinterpret_cast<double *>(base + o_part);
+    s->eigval = reinterpret_cast<double *>(base + o_val);
+    s->eigvec = reinterpret_cast<double *>(base + o_vec);
+    s->status = squat_status_word();
+    if (!s->status) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
+    *out = s;
+    return SQUAT_OK;
+}
+
+int squat_subspace_destroy(squat_subspace *s)
+{
+    if (!s) return SQUAT_OK;
+    cudaError_t e = cudaFree(s->Wt);     // Wt is the base of the single allocation
+    delete s;
+    return e == cudaSuccess ? SQUAT_OK : squat_cuda_fail(e);
+}
+
+int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
+                         long long stride_h, long long stride_t, int rank_r, double lambda,
+                         int block_g, void *stream)
+{
+    if (!s || !q || !valid_dtype(dtype) || !aligned16(q)) return SQUAT_ERR_INVALID_ARG;
+    if (n_q_heads <= 0 || n_tokens <= 0) return SQUAT_ERR_INVALID_ARG;
+    if (n_q_heads % s->n_kv_heads != 0) return SQUAT_ERR_SHAPE;
+    if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
+    if ((long long)rank_r > (long long)n_tokens * (n_q_heads / s->n_kv_heads)) return SQUAT_ERR_SHAPE;
+    if (!(lambda >= 0.0) || !std::isfinite(lambda)) return SQUAT_ERR_INVALID_ARG;
+    if (block_g <= 0 || D % block_g != 0) return SQUAT_ERR_SHAPE;
+    const long long vec = 16 / (long long)elem_size(dtype);
+    if (stride_t < D || stride_h < 0 || stride_t % vec || stride_h % vec) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = squat_launch_gram(s, q, dtype, n_q_heads, n_tokens, stride_h, stride_t, st);
+    if (rc != SQUAT_OK) return rc;
+    rc = squat_launch_eig(s, st);
+    if (rc != SQUAT_OK) return rc;
+    return squat_launch_assemble(s, rank_r, lambda, block_g, st);
+}
+
+int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,
+                          double *eigval_host, double *eigvec_host)
+{
+    if (!s) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t hdd = (size_t)s->n_kv_heads * D * D;
+    std::vector<float> wt;
+    if (W_host) {
+        wt.resize(hdd);
+        SQUAT_CUDA(cudaMemcpyAsync(wt.data(), s->Wt, hdd * sizeof(float), cudaMemcpyDeviceToHost, st));
+    }
+    if (gram_host) SQUAT_CUDA(cudaMemcpyAsync(gram_host, s->gram, hdd * sizeof(double), cudaMemcpyDeviceToHost, st));
+    if (eigval_host) SQUAT_CUDA(cudaMemcpyAsync(eigval_host, s->eigval, (size_t)s->n_kv_heads * D * sizeof(double), cudaMemcpyDeviceToHost, st));
+    if (eigvec_host) SQUAT_CUDA(cudaMemcpyAsync(eigvec_host, s->eigvec, hdd * sizeof(double), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaStreamSynchronize(st));
+    if (W_host)
+        for (int h = 0; h < s->n_kv_heads; ++h)
+            for (int j = 0; j < D; ++j)
+                for (int jp = 0; jp < D; ++jp)
+                    W_host[((size_t)h * D + jp) * D + j] = wt[((size_t)h * D + j) * D + jp];
+    return SQUAT_OK;
+}
+
+int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
+{
+    if (!s || !W_host) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t hdd = (size_t)s->n_kv_heads * D * D;
+    std::vector<float> wt(hdd);
+    for (int h = 0; h < s->n_kv_heads; ++h)
+        for (int j = 0; j < D; ++j)
+            for (int jp = 0; jp < D; ++jp)
+                wt[((size_t)h * D + j) * D + jp] = W_host[((size_t)h * D + jp) * D + j];
+    SQUAT_CUDA(cudaMemcpyAsync(s->Wt, wt.data(), hdd * sizeof(float), cudaMemcpyHostToDevice, st));
+    SQUAT_CUDA(cudaStreamSynchronize(st));
+    return SQUAT_OK;
+}
+
+int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
+                        int n_tokens, int head_dim, long long stride_b, long long stride_h,
+                        long long stride_t, int bits, int group_size, unsigned char *codes,
+                        float *scales, float *zeros, long long out_stride_b, long long out_stride_h,
+                        void *stream)
+{
+    if (!s) return SQUAT_ERR_INVALID_ARG;
+    int rc = check_quant_args(k, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
+                              group_size, codes, scales, zeros, out_stride_b, out_stride_h);
+    if (rc != SQUAT_OK) return rc;
+    if (head_dim != D) return SQUAT_ERR_UNSUPPORTED;
+    if (n_kv_heads != s->n_kv_heads) return SQUAT_ERR_SHAPE;
+    if (n_tokens % group_size != 0 || out_stride_b % group_size != 0 || out_stride_h % group_size != 0)
+        return SQUAT_ERR_SHAPE;
+    return squat_launch_quant_keys(s->Wt, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
+                                   group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status,
+                                   static_cast<cudaStream_t>(stream));
+}
+
+int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
+                          int head_dim, long long stride_b, long long stride_h, long long stride_t,
+                          int bits, int group_size, unsigned char *codes, float *scales, float *zeros,
+                          long long out_stride_b, long long out_stride_h, void *stream)
+{
+    int rc = check_quant_args(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
+                              group_size, codes, scales, zeros, out_stride_b, out_stride_h);
+    if (rc != SQUAT_OK) return rc;
+    if (head_dim % group_size != 0 || (head_dim * bits) % 64 != 0) return SQUAT_ERR_SHAPE;
+    unsigned *status = squat_status_word();
+    if (!status) return SQUAT_ERR_CUDA;
+    return squat_launch_quant_values(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t,
+                                     bits, group_size, codes, scales, zeros, out_stride_b, out_stride_h, status,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+int squat_dequantize(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+                     int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                     long long in_stride_b, long long in_stride_h, void *out, int out_dtype, void *stream)
+{
+    if (!codes || !scales || !zeros || !out || !valid_dtype(out_dtype)) return SQUAT_ERR_INVALID_ARG;
+    if (kind != SQUAT_KEYS && kind != SQUAT_VALUES) return SQUAT_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(scales) || !aligned16(zeros) || !aligned16(out)) return SQUAT_ERR_INVALID_ARG;
+    if (batch < 0 || n_kv_heads <= 0 || n_tokens < 0 || head_dim <= 0 || in_stride_b < 0 || in_stride_h < 0)
+        return SQUAT_ERR_INVALID_ARG;
+    if (bits != 2 && bits != 4) return SQUAT_ERR_UNSUPPORTED;
+    if (group_size != 32 && group_size != 64 && group_size != 128) return SQUAT_ERR_UNSUPPORTED;
+    if (head_dim % 16 != 0) return SQUAT_ERR_SHAPE;
+    if (kind == SQUAT_KEYS && (n_tokens % group_size || in_stride_b % group_size || in_stride_h % group_size))
+        return SQUAT_ERR_SHAPE;
+    if (kind == SQUAT_VALUES && head_dim % group_size) return SQUAT_ERR_SHAPE;
+    return squat_launch_dequant(kind, codes, scales, zeros, batch, n_kv_heads, n_tokens, head_dim, bits, group_size,
+                                in_stride_b, in_stride_h, out, out_dtype, static_cast<cudaStream_t>(stream));
+}
+
+int squat_get_device_status(void *stream, unsigned *flags, int clear)
+{
+    if (!flags) return SQUAT_ERR_INVALID_ARG;
+    unsigned *w = squat_status_word();
+    if (!w) return SQUAT_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SQUAT_CUDA(cudaMemcpyAsync(flags, w, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+    if (clear) SQUAT_CUDA(cudaMemsetAsync(w, 0, sizeof(unsigned), st));
+    SQUAT_CUDA(cudaStreamSynchronize(st));
+    return SQUAT_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Whole write path from host buffers.
+namespace {
+struct HostPathLayout {
+    size_t q, k, v, kc, ks, kz, vc, vs, vz, total;
+};
+HostPathLayout host_layout(int dtype, int batch, int n_q, int H, int T, int d, int bits, int G)
+{
+    HostPathLayout L;
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
+    const size_t es = elem_size(dtype);
+    const size_t toks = (size_t)batch * H * T;
+    L.q = carve((size_t)n_q * T * d * es);
+    L.k = carve(toks * d * es);
+    L.v = carve(toks * d * es);
+    L.kc = carve(toks * d * bits / 8);
+    L.ks = carve(toks / G * d * sizeof(float));
+    L.kz = carve(toks / G * d * sizeof(float));
+    L.vc = carve(toks * d * bits / 8);
+    L.vs = carve(toks * (d / G) * sizeof(float));
+    L.vz = carve(toks * (d / G) * sizeof(float));
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t squat_write_path_workspace_bytes(int dtype, int batch, int n_q_heads, int n_kv_heads,
+                                        int n_tokens, int head_dim, int bits, int group_size)
+{
+    if (!valid_dtype(dtype) || batch <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_tokens <= 0 || head_dim <= 0 ||
+        (bits != 2 && bits != 4) || group_size <= 0)
+        return 0;
+    return host_layout(dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, bits, group_size).total;
+}
+
+int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
+                          int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
+                          int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
+                          unsigned char *k_codes_host, float *k_scales_host, float *k_zeros_host,
+                          unsigned char *v_codes_host, float *v_scales_host, float *v_zeros_host,
+                          void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!s || !q_host || !k_host || !v_host || !k_codes_host || !k_scales_host || !k_zeros_host || !v_codes_host ||
+        !v_scales_host || !v_zeros_host || !workspace || !valid_dtype(dtype))
+        return SQUAT_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQUAT_ERR_INVALID_ARG;
+    if (batch <= 0 || n_tokens <= 0 || head_dim != D || n_kv_heads != s->n_kv_heads) return SQUAT_ERR_SHAPE;
+    if ((bits != 2 && bits != 4) || (group_size != 32 && group_size != 64 && group_size != 128))
+        return SQUAT_ERR_UNSUPPORTED;
+    if (n_tokens % group_size) return SQUAT_ERR_SHAPE;
+    const HostPathLayout L = host_layout(dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, bits, group_size);
+    if (workspace_bytes < L.total) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *w = static_cast<char *>(workspace);
+    const size_t es = elem_size(dtype);
+    const size_t toks = (size_t)batch * n_kv_heads * n_tokens;
+    const long long T = n_tokens, d = head_dim;
+    SQUAT_CUDA(cudaMemcpyAsync(w + L.q, q_host, (size_t)n_q_heads * T * d * es, cudaMemcpyHostToDevice, st));
+    SQUAT_CUDA(cudaMemcpyAsync(w + L.k, k_host, toks * d * es, cudaMemcpyHostToDevice, st));
+    SQUAT_CUDA(cudaMemcpyAsync(w + L.v, v_host, toks * d * es, cudaMemcpyHostToDevice, st));
+    int rc = squat_build_subspace(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g, stream);
+    if (rc != SQUAT_OK) return rc;
+    rc = squat_quantize_keys(s, w + L.k, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
+                             T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.kc),
+                             reinterpret_cast<float *>(w + L.ks), reinterpret_cast<float *>(w + L.kz),
+                             (long long)n_kv_heads * T, T, stream);
+    if (rc != SQUAT_OK) return rc;
+    rc = squat_quantize_values(w + L.v, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
+                               T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.vc),
+                               reinterpret_cast<float *>(w + L.vs), reinterpret_cast<float *>(w + L.vz),
+                               (long long)n_kv_heads * T, T, stream);
+    if (rc != SQUAT_OK) return rc;
+    SQUAT_CUDA(cudaMemcpyAsync(k_codes_host, w + L.kc, toks * d * bits / 8, cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(k_scales_host, w + L.ks, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(k_zeros_host, w + L.kz, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(v_codes_host, w + L.vc, toks * d * bits / 8, cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(v_scales_host, w + L.vs, toks * (d / group_size) * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(v_zeros_host, w + L.vz, toks * (d / group_size) * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaStreamSynchronize(st));
+    return SQUAT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,52 @@
+// Internal declarations shared by the translation units of libsquat (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/squat.h"
+
+#define SQUAT_D 128   // the only head dimension the key path and the subspace build are built for
+
+struct squat_subspace {
+    int n_kv_heads;
+    int head_dim;
+    int device;
+    int gram_chunks_cap;   // capacity (in row chunks per head) of gram_partial
+    float *Wt;             // [H, d, d] float32, Wt[h][j][j'] = W[j'][j]  (row j = update vector of channel j)
+    double *gram;          // [H, d, d] Gram matrices
+    double *gram_partial;  // [chunks, H, d, d] per-chunk partial Gram matrices (deterministic reduction)
+    double *eigval;        // [H, d] descending
+    double *eigvec;        // [H, d, d], row i = eigenvector i
+    unsigned *status;      // device status word of this device
+};
+
+// ---- host-side helpers (api.cu) ------------------------------------------------------
+int squat_cuda_fail(cudaError_t e);          // records the error text, returns SQUAT_ERR_CUDA
+unsigned *squat_status_word();               // device address of the status word of the current device
+void squat_count_launch(unsigned n = 1);
+#define SQUAT_CUDA(call) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) return squat_cuda_fail(e__); } while (0)
+#define SQUAT_LAUNCH_CHECK() do { cudaError_t e__ = cudaGetLastError(); if (e__ != cudaSuccess) return squat_cuda_fail(e__); } while (0)
+
+// ---- kernel launchers (one per .cu) ---------------------------------------------------
+int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
+                      long long stride_h, long long stride_t, cudaStream_t st);
+int squat_launch_eig(squat_subspace *s, cudaStream_t st);
+int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st);
+
+int squat_launch_quant_keys(const float *Wt, const void *k, int dtype, int batch, int H, int T,
+                            long long sb, long long sh, long long st_, int bits, int G,
+                            unsigned char *codes, float *scales, float *zeros,
+                            long long osb, long long osh, unsigned *status, cudaStream_t st);
+int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T, int d,
+                              long long sb, long long sh, long long st_, int bits, int G,
+                              unsigned char *codes, float *scales, float *zeros,
+                              long long osb, long long osh, unsigned *status, cudaStream_t st);
+int squat_launch_dequant(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+                         int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
+                         void *out, int out_dtype, cudaStream_t st);
+
+// ---- small device helpers --------------------------------------------------------------
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint4 ldg128(const void *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }

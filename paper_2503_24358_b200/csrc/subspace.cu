@@ -1,0 +1,355 @@
+// Step 1 of the write path: query subspace and update matrices, all in fp64.
+//
+//   gram_kernel      M_h = Qc^T Qc for the stacked prompt queries of KV head h (Section 3.2;
+//                    Algorithm 1 line 5 needs only the right singular vectors and singular values
+//                    of Qc, i.e. the eigen-pairs of M_h; GQA stacking rule of Appendix C).
+//   eig_kernel       eigen-decomposition of M_h by one-sided (Hestenes) Jacobi on the columns of
+//                    M_h itself: rotations make the columns orthogonal, which leaves M V = V diag(mu);
+//                    column norms are the eigenvalues sigma_i^2, normalised columns the v_i.
+//   assemble_kernel  P_inv = (I + lambda Qhat^T Qhat)^{-1} = I - sum_i s_i/(1+s_i) v_i v_i^T with
+//                    s_i = lambda sigma_i^2 (Woodbury with orthonormal v_i; footnote of Prop. 4),
+//                    then the update matrices B_t H_t of Lemma 3 read off the LDL^T factorisation
+//                    P_inv = (I+W) D (I+W)^T: for g = 1, I+W is its unit lower factor (this equals
+//                    the chain of Prop. 2 / Lemma 4 followed by B_t h_t, which the CPU oracle runs
+//                    literally); for g > 1 each block column is multiplied by the inverse of its
+//                    unit-lower diagonal block, which turns the scalar factor into the block one.
+//
+// The cut at rank r can fall between nearly equal eigenvalues whose directions still carry
+// weight lambda sigma^2, so single precision anywhere in this step changes quantized codes
+// downstream; products of bf16 inputs are exact in fp64 and everything stays fp64 until W is
+// rounded to float32 at the very end.
+#include "squat_internal.cuh"
+
+namespace {
+
+constexpr int D = SQUAT_D;
+
+// ------------------------------------------------------------------------------------- Gram
+constexpr int GRAM_THREADS = 160;   // 136 upper-triangular 8x8 tiles of the 16x16 tile grid, 5 warps
+constexpr int GRAM_ROWS = 32;       // rows staged in shared memory per step
+
+template <bool BF16>
+__global__ void __launch_bounds__(GRAM_THREADS) gram_kernel(
+    const void *__restrict__ q, int n_tokens, int q_per_kv, long long stride_h, long long stride_t,
+    int rows_per_chunk, double *__restrict__ partial /* [chunks, H, D, D] */)
+{
+    __shared__ __align__(16) double rows[GRAM_ROWS][D];
+    const int h = blockIdx.y, chunk = blockIdx.x, H = gridDim.y;
+    const long long N = (long long)n_tokens * q_per_kv;
+    const long long row_lo = (long long)chunk * rows_per_chunk;
+    long long row_hi = row_lo + rows_per_chunk;
+    if (row_hi > N) row_hi = N;
+
+    // tile of this thread: (ti <= tj) in the 16 x 16 grid of 8 x 8 tiles
+    int ti = 0, tj = 0;
+    {
+        int t = threadIdx.x, rowlen = 16;
+        while (t >= rowlen && ti < 15) { t -= rowlen; --rowlen; ++ti; }
+        tj = ti + t;
+    }
+    const bool active = threadIdx.x < 136;
+    double acc[8][8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b) acc[a][b] = 0.0;
+
+    for (long long r0 = row_lo; r0 < row_hi; r0 += GRAM_ROWS) {
+        __syncthreads();
+        // stage GRAM_ROWS rows, 8 elements per thread per step
+        for (int idx = threadIdx.x; idx < GRAM_ROWS * (D / 8); idx += GRAM_THREADS) {
+            const int rr = idx / (D / 8), c8 = idx % (D / 8);
+            const long long n = r0 + rr;
+            double v[8];
+            if (n < row_hi) {
+                const long long hq = (long long)h * q_per_kv + n / n_tokens;
+                const long long t = n % n_tokens;
+                const long long off = hq * stride_h + t * stride_t + c8 * 8;
+                if (BF16) {
+                    const uint4 u = ldg128(reinterpret_cast<const __nv_bfloat16 *>(q) + off);
+                    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        v[2 * k] = (double)bf16lo_to_f32(w[k]);
+                        v[2 * k + 1] = (double)bf16hi_to_f32(w[k]);
+                    }
+                } else {
+                    const float4 a = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(q) + off));
+                    const float4 b = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(q) + off) + 1);
+                    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+                    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[k] = 0.0;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) rows[rr][c8 * 8 + k] = v[k];
+        }
+        __syncthreads();
+        if (active) {
+#pragma unroll 4
+            for (int rr = 0; rr < GRAM_ROWS; ++rr) {
+                double a[8], b[8];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const double2 va = *reinterpret_cast<const double2 *>(&rows[rr][ti * 8 + 2 * k]);
+                    const double2 vb = *reinterpret_cast<const double2 *>(&rows[rr][tj * 8 + 2 * k]);
+                    a[2 * k] = va.x; a[2 * k + 1] = va.y;
+                    b[2 * k] = vb.x; b[2 * k + 1] = vb.y;
+                }
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+#pragma unroll
+                    for (int y = 0; y < 8; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
+            }
+        }
+    }
+    if (active) {
+        double *out = partial + ((long long)chunk * H + h) * D * D;
+#pragma unroll
+        for (int x = 0; x < 8; ++x)
+#pragma unroll
+            for (int y = 0; y < 8; ++y) out[(ti * 8 + x) * D + tj * 8 + y] = acc[x][y];
+    }
+}
+
+// Sums the per-chunk partials in a fixed order and mirrors the upper tiles: gram[h] full symmetric.
+__global__ void gram_reduce_kernel(const double *__restrict__ partial, int chunks, int H, double *__restrict__ gram)
+{
+    const int h = blockIdx.y;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= D * D) return;
+    int a = idx / D, b = idx % D;
+    if (a / 8 > b / 8) { const int t = a; a = b; b = t; }       // read from the stored upper tile
+    double s = 0.0;
+    for (int c = 0; c < chunks; ++c) s += partial[((long long)c * H + h) * D * D + a * D + b];
+    gram[(long long)h * D * D + idx] = s;
+}
+
+// ------------------------------------------------------------------------------------- eigen
+constexpr int EIG_THREADS = 512;    // 64 column pairs x 8 lanes
+constexpr int EIG_LD = D + 2;       // padded column stride (doubles)
+constexpr int EIG_MAX_SWEEPS = 40;
+
+__device__ __forceinline__ double team8_sum(double v)
+{
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    return v;
+}
+
+__global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
+    const double *__restrict__ gram, double *__restrict__ eigval, double *__restrict__ eigvec,
+    unsigned *__restrict__ status)
+{
+    extern __shared__ __align__(16) double sm[];
+    double *Gs = sm;                       // column-major: Gs[col * EIG_LD + row]
+    double *nrm = sm + D * EIG_LD;         // squared column norms
+    int *rank = reinterpret_cast<int *>(nrm + D);
+    const int h = blockIdx.x, tid = threadIdx.x;
+    const int team = tid >> 3, l8 = tid & 7;
+    const double *M = gram + (long long)h * D * D;
+
+    for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
+        const int r = idx / D, c = idx % D;
+        Gs[c * EIG_LD + r] = M[idx];       // M symmetric: row/column choice is immaterial
+    }
+    __syncthreads();
+    double trace = 0.0;
+    for (int i = 0; i < D; ++i) trace += Gs[i * EIG_LD + i];
+    const double null_thr = (1e-14 * trace) * (1e-14 * trace);
+    const double tol2 = 1e-14 * 1e-14;
+
+    bool converged = false;
+    for (int sweep = 0; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
+        // refresh the squared norms from the columns (cached values drift by rounding)
+        for (int col = tid >> 3; col < D; col += EIG_THREADS / 8) {
+            double s = 0.0;
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i) { const double v = Gs[col * EIG_LD + l8 + 8 * i]; s = fma(v, v, s); }
+            s = team8_sum(s);
+            if (l8 == 0) nrm[col] = s;
+        }
+        __syncthreads();
+        int any_rot = 0;
+        for (int round = 0; round < D - 1; ++round) {
+            int p, q;
+            if (team == 0) { p = D - 1; q = round; }
+            else { p = (round + team) % (D - 1); q = (round - team + (D - 1)) % (D - 1); }
+            double *gp = Gs + p * EIG_LD + l8, *gq = Gs + q * EIG_LD + l8;
+            double a[D / 8], b[D / 8];
+            double gam = 0.0;
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i) { a[i] = gp[8 * i]; b[i] = gq[8 * i]; gam = fma(a[i], b[i], gam); }
+            gam = team8_sum(gam);
+            const double alpha = nrm[p], beta = nrm[q];
+            int rot = 0;
+            if (alpha > null_thr && beta > null_thr && gam * gam > tol2 * alpha * beta) {
+                // t = tan of the rotation angle: smaller root of t^2 + 2 zeta t - 1 = 0, zeta = (beta-alpha)/(2 gam)
+                const double diff = beta - alpha;
+                const double den = fabs(diff) + sqrt(fma(diff, diff, 4.0 * gam * gam));
+                double t = 2.0 * gam / den;
+                if (diff < 0.0) t = -t;
+                const double c = rsqrt(fma(t, t, 1.0));
+                const double s = t * c;
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) {
+                    gp[8 * i] = c * a[i] - s * b[i];
+                    gq[8 * i] = s * a[i] + c * b[i];
+                }
+                if (l8 == 0) { nrm[p] = alpha - t * gam; nrm[q] = beta + t * gam; }
+                rot = 1;
+            }
+            any_rot |= __syncthreads_or(rot);
+        }
+        converged = (any_rot == 0);
+    }
+    if (!converged && tid == 0) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
+
+    // exact norms, ranks (descending, ties by column index), normalised output
+    for (int col = tid >> 3; col < D; col += EIG_THREADS / 8) {
+        double s = 0.0;
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) { const double v = Gs[col * EIG_LD + l8 + 8 * i]; s = fma(v, v, s); }
+        s = team8_sum(s);
+        if (l8 == 0) nrm[col] = sqrt(s);
+    }
+    __syncthreads();
+    if (tid < D) {
+        const double mine = nrm[tid];
+        int rk = 0;
+        for (int j = 0; j < D; ++j) {
+            const double o = nrm[j];
+            rk += (o > mine) || (o == mine && j < tid);
+        }
+        rank[tid] = rk;
+        eigval[(long long)h * D + rk] = mine;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
+        const int col = idx / D, r = idx % D;
+        const double mu = nrm[col];
+        const double v = mu > 0.0 ? Gs[col * EIG_LD + r] / mu : 0.0;
+        eigvec[(long long)h * D * D + (long long)rank[col] * D + r] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------- assemble
+constexpr int ASM_THREADS = 512;
+constexpr int ASM_LD = D + 1;
+
+__global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
+    const double *__restrict__ eigval, const double *__restrict__ eigvec, int rank_r, double lambda, int g,
+    float *__restrict__ Wt)
+{
+    extern __shared__ __align__(16) double sm[];
+    double *A = sm;                         // A[row * ASM_LD + col]
+    double *colv = sm + D * ASM_LD;         // column j before scaling
+    double *lcol = colv + D;                // column j of L
+    double *coef = lcol + D;                // s_i / (1 + s_i)
+    const int h = blockIdx.x, tid = threadIdx.x;
+    const double *V = eigvec + (long long)h * D * D;
+
+    if (tid < D) {
+        double mu = eigval[(long long)h * D + tid];
+        if (!(mu > 0.0)) mu = 0.0;
+        const double s = lambda * mu;
+        coef[tid] = (tid < rank_r) ? s / (1.0 + s) : 0.0;
+    }
+    __syncthreads();
+    // P_inv = I - sum_{i<r} coef_i v_i v_i^T
+    for (int idx = tid; idx < D * D; idx += ASM_THREADS) {
+        const int a = idx / D, b = idx % D;
+        double s = (a == b) ? 1.0 : 0.0;
+        for (int i = 0; i < rank_r; ++i) s = fma(-coef[i] * V[i * D + a], V[i * D + b], s);
+        A[a * ASM_LD + b] = s;
+    }
+    __syncthreads();
+    // in-place LDL^T (right-looking): afterwards the strict lower triangle of A holds L
+    for (int j = 0; j < D - 1; ++j) {
+        if (tid > j && tid < D) {
+            const double v = A[tid * ASM_LD + j];
+            colv[tid] = v;
+            lcol[tid] = v / A[j * ASM_LD + j];
+        }
+        __syncthreads();
+        const int n = D - 1 - j;
+        for (int idx = tid; idx < n * n; idx += ASM_THREADS) {
+            const int i = j + 1 + idx / n, k = j + 1 + idx % n;
+            A[i * ASM_LD + k] = fma(-lcol[i], colv[k], A[i * ASM_LD + k]);
+        }
+        if (tid > j && tid < D) A[tid * ASM_LD + j] = lcol[tid];
+        __syncthreads();
+    }
+    // g > 1: block column t becomes L[rest, blk] * inverse(unit-lower diagonal block)
+    if (g > 1) {
+        const int T = D / g;
+        for (int idx = tid; idx < D * (T - 1); idx += ASM_THREADS) {
+            const int row = idx % D, t = idx / D;          // block t: columns [t*g, (t+1)*g)
+            const int c0 = t * g;
+            if (row < c0 + g) continue;
+            double *x = A + row * ASM_LD + c0;
+            for (int c = g - 2; c >= 0; --c) {
+                double s = x[c];
+                for (int cp = c + 1; cp < g; ++cp) s = fma(-x[cp], A[(c0 + cp) * ASM_LD + c0 + c], s);
+                x[c] = s;
+            }
+        }
+        __syncthreads();
+    }
+    // Wt[j][j'] = W[j'][j]: zero on and above the block diagonal
+    float *out = Wt + (long long)h * D * D;
+    for (int idx = tid; idx < D * D; idx += ASM_THREADS) {
+        const int j = idx / D, jp = idx % D;
+        const int blk_end = (j / g + 1) * g;
+        out[idx] = (jp >= blk_end) ? (float)A[jp * ASM_LD + j] : 0.0f;
+    }
+}
+
+}  // namespace
+
+int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
+                      long long stride_h, long long stride_t, cudaStream_t st)
+{
+    const int H = s->n_kv_heads, qpk = n_q_heads / H;
+    const long long N = (long long)n_tokens * qpk;
+    int chunks = s->gram_chunks_cap;
+    long long rows_per_chunk = (N + chunks - 1) / chunks;
+    rows_per_chunk = (rows_per_chunk + GRAM_ROWS - 1) / GRAM_ROWS * GRAM_ROWS;
+    if (rows_per_chunk < 2 * GRAM_ROWS) rows_per_chunk = 2 * GRAM_ROWS;
+    chunks = (int)((N + rows_per_chunk - 1) / rows_per_chunk);
+    if (chunks < 1) chunks = 1;
+    dim3 grid(chunks, H);
+    if (dtype == SQUAT_BF16)
+        gram_kernel<true><<<grid, GRAM_THREADS, 0, st>>>(q, n_tokens, qpk, stride_h, stride_t, (int)rows_per_chunk, s->gram_partial);
+    else
+        gram_kernel<false><<<grid, GRAM_THREADS, 0, st>>>(q, n_tokens, qpk, stride_h, stride_t, (int)rows_per_chunk, s->gram_partial);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    gram_reduce_kernel<<<dim3(D * D / 256, H), 256, 0, st>>>(s->gram_partial, chunks, H, s->gram);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}
+
+int squat_launch_eig(squat_subspace *s, cudaStream_t st)
+{
+    const size_t smem = sizeof(double) * (D * EIG_LD + D) + sizeof(int) * D;
+    SQUAT_CUDA(cudaFuncSetAttribute(eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    eig_kernel<<<s->n_kv_heads, EIG_THREADS, smem, st>>>(s->gram, s->eigval, s->eigvec, s->status);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}
+
+int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st)
+{
+    const size_t smem = sizeof(double) * (D * ASM_LD + 3 * D);
+    SQUAT_CUDA(cudaFuncSetAttribute(assemble_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}

@@ -1,0 +1,257 @@
+// Per-token value quantization (Section 2 "Quantization"; Appendix C: d channels of a token in
+// d/G groups of G) and dequantization (deq(c) = c * Delta + m) for both cache layouts.
+//
+// HBM-bound streaming kernels.  One thread owns one (token, channel-group): it reads its G
+// consecutive channels with 128-bit loads (consecutive lanes read consecutive 16*G/8-byte
+// pieces, so a warp covers a contiguous span), reduces min/max in registers, and writes
+// G*b/8 code bytes plus one scale and one zero -- all contiguous across the warp.
+//
+// The rounding decision is the IEEE binary32 sequence  Delta = (M-m)/L, t = (x-m)/Delta,
+// c = clamp(rint(t), 0, L).  The fast path multiplies by RN(1/Delta) and rounds once; it can
+// differ from the sequence above only when t is within ~1e-6 of a half-integer, so any
+// element within 1e-5 of one is redone with a correctly rounded division.
+#include "squat_internal.cuh"
+
+namespace {
+
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
+constexpr float kTieBand = 0.5f - 1e-5f;
+
+template <int G, int BITS, bool BF16>
+__global__ void __launch_bounds__(256) quant_values_kernel(
+    const void *__restrict__ v, long long n_units, int H, int T, int ng,
+    long long sb, long long sh, long long st, unsigned char *__restrict__ codes,
+    float *__restrict__ scales, float *__restrict__ zeros, long long osb, long long osh,
+    int row_bytes, unsigned *__restrict__ status)
+{
+    constexpr float L = float((1 << BITS) - 1);
+    constexpr int PER_WORD = 32 / BITS;
+    constexpr int NWORDS = G / PER_WORD;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < n_units; u += stride) {
+        const int q = (int)(u % ng);
+        const long long tok = u / ng;
+        const int t = (int)(tok % T);
+        const long long bh = tok / T;
+        const int h = (int)(bh % H);
+        const long long b = bh / H;
+        const long long in_off = b * sb + h * sh + (long long)t * st + (long long)q * G;
+        const long long out_tok = b * osb + h * osh + t;
+
+        float x[G];
+        float m, Mx;
+        if (BF16) {
+            const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(v) + in_off);
+            __nv_bfloat162 mn2, mx2;
+#pragma unroll
+            for (int i = 0; i < G / 8; ++i) {
+                const uint4 r = ldg128(p + i);
+                const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    x[i * 8 + 2 * k] = bf16lo_to_f32(w[k]);
+                    x[i * 8 + 2 * k + 1] = bf16hi_to_f32(w[k]);
+                    __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[k]);
+                    if (i == 0 && k == 0) { mn2 = pr; mx2 = pr; }
+                    else { mn2 = __hmin2(mn2, pr); mx2 = __hmax2(mx2, pr); }
+                }
+            }
+            m = fminf(__low2float(mn2), __high2float(mn2));
+            Mx = fmaxf(__low2float(mx2), __high2float(mx2));
+        } else {
+            const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(v) + in_off);
+#pragma unroll
+            for (int i = 0; i < G / 4; ++i) {
+                const uint4 r = ldg128(p + i);
+                x[i * 4 + 0] = __uint_as_float(r.x);
+                x[i * 4 + 1] = __uint_as_float(r.y);
+                x[i * 4 + 2] = __uint_as_float(r.z);
+                x[i * 4 + 3] = __uint_as_float(r.w);
+            }
+            m = x[0]; Mx = x[0];
+#pragma unroll
+            for (int i = 1; i < G; ++i) { m = fminf(m, x[i]); Mx = fmaxf(Mx, x[i]); }
+        }
+
+        const float delta = __fdiv_rn(__fsub_rn(Mx, m), L);
+        const bool ok = delta > 0.0f && delta < __int_as_float(0x7f800000);
+        const float rcp = ok ? __frcp_rn(delta) : 0.0f;
+        if (!ok) atomicOr(status, delta == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
+
+        uint32_t words[NWORDS];
+        float worst = 0.0f;
+#pragma unroll
+        for (int wd = 0; wd < NWORDS; ++wd) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int k = 0; k < PER_WORD; ++k) {
+                const float dlt = __fsub_rn(x[wd * PER_WORD + k], m);
+                const float y = __fmaf_rn(dlt, rcp, kMagic);
+                const float c = __fsub_rn(y, kMagic);
+                const float res = __fmaf_rn(dlt, rcp, -c);
+                worst = fmaxf(worst, fabsf(res));
+                acc |= (__float_as_uint(y) & ((1u << BITS) - 1u)) << (k * BITS);
+            }
+            words[wd] = acc;
+        }
+        if (worst >= kTieBand && ok) {
+            // some element sits next to a rounding midpoint: redo the group with exact divisions
+#pragma unroll
+            for (int wd = 0; wd < NWORDS; ++wd) {
+                uint32_t acc = 0;
+#pragma unroll
+                for (int k = 0; k < PER_WORD; ++k) {
+                    const float tt = __fdiv_rn(__fsub_rn(x[wd * PER_WORD + k], m), delta);
+                    const float c = fminf(fmaxf(rintf(tt), 0.0f), L);
+                    acc |= ((uint32_t)(int)c) << (k * BITS);
+                }
+                words[wd] = acc;
+            }
+        }
+
+        unsigned char *cp = codes + out_tok * row_bytes + (long long)q * (G * BITS / 8);
+        if (NWORDS % 4 == 0) {
+#pragma unroll
+            for (int i = 0; i < NWORDS / 4; ++i)
+                reinterpret_cast<uint4 *>(cp)[i] = make_uint4(words[4 * i], words[4 * i + 1], words[4 * i + 2], words[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < NWORDS / 2; ++i)
+                reinterpret_cast<uint2 *>(cp)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
+        }
+        scales[out_tok * ng + q] = delta;
+        zeros[out_tok * ng + q] = m;
+    }
+}
+
+// One thread dequantizes 16 consecutive channels of one token.
+template <int BITS, bool KEYS, bool OUT_BF16>
+__global__ void __launch_bounds__(256) dequant_kernel(
+    const unsigned char *__restrict__ codes, const float *__restrict__ scales, const float *__restrict__ zeros,
+    long long n_units, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
+{
+    const int per_tok = d / 16;
+    const int row_bytes = d * BITS / 8;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < n_units; u += stride) {
+        const int c16 = (int)(u % per_tok);
+        const long long tok = u / per_tok;
+        const int t = (int)(tok % T);
+        const long long bh = tok / T;
+        const int h = (int)(bh % H);
+        const long long b = bh / H;
+        const long long in_tok = b * isb + h * ish + t;
+        const unsigned char *cp = codes + in_tok * row_bytes + c16 * (16 * BITS / 8);
+        uint32_t w[2];
+        if (BITS == 2) { w[0] = *reinterpret_cast<const uint32_t *>(cp); w[1] = 0; }
+        else { const uint2 r = *reinterpret_cast<const uint2 *>(cp); w[0] = r.x; w[1] = r.y; }
+        float sc[16], zr[16];
+        if (KEYS) {
+            const long long base = (b * (isb / G) + h * (ish / G) + t / G) * d + c16 * 16;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 s4 = __ldg(reinterpret_cast<const float4 *>(scales + base) + i);
+                const float4 z4 = __ldg(reinterpret_cast<const float4 *>(zeros + base) + i);
+                sc[4 * i] = s4.x; sc[4 * i + 1] = s4.y; sc[4 * i + 2] = s4.z; sc[4 * i + 3] = s4.w;
+                zr[4 * i] = z4.x; zr[4 * i + 1] = z4.y; zr[4 * i + 2] = z4.z; zr[4 * i + 3] = z4.w;
+            }
+        } else {
+            const long long mi = in_tok * (d / G) + (c16 * 16) / G;
+            const float s = __ldg(scales + mi), z = __ldg(zeros + mi);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { sc[i] = s; zr[i] = z; }
+        }
+        float y[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int bit = i * BITS;
+            const float c = (float)((w[bit / 32] >> (bit % 32)) & ((1u << BITS) - 1u));
+            y[i] = __fmaf_rn(c, sc[i], zr[i]);
+        }
+        const long long o = ((bh * T) + t) * d + c16 * 16;
+        if (OUT_BF16) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                __nv_bfloat162 p2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                pk[i] = *reinterpret_cast<uint32_t *>(&p2);
+            }
+            uint4 *op = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(out) + o);
+            op[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            op[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        } else {
+            float4 *op = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + o);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) op[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+        }
+    }
+}
+
+int grid_for(long long n_threads, int block)
+{
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    long long blocks = (n_threads + block - 1) / block;
+    const long long cap = (long long)sms * 8;           // a multiple of the SM count; grid-stride covers the rest
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+template <int G, int BITS>
+int launch_values(const void *v, int dtype, long long n_units, int H, int T, int ng, long long sb, long long sh,
+                  long long st_, unsigned char *codes, float *scales, float *zeros, long long osb, long long osh,
+                  int row_bytes, unsigned *status, cudaStream_t st)
+{
+    const int grid = grid_for(n_units, 256);
+    if (dtype == SQUAT_BF16)
+        quant_values_kernel<G, BITS, true><<<grid, 256, 0, st>>>(v, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status);
+    else
+        quant_values_kernel<G, BITS, false><<<grid, 256, 0, st>>>(v, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}
+
+}  // namespace
+
+int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T, int d,
+                              long long sb, long long sh, long long st_, int bits, int G,
+                              unsigned char *codes, float *scales, float *zeros,
+                              long long osb, long long osh, unsigned *status, cudaStream_t st)
+{
+    const int ng = d / G;
+    const long long n_units = (long long)batch * H * T * ng;
+    if (n_units == 0) return SQUAT_OK;
+    const int row_bytes = d * bits / 8;
+#define SQ_V(GG, BB) return launch_values<GG, BB>(v, dtype, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status, st)
+    if (bits == 2) { if (G == 32) SQ_V(32, 2); if (G == 64) SQ_V(64, 2); if (G == 128) SQ_V(128, 2); }
+    if (bits == 4) { if (G == 32) SQ_V(32, 4); if (G == 64) SQ_V(64, 4); if (G == 128) SQ_V(128, 4); }
+#undef SQ_V
+    return SQUAT_ERR_UNSUPPORTED;
+}
+
+int squat_launch_dequant(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+                         int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
+                         void *out, int out_dtype, cudaStream_t st)
+{
+    const long long n_units = (long long)batch * H * T * (d / 16);
+    if (n_units == 0) return SQUAT_OK;
+    const int grid = grid_for(n_units, 256);
+#define SQ_D(BB, KK, OO) dequant_kernel<BB, KK, OO><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out)
+    const bool keys = kind == SQUAT_KEYS, obf = out_dtype == SQUAT_BF16;
+    if (bits == 2) {
+        if (keys) { if (obf) SQ_D(2, true, true); else SQ_D(2, true, false); }
+        else { if (obf) SQ_D(2, false, true); else SQ_D(2, false, false); }
+    } else if (bits == 4) {
+        if (keys) { if (obf) SQ_D(4, true, true); else SQ_D(4, true, false); }
+        else { if (obf) SQ_D(4, false, true); else SQ_D(4, false, false); }
+    } else {
+        return SQUAT_ERR_UNSUPPORTED;
+    }
+#undef SQ_D
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}

@@ -1,0 +1,128 @@
+"""Helpers of the GPU-vs-oracle parity tests: tensor marshalling and the comparison protocol.
+
+Protocol for keys.  The key quantizer rounds values that earlier roundings have corrected, so a
+rounding tie resolved the other way (legitimate: both neighbours are nearest) changes everything
+downstream of it in that token, and through the shared min/max possibly in its group.  Codes are
+therefore compared like this: per group, find the earliest channel where GPU and oracle codes
+differ; every differing element of that channel must be a tie in the oracle's own arithmetic
+(|frac((x - zero)/scale) - 0.5| < 1e-5) and differ by exactly one level; force the GPU's choice
+there, re-run the oracle on that group, repeat.  The run passes iff every forced decision was such
+a tie and nothing differs afterwards.  The raw (pre-replay) identical fraction is reported too and
+must be >= 99.9 %.
+"""
+import numpy as np
+import torch
+
+import oracle
+import squat_inputs as si
+
+TIE_BAND = 1e-5
+
+
+def to_torch(a: np.ndarray, dtype: str, device="cuda") -> torch.Tensor:
+    """Generator output (float32 array or uint16 bf16 bit patterns) -> torch tensor on device."""
+    if dtype == "f32":
+        return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+    return t.to(device)
+
+
+def from_torch_bf16(t: torch.Tensor) -> np.ndarray:
+    """torch bf16 tensor -> float32 numpy, exact."""
+    return si.bf16_bits_to_f32(t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16))
+
+
+def stacked_queries(cfg, h, n_tokens=None) -> np.ndarray:
+    """Rows = all prompt tokens of the query heads feeding KV head h (float64, exact widening)."""
+    qs = [si.to_f32(si.gen_queries_head(cfg, hq, n_tokens), cfg.dtype)
+          for hq in range(h * cfg.q_per_kv, (h + 1) * cfg.q_per_kv)]
+    return np.concatenate(qs, axis=0).astype(np.float64)
+
+
+def oracle_mats(cfg, h, n_tokens=None, rank_r=None, lam=None, g=None):
+    return oracle.build_W(stacked_queries(cfg, h, n_tokens), cfg.rank_r if rank_r is None else rank_r,
+                          cfg.lam if lam is None else lam, cfg.block_g if g is None else g)
+
+
+def alloc_key_outputs(B, H, T, d, bits, G, device="cuda"):
+    codes = torch.empty((B, H, T, d * bits // 8), dtype=torch.uint8, device=device)
+    scales = torch.empty((B, H, T // G, d), dtype=torch.float32, device=device)
+    zeros = torch.empty((B, H, T // G, d), dtype=torch.float32, device=device)
+    return codes, scales, zeros
+
+
+def alloc_value_outputs(B, H, T, d, bits, G, device="cuda"):
+    codes = torch.empty((B, H, T, d * bits // 8), dtype=torch.uint8, device=device)
+    scales = torch.empty((B, H, T, d // G), dtype=torch.float32, device=device)
+    zeros = torch.empty((B, H, T, d // G), dtype=torch.float32, device=device)
+    return codes, scales, zeros
+
+
+def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=None, Qhat=None, max_replays=64):
+    """Compares one (batch, head) unit.  K64 [n,d] float64; gpu_codes [n,d] unpacked uint8;
+    gpu_scale/zero [n/G, d] float32; gpu_deq [n,d] float32 (optional).  Returns a dict of statistics;
+    raises AssertionError with a precise message on any violation of the protocol."""
+    n, d = K64.shape
+    base = oracle.quant_keys(K64, G, bits, W64, want_tval=True)
+    raw_equal = int((base["codes"] == gpu_codes).sum())
+    ties = 0
+    final_codes = base["codes"].copy()
+    final_khat = base["Khat"].copy()
+    final_scale, final_zero = base["scale"].copy(), base["zero"].copy()
+    bad_groups = np.unique(np.nonzero(base["codes"] != gpu_codes)[0] // G)
+    for grp in bad_groups:
+        lo, hi = grp * G, (grp + 1) * G
+        force = -np.ones((G, d), dtype=np.int16)
+        o = {k: v[lo:hi] if k in ("codes", "Khat", "tval") else v[grp:grp + 1] for k, v in base.items()}
+        for _ in range(max_replays):
+            diff = o["codes"] != gpu_codes[lo:hi]
+            if not diff.any():
+                break
+            j0 = int(np.nonzero(diff.any(axis=0))[0][0])
+            for i in np.nonzero(diff[:, j0])[0]:
+                t = o["tval"][i, j0]
+                frac = abs((t - np.floor(t)) - 0.5)
+                cg, co = int(gpu_codes[lo + i, j0]), int(o["codes"][i, j0])
+                assert abs(cg - co) == 1 and frac < TIE_BAND, (
+                    f"non-tie mismatch: group {grp} token {i} channel {j0}: gpu {cg} oracle {co} "
+                    f"t={t!r} |frac-0.5|={frac:.3e}")
+                force[i, j0] = cg
+                ties += 1
+            o = oracle.quant_keys(K64[lo:hi], G, bits, W64, force=force, want_tval=True)
+        else:
+            raise AssertionError(f"group {grp}: replay did not converge")
+        final_codes[lo:hi] = o["codes"]
+        final_khat[lo:hi] = o["Khat"]
+        final_scale[grp], final_zero[grp] = o["scale"][0], o["zero"][0]
+    assert np.array_equal(final_codes, gpu_codes)
+    stats = {"elements": n * d, "raw_equal": raw_equal, "ties": ties, "raw_fraction": raw_equal / (n * d)}
+    # scale / zero: float32 roundings of fp64 vs fp32 working values
+    sc_err = np.abs(gpu_scale.astype(np.float64) - final_scale).max() / max(np.abs(final_scale).max(), 1e-30)
+    zr_err = np.abs(gpu_zero.astype(np.float64) - final_zero).max() / max(np.abs(final_zero).max(), 1e-30)
+    stats["scale_rel_err"], stats["zero_rel_err"] = float(sc_err), float(zr_err)
+    assert sc_err < 1e-4 and zr_err < 1e-4, (sc_err, zr_err)
+    if gpu_deq is not None:
+        rel = np.linalg.norm(gpu_deq.astype(np.float64) - final_khat) / np.linalg.norm(final_khat)
+        stats["deq_rel_fro"] = float(rel)
+        assert rel < 1e-3, rel
+        if Qhat is not None and Qhat.shape[0] > 0:
+            pg = np.linalg.norm((gpu_deq.astype(np.float64) - K64) @ Qhat.T)
+            po = np.linalg.norm((final_khat - K64) @ Qhat.T)
+            stats["proj_rel"] = float(abs(pg - po) / po)
+            assert abs(pg - po) <= 1e-3 * po, (pg, po)
+    return stats
+
+
+def rtn_per_channel_f32(K32, G, bits):
+    """Per-channel round-to-nearest over groups of G tokens in binary32, through the oracle's
+    per-token routine applied to the transposed groups."""
+    n, d = K32.shape
+    codes = np.empty((n, d), dtype=np.uint8)
+    scale = np.empty((n // G, d), dtype=np.float32)
+    zero = np.empty((n // G, d), dtype=np.float32)
+    for grp in range(n // G):
+        blk = np.ascontiguousarray(K32[grp * G:(grp + 1) * G].T)      # [d, G]
+        o = oracle.quant_values_f32(blk, G, bits)
+        codes[grp * G:(grp + 1) * G] = o["codes"].T
+        scale[grp], zero[grp] = o["scale"][:, 0], o["zero"][:, 0]
+    return codes, scale, zero
