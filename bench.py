@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the SQuat KV-cache write path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
+
+One "step" is one pass of the whole write path over one layer-batch of synthetic input:
+subspace build (Gram, eigen-decomposition, update matrices) -> key quantization -> value
+quantization -> dequantization of both (the read-back).  Default workload: config 1, the
+Llama-2-7B-shaped layer (32 heads x 4096 tokens x 128, bf16, r = 32, 2 bits, G = 32).
+Inputs are resident in HBM before the timed region; L2 is flushed between steps; every step
+and every stage is timed with CUDA events on the launching stream; with N > 1 ranks each
+rank processes its own replica of the workload (the path has no exchange step) and the
+slowest rank's time counts.  Prints ONE JSON line on rank 0.
+
+`--impl reference` times the CPU oracle (plain single-threaded fp64 C, as it stands) on a bounded
+sample of the same workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import squat_inputs as si  # noqa: E402
+
+METRIC = "key vectors quantized/sec (whole write path: subspace build + keys + values + dequantize)"
+UNIT = "key_vectors/s"
+
+# Nominal FP32 peak of a B200: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz (max SM clock).
+SM_COUNT, FMA_LANES, SM_MAX_GHZ = 148, 128, 1.965
+ALU_PEAK_TFLOPS = SM_COUNT * FMA_LANES * 2 * SM_MAX_GHZ / 1e3
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the key kernel, from the ncu capture
+# summarised under profiles/ (None until a capture exists for that workload).
+NCU_KEY_KERNEL_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- algorithmic counts
+def key_flops_per_vector(d, g):
+    """2 x FMAs of the dense block-triangular update (Eq. (3) / Eq. (update_block))."""
+    T = d // g
+    return 2 * sum(g * (d - t * g) for t in range(1, T))
+
+
+def bytes_per_vector(d, bits, G, elem_bytes):
+    """Algorithmic HBM bytes per key (or value) vector: read the vector, write codes + fp32 scale/zero."""
+    return d * elem_bytes + d * bits // 8 + 8 * d // G
+
+
+# --------------------------------------------------------------------------- clocks sampling
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu_index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- distributed glue
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate_over_ranks(local_ms, local_units, device=None):
+    """Whole-job figures: time = max over ranks, units = sum over ranks.  Works on any backend."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return local_ms, local_units
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([float(local_units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(round(u.item()))
+
+
+# --------------------------------------------------------------------------- the CPU oracle legs
+def oracle_pass(cfg, heads, n_tokens):
+    """The oracle's whole path for the given KV heads of sample 0.  Returns key vectors processed."""
+    import oracle
+    for h in heads:
+        qs = [si.to_f32(si.gen_queries_head(cfg, hq, n_tokens), cfg.dtype)
+              for hq in range(h * cfg.q_per_kv, (h + 1) * cfg.q_per_kv)]
+        Qc = np.concatenate(qs, 0).astype(np.float64)
+        K = si.to_f32(si.gen_keys_unit(cfg, 0, h, n_tokens), cfg.dtype)
+        V = si.to_f32(si.gen_values_unit(cfg, 0, h, n_tokens), cfg.dtype)
+        t0 = time.perf_counter()
+        mats = oracle.build_W(Qc, cfg.rank_r, cfg.lam, cfg.block_g)
+        ok = oracle.quant_keys(K.astype(np.float64), cfg.group_size, cfg.bits, mats["W"])
+        ov = oracle.quant_values_f32(V, cfg.group_size, cfg.bits)
+        oracle.dequant_keys(ok["codes"], ok["scale"], ok["zero"], cfg.group_size)
+        oracle.dequant_values(ov["codes"], ov["scale"], ov["zero"], cfg.group_size)
+        yield time.perf_counter() - t0, n_tokens
+
+
+def cpu_baseline(cfg, budget_s=12.0):
+    """Times the oracle (as it stands, 1 thread) on a bounded sample: as many KV heads of sample 0 as fit
+    in the budget (at least one)."""
+    import oracle
+    oracle.build()
+    spent, vecs, heads = 0.0, 0, 0
+    for dt, n in oracle_pass(cfg, range(cfg.n_kv_heads), cfg.n_tokens):
+        spent += dt; vecs += n; heads += 1
+        if spent > budget_s:
+            break
+    return {"value": vecs / spent, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{heads} of {cfg.n_kv_heads} KV heads of sample 0 of {cfg.name} (all {cfg.n_tokens} tokens each): "
+                      f"subspace build + keys + values + dequantize, {spent:.1f} s of CPU time"}
+
+
+def run_reference(args, cfg):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    heads_per_step = 2
+    times = []
+    it = 0
+    for step in range(args.warmup + args.steps):
+        heads = [(it + i) % cfg.n_kv_heads for i in range(heads_per_step)]
+        it += heads_per_step
+        dt = sum(t for t, _ in oracle_pass(cfg, heads, cfg.n_tokens))
+        if step >= args.warmup:
+            times.append(dt)
+    vec_per_step = heads_per_step * cfg.n_tokens
+    total = sum(times)
+    value = vec_per_step * len(times) / total
+    sample = (f"each step = {heads_per_step} KV heads of sample 0 of {cfg.name}, all {cfg.n_tokens} tokens: "
+              "subspace build + keys + values + dequantize")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg), "gpu_launches": 0,
+            "cpu_baseline": {"value": value, "unit": UNIT, "kind": "oracle", "cores": 1, "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": f"config {cfg.index}: {cfg.name}", "dtype": cfg.dtype, "batch": cfg.batch,
+            "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
+            "n_tokens": cfg.n_tokens, "rank_r": cfg.rank_r, "bits": cfg.bits, "group_size": cfg.group_size,
+            "lambda": cfg.lam, "block_g": cfg.block_g, "l2": "flushed between steps (512 MiB write)",
+            "parallelism": "independent replicas per GPU (no collective on the data path)"}
+
+
+# --------------------------------------------------------------------------- the GPU arm
+def run_gpu(args, cfg):
+    import torch
+    import torch.distributed as dist
+    import paper_2503_24358_b200 as sq
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the write path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group(backend="nccl", device_id=dev)
+
+    def to_dev(a, pin=False):
+        if cfg.dtype == "f32":
+            t = torch.from_numpy(np.ascontiguousarray(a))
+        else:
+            t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+        return t.pin_memory() if pin else t.to(dev)
+
+    B, H, T, d, bits, G = cfg.batch, cfg.n_kv_heads, cfg.n_tokens, cfg.head_dim, cfg.bits, cfg.group_size
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    q_np, k_np, v_np = si.gen_queries(cfg), si.gen_keys(cfg), si.gen_values(cfg)
+    q, k, v = to_dev(q_np), to_dev(k_np), to_dev(v_np)
+    kc = torch.empty((B, H, T, d * bits // 8), dtype=torch.uint8, device=dev)
+    ks = torch.empty((B, H, T // G, d), dtype=torch.float32, device=dev)
+    kz = torch.empty_like(ks)
+    vc = torch.empty_like(kc)
+    vs = torch.empty((B, H, T, d // G), dtype=torch.float32, device=dev)
+    vz = torch.empty_like(vs)
+    kd = torch.empty((B, H, T, d), dtype=tdt, device=dev)
+    vd = torch.empty_like(kd)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    s = sq.Subspace(H, d)
+    stream = torch.cuda.current_stream()
+
+    stage_names = ["build_subspace", "quantize_keys", "quantize_values", "dequantize"]
+
+    def step(ev=None):
+        if ev: ev[0].record(stream)
+        sq.squat_build_subspace(s, q, cfg.rank_r, cfg.lam, cfg.block_g)
+        if ev: ev[1].record(stream)
+        sq.squat_quantize_keys(s, k, bits, G, kc, ks, kz)
+        if ev: ev[2].record(stream)
+        sq.squat_quantize_values(v, bits, G, vc, vs, vz)
+        if ev: ev[3].record(stream)
+        sq.squat_dequantize(sq.SQUAT_KEYS, kc, ks, kz, B, H, T, d, bits, G, kd)
+        sq.squat_dequantize(sq.SQUAT_VALUES, vc, vs, vz, B, H, T, d, bits, G, vd)
+        if ev: ev[4].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = sq.squat_kernel_launch_count()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush.zero_()                      # evict inputs and outputs from L2 (not part of a step's time)
+        step(events[i])
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    wall = time.perf_counter() - wall0
+    launches = sq.squat_kernel_launch_count() - launches0
+    step_ms = [e[0].elapsed_time(e[4]) for e in events]
+    stage_ms = {n: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in events) for i, n in enumerate(stage_names)}
+    local_ms = sum(step_ms)
+    vec_per_step = cfg.key_vectors()
+    total_ms, total_units = aggregate_over_ranks(local_ms, vec_per_step * args.steps, dev)
+    flags = sq.squat_get_device_status(clear=True)
+
+    # ---- end to end from host buffers through squat_write_path_host --------------------------------
+    qh, kh, vh = to_dev(q_np, pin=True), to_dev(k_np, pin=True), to_dev(v_np, pin=True)
+    outs_h = [torch.empty_like(t, device="cpu").pin_memory() for t in (kc, ks, kz, vc, vs, vz)]
+    ws = torch.empty(sq.squat_write_path_workspace_bytes(tdt, B, cfg.n_q_heads, H, T, d, bits, G), dtype=torch.uint8,
+                     device=dev)
+    h2d = sum(t.numel() * t.element_size() for t in (qh, kh, vh))
+    d2h = sum(t.numel() * t.element_size() for t in outs_h)
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws)
+    e2e_ms = []
+    for _ in range(e2e_steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws)
+        e2e_ms.append(1e3 * (time.perf_counter() - t0))        # the call synchronises its stream
+    e2e_total_ms, e2e_units = aggregate_over_ranks(sum(e2e_ms), vec_per_step * e2e_steps, dev)
+    clocks = sampler.stop() if rank == 0 else None
+
+    if rank == 0:
+        peaks = measured_peaks()
+        elem = 4 if cfg.dtype == "f32" else 2
+        key_ms = stage_ms["quantize_keys"]
+        flops = key_flops_per_vector(d, cfg.block_g) * vec_per_step
+        kbytes = bytes_per_vector(d, bits, G, elem) * vec_per_step
+        alu_time_ms = flops / (ALU_PEAK_TFLOPS * 1e12) * 1e3
+        hbm_time_ms = kbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        if alu_time_ms >= hbm_time_ms:
+            roof = {"bound": "alu", "achieved": flops / (key_ms * 1e-3) / 1e12, "peak": ALU_PEAK_TFLOPS,
+                    "unit": "TFLOP/s", "peak_source": "nominal: 148 SM x 128 FMA/clk x 2 x 1.965 GHz"}
+        else:
+            roof = {"bound": "hbm", "achieved": kbytes / (key_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "peak_source": peaks["source"]}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = NCU_KEY_KERNEL_TRAFFIC_BYTES.get(cfg.index)
+        roof["kernel"] = "quant_keys_kernel"
+        roof["ms_per_launch"] = key_ms
+        roof["key_vectors_per_s"] = vec_per_step / (key_ms * 1e-3)
+        roof["kv_input_gbs"] = vec_per_step * d * elem / (key_ms * 1e-3) / 1e9
+        roof["hbm_frac_of_" + peaks["source"]] = kbytes / (key_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]
+        # the HBM-bound stages, for the record
+        vbytes = bytes_per_vector(d, bits, G, elem) * vec_per_step
+        dq_bytes = 2 * (d * bits // 8 + 8 * d // G + d * elem) * vec_per_step
+        stages = {n: {"ms": stage_ms[n], "share": stage_ms[n] / statistics.mean(step_ms)} for n in stage_names}
+        stages["quantize_values"]["hbm_gbs"] = vbytes / (stage_ms["quantize_values"] * 1e-3) / 1e9
+        stages["quantize_values"]["hbm_frac"] = stages["quantize_values"]["hbm_gbs"] / peaks["hbm_gbs"]
+        stages["dequantize"]["hbm_gbs"] = dq_bytes / (stage_ms["dequantize"] * 1e-3) / 1e9
+        stages["dequantize"]["hbm_frac"] = stages["dequantize"]["hbm_gbs"] / peaks["hbm_gbs"]
+        line = {
+            "metric": METRIC, "value": total_units / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg),
+            "kv_ingested_gbs": 2 * vec_per_step * world * d * elem / (total_ms / args.steps * 1e-3) / 1e9,
+            "roofline": roof, "stages": stages,
+            "e2e": {"value": e2e_units / (e2e_total_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total_ms / e2e_steps,
+                    "api": "squat_write_path_host (pinned host buffers; build + keys + values)"},
+            "gpu_launches": int(launches), "wall_s_timed_region": wall, "device_status_flags": int(flags),
+            "clocks": clocks,
+            "cpu_baseline": cpu_baseline(cfg) if world == 1 else None,
+        }
+        print(json.dumps(line))
+    s.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=1, help="workload index (default 1: Llama-2-7B-shaped layer)")
+    ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
+    args = ap.parse_args()
+    cfg = si.get_config(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_gpu(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

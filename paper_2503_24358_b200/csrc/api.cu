@@ -29,9 +29,10 @@ int check_quant_args(const void *x, int dtype, int batch, int H, int T, int d, l
                      long long st, int bits, int G, const void *codes, const void *scales, const void *zeros,
                      long long osb, long long osh)
 {
-    if (!x || !codes || !scales || !zeros || !valid_dtype(dtype)) return SQUAT_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || batch < 0 || H <= 0 || T < 0 || d <= 0) return SQUAT_ERR_INVALID_ARG;
+    const bool empty = batch == 0 || T == 0;             // nothing will be read or written
+    if (!empty && (!x || !codes || !scales || !zeros)) return SQUAT_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(codes) || !aligned16(scales) || !aligned16(zeros)) return SQUAT_ERR_INVALID_ARG;
-    if (batch < 0 || H <= 0 || T < 0 || d <= 0) return SQUAT_ERR_INVALID_ARG;
     if (bits != 2 && bits != 4) return SQUAT_ERR_UNSUPPORTED;
     if (G != 32 && G != 64 && G != 128) return SQUAT_ERR_UNSUPPORTED;
     if (sb < 0 || sh < 0 || st < d || osb < 0 || osh < 0) return SQUAT_ERR_INVALID_ARG;
@@ -202,6 +203,7 @@ int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int b
     if (n_kv_heads != s->n_kv_heads) return SQUAT_ERR_SHAPE;
     if (n_tokens % group_size != 0 || out_stride_b % group_size != 0 || out_stride_h % group_size != 0)
         return SQUAT_ERR_SHAPE;
+    if (batch == 0 || n_tokens == 0) return SQUAT_OK;
     return squat_launch_quant_keys(s->Wt, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
                                    group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status,
                                    static_cast<cudaStream_t>(stream));
@@ -216,6 +218,7 @@ int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, i
                               group_size, codes, scales, zeros, out_stride_b, out_stride_h);
     if (rc != SQUAT_OK) return rc;
     if (head_dim % group_size != 0 || (head_dim * bits) % 64 != 0) return SQUAT_ERR_SHAPE;
+    if (batch == 0 || n_tokens == 0) return SQUAT_OK;
     unsigned *status = squat_status_word();
     if (!status) return SQUAT_ERR_CUDA;
     return squat_launch_quant_values(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t,
@@ -227,8 +230,8 @@ int squat_dequantize(int kind, const unsigned char *codes, const float *scales, 
                      int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
                      long long in_stride_b, long long in_stride_h, void *out, int out_dtype, void *stream)
 {
-    if (!codes || !scales || !zeros || !out || !valid_dtype(out_dtype)) return SQUAT_ERR_INVALID_ARG;
-    if (kind != SQUAT_KEYS && kind != SQUAT_VALUES) return SQUAT_ERR_INVALID_ARG;
+    if (!valid_dtype(out_dtype) || (kind != SQUAT_KEYS && kind != SQUAT_VALUES)) return SQUAT_ERR_INVALID_ARG;
+    if (batch != 0 && n_tokens != 0 && (!codes || !scales || !zeros || !out)) return SQUAT_ERR_INVALID_ARG;
     if (!aligned16(codes) || !aligned16(scales) || !aligned16(zeros) || !aligned16(out)) return SQUAT_ERR_INVALID_ARG;
     if (batch < 0 || n_kv_heads <= 0 || n_tokens < 0 || head_dim <= 0 || in_stride_b < 0 || in_stride_h < 0)
         return SQUAT_ERR_INVALID_ARG;

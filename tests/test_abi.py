@@ -50,6 +50,7 @@ def test_argument_errors_come_back_as_status_codes(lib):
     a = ctypes.c_void_p(4096)          # never dereferenced: validation fails first
     mis = ctypes.c_void_p(4100)
     assert lib.squat_quantize_values(z, 1, 1, 1, 32, 128, 0, 0, 128, 2, 32, a, a, a, 0, 0, None) == 1
+    assert lib.squat_quantize_values(z, 1, 1, 1, 0, 128, 0, 0, 128, 2, 32, z, z, z, 0, 0, None) == 0      # empty: no-op
     assert lib.squat_quantize_values(mis, 1, 1, 1, 32, 128, 0, 0, 128, 2, 32, a, a, a, 0, 0, None) == 1
     assert lib.squat_quantize_values(a, 1, 1, 1, 32, 128, 0, 0, 128, 3, 32, a, a, a, 0, 0, None) == 3
     assert lib.squat_quantize_values(a, 1, 1, 1, 32, 128, 0, 0, 128, 2, 48, a, a, a, 0, 0, None) == 3
