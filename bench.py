@@ -274,6 +274,7 @@ def run_gpu(args, cfg):
     if world > 1:
         dist.barrier()
     wall = time.perf_counter() - wall0
+    clocks = sampler.stop() if rank == 0 else None
     launches = sq.squat_kernel_launch_count() - launches0
     step_ms = [e[0].elapsed_time(e[4]) for e in events]
     stage_ms = {n: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in events) for i, n in enumerate(stage_names)}
@@ -283,6 +284,23 @@ def run_gpu(args, cfg):
     flags = sq.squat_get_device_status(clear=True)
 
     # ---- end to end from host buffers through squat_write_path_host --------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, cfg, sq, s, (q_np, k_np, v_np), (kc, ks, kz, vc, vs, vz), to_dev, flush, tdt, dev,
+                      vec_per_step)
+    if rank == 0:
+        report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches,
+               wall, flags, clocks)
+    s.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, cfg, sq, s, host_np, dev_outs, to_dev, flush, tdt, dev, vec_per_step):
+    import torch
+    B, H, T, d, bits, G = cfg.batch, cfg.n_kv_heads, cfg.n_tokens, cfg.head_dim, cfg.bits, cfg.group_size
+    q_np, k_np, v_np = host_np
+    kc, ks, kz, vc, vs, vz = dev_outs
     qh, kh, vh = to_dev(q_np, pin=True), to_dev(k_np, pin=True), to_dev(v_np, pin=True)
     outs_h = [torch.empty_like(t, device="cpu").pin_memory() for t in (kc, ks, kz, vc, vs, vz)]
     ws = torch.empty(sq.squat_write_path_workspace_bytes(tdt, B, cfg.n_q_heads, H, T, d, bits, G), dtype=torch.uint8,
@@ -300,9 +318,15 @@ def run_gpu(args, cfg):
         sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws)
         e2e_ms.append(1e3 * (time.perf_counter() - t0))        # the call synchronises its stream
     e2e_total_ms, e2e_units = aggregate_over_ranks(sum(e2e_ms), vec_per_step * e2e_steps, dev)
-    clocks = sampler.stop() if rank == 0 else None
+    return {"value": e2e_units / (e2e_total_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total_ms / e2e_steps,
+            "api": "squat_write_path_host (pinned host buffers; build + keys + values)"}
 
-    if rank == 0:
+
+def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches, wall,
+           flags, clocks):
+    d, bits, G = cfg.head_dim, cfg.bits, cfg.group_size
+    if True:
         peaks = measured_peaks()
         elem = 4 if cfg.dtype == "f32" else 2
         key_ms = stage_ms["quantize_keys"]
@@ -338,17 +362,12 @@ def run_gpu(args, cfg):
             "config": workload_config(cfg),
             "kv_ingested_gbs": 2 * vec_per_step * world * d * elem / (total_ms / args.steps * 1e-3) / 1e9,
             "roofline": roof, "stages": stages,
-            "e2e": {"value": e2e_units / (e2e_total_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total_ms / e2e_steps,
-                    "api": "squat_write_path_host (pinned host buffers; build + keys + values)"},
+            "e2e": e2e,
             "gpu_launches": int(launches), "wall_s_timed_region": wall, "device_status_flags": int(flags),
             "clocks": clocks,
-            "cpu_baseline": cpu_baseline(cfg) if world == 1 else None,
+            "cpu_baseline": cpu_baseline(cfg) if (world == 1 and not args.no_cpu_baseline) else None,
         }
         print(json.dumps(line))
-    s.close()
-    if world > 1:
-        dist.destroy_process_group()
 
 
 def main():
@@ -358,6 +377,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="workload index (default 1: Llama-2-7B-shaped layer)")
     ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     args = ap.parse_args()
     cfg = si.get_config(args.config)
     if args.impl == "reference":

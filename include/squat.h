@@ -87,6 +87,9 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
 int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,
                           double *eigval_host, double *eigvec_host);
 int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream);
+/* Diagnostics of the last build: Jacobi sweeps the eigensolver ran for each head.  Synchronises
+ * `stream`.  sweeps_host is a host array of n_kv_heads ints. */
+int squat_subspace_eig_sweeps(const squat_subspace *s, void *stream, int *sweeps_host);
 
 /*
  * Step 2 -- key quantization with error feedback  (Algorithm 1, function Quant; Eq. (3) and

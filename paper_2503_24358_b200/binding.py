@@ -19,7 +19,7 @@ FLAG_NONFINITE, FLAG_ZERO_RANGE, FLAG_NO_CONVERGE = 1, 2, 4
 
 EXPORTED_SYMBOLS = (
     "squat_subspace_create", "squat_subspace_destroy", "squat_build_subspace", "squat_subspace_export",
-    "squat_subspace_import", "squat_quantize_keys", "squat_quantize_values", "squat_dequantize",
+    "squat_subspace_import", "squat_subspace_eig_sweeps", "squat_quantize_keys", "squat_quantize_values", "squat_dequantize",
     "squat_write_path_workspace_bytes", "squat_write_path_host", "squat_get_device_status",
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error",
 )
@@ -51,6 +51,7 @@ def _load():
         lib.squat_build_subspace.argtypes = [vp, vp, i, i, i, ll, ll, i, dbl, i, vp]
         lib.squat_subspace_export.argtypes = [vp, vp, vp, vp, vp, vp]
         lib.squat_subspace_import.argtypes = [vp, vp, vp]
+        lib.squat_subspace_eig_sweeps.argtypes = [vp, vp, vp]
         lib.squat_quantize_keys.argtypes = [vp, vp, i, i, i, i, i, ll, ll, ll, i, i, vp, vp, vp, ll, ll, vp]
         lib.squat_quantize_values.argtypes = [vp, i, i, i, i, i, ll, ll, ll, i, i, vp, vp, vp, ll, ll, vp]
         lib.squat_dequantize.argtypes = [i, vp, vp, vp, i, i, i, i, i, i, ll, ll, vp, i, vp]
@@ -149,6 +150,15 @@ def squat_subspace_import(s: Subspace, W, stream=None):
         raise ValueError("W must be [n_kv_heads, d, d]")
     _check(_load().squat_subspace_import(s.handle, W.ctypes.data_as(ctypes.c_void_p), _stream(stream)),
            "squat_subspace_import")
+
+
+def squat_subspace_eig_sweeps(s: Subspace, stream=None):
+    """Jacobi sweeps the eigensolver ran for each head in the last build (diagnostic)."""
+    import numpy as np
+    out = np.zeros(s.n_kv_heads, dtype=np.int32)
+    _check(_load().squat_subspace_eig_sweeps(s.handle, _stream(stream), out.ctypes.data_as(ctypes.c_void_p)),
+           "squat_subspace_eig_sweeps")
+    return out
 
 
 def _check_bhtd(x, name):

@@ -108,6 +108,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     const size_t o_part = carve(hdd * sizeof(double) * s->gram_chunks_cap);
     const size_t o_val = carve((size_t)n_kv_heads * D * sizeof(double));
     const size_t o_vec = carve(hdd * sizeof(double));
+    const size_t o_swp = carve((size_t)n_kv_heads * sizeof(int));
     char *base = nullptr;
     if (cudaMalloc(&base, off) != cudaSuccess) { cudaGetLastError(); delete s; return SQUAT_ERR_ALLOC; }
     if (cudaMemset(base, 0, off) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
@@ -116,6 +117,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     s->gram_partial = reinterpret_cast<double *>(base + o_part);
     s->eigval = reinterpret_cast<double *>(base + o_val);
     s->eigvec = reinterpret_cast<double *>(base + o_vec);
+    s->eig_sweeps = reinterpret_cast<int *>(base + o_swp);
     s->status = squat_status_word();
     if (!s->status) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
     *out = s;
@@ -171,6 +173,15 @@ int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, 
             for (int j = 0; j < D; ++j)
                 for (int jp = 0; jp < D; ++jp)
                     W_host[((size_t)h * D + jp) * D + j] = wt[((size_t)h * D + j) * D + jp];
+    return SQUAT_OK;
+}
+
+int squat_subspace_eig_sweeps(const squat_subspace *s, void *stream, int *sweeps_host)
+{
+    if (!s || !sweeps_host) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SQUAT_CUDA(cudaMemcpyAsync(sweeps_host, s->eig_sweeps, (size_t)s->n_kv_heads * sizeof(int), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;
 }
 

@@ -4,17 +4,25 @@
 //
 // Mapping.  A group is G consecutive tokens of one (batch, head); its channels must be visited in
 // order, and each channel's grid needs min/max over the group's tokens.  So: lane = token, one warp
-// (G = 32) or a team of G/32 warps per group, and the token's whole 128-channel working row lives
-// in that lane's registers as 64 packed float pairs.  Channel j:
-//     m, M   = warp min / max (redux.sync on f32)              -> scale = (M-m)/L, zero = m
-//     c      = clamp(rint((x_j - m)/scale))                     (binary32 sequence, see values.cu)
-//     e      = fma(c, scale, -(x_j - m))                        (= deq(qtz(x_j)) - x_j)
-//     x_j'  += e * W[j'][j]  for j' > j                          packed fma.rn.f32x2, W row j is a
-//                                                               shared-memory broadcast (LDS.128)
-// The loop over j is fully unrolled so every register index is static.  The d x d matrix of the
-// CTA's current head sits in shared memory (64 KB, stored transposed: row j = update vector of j).
+// (G = 32) or a team of G/32 warps per group.  The 128 channels are processed in 4 blocks of 32:
+//
+//   left-looking trailing update (runtime loop, tiny code):
+//       x_blk[c] = k[c] + sum_{j < block start} e_j * W[c][j]
+//     e_j of earlier channels sit in shared memory ([channel][lane], read conflict-free), the row of
+//     W is a shared-memory broadcast (LDS.128), the 32 values of the block live in registers as 16
+//     packed pairs updated with fma.rn.f32x2.
+//   in-block triangle (32 channels, unrolled so every register index is static; the same code
+//   serves all 4 blocks):
+//       m, M  = warp min / max (redux.sync on f32)         -> scale = (M-m)/L, zero = m
+//       c     = clamp(rint((x_j - m)/scale))                (binary32 sequence, see values.cu)
+//       e     = fma(c, scale, -(x_j - m))                   (= deq(qtz(x_j)) - x_j)
+//       x_j' += e * W[j'][j]  for the later channels j' of the block; e goes to shared memory.
+//
+// The update matrix of the CTA's current head is kept in shared memory as 4 column panels
+// (panel b = W^T[0 .. 32b+31][32b .. 32b+31], 40 KB in all: only the lower triangle is ever read).
 // CTAs are persistent: each takes a contiguous range of groups ordered head-major, so W is
-// reloaded only when the range crosses a head.
+// reloaded only when the range crosses a head.  14 warps per SM x 2 rounds cover the 27.7 groups
+// per SM of the 32-head x 4096-token workload.
 //
 // Work per key vector: 8128 fp32 FMA (dense triangle, g = 1) -> bound by the FP32 pipes, not HBM.
 #include "squat_internal.cuh"
@@ -22,10 +30,14 @@
 namespace {
 
 constexpr int D = SQUAT_D;
-constexpr int NPAIR = D / 2;
-constexpr float kMagic = 12582912.0f;
+constexpr int BLK = 32;                   // channels per block
+constexpr int NBLK = D / BLK;             // 4
+constexpr int PANEL_FLOATS = BLK * BLK * (NBLK * (NBLK + 1) / 2);   // 10 blocks of 32 x 32
+constexpr int E_ROWS = D - BLK;           // errors of the last block are never read
+constexpr float kMagic = 12582912.0f;     // 1.5 * 2^23
 constexpr float kTieBand = 0.5f - 1e-5f;
-constexpr int KEY_THREADS = 384;
+constexpr int KEY_WARPS = 14;
+constexpr int KEY_THREADS = KEY_WARPS * 32;
 
 typedef unsigned long long u64;
 
@@ -39,12 +51,14 @@ __device__ __forceinline__ float lo_of(u64 v)
 {
     float lo, hi;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    (void)hi;
     return lo;
 }
 __device__ __forceinline__ float hi_of(u64 v)
 {
     float lo, hi;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    (void)lo;
     return hi;
 }
 __device__ __forceinline__ u64 ffma2(u64 a, u64 b, u64 c)
@@ -91,7 +105,7 @@ __device__ __noinline__ float exact_code(float dlt, float scale)
 }
 
 struct KeyParams {
-    const float *Wt;          // [H, D, D] transposed update matrices
+    const float *Wt;          // [H, D, D] transposed update matrices: Wt[j][j'] = W[j'][j]
     const void *k;
     long long sb, sh, st;     // element strides of k
     unsigned char *codes;
@@ -103,22 +117,62 @@ struct KeyParams {
     unsigned *status;
 };
 
+template <bool BF16>
+struct RawBlock {             // one block (32 channels) of one token as loaded from global memory
+    uint4 v[BF16 ? 4 : 8];
+};
+
+template <bool BF16>
+__device__ __forceinline__ void load_raw(RawBlock<BF16> &r, const void *row, int b)
+{
+    if (BF16) {
+        const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(row) + b * BLK);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r.v[i] = ldg128(p + i);
+    } else {
+        const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(row) + b * BLK);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r.v[i] = ldg128(p + i);
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void unpack_raw(const RawBlock<BF16> &r, u64 (&xp)[BLK / 2])
+{
+    if (BF16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            xp[4 * i + 0] = pack2(bf16lo_to_f32(r.v[i].x), bf16hi_to_f32(r.v[i].x));
+            xp[4 * i + 1] = pack2(bf16lo_to_f32(r.v[i].y), bf16hi_to_f32(r.v[i].y));
+            xp[4 * i + 2] = pack2(bf16lo_to_f32(r.v[i].z), bf16hi_to_f32(r.v[i].z));
+            xp[4 * i + 3] = pack2(bf16lo_to_f32(r.v[i].w), bf16hi_to_f32(r.v[i].w));
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            xp[2 * i + 0] = pack2(__uint_as_float(r.v[i].x), __uint_as_float(r.v[i].y));
+            xp[2 * i + 1] = pack2(__uint_as_float(r.v[i].z), __uint_as_float(r.v[i].w));
+        }
+    }
+}
+
 template <int BITS, int NW, bool BF16>
 __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyParams p)
 {
-    constexpr float L = float((1 << BITS) - 1);
     constexpr int G = 32 * NW;
-    constexpr int NTEAMS = KEY_THREADS / 32 / NW;
-    constexpr int NWORDS = D * BITS / 32;
+    constexpr int NTEAMS = KEY_WARPS / NW;
+    constexpr int WORDS_PER_BLK = BLK * BITS / 32;       // 2 (2-bit) or 4 (4-bit)
     constexpr int PER_WORD = 32 / BITS;
     extern __shared__ __align__(16) float smem[];
-    float *Ws = smem;                                    // [D][D]
-    float2 *red = reinterpret_cast<float2 *>(smem + D * D);   // [NTEAMS][2][NW] (min, max)
+    float *Wp = smem;                                    // 4 column panels, PANEL_FLOATS
+    float *Eall = smem + PANEL_FLOATS;                   // [KEY_WARPS][E_ROWS][32]
+    float2 *red = reinterpret_cast<float2 *>(Eall + KEY_WARPS * E_ROWS * 32);   // [NTEAMS][2][NW]
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int team = warp / NW;
     const int wteam = warp % NW;
+    float *Ew = Eall + warp * (E_ROWS * 32) + lane;      // this lane's column of the warp's error store
 
     const long long lo = p.total_groups * blockIdx.x / gridDim.x;
     const long long hi = p.total_groups * (blockIdx.x + 1) / gridDim.x;
@@ -132,105 +186,120 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
 
         __syncthreads();                                 // everyone is done with the previous head's W
         {
-            const float4 *src = reinterpret_cast<const float4 *>(p.Wt + (long long)h * D * D);
-            float4 *dst = reinterpret_cast<float4 *>(Ws);
-            for (int i = threadIdx.x; i < D * D / 4; i += KEY_THREADS) dst[i] = __ldg(src + i);
+            // panel cb holds rows j = 0 .. 32 cb + 31 of W^T restricted to columns 32 cb .. 32 cb + 31
+            const float *src = p.Wt + (long long)h * D * D;
+            for (int i = threadIdx.x; i < PANEL_FLOATS / 4; i += KEY_THREADS) {
+                int f = i * 4, cb = 0;
+                while (f >= BLK * BLK * (cb + 1)) { f -= BLK * BLK * (cb + 1); ++cb; }
+                const int j = f / BLK, c = f % BLK;
+                reinterpret_cast<float4 *>(Wp)[i] = __ldg(reinterpret_cast<const float4 *>(src + j * D + cb * BLK + c));
+            }
         }
         __syncthreads();
 
-        for (long long gi = pos + team; gi < seg_end; gi += NTEAMS) {
-            const long long in_head = gi - (long long)h * groups_per_head;
-            const int b = (int)(in_head / p.groups_per_bh);
-            const int grp = (int)(in_head % p.groups_per_bh);
-            const int tok = grp * G + wteam * 32 + lane;
+        if (team < NTEAMS) {
+            for (long long gi = pos + team; gi < seg_end; gi += NTEAMS) {
+                const long long in_head = gi - (long long)h * groups_per_head;
+                const int b = (int)(in_head / p.groups_per_bh);
+                const int grp = (int)(in_head % p.groups_per_bh);
+                const int tok = grp * G + wteam * 32 + lane;
+                const long long row_off = (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st;
+                const void *row = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row_off)
+                                       : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row_off);
+                const long long out_tok0 = (long long)b * p.osb + (long long)h * p.osh;
+                float *sc_out = p.scales + (out_tok0 / G + grp) * D;
+                float *zr_out = p.zeros + (out_tok0 / G + grp) * D;
+                unsigned char *cp = p.codes + (out_tok0 + tok) * (D * BITS / 8);
+                unsigned flags = 0;
 
-            // ---- load this lane's token row into registers --------------------------------
-            u64 xp[NPAIR];
-            if (BF16) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    reinterpret_cast<const __nv_bfloat16 *>(p.k) + (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st);
-#pragma unroll
-                for (int i = 0; i < D / 8; ++i) {
-                    const uint4 r = ldg128(src + i);
-                    xp[4 * i + 0] = pack2(bf16lo_to_f32(r.x), bf16hi_to_f32(r.x));
-                    xp[4 * i + 1] = pack2(bf16lo_to_f32(r.y), bf16hi_to_f32(r.y));
-                    xp[4 * i + 2] = pack2(bf16lo_to_f32(r.z), bf16hi_to_f32(r.z));
-                    xp[4 * i + 3] = pack2(bf16lo_to_f32(r.w), bf16hi_to_f32(r.w));
-                }
-            } else {
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    reinterpret_cast<const float *>(p.k) + (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st);
-#pragma unroll
-                for (int i = 0; i < D / 4; ++i) {
-                    const uint4 r = ldg128(src + i);
-                    xp[2 * i + 0] = pack2(__uint_as_float(r.x), __uint_as_float(r.y));
-                    xp[2 * i + 1] = pack2(__uint_as_float(r.z), __uint_as_float(r.w));
-                }
-            }
+                RawBlock<BF16> raw;
+                load_raw<BF16>(raw, row, 0);
 
-            const long long out_tok0 = (long long)b * p.osb + (long long)h * p.osh;   // token offset of (b, h)
-            float *sc_out = p.scales + (out_tok0 / G + grp) * D;
-            float *zr_out = p.zeros + (out_tok0 / G + grp) * D;
-            uint32_t cw[NWORDS];
-            float my_scale = 0.0f, my_zero = 0.0f;
-            unsigned flags = 0;
+                for (int blk = 0; blk < NBLK; ++blk) {
+                    u64 xp[BLK / 2];
+                    unpack_raw<BF16>(raw, xp);
+                    if (blk + 1 < NBLK) load_raw<BF16>(raw, row, blk + 1);          // prefetch the next block
 
-            // ---- the sequential sweep over channels ---------------------------------------
+                    const float *panel = Wp + (blk * (blk + 1) / 2) * (BLK * BLK);
+                    // ---- left-looking update from all earlier channels ------------------------
+                    const int nprev = blk * BLK;
+#pragma unroll 4
+                    for (int j = 0; j < nprev; ++j) {
+                        const float e = Ew[j * 32];
+                        const u64 ee = pack2(e, e);
+                        const ulonglong2 *w = reinterpret_cast<const ulonglong2 *>(panel + j * BLK);
 #pragma unroll
-            for (int j = 0; j < D; ++j) {
-                const float xj = (j & 1) ? hi_of(xp[j >> 1]) : lo_of(xp[j >> 1]);
-                float m = warp_min(xj);
-                float Mx = warp_max(xj);
-                if (NW > 1) {
-                    float2 *slot = red + (team * 2 + (j & 1)) * NW;
-                    if (lane == 0) slot[wteam] = make_float2(m, Mx);
-                    team_barrier(1 + team, 32 * NW);
+                        for (int q = 0; q < BLK / 4; ++q) {
+                            const ulonglong2 wv = w[q];
+                            xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
+                            xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
+                        }
+                    }
+
+                    // ---- sequential sweep over the block's 32 channels ------------------------
+                    const float *diag = panel + nprev * BLK;
+                    float *Eblk = Ew + nprev * 32;
+                    uint32_t cw[WORDS_PER_BLK];
+                    float my_scale = 0.0f, my_zero = 0.0f;
 #pragma unroll
-                    for (int w = 0; w < NW; ++w) {
-                        const float2 o = slot[w];
-                        m = fminf(m, o.x);
-                        Mx = fmaxf(Mx, o.y);
+                    for (int jj = 0; jj < BLK; ++jj) {
+                        const float xj = (jj & 1) ? hi_of(xp[jj >> 1]) : lo_of(xp[jj >> 1]);
+                        float m = warp_min(xj);
+                        float Mx = warp_max(xj);
+                        if (NW > 1) {
+                            float2 *slot = red + (team * 2 + (jj & 1)) * NW;
+                            if (lane == 0) slot[wteam] = make_float2(m, Mx);
+                            team_barrier(1 + team, 32 * NW);
+#pragma unroll
+                            for (int w = 0; w < NW; ++w) {
+                                const float2 o = slot[w];
+                                m = fminf(m, o.x);
+                                Mx = fmaxf(Mx, o.y);
+                            }
+                        }
+                        const float scale = div_by_levels<BITS>(__fsub_rn(Mx, m));
+                        const bool ok = scale > 0.0f && scale < __int_as_float(0x7f800000);
+                        if (!ok) flags |= (scale == 0.0f) ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE;
+                        const float rcp = ok ? __frcp_rn(scale) : 0.0f;
+                        const float dlt = __fsub_rn(xj, m);
+                        const float y = __fmaf_rn(dlt, rcp, kMagic);
+                        float c = __fsub_rn(y, kMagic);
+                        const float res = __fmaf_rn(dlt, rcp, -c);
+                        uint32_t cbits = __float_as_uint(y) & ((1u << BITS) - 1u);
+                        if (__any_sync(0xffffffffu, fabsf(res) >= kTieBand) && ok) {
+                            if (fabsf(res) >= kTieBand) {
+                                c = exact_code<BITS>(dlt, scale);
+                                cbits = (uint32_t)(int)c;
+                            }
+                        }
+                        const float e = __fmaf_rn(c, scale, -dlt);
+                        if (blk + 1 < NBLK) Eblk[jj * 32] = e;
+                        const u64 ee = pack2(e, e);
+                        const float *wrow = diag + jj * BLK;
+#pragma unroll
+                        for (int q = (jj + 1) / 4; q < BLK / 4; ++q) {
+                            const ulonglong2 wv = *reinterpret_cast<const ulonglong2 *>(wrow + 4 * q);
+                            if (2 * q >= (jj + 1) / 2) xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
+                            xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
+                        }
+                        if (jj % PER_WORD == 0) cw[jj / PER_WORD] = cbits;
+                        else cw[jj / PER_WORD] |= cbits << ((jj % PER_WORD) * BITS);
+                        if (lane == jj) { my_scale = scale; my_zero = m; }
+                    }
+
+                    // ---- this block's outputs -----------------------------------------------
+                    if (WORDS_PER_BLK == 2)
+                        *reinterpret_cast<uint2 *>(cp + blk * (BLK * BITS / 8)) = make_uint2(cw[0], cw[1]);
+                    else
+                        *reinterpret_cast<uint4 *>(cp + blk * (BLK * BITS / 8)) =
+                            make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
+                    if (wteam == 0) {
+                        sc_out[blk * BLK + lane] = my_scale;
+                        zr_out[blk * BLK + lane] = my_zero;
                     }
                 }
-                const float scale = div_by_levels<BITS>(__fsub_rn(Mx, m));
-                const bool ok = scale > 0.0f && scale < __int_as_float(0x7f800000);
-                if (!ok) flags |= (scale == 0.0f) ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE;
-                const float rcp = ok ? __frcp_rn(scale) : 0.0f;
-                const float dlt = __fsub_rn(xj, m);
-                const float y = __fmaf_rn(dlt, rcp, kMagic);
-                float c = __fsub_rn(y, kMagic);
-                const float res = __fmaf_rn(dlt, rcp, -c);
-                if (__any_sync(0xffffffffu, fabsf(res) >= kTieBand) && ok) {
-                    if (fabsf(res) >= kTieBand) c = exact_code<BITS>(dlt, scale);
-                }
-                const float e = __fmaf_rn(c, scale, -dlt);
-                const u64 ee = pack2(e, e);
-
-                // push the error onto the later channels:  x[j'] += e * W[j'][j]
-                const float *wrow = Ws + j * D;
-#pragma unroll
-                for (int q = (j + 1) / 4; q < D / 4; ++q) {
-                    const ulonglong2 w = *reinterpret_cast<const ulonglong2 *>(wrow + 4 * q);
-                    if (2 * q >= (j + 1) / 2) xp[2 * q] = ffma2(ee, w.x, xp[2 * q]);
-                    xp[2 * q + 1] = ffma2(ee, w.y, xp[2 * q + 1]);
-                }
-
-                // bookkeeping: code bits, and the (scale, zero) of channel j parked in lane j % 32
-                const uint32_t cbits = (uint32_t)(int)c;
-                if (j % PER_WORD == 0) cw[j / PER_WORD] = cbits;
-                else cw[j / PER_WORD] |= cbits << ((j % PER_WORD) * BITS);
-                if (lane == (j & 31)) { my_scale = scale; my_zero = m; }
-                if ((j & 31) == 31 && wteam == 0) {
-                    sc_out[(j & ~31) + lane] = my_scale;
-                    zr_out[(j & ~31) + lane] = my_zero;
-                }
+                if (flags) atomicOr(p.status, flags);
             }
-
-            // ---- write this token's packed codes -------------------------------------------
-            uint4 *cp = reinterpret_cast<uint4 *>(p.codes + (out_tok0 + tok) * (D * BITS / 8));
-#pragma unroll
-            for (int i = 0; i < NWORDS / 4; ++i) cp[i] = make_uint4(cw[4 * i], cw[4 * i + 1], cw[4 * i + 2], cw[4 * i + 3]);
-            if (flags) atomicOr(p.status, flags);
         }
         pos = seg_end;
     }
@@ -242,8 +311,8 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    constexpr int NTEAMS = KEY_THREADS / 32 / NW;
-    const size_t smem = sizeof(float) * D * D + sizeof(float2) * NTEAMS * 2 * NW;
+    constexpr int NTEAMS = KEY_WARPS / NW;
+    const size_t smem = sizeof(float) * (PANEL_FLOATS + KEY_WARPS * E_ROWS * 32) + sizeof(float2) * NTEAMS * 2 * NW;
     long long want = (p.total_groups + NTEAMS - 1) / NTEAMS;
     const int grid = (int)(want < sms ? want : sms);
     if (dtype == SQUAT_BF16) {

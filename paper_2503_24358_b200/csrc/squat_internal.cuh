@@ -17,6 +17,7 @@ struct squat_subspace {
     double *gram_partial;  // [chunks, H, d, d] per-chunk partial Gram matrices (deterministic reduction)
     double *eigval;        // [H, d] descending
     double *eigvec;        // [H, d, d], row i = eigenvector i
+    int *eig_sweeps;       // [H] sweeps of the last eigen-decomposition
     unsigned *status;      // device status word of this device
 };
 

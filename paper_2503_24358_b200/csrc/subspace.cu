@@ -142,7 +142,7 @@ __device__ __forceinline__ double team8_sum(double v)
 
 __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
     const double *__restrict__ gram, double *__restrict__ eigval, double *__restrict__ eigvec,
-    unsigned *__restrict__ status)
+    int *__restrict__ sweeps_out, unsigned *__restrict__ status)
 {
     extern __shared__ __align__(16) double sm[];
     double *Gs = sm;                       // column-major: Gs[col * EIG_LD + row]
@@ -163,7 +163,8 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
     const double tol2 = 1e-14 * 1e-14;
 
     bool converged = false;
-    for (int sweep = 0; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
+    int sweep = 0;
+    for (; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
         // refresh the squared norms from the columns (cached values drift by rounding)
         for (int col = tid >> 3; col < D; col += EIG_THREADS / 8) {
             double s = 0.0;
@@ -206,7 +207,10 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
         }
         converged = (any_rot == 0);
     }
-    if (!converged && tid == 0) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
+    if (tid == 0) {
+        sweeps_out[h] = sweep;
+        if (!converged) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
+    }
 
     // exact norms, ranks (descending, ties by column index), normalised output
     for (int col = tid >> 3; col < D; col += EIG_THREADS / 8) {
@@ -338,7 +342,7 @@ int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 {
     const size_t smem = sizeof(double) * (D * EIG_LD + D) + sizeof(int) * D;
     SQUAT_CUDA(cudaFuncSetAttribute(eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    eig_kernel<<<s->n_kv_heads, EIG_THREADS, smem, st>>>(s->gram, s->eigval, s->eigvec, s->status);
+    eig_kernel<<<s->n_kv_heads, EIG_THREADS, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
