@@ -14,7 +14,7 @@
 //   in-block triangle (32 channels, unrolled so every register index is static; the same code
 //   serves all 4 blocks):
 //       m, M  = warp min / max (redux.sync on f32)         -> scale = (M-m)/L, zero = m
-//       c     = clamp(rint((x_j - m)/scale))                (binary32 sequence, see values.cu)
+//       c     = rint((x_j - m)/scale), decided exactly through the remainder c*scale - (x_j - m)
 //       e     = fma(c, scale, -(x_j - m))                   (= deq(qtz(x_j)) - x_j)
 //       x_j' += e * W[j'][j]  for the later channels j' of the block; e goes to shared memory.
 //
@@ -35,7 +35,6 @@ constexpr int NBLK = D / BLK;             // 4
 constexpr int PANEL_FLOATS = BLK * BLK * (NBLK * (NBLK + 1) / 2);   // 10 blocks of 32 x 32
 constexpr int E_ROWS = D - BLK;           // errors of the last block are never read
 constexpr float kMagic = 12582912.0f;     // 1.5 * 2^23
-constexpr float kTieBand = 0.5f - 1e-5f;
 constexpr int KEY_WARPS = 14;
 constexpr int KEY_THREADS = KEY_WARPS * 32;
 
@@ -94,14 +93,6 @@ __device__ __forceinline__ float div_by_levels(float rng)
     const float q = __fmul_rn(rng, invL);
     const float r = __fmaf_rn(-L, q, rng);
     return __fmaf_rn(r, invL, q);
-}
-
-// Slow path for an element within 1e-5 of a rounding midpoint: the exact binary32 sequence.
-template <int BITS>
-__device__ __noinline__ float exact_code(float dlt, float scale)
-{
-    constexpr float L = float((1 << BITS) - 1);
-    return fminf(fmaxf(rintf(__fdiv_rn(dlt, scale)), 0.0f), L);
 }
 
 struct KeyParams {
@@ -163,6 +154,7 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
     constexpr int NTEAMS = KEY_WARPS / NW;
     constexpr int WORDS_PER_BLK = BLK * BITS / 32;       // 2 (2-bit) or 4 (4-bit)
     constexpr int PER_WORD = 32 / BITS;
+    constexpr float L = float((1 << BITS) - 1);
     extern __shared__ __align__(16) float smem[];
     float *Wp = smem;                                    // 4 column panels, PANEL_FLOATS
     float *Eall = smem + PANEL_FLOATS;                   // [KEY_WARPS][E_ROWS][32]
@@ -210,7 +202,6 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                 float *sc_out = p.scales + (out_tok0 / G + grp) * D;
                 float *zr_out = p.zeros + (out_tok0 / G + grp) * D;
                 unsigned char *cp = p.codes + (out_tok0 + tok) * (D * BITS / 8);
-                unsigned flags = 0;
 
                 RawBlock<BF16> raw;
                 load_raw<BF16>(raw, row, 0);
@@ -257,22 +248,25 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                                 Mx = fmaxf(Mx, o.y);
                             }
                         }
-                        const float scale = div_by_levels<BITS>(__fsub_rn(Mx, m));
-                        const bool ok = scale > 0.0f && scale < __int_as_float(0x7f800000);
-                        if (!ok) flags |= (scale == 0.0f) ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE;
-                        const float rcp = ok ? __frcp_rn(scale) : 0.0f;
+                        // Decision.  c0 = rint((x - m) * r) with r ~ L/(M-m) from the hardware reciprocal can be off
+                        // by one next to a rounding midpoint; the remainder e0 = c0*scale - (x - m) is exact there,
+                        // so comparing it with +-scale/2 settles the rounding exactly as real arithmetic on the
+                        // stored float32 scale would; an exact tie goes to the even code (the threshold of an odd c0
+                        // is lowered by one ulp, so "remainder == scale/2" moves it and an even c0 stays).
+                        const float rng = __fsub_rn(Mx, m);
+                        const float scale = div_by_levels<BITS>(rng);
+                        const float half = 0.5f * scale;
+                        float rcp;
+                        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(rng));
+                        rcp = (rng > 1e-30f) ? rcp * L : 0.0f;          // constant (or absurdly tight) group: code 0
                         const float dlt = __fsub_rn(xj, m);
-                        const float y = __fmaf_rn(dlt, rcp, kMagic);
-                        float c = __fsub_rn(y, kMagic);
-                        const float res = __fmaf_rn(dlt, rcp, -c);
-                        uint32_t cbits = __float_as_uint(y) & ((1u << BITS) - 1u);
-                        if (__any_sync(0xffffffffu, fabsf(res) >= kTieBand) && ok) {
-                            if (fabsf(res) >= kTieBand) {
-                                c = exact_code<BITS>(dlt, scale);
-                                cbits = (uint32_t)(int)c;
-                            }
-                        }
-                        const float e = __fmaf_rn(c, scale, -dlt);
+                        const float y0 = __fmaf_rn(dlt, rcp, kMagic);
+                        const float e0 = __fmaf_rn(__fsub_rn(y0, kMagic), scale, -dlt);
+                        const float thr = __uint_as_float(__float_as_uint(half) - (__float_as_uint(y0) & 1u));
+                        const float adj = (e0 > thr) ? -1.0f : ((e0 < -thr) ? 1.0f : 0.0f);
+                        const float y = __fadd_rn(y0, adj);
+                        const float e = __fmaf_rn(adj, scale, e0);
+                        const uint32_t cbits = __float_as_uint(y) & ((1u << BITS) - 1u);
                         if (blk + 1 < NBLK) Eblk[jj * 32] = e;
                         const u64 ee = pack2(e, e);
                         const float *wrow = diag + jj * BLK;
@@ -296,9 +290,10 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                     if (wteam == 0) {
                         sc_out[blk * BLK + lane] = my_scale;
                         zr_out[blk * BLK + lane] = my_zero;
+                        if (!(my_scale > 0.0f && my_scale < __int_as_float(0x7f800000)))
+                            atomicOr(p.status, my_scale == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
                     }
                 }
-                if (flags) atomicOr(p.status, flags);
             }
         }
         pos = seg_end;
