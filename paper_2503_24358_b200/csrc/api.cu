@@ -94,6 +94,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     memset(s, 0, sizeof(*s));
     s->n_kv_heads = n_kv_heads;
     s->head_dim = head_dim;
+    s->exact_blocks = D / 32;            // W starts as zero: every channel is uncorrected
     int sms = 148;
     if (cudaGetDevice(&s->device) != cudaSuccess) { delete s; return SQUAT_ERR_CUDA; }
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, s->device);
@@ -150,6 +151,8 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
     if (rc != SQUAT_OK) return rc;
     rc = squat_launch_eig(s, st);
     if (rc != SQUAT_OK) return rc;
+    // channels of the first g-block are never corrected; with r = 0 or lambda = 0, W = 0 and none is
+    s->exact_blocks = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
     return squat_launch_assemble(s, rank_r, lambda, block_g, st);
 }
 
@@ -195,6 +198,15 @@ int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
         for (int j = 0; j < D; ++j)
             for (int jp = 0; jp < D; ++jp)
                 wt[((size_t)h * D + j) * D + jp] = W_host[((size_t)h * D + jp) * D + j];
+    // channel j' is uncorrected if row j' of W is zero in every head (channel 0 always is); the blocks that
+    // hold the leading run of uncorrected channels need the exact rounding decision
+    int uncorrected = D;
+    for (int h = 0; h < s->n_kv_heads; ++h)
+        for (int jp = 0; jp < uncorrected; ++jp)
+            for (int j = 0; j < D; ++j)
+                if (W_host[((size_t)h * D + jp) * D + j] != 0.0f) { uncorrected = jp; break; }
+    const int exact = (uncorrected + 31) / 32;
+    s->exact_blocks = exact;
     SQUAT_CUDA(cudaMemcpyAsync(s->Wt, wt.data(), hdd * sizeof(float), cudaMemcpyHostToDevice, st));
     SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;
@@ -216,7 +228,7 @@ int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int b
         return SQUAT_ERR_SHAPE;
     if (batch == 0 || n_tokens == 0) return SQUAT_OK;
     return squat_launch_quant_keys(s->Wt, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
-                                   group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status,
+                                   group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status, s->exact_blocks,
                                    static_cast<cudaStream_t>(stream));
 }
 

@@ -7,10 +7,12 @@
 // (G = 32) or a team of G/32 warps per group.  The 128 channels are processed in 4 blocks of 32:
 //
 //   left-looking trailing update (runtime loop, tiny code):
-//       x_blk[c] = k[c] + sum_{j < block start} e_j * W[c][j]
-//     e_j of earlier channels sit in shared memory ([channel][lane], read conflict-free), the row of
-//     W is a shared-memory broadcast (LDS.128), the 32 values of the block live in registers as 16
-//     packed pairs updated with fma.rn.f32x2.
+//       x_blk[tok][c] = k[tok][c] + sum_{j < block start} e_j[tok] * W[c][j]
+//     a (32 tokens x J) x (J x 32 channels) product, register-tiled: each lane owns 4 tokens x 8
+//     channels, reads 4 errors (one LDS.128 of the [channel][token] error store) and 8 entries of
+//     W^T (two LDS.128) per j and issues 16 packed fma.rn.f32x2 -- 6 shared-memory wavefronts per
+//     j instead of 17 with one token per lane, which would make shared memory the bound.  The tile
+//     is then transposed through shared memory to one token per lane for the sequential part.
 //   in-block triangle (32 channels, unrolled so every register index is static; the same code
 //   serves all 4 blocks):
 //       m, M  = warp min / max (redux.sync on f32)         -> scale = (M-m)/L, zero = m
@@ -106,44 +108,115 @@ struct KeyParams {
     int groups_per_bh;        // T / G
     long long total_groups;   // H * B * groups_per_bh, ordered (h, b, grp)
     unsigned *status;
+    int exact_blocks;         // leading 32-channel blocks that no earlier channel corrects (see sweep_block)
+};
+
+// One lane's share of a 32-token x 32-channel block in the trailing-update layout: 4 tokens x 8 channels.
+template <bool BF16>
+struct RawTile {
+    uint4 v[BF16 ? 4 : 8];      // per token: 8 channels = 16 B (bf16) or 32 B (f32)
 };
 
 template <bool BF16>
-struct RawBlock {             // one block (32 channels) of one token as loaded from global memory
-    uint4 v[BF16 ? 4 : 8];
-};
-
-template <bool BF16>
-__device__ __forceinline__ void load_raw(RawBlock<BF16> &r, const void *row, int b)
+__device__ __forceinline__ void load_tile(RawTile<BF16> &r, const void *row0, long long st, int chan)
 {
+    // row0: first of the lane's 4 consecutive tokens; st: token stride in elements; chan: first channel
     if (BF16) {
-        const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(row) + b * BLK);
+        const __nv_bfloat16 *p = reinterpret_cast<const __nv_bfloat16 *>(row0) + chan;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) r.v[i] = ldg128(p + i);
+        for (int i = 0; i < 4; ++i) r.v[i] = ldg128(p + i * st);
     } else {
-        const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(row) + b * BLK);
+        const float *p = reinterpret_cast<const float *>(row0) + chan;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) r.v[i] = ldg128(p + i);
+        for (int i = 0; i < 4; ++i) {
+            r.v[2 * i] = ldg128(p + i * st);
+            r.v[2 * i + 1] = ldg128(p + i * st + 4);
+        }
     }
 }
 
 template <bool BF16>
-__device__ __forceinline__ void unpack_raw(const RawBlock<BF16> &r, u64 (&xp)[BLK / 2])
+__device__ __forceinline__ void unpack_tile(const RawTile<BF16> &r, u64 (&acc)[4][4])
 {
-    if (BF16) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            xp[4 * i + 0] = pack2(bf16lo_to_f32(r.v[i].x), bf16hi_to_f32(r.v[i].x));
-            xp[4 * i + 1] = pack2(bf16lo_to_f32(r.v[i].y), bf16hi_to_f32(r.v[i].y));
-            xp[4 * i + 2] = pack2(bf16lo_to_f32(r.v[i].z), bf16hi_to_f32(r.v[i].z));
-            xp[4 * i + 3] = pack2(bf16lo_to_f32(r.v[i].w), bf16hi_to_f32(r.v[i].w));
+    for (int i = 0; i < 4; ++i) {
+        if (BF16) {
+            acc[i][0] = pack2(bf16lo_to_f32(r.v[i].x), bf16hi_to_f32(r.v[i].x));
+            acc[i][1] = pack2(bf16lo_to_f32(r.v[i].y), bf16hi_to_f32(r.v[i].y));
+            acc[i][2] = pack2(bf16lo_to_f32(r.v[i].z), bf16hi_to_f32(r.v[i].z));
+            acc[i][3] = pack2(bf16lo_to_f32(r.v[i].w), bf16hi_to_f32(r.v[i].w));
+        } else {
+            acc[i][0] = pack2(__uint_as_float(r.v[2 * i].x), __uint_as_float(r.v[2 * i].y));
+            acc[i][1] = pack2(__uint_as_float(r.v[2 * i].z), __uint_as_float(r.v[2 * i].w));
+            acc[i][2] = pack2(__uint_as_float(r.v[2 * i + 1].x), __uint_as_float(r.v[2 * i + 1].y));
+            acc[i][3] = pack2(__uint_as_float(r.v[2 * i + 1].z), __uint_as_float(r.v[2 * i + 1].w));
         }
-    } else {
+    }
+}
+
+// The sequential part: the 32 channels of one block, one token per lane, values in xp (16 packed pairs).
+// For every channel: grid from the warp (team) min / max, rounding decision, error e; e is pushed onto the
+// later channels of the block through the diagonal 32 x 32 block of W^T and stored for the later blocks.
+//
+// Rounding decision.  t = (x - m) / scale is formed as (x - m) * L * rcp(M - m) with the hardware reciprocal,
+// so c0 = rint(t) can be off by one when t is within ~1e-6 of a rounding midpoint.  Channels that earlier
+// channels have corrected hold generic float32 values and such near-ties are as rare as that bound; but
+// channels nothing has corrected yet (the first g channels, or all of them when W = 0) hold raw bf16 / f32
+// inputs, where exact ties are structural (x exactly half way between min and max).  For those blocks
+// (EXACT) the remainder e0 = c0*scale - (x - m), which is exact next to a midpoint, is compared with
+// +-scale/2: that settles the rounding exactly as real arithmetic on the stored float32 scale would, ties
+// going to the even code (the threshold of an odd c0 is one ulp lower, so "remainder == scale/2" moves it).
+template <int BITS, int NW, bool EXACT>
+__device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, float *Eblk, bool store_e,
+                                            int lane, int team, int wteam, float2 *red,
+                                            uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
+{
+    constexpr int PER_WORD = 32 / BITS;
+    constexpr float L = float((1 << BITS) - 1);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            xp[2 * i + 0] = pack2(__uint_as_float(r.v[i].x), __uint_as_float(r.v[i].y));
-            xp[2 * i + 1] = pack2(__uint_as_float(r.v[i].z), __uint_as_float(r.v[i].w));
+    for (int jj = 0; jj < BLK; ++jj) {
+        const float xj = (jj & 1) ? hi_of(xp[jj >> 1]) : lo_of(xp[jj >> 1]);
+        float m = warp_min(xj);
+        float Mx = warp_max(xj);
+        if (NW > 1) {
+            float2 *slot = red + (team * 2 + (jj & 1)) * NW;
+            if (lane == 0) slot[wteam] = make_float2(m, Mx);
+            team_barrier(1 + team, 32 * NW);
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const float2 o = slot[w];
+                m = fminf(m, o.x);
+                Mx = fmaxf(Mx, o.y);
+            }
         }
+        const float rng = __fsub_rn(Mx, m);
+        const float dlt = __fsub_rn(xj, m);
+        const float dltL = __fmul_rn(dlt, L);
+        float rcp;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(fmaxf(rng, 1e-30f)));   // constant group: dlt = 0 -> code 0
+        const float scale = div_by_levels<BITS>(rng);
+        const float y0 = __fmaf_rn(dltL, rcp, kMagic);
+        float e = __fmaf_rn(__fsub_rn(y0, kMagic), scale, -dlt);
+        float y = y0;
+        if (EXACT) {
+            const float thr = __uint_as_float(__float_as_uint(0.5f * scale) - (__float_as_uint(y0) & 1u));
+            const float adj = (e > thr) ? -1.0f : ((e < -thr) ? 1.0f : 0.0f);
+            y = __fadd_rn(y0, adj);
+            e = __fmaf_rn(adj, scale, e);
+        }
+        const uint32_t cbits = __float_as_uint(y) & ((1u << BITS) - 1u);
+        if (store_e) Eblk[jj * 32] = e;
+        const u64 ee = pack2(e, e);
+        const float *wrow = diag + jj * BLK;
+#pragma unroll
+        for (int q = (jj + 1) / 4; q < BLK / 4; ++q) {
+            const ulonglong2 wv = *reinterpret_cast<const ulonglong2 *>(wrow + 4 * q);
+            if (2 * q >= (jj + 1) / 2) xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
+            xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
+        }
+        if (jj % PER_WORD == 0) cw[jj / PER_WORD] = cbits;
+        else cw[jj / PER_WORD] |= cbits << ((jj % PER_WORD) * BITS);
+        if (lane == jj) { my_scale = scale; my_zero = m; }
     }
 }
 
@@ -153,8 +226,6 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
     constexpr int G = 32 * NW;
     constexpr int NTEAMS = KEY_WARPS / NW;
     constexpr int WORDS_PER_BLK = BLK * BITS / 32;       // 2 (2-bit) or 4 (4-bit)
-    constexpr int PER_WORD = 32 / BITS;
-    constexpr float L = float((1 << BITS) - 1);
     extern __shared__ __align__(16) float smem[];
     float *Wp = smem;                                    // 4 column panels, PANEL_FLOATS
     float *Eall = smem + PANEL_FLOATS;                   // [KEY_WARPS][E_ROWS][32]
@@ -195,36 +266,92 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                 const int b = (int)(in_head / p.groups_per_bh);
                 const int grp = (int)(in_head % p.groups_per_bh);
                 const int tok = grp * G + wteam * 32 + lane;
-                const long long row_off = (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st;
-                const void *row = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row_off)
-                                       : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row_off);
                 const long long out_tok0 = (long long)b * p.osb + (long long)h * p.osh;
                 float *sc_out = p.scales + (out_tok0 / G + grp) * D;
                 float *zr_out = p.zeros + (out_tok0 / G + grp) * D;
                 unsigned char *cp = p.codes + (out_tok0 + tok) * (D * BITS / 8);
 
-                RawBlock<BF16> raw;
-                load_raw<BF16>(raw, row, 0);
+                // trailing-update layout: this lane owns tokens 4 tr .. 4 tr + 3 and channels 8 cr .. 8 cr + 7 of a block
+                const int tr = lane >> 2, cr = lane & 3;
+                const long long row0_off = (long long)b * p.sb + (long long)h * p.sh +
+                                           (long long)(grp * G + wteam * 32 + 4 * tr) * p.st;
+                const void *row0 = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row0_off)
+                                        : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row0_off);
+                RawTile<BF16> raw;
+                load_tile<BF16>(raw, row0, p.st, 8 * cr);
 
                 for (int blk = 0; blk < NBLK; ++blk) {
-                    u64 xp[BLK / 2];
-                    unpack_raw<BF16>(raw, xp);
-                    if (blk + 1 < NBLK) load_raw<BF16>(raw, row, blk + 1);          // prefetch the next block
-
                     const float *panel = Wp + (blk * (blk + 1) / 2) * (BLK * BLK);
-                    // ---- left-looking update from all earlier channels ------------------------
                     const int nprev = blk * BLK;
-#pragma unroll 4
-                    for (int j = 0; j < nprev; ++j) {
-                        const float e = Ew[j * 32];
-                        const u64 ee = pack2(e, e);
-                        const ulonglong2 *w = reinterpret_cast<const ulonglong2 *>(panel + j * BLK);
+                    u64 xp[BLK / 2];
+                    {
+                        // ---- left-looking update from all earlier channels, as a register-tiled product:
+                        //      acc[token][channel pair] = k + sum_j e_j[token] * W^T[j][channel]
+                        u64 acc[4][4];
+                        unpack_tile<BF16>(raw, acc);
+                        if (blk + 1 < NBLK) load_tile<BF16>(raw, row0, p.st, (blk + 1) * BLK + 8 * cr);   // prefetch
+                        const float *e_ptr = Ew - lane + 4 * tr;          // E[j][4 tr .. 4 tr + 3]
+                        const float *w_ptr = panel + 8 * cr;              // W^T[j][8 cr .. 8 cr + 7]
+                        // software-pipelined over j: the operands of the next 2 steps are loaded while the current 2
+                        // steps' 32 packed FMAs issue (warps issue in order, so the loads must be hoisted by hand)
+                        constexpr int PF = 2;
+                        float4 ea[PF], eb[PF];
+                        ulonglong2 wa[PF][2], wb[PF][2];
+                        auto loadn = [&](float4 (&ev)[PF], ulonglong2 (&wv)[PF][2], int j0) {
+#pragma unroll
+                            for (int u = 0; u < PF; ++u) {
+                                ev[u] = *reinterpret_cast<const float4 *>(e_ptr + (j0 + u) * 32);
+                                wv[u][0] = *reinterpret_cast<const ulonglong2 *>(w_ptr + (j0 + u) * BLK);
+                                wv[u][1] = *reinterpret_cast<const ulonglong2 *>(w_ptr + (j0 + u) * BLK + 4);
+                            }
+                        };
+                        auto fman = [&](const float4 (&ev)[PF], const ulonglong2 (&wv)[PF][2]) {
+#pragma unroll
+                            for (int u = 0; u < PF; ++u) {
+                                const float e[4] = {ev[u].x, ev[u].y, ev[u].z, ev[u].w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const u64 ee = pack2(e[i], e[i]);
+                                    acc[i][0] = ffma2(ee, wv[u][0].x, acc[i][0]);
+                                    acc[i][1] = ffma2(ee, wv[u][0].y, acc[i][1]);
+                                    acc[i][2] = ffma2(ee, wv[u][1].x, acc[i][2]);
+                                    acc[i][3] = ffma2(ee, wv[u][1].y, acc[i][3]);
+                                }
+                            }
+                        };
+                        if (nprev > 0) {
+                            loadn(ea, wa, 0);
+#pragma unroll 1
+                            for (int j = 0; j < nprev; j += 2 * PF) {        // nprev is a multiple of 32
+                                loadn(eb, wb, j + PF);
+                                fman(ea, wa);
+                                loadn(ea, wa, (j + 2 * PF < nprev) ? j + 2 * PF : j);   // last reload: redundant, in range
+                                fman(eb, wb);
+                            }
+                        }
+                        // ---- transpose to one token per lane through a 4 KB staging tile (the error rows this
+                        //      block is about to fill; for the last block, rows 0..31, which nothing reads any more).
+                        //      16-byte chunks are swizzled with the token index so the row reads are conflict-free.
+                        float *stage = Ew - lane + ((blk + 1 < NBLK) ? nprev * 32 : 0);
+                        __syncwarp();
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int tok = 4 * tr + i;
+#pragma unroll
+                            for (int v = 0; v < 2; ++v) {
+                                const int phys = (2 * cr + v) ^ (tok & 7);
+                                *reinterpret_cast<ulonglong2 *>(stage + tok * 32 + 4 * phys) =
+                                    make_ulonglong2(acc[i][2 * v], acc[i][2 * v + 1]);
+                            }
+                        }
+                        __syncwarp();
 #pragma unroll
                         for (int q = 0; q < BLK / 4; ++q) {
-                            const ulonglong2 wv = w[q];
-                            xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
-                            xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
+                            const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(stage + lane * 32 + 4 * (q ^ (lane & 7)));
+                            xp[2 * q] = v.x;
+                            xp[2 * q + 1] = v.y;
                         }
+                        __syncwarp();
                     }
 
                     // ---- sequential sweep over the block's 32 channels ------------------------
@@ -232,54 +359,10 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                     float *Eblk = Ew + nprev * 32;
                     uint32_t cw[WORDS_PER_BLK];
                     float my_scale = 0.0f, my_zero = 0.0f;
-#pragma unroll
-                    for (int jj = 0; jj < BLK; ++jj) {
-                        const float xj = (jj & 1) ? hi_of(xp[jj >> 1]) : lo_of(xp[jj >> 1]);
-                        float m = warp_min(xj);
-                        float Mx = warp_max(xj);
-                        if (NW > 1) {
-                            float2 *slot = red + (team * 2 + (jj & 1)) * NW;
-                            if (lane == 0) slot[wteam] = make_float2(m, Mx);
-                            team_barrier(1 + team, 32 * NW);
-#pragma unroll
-                            for (int w = 0; w < NW; ++w) {
-                                const float2 o = slot[w];
-                                m = fminf(m, o.x);
-                                Mx = fmaxf(Mx, o.y);
-                            }
-                        }
-                        // Decision.  c0 = rint((x - m) * r) with r ~ L/(M-m) from the hardware reciprocal can be off
-                        // by one next to a rounding midpoint; the remainder e0 = c0*scale - (x - m) is exact there,
-                        // so comparing it with +-scale/2 settles the rounding exactly as real arithmetic on the
-                        // stored float32 scale would; an exact tie goes to the even code (the threshold of an odd c0
-                        // is lowered by one ulp, so "remainder == scale/2" moves it and an even c0 stays).
-                        const float rng = __fsub_rn(Mx, m);
-                        const float scale = div_by_levels<BITS>(rng);
-                        const float half = 0.5f * scale;
-                        float rcp;
-                        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(rng));
-                        rcp = (rng > 1e-30f) ? rcp * L : 0.0f;          // constant (or absurdly tight) group: code 0
-                        const float dlt = __fsub_rn(xj, m);
-                        const float y0 = __fmaf_rn(dlt, rcp, kMagic);
-                        const float e0 = __fmaf_rn(__fsub_rn(y0, kMagic), scale, -dlt);
-                        const float thr = __uint_as_float(__float_as_uint(half) - (__float_as_uint(y0) & 1u));
-                        const float adj = (e0 > thr) ? -1.0f : ((e0 < -thr) ? 1.0f : 0.0f);
-                        const float y = __fadd_rn(y0, adj);
-                        const float e = __fmaf_rn(adj, scale, e0);
-                        const uint32_t cbits = __float_as_uint(y) & ((1u << BITS) - 1u);
-                        if (blk + 1 < NBLK) Eblk[jj * 32] = e;
-                        const u64 ee = pack2(e, e);
-                        const float *wrow = diag + jj * BLK;
-#pragma unroll
-                        for (int q = (jj + 1) / 4; q < BLK / 4; ++q) {
-                            const ulonglong2 wv = *reinterpret_cast<const ulonglong2 *>(wrow + 4 * q);
-                            if (2 * q >= (jj + 1) / 2) xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
-                            xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
-                        }
-                        if (jj % PER_WORD == 0) cw[jj / PER_WORD] = cbits;
-                        else cw[jj / PER_WORD] |= cbits << ((jj % PER_WORD) * BITS);
-                        if (lane == jj) { my_scale = scale; my_zero = m; }
-                    }
+                    if (blk < p.exact_blocks)
+                        sweep_block<BITS, NW, true>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, cw, my_scale, my_zero);
+                    else
+                        sweep_block<BITS, NW, false>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, cw, my_scale, my_zero);
 
                     // ---- this block's outputs -----------------------------------------------
                     if (WORDS_PER_BLK == 2)
@@ -327,7 +410,7 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
 int squat_launch_quant_keys(const float *Wt, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
                             unsigned char *codes, float *scales, float *zeros,
-                            long long osb, long long osh, unsigned *status, cudaStream_t st)
+                            long long osb, long long osh, unsigned *status, int exact_blocks, cudaStream_t st)
 {
     KeyParams p;
     p.Wt = Wt; p.k = k; p.sb = sb; p.sh = sh; p.st = st_;
@@ -335,6 +418,7 @@ int squat_launch_quant_keys(const float *Wt, const void *k, int dtype, int batch
     p.B = batch; p.H = H; p.T = T; p.groups_per_bh = T / G;
     p.total_groups = (long long)H * batch * (T / G);
     p.status = status;
+    p.exact_blocks = exact_blocks;
     if (p.total_groups == 0) return SQUAT_OK;
     if (bits == 2) {
         if (G == 32) return launch_keys<2, 1>(p, dtype, st);

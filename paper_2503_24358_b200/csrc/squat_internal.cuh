@@ -12,6 +12,7 @@ struct squat_subspace {
     int head_dim;
     int device;
     int gram_chunks_cap;   // capacity (in row chunks per head) of gram_partial
+    int exact_blocks;      // leading 32-channel blocks of W that receive no correction (4 when W = 0)
     float *Wt;             // [H, d, d] float32, Wt[h][j][j'] = W[j'][j]  (row j = update vector of channel j)
     double *gram;          // [H, d, d] Gram matrices
     double *gram_partial;  // [chunks, H, d, d] per-chunk partial Gram matrices (deterministic reduction)
@@ -37,7 +38,7 @@ int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int bloc
 int squat_launch_quant_keys(const float *Wt, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
                             unsigned char *codes, float *scales, float *zeros,
-                            long long osb, long long osh, unsigned *status, cudaStream_t st);
+                            long long osb, long long osh, unsigned *status, int exact_blocks, cudaStream_t st);
 int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T, int d,
                               long long sb, long long sh, long long st_, int bits, int G,
                               unsigned char *codes, float *scales, float *zeros,
