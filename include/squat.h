@@ -151,6 +151,32 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
                           unsigned char *v_codes_host, float *v_scales_host, float *v_zeros_host,
                           void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Gram matrices of the stacked prompt queries without any allocation.  (The paper has no counterpart:
+ * this entry exists for callers that must not allocate.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they need the Gram step: code that
+ * runs inside a memory-pool or allocator callback, inside a region where the framework has frozen its
+ * allocator (for instance while it records work for later replay), or in a process whose device memory
+ * has been handed out completely to a serving engine.  squat_subspace_create allocates its scratch; this
+ * entry does not.  It computes, for every KV head h, M_h = Qc^T Qc in fp64 (the first stage of
+ * squat_build_subspace, same kernels, same layout of q) into the caller's gram_out
+ * [n_kv_heads, d, d] (device, float64), keeping its intermediate per-chunk partial sums in a fixed
+ * 8 MiB array that is part of the library image on every GPU that loads it.
+ *
+ * Limits and rules:
+ *   - n_kv_heads <= 64 (one 128 KiB partial per head and row chunk, 64 in all); more heads are rejected
+ *     with SQUAT_ERR_UNSUPPORTED and nothing is launched.  head_dim must be 128.
+ *   - no cudaMalloc, cudaFree or other allocating call is made, on any call.
+ *   - the first call on each device looks up the array's device address (with that device current) and
+ *     keeps it; make that first call outside any stream capture.
+ *   - all calls share the one array.  It keeps whatever the previous call left; every element a call reads
+ *     it has written first, so results never depend on earlier calls -- but two calls whose kernels overlap
+ *     on the GPU (different streams, or different threads) race on it.  Serialise them.
+ */
+int squat_gram_static(const void *q, int dtype, int n_q_heads, int n_kv_heads, int n_tokens, int head_dim,
+                      long long stride_h, long long stride_t, double *gram_out, void *stream);
+
 /* Reads (and clears when `clear` != 0) the device status word of the current device.
  * Synchronises `stream`.  flags is a host pointer. */
 int squat_get_device_status(void *stream, unsigned *flags, int clear);

@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = (
     "squat_subspace_create", "squat_subspace_destroy", "squat_build_subspace", "squat_subspace_export",
     "squat_subspace_import", "squat_subspace_eig_sweeps", "squat_quantize_keys", "squat_quantize_values", "squat_dequantize",
     "squat_write_path_workspace_bytes", "squat_write_path_host", "squat_get_device_status",
-    "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error",
+    "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
 )
 
 _lib = None
@@ -59,6 +59,7 @@ def _load():
         lib.squat_write_path_workspace_bytes.restype = c.c_size_t
         lib.squat_write_path_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, dbl, i, i, i,
                                               vp, vp, vp, vp, vp, vp, vp, c.c_size_t, vp]
+        lib.squat_gram_static.argtypes = [vp, i, i, i, i, i, ll, ll, vp, vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
         lib.squat_status_string.argtypes = [i]
@@ -225,6 +226,19 @@ def squat_write_path_host(s: Subspace, q, k, v, rank_r, lam, block_g, bits, grou
                                          hp(v_codes), hp(v_scales), hp(v_zeros), _dev(workspace, "workspace"),
                                          workspace.numel() * workspace.element_size(), _stream(stream)),
            "squat_write_path_host")
+
+
+def squat_gram_static(q: torch.Tensor, n_kv_heads: int, gram_out: torch.Tensor, stream=None):
+    """Gram matrices of the stacked queries into gram_out [n_kv_heads, d, d] (float64, CUDA) without any
+    allocation: for callers that cannot call cudaMalloc (allocator callbacks, frozen allocators, processes
+    whose device memory is fully handed out).  At most 64 KV heads; calls must not overlap on the GPU."""
+    if q.dim() != 3 or q.stride(2) != 1:
+        raise ValueError("q must be [n_q_heads, n_tokens, head_dim] with contiguous last dim")
+    if gram_out.dtype != torch.float64 or not gram_out.is_contiguous():
+        raise ValueError("gram_out must be a contiguous float64 tensor")
+    _check(_load().squat_gram_static(_dev(q, "q"), _dtype_code(q), q.shape[0], n_kv_heads, q.shape[1], q.shape[2],
+                                     q.stride(0), q.stride(1), _dev(gram_out, "gram_out"), _stream(stream)),
+           "squat_gram_static")
 
 
 def squat_get_device_status(clear: bool = True, stream=None) -> int:

@@ -357,3 +357,63 @@ int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int bloc
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
 }
+
+// ------------------------------------------------------------------------- allocation-free Gram entry
+// Scratch for squat_gram_static: the per-chunk partial Gram matrices live in this fixed array instead of
+// memory obtained from cudaMalloc.  64 units of one d x d fp64 matrix = 8 MiB, held by every GPU that loads
+// the library until the process exits.
+namespace {
+constexpr int GRAM_STATIC_MAX_UNITS = 64;            // n_kv_heads x row chunks
+static __device__ __align__(256) double g_gram_static_scratch[(size_t)GRAM_STATIC_MAX_UNITS * D * D];
+double *g_gram_static_ptr[64] = {nullptr};           // device address of the array, per device ordinal
+}  // namespace
+
+extern "C" int squat_gram_static(const void *q, int dtype, int n_q_heads, int n_kv_heads, int n_tokens,
+                                 int head_dim, long long stride_h, long long stride_t, double *gram_out,
+                                 void *stream)
+{
+    if (!q || !gram_out || (dtype != SQUAT_F32 && dtype != SQUAT_BF16)) return SQUAT_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(gram_out) & 15u)) return SQUAT_ERR_INVALID_ARG;
+    if (n_q_heads <= 0 || n_kv_heads <= 0 || n_tokens <= 0) return SQUAT_ERR_INVALID_ARG;
+    if (head_dim != D) return SQUAT_ERR_UNSUPPORTED;
+    if (n_kv_heads > GRAM_STATIC_MAX_UNITS) return SQUAT_ERR_UNSUPPORTED;      // beyond the fixed scratch
+    if (n_q_heads % n_kv_heads != 0) return SQUAT_ERR_SHAPE;
+    const long long vec = dtype == SQUAT_BF16 ? 8 : 4;
+    if (stride_t < D || stride_h < 0 || stride_t % vec || stride_h % vec) return SQUAT_ERR_INVALID_ARG;
+
+    // set-up, once per device, with that device current: the array's name is only a host-side handle here;
+    // kernels must be given the device address that cudaGetSymbolAddress reports
+    int dev = 0;
+    SQUAT_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SQUAT_ERR_UNSUPPORTED;
+    if (!g_gram_static_ptr[dev]) {
+        double *ptr = nullptr;
+        SQUAT_CUDA(cudaGetSymbolAddress((void **)&ptr, g_gram_static_scratch));
+        g_gram_static_ptr[dev] = ptr;
+    }
+    double *partial = g_gram_static_ptr[dev];
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int H = n_kv_heads, qpk = n_q_heads / H;
+    const long long N = (long long)n_tokens * qpk;
+    int chunks = GRAM_STATIC_MAX_UNITS / H;                                   // >= 1
+    long long rows_per_chunk = (N + chunks - 1) / chunks;
+    rows_per_chunk = (rows_per_chunk + GRAM_ROWS - 1) / GRAM_ROWS * GRAM_ROWS;
+    if (rows_per_chunk < 2 * GRAM_ROWS) rows_per_chunk = 2 * GRAM_ROWS;
+    chunks = (int)((N + rows_per_chunk - 1) / rows_per_chunk);
+    if (chunks < 1) chunks = 1;
+    // every element the reduction reads is written by this call's first kernel, so nothing left in the
+    // array by an earlier call is ever seen and nothing needs clearing
+    dim3 grid(chunks, H);
+    if (dtype == SQUAT_BF16)
+        gram_kernel<true><<<grid, GRAM_THREADS, 0, st>>>(q, n_tokens, qpk, stride_h, stride_t, (int)rows_per_chunk, partial);
+    else
+        gram_kernel<false><<<grid, GRAM_THREADS, 0, st>>>(q, n_tokens, qpk, stride_h, stride_t, (int)rows_per_chunk, partial);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    gram_reduce_kernel<<<dim3(D * D / 256, H), 256, 0, st>>>(partial, chunks, H, gram_out);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}
+
