@@ -3,9 +3,10 @@
 //   gram_kernel      M_h = Qc^T Qc for the stacked prompt queries of KV head h (Section 3.2;
 //                    Algorithm 1 line 5 needs only the right singular vectors and singular values
 //                    of Qc, i.e. the eigen-pairs of M_h; GQA stacking rule of Appendix C).
-//   eig_kernel       eigen-decomposition of M_h by one-sided (Hestenes) Jacobi on the columns of
-//                    M_h itself: rotations make the columns orthogonal, which leaves M V = V diag(mu);
-//                    column norms are the eigenvalues sigma_i^2, normalised columns the v_i.
+//   eig_kernel       eigen-decomposition of M_h: Cholesky M_h + shift I = L L^T, then one-sided (Hestenes)
+//                    Jacobi on the columns of L: rotations make the columns orthogonal, L V = U Sigma;
+//                    the normalised columns U are the eigenvectors v_i of M_h and the squared column
+//                    norms, minus the shift, its eigenvalues sigma_i^2.
 //   assemble_kernel  P_inv = (I + lambda Qhat^T Qhat)^{-1} = I - sum_i s_i/(1+s_i) v_i v_i^T with
 //                    s_i = lambda sigma_i^2 (Woodbury with orthonormal v_i; footnote of Prop. 4),
 //                    then the update matrices B_t H_t of Lemma 3 read off the LDL^T factorisation
@@ -128,12 +129,15 @@ __global__ void gram_reduce_kernel(const double *__restrict__ partial, int chunk
 }
 
 // ------------------------------------------------------------------------------------- eigen
-constexpr int EIG_THREADS = 512;    // 64 column pairs x 8 lanes
+constexpr int EIG_THREADS = 1024;   // 64 column pairs x 16 lanes
+constexpr int EIG_TEAM = 16;        // lanes per column pair
+constexpr int EIG_RPL = D / EIG_TEAM; // rows per lane
 constexpr int EIG_LD = D + 2;       // padded column stride (doubles)
 constexpr int EIG_MAX_SWEEPS = 40;
 
-__device__ __forceinline__ double team8_sum(double v)
+__device__ __forceinline__ double team_sum(double v)
 {
+    v += __shfl_xor_sync(0xffffffffu, v, 8);
     v += __shfl_xor_sync(0xffffffffu, v, 1);
     v += __shfl_xor_sync(0xffffffffu, v, 2);
     v += __shfl_xor_sync(0xffffffffu, v, 4);
@@ -149,7 +153,7 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
     double *nrm = sm + D * EIG_LD;         // squared column norms
     int *rank = reinterpret_cast<int *>(nrm + D);
     const int h = blockIdx.x, tid = threadIdx.x;
-    const int team = tid >> 3, l8 = tid & 7;
+    const int team = tid >> 4, l8 = tid & (EIG_TEAM - 1);
     const double *M = gram + (long long)h * D * D;
 
     for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
@@ -159,53 +163,85 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
     __syncthreads();
     double trace = 0.0;
     for (int i = 0; i < D; ++i) trace += Gs[i * EIG_LD + i];
-    const double null_thr = (1e-14 * trace) * (1e-14 * trace);
+    // Preconditioning: M + shift*I = L L^T (Cholesky), then Jacobi on the columns of L instead of M.  The left
+    // singular vectors of L are the eigenvectors of M, its singular values sqrt(mu + shift); L has the square
+    // root of M's condition number and L^T L is much closer to diagonal than M^2, which roughly halves the
+    // sweeps.  The shift (1e-12 of the trace) keeps the factorisation defined for rank-deficient M and is
+    // subtracted from the eigenvalues at the end; eigenvectors are unaffected by it.
+    const double shift = trace > 0.0 ? 1e-12 * trace : 1e-300;
+    __syncthreads();
+    if (tid < D) Gs[tid * EIG_LD + tid] += shift;
+    double *lcol = nrm;                     // reused as the current column of L during the factorisation
+    for (int j = 0; j < D; ++j) {
+        __syncthreads();
+        const double ajj = Gs[j * EIG_LD + j];
+        const double ljj = sqrt(ajj > 0.0 ? ajj : shift);
+        if (tid >= j && tid < D) lcol[tid] = (tid == j) ? ljj : Gs[j * EIG_LD + tid] / ljj;
+        __syncthreads();
+        const int n = D - 1 - j;            // trailing block: rows/cols j+1 .. D-1, lower triangle (row >= col)
+        for (int idx = tid; idx < n * n; idx += EIG_THREADS) {
+            const int c = j + 1 + idx / n, r = j + 1 + idx % n;
+            if (r >= c) Gs[c * EIG_LD + r] = fma(-lcol[r], lcol[c], Gs[c * EIG_LD + r]);
+        }
+        if (tid >= j && tid < D) Gs[j * EIG_LD + tid] = lcol[tid];
+    }
+    __syncthreads();
+    for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
+        const int c = idx / D, r = idx % D;
+        if (r < c) Gs[c * EIG_LD + r] = 0.0;            // L is lower triangular
+    }
+    __syncthreads();
+    const double null_thr = 4.0 * shift;                // squared norm of a column that is numerically null
     const double tol2 = 1e-14 * 1e-14;
 
     bool converged = false;
     int sweep = 0;
     for (; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
         // refresh the squared norms from the columns (cached values drift by rounding)
-        for (int col = tid >> 3; col < D; col += EIG_THREADS / 8) {
+        for (int col = tid >> 4; col < D; col += EIG_THREADS / EIG_TEAM) {
             double s = 0.0;
 #pragma unroll
-            for (int i = 0; i < D / 8; ++i) { const double v = Gs[col * EIG_LD + l8 + 8 * i]; s = fma(v, v, s); }
-            s = team8_sum(s);
+            for (int i = 0; i < EIG_RPL; ++i) { const double v = Gs[col * EIG_LD + l8 + EIG_TEAM * i]; s = fma(v, v, s); }
+            s = team_sum(s);
             if (l8 == 0) nrm[col] = s;
         }
         __syncthreads();
-        int any_rot = 0;
+        // Largest cos^2 between two columns seen at the start of their rotation in this sweep.  Jacobi converges
+        // quadratically, so once every pair starts a sweep below 1e-7 the sweep leaves them below ~1e-14: done.
+        int big = 0;
         for (int round = 0; round < D - 1; ++round) {
             int p, q;
             if (team == 0) { p = D - 1; q = round; }
             else { p = (round + team) % (D - 1); q = (round - team + (D - 1)) % (D - 1); }
             double *gp = Gs + p * EIG_LD + l8, *gq = Gs + q * EIG_LD + l8;
-            double a[D / 8], b[D / 8];
-            double gam = 0.0;
+            double a[EIG_RPL], b[EIG_RPL];
+            double gam0 = 0.0, gam1 = 0.0;
 #pragma unroll
-            for (int i = 0; i < D / 8; ++i) { a[i] = gp[8 * i]; b[i] = gq[8 * i]; gam = fma(a[i], b[i], gam); }
-            gam = team8_sum(gam);
+            for (int i = 0; i < EIG_RPL; ++i) { a[i] = gp[EIG_TEAM * i]; b[i] = gq[EIG_TEAM * i]; }
+#pragma unroll
+            for (int i = 0; i < EIG_RPL; i += 2) { gam0 = fma(a[i], b[i], gam0); gam1 = fma(a[i + 1], b[i + 1], gam1); }
+            const double gam = team_sum(gam0 + gam1);
             const double alpha = nrm[p], beta = nrm[q];
-            int rot = 0;
-            if (alpha > null_thr && beta > null_thr && gam * gam > tol2 * alpha * beta) {
+            const double g2 = gam * gam, ab = alpha * beta;
+            if ((alpha > null_thr || beta > null_thr) && g2 > tol2 * ab) {
                 // t = tan of the rotation angle: smaller root of t^2 + 2 zeta t - 1 = 0, zeta = (beta-alpha)/(2 gam)
                 const double diff = beta - alpha;
-                const double den = fabs(diff) + sqrt(fma(diff, diff, 4.0 * gam * gam));
+                const double den = fabs(diff) + sqrt(fma(diff, diff, 4.0 * g2));
                 double t = 2.0 * gam / den;
                 if (diff < 0.0) t = -t;
                 const double c = rsqrt(fma(t, t, 1.0));
                 const double s = t * c;
 #pragma unroll
-                for (int i = 0; i < D / 8; ++i) {
-                    gp[8 * i] = c * a[i] - s * b[i];
-                    gq[8 * i] = s * a[i] + c * b[i];
+                for (int i = 0; i < EIG_RPL; ++i) {
+                    gp[EIG_TEAM * i] = c * a[i] - s * b[i];
+                    gq[EIG_TEAM * i] = s * a[i] + c * b[i];
                 }
                 if (l8 == 0) { nrm[p] = alpha - t * gam; nrm[q] = beta + t * gam; }
-                rot = 1;
+                if (g2 > 1e-14 * ab) big = 1;
             }
-            any_rot |= __syncthreads_or(rot);
+            big = __syncthreads_or(big);
         }
-        converged = (any_rot == 0);
+        converged = (big == 0);
     }
     if (tid == 0) {
         sweeps_out[h] = sweep;
@@ -213,12 +249,12 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
     }
 
     // exact norms, ranks (descending, ties by column index), normalised output
-    for (int col = tid >> 3; col < D; col += EIG_THREADS / 8) {
+    for (int col = tid >> 4; col < D; col += EIG_THREADS / EIG_TEAM) {
         double s = 0.0;
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i) { const double v = Gs[col * EIG_LD + l8 + 8 * i]; s = fma(v, v, s); }
-        s = team8_sum(s);
-        if (l8 == 0) nrm[col] = sqrt(s);
+        for (int i = 0; i < EIG_RPL; ++i) { const double v = Gs[col * EIG_LD + l8 + EIG_TEAM * i]; s = fma(v, v, s); }
+        s = team_sum(s);
+        if (l8 == 0) nrm[col] = sqrt(s);                 // singular value of L: sqrt(mu + shift)
     }
     __syncthreads();
     if (tid < D) {
@@ -229,7 +265,8 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
             rk += (o > mine) || (o == mine && j < tid);
         }
         rank[tid] = rk;
-        eigval[(long long)h * D + rk] = mine;
+        const double mu_out = mine * mine - shift;
+        eigval[(long long)h * D + rk] = mu_out > 0.0 ? mu_out : 0.0;
     }
     __syncthreads();
     for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
