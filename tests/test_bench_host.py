@@ -1,0 +1,64 @@
+"""CPU tests of bench.py's host-side logic: the world-size-2 aggregation (gloo), the algorithmic
+counts behind the roofline, and the reference (oracle) arm's JSON line."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        # rank r took (10 + 5 r) ms for 1000 (r + 1) units: job time = slowest rank, job units = sum
+        ms, units = bench.aggregate_over_ranks(10.0 + 5.0 * rank, 1000 * (rank + 1))
+        out[rank] = (ms, units)
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_aggregate_over_ranks_gloo_world_size_2():
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_worker, args=(2, 29611, out), nprocs=2, join=True)
+    assert out[0] == out[1] == (15.0, 3000)
+
+
+def test_aggregate_without_process_group_is_identity():
+    assert bench.aggregate_over_ranks(3.5, 42) == (3.5, 42)
+
+
+def test_algorithmic_counts():
+    assert bench.key_flops_per_vector(128, 1) == 2 * 8128
+    assert bench.key_flops_per_vector(128, 32) == 2 * 6144
+    assert bench.key_flops_per_vector(128, 64) == 2 * 4096
+    assert bench.bytes_per_vector(128, 2, 32, 2) == 320
+    assert bench.bytes_per_vector(128, 4, 128, 2) == 328
+    assert abs(bench.ALU_PEAK_TFLOPS - 74.45) < 0.01
+
+
+def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
+    env = dict(os.environ, RANK="0", WORLD_SIZE="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "0",
+                        "--steps", "2", "--warmup", "1"], capture_output=True, text=True, env=env, timeout=600)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "key_vectors/s" and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["value"] == d["value"]
+    env["RANK"], env["WORLD_SIZE"] = "1", "2"
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "0"],
+                       capture_output=True, text=True, env=env, timeout=600)
+    assert r.returncode == 0 and r.stdout.strip() == ""
