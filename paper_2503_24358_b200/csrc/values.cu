@@ -17,6 +17,38 @@ namespace {
 constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
 constexpr float kTieBand = 0.5f - 1e-5f;
 
+typedef unsigned long long u64;
+__device__ __forceinline__ u64 pk2(float lo, float hi) { u64 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void unpk2(u64 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ u64 sub2(u64 a, u64 b) { u64 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) { u64 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+
+// Exact binary32 decision for one element next to a rounding midpoint (rare; kept out of line).
+template <int BITS>
+__device__ __noinline__ uint32_t exact_code_bits(float dlt, float delta)
+{
+    constexpr float L = float((1 << BITS) - 1);
+    return (uint32_t)(int)fminf(fmaxf(rintf(__fdiv_rn(dlt, delta)), 0.0f), L);
+}
+
+template <int G, bool BF16>
+struct ValRaw {
+    static constexpr int NV = BF16 ? G / 8 : G / 4;      // 128-bit pieces of one group
+    uint4 v[NV];
+    __device__ __forceinline__ float get(int i) const     // channel i of the group, exact widening
+    {
+        if (BF16) {
+            const uint4 &r = v[i / 8];
+            const uint32_t w = (i % 8) / 2 == 0 ? r.x : (i % 8) / 2 == 1 ? r.y : (i % 8) / 2 == 2 ? r.z : r.w;
+            return (i & 1) ? bf16hi_to_f32(w) : bf16lo_to_f32(w);
+        } else {
+            const uint4 &r = v[i / 4];
+            const uint32_t w = i % 4 == 0 ? r.x : i % 4 == 1 ? r.y : i % 4 == 2 ? r.z : r.w;
+            return __uint_as_float(w);
+        }
+    }
+};
+
 template <int G, int BITS, bool BF16>
 __global__ void __launch_bounds__(256) quant_values_kernel(
     const void *__restrict__ v, long long n_units, int H, int T, int ng,
@@ -27,31 +59,52 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
     constexpr float L = float((1 << BITS) - 1);
     constexpr int PER_WORD = 32 / BITS;
     constexpr int NWORDS = G / PER_WORD;
+    using Raw = ValRaw<G, BF16>;
+    constexpr bool PREFETCH = false;              // keep the next unit's data in flight while this one computes
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < n_units; u += stride) {
+
+    auto in_ptr = [&](long long u) -> const uint4 * {
         const int q = (int)(u % ng);
         const long long tok = u / ng;
         const int t = (int)(tok % T);
         const long long bh = tok / T;
-        const int h = (int)(bh % H);
-        const long long b = bh / H;
-        const long long in_off = b * sb + h * sh + (long long)t * st + (long long)q * G;
-        const long long out_tok = b * osb + h * osh + t;
+        const long long off = (bh / H) * sb + (bh % H) * sh + (long long)t * st + (long long)q * G;
+        return BF16 ? reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(v) + off)
+                    : reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(v) + off);
+    };
+    auto load = [&](Raw &r, long long u) {
+        const uint4 *p = in_ptr(u);
+#pragma unroll
+        for (int i = 0; i < Raw::NV; ++i) r.v[i] = ldg128(p + i);
+    };
 
-        float x[G];
+    long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    Raw nxt;
+    if (PREFETCH && u < n_units) load(nxt, u);
+    for (; u < n_units; u += stride) {
+        Raw raw;
+        if (PREFETCH) {
+            raw = nxt;
+            if (u + stride < n_units) load(nxt, u + stride);
+        } else {
+            load(raw, u);
+        }
+        const int q = (int)(u % ng);
+        const long long tok = u / ng;
+        const int t = (int)(tok % T);
+        const long long bh = tok / T;
+        const long long out_tok = (bh / H) * osb + (bh % H) * osh + t;
+
         float m, Mx;
         if (BF16) {
-            const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(v) + in_off);
+            // min / max on packed bf16 pairs (exact), then across the pair
             __nv_bfloat162 mn2, mx2;
 #pragma unroll
-            for (int i = 0; i < G / 8; ++i) {
-                const uint4 r = ldg128(p + i);
-                const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+            for (int i = 0; i < Raw::NV; ++i) {
+                const uint32_t w[4] = {raw.v[i].x, raw.v[i].y, raw.v[i].z, raw.v[i].w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    x[i * 8 + 2 * k] = bf16lo_to_f32(w[k]);
-                    x[i * 8 + 2 * k + 1] = bf16hi_to_f32(w[k]);
-                    __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[k]);
+                    const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[k]);
                     if (i == 0 && k == 0) { mn2 = pr; mx2 = pr; }
                     else { mn2 = __hmin2(mn2, pr); mx2 = __hmax2(mx2, pr); }
                 }
@@ -59,18 +112,9 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
             m = fminf(__low2float(mn2), __high2float(mn2));
             Mx = fmaxf(__low2float(mx2), __high2float(mx2));
         } else {
-            const uint4 *p = reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(v) + in_off);
+            m = raw.get(0); Mx = m;
 #pragma unroll
-            for (int i = 0; i < G / 4; ++i) {
-                const uint4 r = ldg128(p + i);
-                x[i * 4 + 0] = __uint_as_float(r.x);
-                x[i * 4 + 1] = __uint_as_float(r.y);
-                x[i * 4 + 2] = __uint_as_float(r.z);
-                x[i * 4 + 3] = __uint_as_float(r.w);
-            }
-            m = x[0]; Mx = x[0];
-#pragma unroll
-            for (int i = 1; i < G; ++i) { m = fminf(m, x[i]); Mx = fmaxf(Mx, x[i]); }
+            for (int i = 1; i < G; ++i) { m = fminf(m, raw.get(i)); Mx = fmaxf(Mx, raw.get(i)); }
         }
 
         const float delta = __fdiv_rn(__fsub_rn(Mx, m), L);
@@ -78,35 +122,35 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
         const float rcp = ok ? __frcp_rn(delta) : 0.0f;
         if (!ok) atomicOr(status, delta == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
 
+        // two channels per instruction (packed f32x2): dlt = x - m, y = dlt * rcp + magic, c = y - magic,
+        // res = dlt * rcp - c; each half is the same IEEE operation as its scalar form
+        const u64 m2 = pk2(m, m), rcp2 = pk2(rcp, rcp), magic2 = pk2(kMagic, kMagic);
         uint32_t words[NWORDS];
-        float worst = 0.0f;
 #pragma unroll
         for (int wd = 0; wd < NWORDS; ++wd) {
             uint32_t acc = 0;
 #pragma unroll
-            for (int k = 0; k < PER_WORD; ++k) {
-                const float dlt = __fsub_rn(x[wd * PER_WORD + k], m);
-                const float y = __fmaf_rn(dlt, rcp, kMagic);
-                const float c = __fsub_rn(y, kMagic);
-                const float res = __fmaf_rn(dlt, rcp, -c);
-                worst = fmaxf(worst, fabsf(res));
-                acc |= (__float_as_uint(y) & ((1u << BITS) - 1u)) << (k * BITS);
+            for (int k = 0; k < PER_WORD; k += 2) {
+                const int i = wd * PER_WORD + k;
+                const u64 dlt2 = sub2(pk2(raw.get(i), raw.get(i + 1)), m2);
+                const u64 y2 = fma2(dlt2, rcp2, magic2);
+                const u64 nc2 = sub2(magic2, y2);                       // -(y - magic), exact
+                const u64 res2 = fma2(dlt2, rcp2, nc2);
+                float ylo, yhi, rlo, rhi;
+                unpk2(y2, ylo, yhi);
+                unpk2(res2, rlo, rhi);
+                uint32_t cb0 = __float_as_uint(ylo) & ((1u << BITS) - 1u);
+                uint32_t cb1 = __float_as_uint(yhi) & ((1u << BITS) - 1u);
+                // next to a rounding midpoint (structural with coarse bf16 data): the exact sequence decides
+                if (fmaxf(fabsf(rlo), fabsf(rhi)) >= kTieBand && ok) {
+                    float dlo, dhi;
+                    unpk2(dlt2, dlo, dhi);
+                    if (fabsf(rlo) >= kTieBand) cb0 = exact_code_bits<BITS>(dlo, delta);
+                    if (fabsf(rhi) >= kTieBand) cb1 = exact_code_bits<BITS>(dhi, delta);
+                }
+                acc |= (cb0 | (cb1 << BITS)) << (k * BITS);
             }
             words[wd] = acc;
-        }
-        if (worst >= kTieBand && ok) {
-            // some element sits next to a rounding midpoint: redo the group with exact divisions
-#pragma unroll
-            for (int wd = 0; wd < NWORDS; ++wd) {
-                uint32_t acc = 0;
-#pragma unroll
-                for (int k = 0; k < PER_WORD; ++k) {
-                    const float tt = __fdiv_rn(__fsub_rn(x[wd * PER_WORD + k], m), delta);
-                    const float c = fminf(fmaxf(rintf(tt), 0.0f), L);
-                    acc |= ((uint32_t)(int)c) << (k * BITS);
-                }
-                words[wd] = acc;
-            }
         }
 
         unsigned char *cp = codes + out_tok * row_bytes + (long long)q * (G * BITS / 8);
@@ -124,30 +168,30 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
     }
 }
 
-// One thread dequantizes 16 consecutive channels of one token.
+// One thread dequantizes 16 consecutive channels of 4 consecutive tokens (same key group, so the 16
+// scales and zeros are read once for the four).  Codes become floats through the 2^23 trick
+// (exact), then one fma each: deq(c) = fma(c, scale, zero), rounded once.
 template <int BITS, bool KEYS, bool OUT_BF16>
 __global__ void __launch_bounds__(256) dequant_kernel(
     const unsigned char *__restrict__ codes, const float *__restrict__ scales, const float *__restrict__ zeros,
     long long n_units, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
 {
+    constexpr int TOK = 4;
     const int per_tok = d / 16;
+    const int tq_per_row = (T + TOK - 1) / TOK;
     const int row_bytes = d * BITS / 8;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < n_units; u += stride) {
         const int c16 = (int)(u % per_tok);
-        const long long tok = u / per_tok;
-        const int t = (int)(tok % T);
-        const long long bh = tok / T;
+        const long long r = u / per_tok;
+        const int t0 = (int)(r % tq_per_row) * TOK;
+        const long long bh = r / tq_per_row;
         const int h = (int)(bh % H);
         const long long b = bh / H;
-        const long long in_tok = b * isb + h * ish + t;
-        const unsigned char *cp = codes + in_tok * row_bytes + c16 * (16 * BITS / 8);
-        uint32_t w[2];
-        if (BITS == 2) { w[0] = *reinterpret_cast<const uint32_t *>(cp); w[1] = 0; }
-        else { const uint2 r = *reinterpret_cast<const uint2 *>(cp); w[0] = r.x; w[1] = r.y; }
+        const long long in_tok0 = b * isb + h * ish;
         float sc[16], zr[16];
         if (KEYS) {
-            const long long base = (b * (isb / G) + h * (ish / G) + t / G) * d + c16 * 16;
+            const long long base = (b * (isb / G) + h * (ish / G) + t0 / G) * d + c16 * 16;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float4 s4 = __ldg(reinterpret_cast<const float4 *>(scales + base) + i);
@@ -155,34 +199,45 @@ __global__ void __launch_bounds__(256) dequant_kernel(
                 sc[4 * i] = s4.x; sc[4 * i + 1] = s4.y; sc[4 * i + 2] = s4.z; sc[4 * i + 3] = s4.w;
                 zr[4 * i] = z4.x; zr[4 * i + 1] = z4.y; zr[4 * i + 2] = z4.z; zr[4 * i + 3] = z4.w;
             }
-        } else {
-            const long long mi = in_tok * (d / G) + (c16 * 16) / G;
-            const float s = __ldg(scales + mi), z = __ldg(zeros + mi);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) { sc[i] = s; zr[i] = z; }
         }
-        float y[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int bit = i * BITS;
-            const float c = (float)((w[bit / 32] >> (bit % 32)) & ((1u << BITS) - 1u));
-            y[i] = __fmaf_rn(c, sc[i], zr[i]);
-        }
-        const long long o = ((bh * T) + t) * d + c16 * 16;
-        if (OUT_BF16) {
-            uint32_t pk[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                __nv_bfloat162 p2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
-                pk[i] = *reinterpret_cast<uint32_t *>(&p2);
+        for (int tt = 0; tt < TOK; ++tt) {
+            const int t = t0 + tt;
+            if (t >= T) break;
+            const unsigned char *cp = codes + (in_tok0 + t) * row_bytes + c16 * (16 * BITS / 8);
+            uint32_t w[2];
+            if (BITS == 2) { w[0] = __ldg(reinterpret_cast<const uint32_t *>(cp)); w[1] = 0; }
+            else { const uint2 rr = __ldg(reinterpret_cast<const uint2 *>(cp)); w[0] = rr.x; w[1] = rr.y; }
+            float s1 = 0.0f, z1 = 0.0f;
+            if (!KEYS) {
+                const long long mi = (in_tok0 + t) * (d / G) + (c16 * 16) / G;
+                s1 = __ldg(scales + mi);
+                z1 = __ldg(zeros + mi);
             }
-            uint4 *op = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(out) + o);
-            op[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            op[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-        } else {
-            float4 *op = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + o);
+            float y[16];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) op[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+            for (int i = 0; i < 16; ++i) {
+                const int bit = i * BITS;
+                const uint32_t cb = (w[bit / 32] >> (bit % 32)) & ((1u << BITS) - 1u);
+                const float c = __fsub_rn(__uint_as_float(0x4B000000u | cb), 8388608.0f);     // exact int -> float
+                y[i] = KEYS ? __fmaf_rn(c, sc[i], zr[i]) : __fmaf_rn(c, s1, z1);
+            }
+            const long long o = ((bh * T) + t) * d + c16 * 16;
+            if (OUT_BF16) {
+                uint32_t pk[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    __nv_bfloat162 p2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                    pk[i] = *reinterpret_cast<uint32_t *>(&p2);
+                }
+                uint4 *op = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(out) + o);
+                op[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                op[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            } else {
+                float4 *op = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + o);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) op[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+            }
         }
     }
 }
@@ -236,7 +291,7 @@ int squat_launch_dequant(int kind, const unsigned char *codes, const float *scal
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
                          void *out, int out_dtype, cudaStream_t st)
 {
-    const long long n_units = (long long)batch * H * T * (d / 16);
+    const long long n_units = (long long)batch * H * ((T + 3) / 4) * (d / 16);     // 4 tokens x 16 channels per thread
     if (n_units == 0) return SQUAT_OK;
     const int grid = grid_for(n_units, 256);
 #define SQ_D(BB, KK, OO) dequant_kernel<BB, KK, OO><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out)
