@@ -3,7 +3,7 @@
 //   gram_kernel      M_h = Qc^T Qc for the stacked prompt queries of KV head h (Section 3.2;
 //                    Algorithm 1 line 5 needs only the right singular vectors and singular values
 //                    of Qc, i.e. the eigen-pairs of M_h; GQA stacking rule of Appendix C).
-//   eig_kernel       eigen-decomposition of M_h: Cholesky M_h + shift I = L L^T, then one-sided (Hestenes)
+//   eig_cluster_kernel  eigen-decomposition of M_h: Cholesky M_h + shift I = L L^T, then one-sided (Hestenes)
 //                    Jacobi on the columns of L: rotations make the columns orthogonal, L V = U Sigma;
 //                    the normalised columns U are the eigenvectors v_i of M_h and the squared column
 //                    norms, minus the shift, its eigenvalues sigma_i^2.
@@ -19,6 +19,7 @@
 // weight lambda sigma^2, so single precision anywhere in this step changes quantized codes
 // downstream; products of bf16 inputs are exact in fp64 and everything stays fp64 until W is
 // rounded to float32 at the very end.
+#include <cooperative_groups.h>
 #include "squat_internal.cuh"
 
 namespace {
@@ -129,102 +130,140 @@ __global__ void gram_reduce_kernel(const double *__restrict__ partial, int chunk
 }
 
 // ------------------------------------------------------------------------------------- eigen
-constexpr int EIG_THREADS = 1024;   // 64 column pairs x 16 lanes
-constexpr int EIG_TEAM = 16;        // lanes per column pair
-constexpr int EIG_RPL = D / EIG_TEAM; // rows per lane
-constexpr int EIG_LD = D + 2;       // padded column stride (doubles)
+constexpr int EIG_LD = D + 2;       // padded column stride (doubles) of the full matrix
 constexpr int EIG_MAX_SWEEPS = 40;
 
-__device__ __forceinline__ double team_sum(double v)
+// Eigen-decomposition of M: Cholesky M + shift I = L L^T, then one-sided (Hestenes) Jacobi on the columns of L
+// (cyclic tournament order, 64 disjoint column pairs per round, cached squared norms, rotations skipped below
+// 1e-14 relative).  L has the square root of M's condition number and L^T L is much closer to diagonal than
+// M^2, which cuts the sweeps (14 -> 10 on the 4096-token workload).  The shift (1e-12 of the trace) keeps
+// the factorisation defined for rank-deficient M and is subtracted from the eigenvalues at the end;
+// eigenvectors are unaffected by it.  Jacobi converges quadratically, so a sweep in which every pair starts
+// below 1e-7 relative leaves them below ~1e-14: that sweep is the last.
+//
+// The rows of L are split over a cluster of 4 CTAs (4 SMs per head instead of 1; a
+// 32-head layer then occupies 128 of the 148 SMs).  Column rotations act on every row independently, so each
+// CTA rotates its own 32-row slice; only the dot product of a column pair needs all rows: every CTA writes its
+// partial sums into the shared memory of all four (distributed shared memory), one hardware cluster barrier
+// per round, and then all four CTAs add the partials in the same order -- every CTA takes bit-identical
+// rotation decisions, so they stay in step without further communication.  The Cholesky factorisation is
+// done redundantly by each CTA on a full copy (it is a small part of the time).
+namespace cg = cooperative_groups;
+constexpr int ECL = 4;                       // CTAs per cluster
+constexpr int ECT = 512;                     // threads per CTA: 64 column pairs x 8 lanes
+constexpr int ESL_ROWS = D / ECL;            // rows per CTA (32)
+constexpr int ESL_LD = ESL_ROWS + 2;         // padded column stride of the slice
+constexpr int ESL_RPL = ESL_ROWS / 8;        // rows per lane (4)
+
+__device__ __forceinline__ double team8_sum(double v)
 {
-    v += __shfl_xor_sync(0xffffffffu, v, 8);
     v += __shfl_xor_sync(0xffffffffu, v, 1);
     v += __shfl_xor_sync(0xffffffffu, v, 2);
     v += __shfl_xor_sync(0xffffffffu, v, 4);
     return v;
 }
 
-__global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
+__global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluster_kernel(
     const double *__restrict__ gram, double *__restrict__ eigval, double *__restrict__ eigvec,
     int *__restrict__ sweeps_out, unsigned *__restrict__ status)
 {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank();
     extern __shared__ __align__(16) double sm[];
-    double *Gs = sm;                       // column-major: Gs[col * EIG_LD + row]
-    double *nrm = sm + D * EIG_LD;         // squared column norms
+    double *Gs = sm;                                   // full matrix for the factorisation: Gs[col * EIG_LD + row]
+    double *Gl = Gs + D * EIG_LD;                      // this CTA's row slice: Gl[col * ESL_LD + r]
+    double *gpart = Gl + D * ESL_LD;                   // [2 parities][ECL sources][64 pairs] partial dot products
+    double *npart = gpart + 2 * ECL * 64;              // [ECL sources][D] partial squared norms
+    double *nrm = npart + ECL * D;                     // [D] squared column norms (identical in every CTA)
     int *rank = reinterpret_cast<int *>(nrm + D);
-    const int h = blockIdx.x, tid = threadIdx.x;
-    const int team = tid >> 4, l8 = tid & (EIG_TEAM - 1);
+    const int h = blockIdx.x / ECL, tid = threadIdx.x;
+    const int team = tid >> 3, l8 = tid & 7;
     const double *M = gram + (long long)h * D * D;
 
-    for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
+    for (int idx = tid; idx < D * D; idx += ECT) {
         const int r = idx / D, c = idx % D;
-        Gs[c * EIG_LD + r] = M[idx];       // M symmetric: row/column choice is immaterial
+        Gs[c * EIG_LD + r] = M[idx];
     }
     __syncthreads();
     double trace = 0.0;
     for (int i = 0; i < D; ++i) trace += Gs[i * EIG_LD + i];
-    // Preconditioning: M + shift*I = L L^T (Cholesky), then Jacobi on the columns of L instead of M.  The left
-    // singular vectors of L are the eigenvectors of M, its singular values sqrt(mu + shift); L has the square
-    // root of M's condition number and L^T L is much closer to diagonal than M^2, which roughly halves the
-    // sweeps.  The shift (1e-12 of the trace) keeps the factorisation defined for rank-deficient M and is
-    // subtracted from the eigenvalues at the end; eigenvectors are unaffected by it.
-    const double shift = trace > 0.0 ? 1e-12 * trace : 1e-300;
+    const double shift = trace > 0.0 ? 1e-12 * trace : 1e-300;       // M + shift I = L L^T
     __syncthreads();
     if (tid < D) Gs[tid * EIG_LD + tid] += shift;
-    double *lcol = nrm;                     // reused as the current column of L during the factorisation
+    double *lcol = nrm;
     for (int j = 0; j < D; ++j) {
         __syncthreads();
         const double ajj = Gs[j * EIG_LD + j];
         const double ljj = sqrt(ajj > 0.0 ? ajj : shift);
         if (tid >= j && tid < D) lcol[tid] = (tid == j) ? ljj : Gs[j * EIG_LD + tid] / ljj;
         __syncthreads();
-        const int n = D - 1 - j;            // trailing block: rows/cols j+1 .. D-1, lower triangle (row >= col)
-        for (int idx = tid; idx < n * n; idx += EIG_THREADS) {
+        const int n = D - 1 - j;
+        for (int idx = tid; idx < n * n; idx += ECT) {
             const int c = j + 1 + idx / n, r = j + 1 + idx % n;
             if (r >= c) Gs[c * EIG_LD + r] = fma(-lcol[r], lcol[c], Gs[c * EIG_LD + r]);
         }
         if (tid >= j && tid < D) Gs[j * EIG_LD + tid] = lcol[tid];
     }
     __syncthreads();
-    for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
-        const int c = idx / D, r = idx % D;
-        if (r < c) Gs[c * EIG_LD + r] = 0.0;            // L is lower triangular
+    // keep rows [32 crank, 32 crank + 32) of L (lower triangular: zero above the diagonal)
+    for (int idx = tid; idx < D * ESL_ROWS; idx += ECT) {
+        const int c = idx / ESL_ROWS, r = idx % ESL_ROWS, gr = crank * ESL_ROWS + r;
+        Gl[c * ESL_LD + r] = (gr >= c) ? Gs[c * EIG_LD + gr] : 0.0;
     }
-    __syncthreads();
-    const double null_thr = 4.0 * shift;                // squared norm of a column that is numerically null
+    const double null_thr = 4.0 * shift;
     const double tol2 = 1e-14 * 1e-14;
+    cluster.sync();                                    // every CTA's shared memory is set up before remote writes
+
+    double *gpart_remote[ECL], *npart_remote[ECL];
+#pragma unroll
+    for (int r = 0; r < ECL; ++r) {
+        gpart_remote[r] = cluster.map_shared_rank(gpart, r);
+        npart_remote[r] = cluster.map_shared_rank(npart, r);
+    }
+
+    // squared norms of all columns: partial over the local rows, exchanged, summed in rank order
+    auto refresh_norms = [&](bool take_sqrt) {
+        for (int col = team; col < D; col += ECT / 8) {
+            double s = 0.0;
+#pragma unroll
+            for (int i = 0; i < ESL_RPL; ++i) { const double v = Gl[col * ESL_LD + l8 + 8 * i]; s = fma(v, v, s); }
+            s = team8_sum(s);
+            if (l8 < ECL) npart_remote[l8][crank * D + col] = s;
+        }
+        cluster.sync();
+        if (tid < D) {
+            double s = 0.0;
+#pragma unroll
+            for (int r = 0; r < ECL; ++r) s += npart[r * D + tid];
+            nrm[tid] = take_sqrt ? sqrt(s) : s;
+        }
+        cluster.sync();                                // nobody overwrites npart before everyone has read it
+    };
 
     bool converged = false;
     int sweep = 0;
     for (; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
-        // refresh the squared norms from the columns (cached values drift by rounding)
-        for (int col = tid >> 4; col < D; col += EIG_THREADS / EIG_TEAM) {
-            double s = 0.0;
-#pragma unroll
-            for (int i = 0; i < EIG_RPL; ++i) { const double v = Gs[col * EIG_LD + l8 + EIG_TEAM * i]; s = fma(v, v, s); }
-            s = team_sum(s);
-            if (l8 == 0) nrm[col] = s;
-        }
-        __syncthreads();
-        // Largest cos^2 between two columns seen at the start of their rotation in this sweep.  Jacobi converges
-        // quadratically, so once every pair starts a sweep below 1e-7 the sweep leaves them below ~1e-14: done.
+        refresh_norms(false);
         int big = 0;
         for (int round = 0; round < D - 1; ++round) {
             int p, q;
             if (team == 0) { p = D - 1; q = round; }
             else { p = (round + team) % (D - 1); q = (round - team + (D - 1)) % (D - 1); }
-            double *gp = Gs + p * EIG_LD + l8, *gq = Gs + q * EIG_LD + l8;
-            double a[EIG_RPL], b[EIG_RPL];
-            double gam0 = 0.0, gam1 = 0.0;
+            double *gp = Gl + p * ESL_LD + l8, *gq = Gl + q * ESL_LD + l8;
+            double a[ESL_RPL], b[ESL_RPL];
+            double part = 0.0;
 #pragma unroll
-            for (int i = 0; i < EIG_RPL; ++i) { a[i] = gp[EIG_TEAM * i]; b[i] = gq[EIG_TEAM * i]; }
+            for (int i = 0; i < ESL_RPL; ++i) { a[i] = gp[8 * i]; b[i] = gq[8 * i]; part = fma(a[i], b[i], part); }
+            part = team8_sum(part);
+            double *slot = gpart + (round & 1) * (ECL * 64);
+            if (l8 < ECL) gpart_remote[l8][(round & 1) * (ECL * 64) + crank * 64 + team] = part;
+            cluster.sync();
+            double gam = 0.0;
 #pragma unroll
-            for (int i = 0; i < EIG_RPL; i += 2) { gam0 = fma(a[i], b[i], gam0); gam1 = fma(a[i + 1], b[i + 1], gam1); }
-            const double gam = team_sum(gam0 + gam1);
+            for (int r = 0; r < ECL; ++r) gam += slot[r * 64 + team];
             const double alpha = nrm[p], beta = nrm[q];
             const double g2 = gam * gam, ab = alpha * beta;
             if ((alpha > null_thr || beta > null_thr) && g2 > tol2 * ab) {
-                // t = tan of the rotation angle: smaller root of t^2 + 2 zeta t - 1 = 0, zeta = (beta-alpha)/(2 gam)
                 const double diff = beta - alpha;
                 const double den = fabs(diff) + sqrt(fma(diff, diff, 4.0 * g2));
                 double t = 2.0 * gam / den;
@@ -232,31 +271,23 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
                 const double c = rsqrt(fma(t, t, 1.0));
                 const double s = t * c;
 #pragma unroll
-                for (int i = 0; i < EIG_RPL; ++i) {
-                    gp[EIG_TEAM * i] = c * a[i] - s * b[i];
-                    gq[EIG_TEAM * i] = s * a[i] + c * b[i];
+                for (int i = 0; i < ESL_RPL; ++i) {
+                    gp[8 * i] = c * a[i] - s * b[i];
+                    gq[8 * i] = s * a[i] + c * b[i];
                 }
-                if (l8 == 0) { nrm[p] = alpha - t * gam; nrm[q] = beta + t * gam; }
                 if (g2 > 1e-14 * ab) big = 1;
+                if (l8 == 0) { nrm[p] = alpha - t * gam; nrm[q] = beta + t * gam; }
             }
-            big = __syncthreads_or(big);
+            __syncthreads();                           // this round's rotations are visible to the next round's reads
         }
-        converged = (big == 0);
+        converged = (__syncthreads_or(big) == 0);      // identical in every CTA: same gam, alpha, beta everywhere
     }
-    if (tid == 0) {
+    if (tid == 0 && crank == 0) {
         sweeps_out[h] = sweep;
         if (!converged) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
     }
 
-    // exact norms, ranks (descending, ties by column index), normalised output
-    for (int col = tid >> 4; col < D; col += EIG_THREADS / EIG_TEAM) {
-        double s = 0.0;
-#pragma unroll
-        for (int i = 0; i < EIG_RPL; ++i) { const double v = Gs[col * EIG_LD + l8 + EIG_TEAM * i]; s = fma(v, v, s); }
-        s = team_sum(s);
-        if (l8 == 0) nrm[col] = sqrt(s);                 // singular value of L: sqrt(mu + shift)
-    }
-    __syncthreads();
+    refresh_norms(true);                               // nrm = singular values of L = sqrt(mu + shift)
     if (tid < D) {
         const double mine = nrm[tid];
         int rk = 0;
@@ -265,16 +296,19 @@ __global__ void __launch_bounds__(EIG_THREADS, 1) eig_kernel(
             rk += (o > mine) || (o == mine && j < tid);
         }
         rank[tid] = rk;
-        const double mu_out = mine * mine - shift;
-        eigval[(long long)h * D + rk] = mu_out > 0.0 ? mu_out : 0.0;
+        if (crank == 0) {
+            const double mu_out = mine * mine - shift;
+            eigval[(long long)h * D + rk] = mu_out > 0.0 ? mu_out : 0.0;
+        }
     }
     __syncthreads();
-    for (int idx = tid; idx < D * D; idx += EIG_THREADS) {
-        const int col = idx / D, r = idx % D;
+    for (int idx = tid; idx < D * ESL_ROWS; idx += ECT) {
+        const int col = idx / ESL_ROWS, r = idx % ESL_ROWS;
         const double mu = nrm[col];
-        const double v = mu > 0.0 ? Gs[col * EIG_LD + r] / mu : 0.0;
-        eigvec[(long long)h * D * D + (long long)rank[col] * D + r] = v;
+        const double v = mu > 0.0 ? Gl[col * ESL_LD + r] / mu : 0.0;
+        eigvec[(long long)h * D * D + (long long)rank[col] * D + crank * ESL_ROWS + r] = v;
     }
+    cluster.sync();                                    // no CTA exits while a peer may still write into it
 }
 
 // ------------------------------------------------------------------------------------- assemble
@@ -377,9 +411,9 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
 
 int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * EIG_LD + D) + sizeof(int) * D;
-    SQUAT_CUDA(cudaFuncSetAttribute(eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    eig_kernel<<<s->n_kv_heads, EIG_THREADS, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
+    const size_t smem = sizeof(double) * (D * EIG_LD + D * ESL_LD + 2 * ECL * 64 + ECL * D + D) + sizeof(int) * D;
+    SQUAT_CUDA(cudaFuncSetAttribute(eig_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    eig_cluster_kernel<<<s->n_kv_heads * ECL, ECT, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
