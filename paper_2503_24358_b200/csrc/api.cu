@@ -98,7 +98,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     int sms = 148;
     if (cudaGetDevice(&s->device) != cudaSuccess) { delete s; return SQUAT_ERR_CUDA; }
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, s->device);
-    s->gram_chunks_cap = (2 * sms + n_kv_heads - 1) / n_kv_heads;
+    s->gram_chunks_cap = (2 * sms) / n_kv_heads;        // 2 resident CTAs per SM: one wave
     if (s->gram_chunks_cap < 1) s->gram_chunks_cap = 1;
     const size_t hdd = (size_t)n_kv_heads * D * D;
     // one allocation, carved up (256-byte aligned pieces)

@@ -56,39 +56,58 @@ __global__ void __launch_bounds__(GRAM_THREADS) gram_kernel(
 #pragma unroll
         for (int b = 0; b < 8; ++b) acc[a][b] = 0.0;
 
-    for (long long r0 = row_lo; r0 < row_hi; r0 += GRAM_ROWS) {
-        __syncthreads();
-        // stage GRAM_ROWS rows, 8 elements per thread per step
-        for (int idx = threadIdx.x; idx < GRAM_ROWS * (D / 8); idx += GRAM_THREADS) {
+    // Each thread stages up to 4 pieces of 8 elements per step (32 rows x 16 pieces over 160 threads).  The
+    // global loads of step s+1 are issued before the arithmetic of step s, so their latency is hidden.
+    constexpr int NPIECE = (GRAM_ROWS * (D / 8) + GRAM_THREADS - 1) / GRAM_THREADS;
+    uint4 pre[NPIECE][BF16 ? 1 : 2];
+    auto fetch = [&](long long r0) {
+#pragma unroll
+        for (int it = 0; it < NPIECE; ++it) {
+            const int idx = threadIdx.x + it * GRAM_THREADS;
             const int rr = idx / (D / 8), c8 = idx % (D / 8);
             const long long n = r0 + rr;
-            double v[8];
-            if (n < row_hi) {
+            if (idx < GRAM_ROWS * (D / 8) && n < row_hi) {
                 const long long hq = (long long)h * q_per_kv + n / n_tokens;
                 const long long t = n % n_tokens;
                 const long long off = hq * stride_h + t * stride_t + c8 * 8;
                 if (BF16) {
-                    const uint4 u = ldg128(reinterpret_cast<const __nv_bfloat16 *>(q) + off);
-                    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        v[2 * k] = (double)bf16lo_to_f32(w[k]);
-                        v[2 * k + 1] = (double)bf16hi_to_f32(w[k]);
-                    }
+                    pre[it][0] = ldg128(reinterpret_cast<const __nv_bfloat16 *>(q) + off);
                 } else {
-                    const float4 a = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(q) + off));
-                    const float4 b = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(q) + off) + 1);
-                    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-                    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+                    pre[it][0] = ldg128(reinterpret_cast<const float *>(q) + off);
+                    pre[it][BF16 ? 0 : 1] = ldg128(reinterpret_cast<const float *>(q) + off + 4);
                 }
             } else {
+                pre[it][0] = make_uint4(0, 0, 0, 0);
+                pre[it][BF16 ? 0 : 1] = make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+    if (row_lo < row_hi) fetch(row_lo);
+    for (long long r0 = row_lo; r0 < row_hi; r0 += GRAM_ROWS) {
+        __syncthreads();
 #pragma unroll
-                for (int k = 0; k < 8; ++k) v[k] = 0.0;
+        for (int it = 0; it < NPIECE; ++it) {
+            const int idx = threadIdx.x + it * GRAM_THREADS;
+            if (idx >= GRAM_ROWS * (D / 8)) continue;
+            const int rr = idx / (D / 8), c8 = idx % (D / 8);
+            double v[8];
+            if (BF16) {
+                const uint32_t w[4] = {pre[it][0].x, pre[it][0].y, pre[it][0].z, pre[it][0].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    v[2 * k] = (double)bf16lo_to_f32(w[k]);
+                    v[2 * k + 1] = (double)bf16hi_to_f32(w[k]);
+                }
+            } else {
+                const uint4 a = pre[it][0], b = pre[it][BF16 ? 0 : 1];
+                v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y); v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
+                v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y); v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
             }
 #pragma unroll
             for (int k = 0; k < 8; ++k) rows[rr][c8 * 8 + k] = v[k];
         }
         __syncthreads();
+        if (r0 + GRAM_ROWS < row_hi) fetch(r0 + GRAM_ROWS);
         if (active) {
 #pragma unroll 4
             for (int rr = 0; rr < GRAM_ROWS; ++rr) {
