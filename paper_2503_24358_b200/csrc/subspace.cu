@@ -276,19 +276,25 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
             part = team8_sum(part);
             double *slot = gpart + (round & 1) * (ECL * 64);
             if (l8 < ECL) gpart_remote[l8][(round & 1) * (ECL * 64) + crank * 64 + team] = part;
-            cluster.sync();
+            cluster.barrier_arrive();                  // release: the partial sums are visible cluster-wide ...
+            const double alpha = nrm[p], beta = nrm[q];
+            const double ab = alpha * beta, diff = beta - alpha;
+            cluster.barrier_wait();                    // ... once every CTA has arrived
             double gam = 0.0;
 #pragma unroll
             for (int r = 0; r < ECL; ++r) gam += slot[r * 64 + team];
-            const double alpha = nrm[p], beta = nrm[q];
-            const double g2 = gam * gam, ab = alpha * beta;
+            const double g2 = gam * gam;
             if ((alpha > null_thr || beta > null_thr) && g2 > tol2 * ab) {
-                const double diff = beta - alpha;
-                const double den = fabs(diff) + sqrt(fma(diff, diff, 4.0 * g2));
-                double t = 2.0 * gam / den;
-                if (diff < 0.0) t = -t;
-                const double c = rsqrt(fma(t, t, 1.0));
-                const double s = t * c;
+                // Rotation angle theta with tan(2 theta) = 2 gam / (beta - alpha), |theta| <= pi/4, from two
+                // reciprocal square roots (no division, no square root on the serial path):
+                //   cos(2 theta) = |diff| / hypot(diff, 2 gam),  c = sqrt((1 + cos 2theta)/2),  s = sin(2 theta)/(2c)
+                const double inv_r = rsqrt(fma(diff, diff, 4.0 * g2));
+                const double hc = fma(0.5 * fabs(diff), inv_r, 0.5);          // (1 + cos 2theta)/2 = c^2
+                const double inv_c = rsqrt(hc);
+                const double c = hc * inv_c;
+                double s = gam * inv_r * inv_c;                               // |sin 2theta| / (2c), sign of gam
+                if (diff < 0.0) s = -s;
+                const double t = s * inv_c;                                   // tan(theta)
 #pragma unroll
                 for (int i = 0; i < ESL_RPL; ++i) {
                     gp[8 * i] = c * a[i] - s * b[i];
