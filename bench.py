@@ -41,7 +41,7 @@ ALU_PEAK_TFLOPS = SM_COUNT * FMA_LANES * 2 * SM_MAX_GHZ / 1e3
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the key kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists for that workload).
-NCU_KEY_KERNEL_TRAFFIC_BYTES = {}
+NCU_KEY_KERNEL_TRAFFIC_BYTES = {1: 34_950_912, 2: 325_360_640}    # profiles/quant_keys_kernel_config1.md, streaming_kernels_config2.md
 
 
 def measured_peaks():
@@ -194,6 +194,10 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def rank_is_zero():
+    return dist_env()[0] == 0
+
+
 def workload_config(cfg):
     return {"workload": f"config {cfg.index}: {cfg.name}", "dtype": cfg.dtype, "batch": cfg.batch,
             "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
@@ -326,7 +330,7 @@ def run_e2e(args, cfg, sq, s, host_np, dev_outs, to_dev, flush, tdt, dev, vec_pe
 def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches, wall,
            flags, clocks):
     d, bits, G = cfg.head_dim, cfg.bits, cfg.group_size
-    if True:
+    if rank_is_zero():
         peaks = measured_peaks()
         elem = 4 if cfg.dtype == "f32" else 2
         key_ms = stage_ms["quantize_keys"]
