@@ -216,10 +216,10 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
         const double ljj = sqrt(ajj > 0.0 ? ajj : shift);
         if (tid >= j && tid < D) lcol[tid] = (tid == j) ? ljj : Gs[j * EIG_LD + tid] / ljj;
         __syncthreads();
-        const int n = D - 1 - j;
-        for (int idx = tid; idx < n * n; idx += ECT) {
-            const int c = j + 1 + idx / n, r = j + 1 + idx % n;
-            if (r >= c) Gs[c * EIG_LD + r] = fma(-lcol[r], lcol[c], Gs[c * EIG_LD + r]);
+        // trailing update of the lower triangle (row >= col); 2-D thread grid, no index division
+        for (int c = j + 1 + (tid >> 5); c < D; c += ECT / 32) {
+            const double lc = lcol[c];
+            for (int r = c + (tid & 31); r < D; r += 32) Gs[c * EIG_LD + r] = fma(-lcol[r], lc, Gs[c * EIG_LD + r]);
         }
         if (tid >= j && tid < D) Gs[j * EIG_LD + tid] = lcol[tid];
     }
@@ -359,12 +359,44 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
         coef[tid] = (tid < rank_r) ? s / (1.0 + s) : 0.0;
     }
     __syncthreads();
-    // P_inv = I - sum_{i<r} coef_i v_i v_i^T
-    for (int idx = tid; idx < D * D; idx += ASM_THREADS) {
-        const int a = idx / D, b = idx % D;
-        double s = (a == b) ? 1.0 : 0.0;
-        for (int i = 0; i < rank_r; ++i) s = fma(-coef[i] * V[i * D + a], V[i * D + b], s);
-        A[a * ASM_LD + b] = s;
+    // P_inv = I - sum_{i<r} coef_i v_i v_i^T, register-tiled: thread (ta, tb) owns rows 4 ta .. 4 ta + 3 and columns
+    // 8 tb .. 8 tb + 7; the eigenvectors are staged 32 at a time in shared memory behind A
+    {
+        double *U = coef + D;                           // [32][D] staged eigenvectors
+        const int ta = tid >> 4, tb = tid & 15;         // 32 x 16 tiles
+        double acc[4][8];
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 8; ++y) acc[x][y] = (4 * ta + x == 8 * tb + y) ? 1.0 : 0.0;
+        for (int i0 = 0; i0 < rank_r; i0 += 32) {
+            const int ni = rank_r - i0 < 32 ? rank_r - i0 : 32;
+            __syncthreads();
+            for (int idx = tid; idx < ni * D; idx += ASM_THREADS) U[idx] = V[(long long)i0 * D + idx];
+            __syncthreads();
+            for (int i = 0; i < ni; ++i) {
+                const double cf = -coef[i0 + i];
+                double a[4], b[8];
+#pragma unroll
+                for (int x = 0; x < 4; x += 2) {
+                    const double2 v = *reinterpret_cast<const double2 *>(U + i * D + 4 * ta + x);
+                    a[x] = cf * v.x; a[x + 1] = cf * v.y;
+                }
+#pragma unroll
+                for (int y = 0; y < 8; y += 2) {
+                    const double2 v = *reinterpret_cast<const double2 *>(U + i * D + 8 * tb + y);
+                    b[y] = v.x; b[y + 1] = v.y;
+                }
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+#pragma unroll
+                    for (int y = 0; y < 8; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 8; ++y) A[(4 * ta + x) * ASM_LD + 8 * tb + y] = acc[x][y];
     }
     __syncthreads();
     // in-place LDL^T (right-looking): afterwards the strict lower triangle of A holds L
@@ -375,10 +407,10 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
             lcol[tid] = v / A[j * ASM_LD + j];
         }
         __syncthreads();
-        const int n = D - 1 - j;
-        for (int idx = tid; idx < n * n; idx += ASM_THREADS) {
-            const int i = j + 1 + idx / n, k = j + 1 + idx % n;
-            A[i * ASM_LD + k] = fma(-lcol[i], colv[k], A[i * ASM_LD + k]);
+        // trailing update (full square, both triangles kept); 2-D thread grid, no index division
+        for (int i = j + 1 + (tid >> 5); i < D; i += ASM_THREADS / 32) {
+            const double li = lcol[i];
+            for (int k = j + 1 + (tid & 31); k < D; k += 32) A[i * ASM_LD + k] = fma(-li, colv[k], A[i * ASM_LD + k]);
         }
         if (tid > j && tid < D) A[tid * ASM_LD + j] = lcol[tid];
         __syncthreads();
@@ -446,7 +478,7 @@ int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 
 int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * ASM_LD + 3 * D);
+    const size_t smem = sizeof(double) * (D * ASM_LD + 3 * D + 32 * D);
     SQUAT_CUDA(cudaFuncSetAttribute(assemble_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt);
     squat_count_launch();
