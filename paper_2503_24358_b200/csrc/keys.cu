@@ -168,11 +168,12 @@ __device__ __forceinline__ void unpack_tile(const RawTile<BF16> &r, u64 (&acc)[4
 // going to the even code (the threshold of an odd c0 is one ulp lower, so "remainder == scale/2" moves it).
 template <int BITS, int NW, bool EXACT>
 __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, float *Eblk, bool store_e,
-                                            int lane, int team, int wteam, float2 *red,
+                                            int lane, int team, int wteam, float2 *red, float2 *park,
                                             uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
 {
-    constexpr int PER_WORD = 32 / BITS;
     constexpr float L = float((1 << BITS) - 1);
+    constexpr int PER_ACC = 16 / BITS;              // codes accumulated exactly in one float (16 bits of mantissa)
+    float cacc[BLK / PER_ACC];
 #pragma unroll
     for (int jj = 0; jj < BLK; ++jj) {
         const float xj = (jj & 1) ? hi_of(xp[jj >> 1]) : lo_of(xp[jj >> 1]);
@@ -196,15 +197,18 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(fmaxf(rng, 1e-30f)));   // constant group: dlt = 0 -> code 0
         const float scale = div_by_levels<BITS>(rng);
         const float y0 = __fmaf_rn(dltL, rcp, kMagic);
-        float e = __fmaf_rn(__fsub_rn(y0, kMagic), scale, -dlt);
-        float y = y0;
+        float c = __fsub_rn(y0, kMagic);
+        float e = __fmaf_rn(c, scale, -dlt);
         if (EXACT) {
             const float thr = __uint_as_float(__float_as_uint(0.5f * scale) - (__float_as_uint(y0) & 1u));
             const float adj = (e > thr) ? -1.0f : ((e < -thr) ? 1.0f : 0.0f);
-            y = __fadd_rn(y0, adj);
+            c = __fadd_rn(c, adj);
             e = __fmaf_rn(adj, scale, e);
         }
-        const uint32_t cbits = __float_as_uint(y) & ((1u << BITS) - 1u);
+        // pack the code arithmetically: sum of c * 2^(BITS k) is exact in float32 up to 16 bits
+        if (jj % PER_ACC == 0) cacc[jj / PER_ACC] = c;
+        else cacc[jj / PER_ACC] = __fmaf_rn(c, float(1 << ((jj % PER_ACC) * BITS)), cacc[jj / PER_ACC]);
+        park[jj] = make_float2(scale, m);               // same value from every lane; lane jj picks it up below
         if (store_e) Eblk[jj * 32] = e;
         const u64 ee = pack2(e, e);
         const float *wrow = diag + jj * BLK;
@@ -214,10 +218,15 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
             if (2 * q >= (jj + 1) / 2) xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
             xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
         }
-        if (jj % PER_WORD == 0) cw[jj / PER_WORD] = cbits;
-        else cw[jj / PER_WORD] |= cbits << ((jj % PER_WORD) * BITS);
-        if (lane == jj) { my_scale = scale; my_zero = m; }
     }
+    __syncwarp();
+    const float2 sz = park[lane];
+    my_scale = sz.x;
+    my_zero = sz.y;
+    __syncwarp();
+#pragma unroll
+    for (int w = 0; w < BLK * BITS / 32; ++w)
+        cw[w] = (uint32_t)__float2int_rn(cacc[2 * w]) | ((uint32_t)__float2int_rn(cacc[2 * w + 1]) << 16);
 }
 
 template <int BITS, int NW, bool BF16>
@@ -230,6 +239,7 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
     float *Wp = smem;                                    // 4 column panels, PANEL_FLOATS
     float *Eall = smem + PANEL_FLOATS;                   // [KEY_WARPS][E_ROWS][32]
     float2 *red = reinterpret_cast<float2 *>(Eall + KEY_WARPS * E_ROWS * 32);   // [NTEAMS][2][NW]
+    float2 *park = red + NTEAMS * 2 * NW + (threadIdx.x >> 5) * BLK;             // [KEY_WARPS][BLK] (scale, zero) of a block
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -360,9 +370,9 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                     uint32_t cw[WORDS_PER_BLK];
                     float my_scale = 0.0f, my_zero = 0.0f;
                     if (blk < p.exact_blocks)
-                        sweep_block<BITS, NW, true>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, cw, my_scale, my_zero);
+                        sweep_block<BITS, NW, true>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, park, cw, my_scale, my_zero);
                     else
-                        sweep_block<BITS, NW, false>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, cw, my_scale, my_zero);
+                        sweep_block<BITS, NW, false>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, park, cw, my_scale, my_zero);
 
                     // ---- this block's outputs -----------------------------------------------
                     if (WORDS_PER_BLK == 2)
@@ -390,7 +400,7 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     constexpr int NTEAMS = KEY_WARPS / NW;
-    const size_t smem = sizeof(float) * (PANEL_FLOATS + KEY_WARPS * E_ROWS * 32) + sizeof(float2) * NTEAMS * 2 * NW;
+    const size_t smem = sizeof(float) * (PANEL_FLOATS + KEY_WARPS * E_ROWS * 32) + sizeof(float2) * (NTEAMS * 2 * NW + KEY_WARPS * BLK);
     long long want = (p.total_groups + NTEAMS - 1) / NTEAMS;
     const int grid = (int)(want < sms ? want : sms);
     if (dtype == SQUAT_BF16) {
