@@ -182,6 +182,73 @@ __device__ __forceinline__ double team8_sum(double v)
     return v;
 }
 
+__device__ __forceinline__ double team16_sum(double v)
+{
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 8);
+    return v;
+}
+
+// 1/sqrt(x) for a normal positive double: hardware seed y (relative error 2^-22), residual r = 1 - x y^2, and one
+// third-order correction y (1 + r/2 + 3 r^2/8); what is left, about r^3/3, is far below a double's rounding.
+__device__ __forceinline__ double rsqrt_nr(double x)
+{
+    double y;
+    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    const double r = fma(-(x * y), y, 1.0);
+    return fma(y * r, fma(0.375, r, 0.5), y);
+}
+
+// One stage of the Jacobi method on the 4 x 4 Gram matrix g of a 4-column set: the two rotations (P,Q) and (R,S) act
+// on disjoint planes, so both are decided from the current g and applied together, free of branches (the two
+// dependency chains interleave).  A rotation turns col P into c colP - s colQ and col Q into s colP + c colQ with the
+// angle that makes them orthogonal (tan 2theta = 2 g_PQ / (g_QQ - g_PP), |theta| <= pi/4), from two reciprocal
+// square roots.  A pair already orthogonal to 1e-14 relative, or numerically null twice over, keeps c = 1, s = 0.
+struct RotParams { double c, s, t; bool act; };
+
+__device__ __forceinline__ RotParams rot_params(double alpha, double beta, double gam, double null_thr, double tol2, int &big)
+{
+    RotParams p;
+    const double g2 = gam * gam, ab = alpha * beta;
+    p.act = (alpha > null_thr || beta > null_thr) && g2 > tol2 * ab;
+    const double diff = beta - alpha;
+    const double rr = fma(diff, diff, 4.0 * g2);
+    const double inv_r = rsqrt_nr(p.act ? rr : 1.0);
+    const double hc = fma(0.5 * fabs(diff), inv_r, 0.5);              // (1 + cos 2theta)/2 = c^2, in [1/2, 1]
+    const double inv_c = rsqrt_nr(p.act ? hc : 1.0);
+    const double sm = gam * inv_r * inv_c;
+    p.c = p.act ? hc * inv_c : 1.0;
+    p.s = p.act ? (diff < 0.0 ? -sm : sm) : 0.0;
+    p.t = p.s * inv_c;                                                // tan(theta)
+    if (p.act && g2 > 1e-14 * ab) big = 1;
+    return p;
+}
+
+template <int P, int Q, int R, int S>
+__device__ __forceinline__ void gram_stage(double (&g)[4][4], double null_thr, double tol2,
+                                           double &c1, double &s1, double &c2, double &s2, int &big)
+{
+    const RotParams a = rot_params(g[P][P], g[Q][Q], g[P][Q], null_thr, tol2, big);
+    const RotParams b = rot_params(g[R][R], g[S][S], g[R][S], null_thr, tol2, big);
+    const double gpq = g[P][Q], grs = g[R][S];
+    g[P][P] -= a.t * gpq;
+    g[Q][Q] += a.t * gpq;
+    g[R][R] -= b.t * grs;
+    g[S][S] += b.t * grs;
+    g[P][Q] = g[Q][P] = a.act ? 0.0 : gpq;
+    g[R][S] = g[S][R] = b.act ? 0.0 : grs;
+    // the 2 x 2 block between the planes: rotate its (P,Q) index by a, then its (R,S) index by b
+    const double pr = a.c * g[P][R] - a.s * g[Q][R], qr = a.s * g[P][R] + a.c * g[Q][R];
+    const double ps = a.c * g[P][S] - a.s * g[Q][S], qs = a.s * g[P][S] + a.c * g[Q][S];
+    g[P][R] = g[R][P] = b.c * pr - b.s * ps;
+    g[P][S] = g[S][P] = b.s * pr + b.c * ps;
+    g[Q][R] = g[R][Q] = b.c * qr - b.s * qs;
+    g[Q][S] = g[S][Q] = b.s * qr + b.c * qs;
+    c1 = a.c; s1 = a.s; c2 = b.c; s2 = b.s;
+}
+
 __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluster_kernel(
     const double *__restrict__ gram, double *__restrict__ eigval, double *__restrict__ eigvec,
     int *__restrict__ sweeps_out, unsigned *__restrict__ status)
@@ -191,10 +258,11 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
     extern __shared__ __align__(16) double sm[];
     double *Gs = sm;                                   // full matrix for the factorisation: Gs[col * EIG_LD + row]
     double *Gl = Gs + D * EIG_LD;                      // this CTA's row slice: Gl[col * ESL_LD + r]
-    double *gpart = Gl + D * ESL_LD;                   // [2 parities][ECL sources][64 pairs] partial dot products
-    double *npart = gpart + 2 * ECL * 64;              // [ECL sources][D] partial squared norms
-    double *nrm = npart + ECL * D;                     // [D] squared column norms (identical in every CTA)
-    int *rank = reinterpret_cast<int *>(nrm + D);
+    double *gpart = Gl + D * ESL_LD;                   // [2 parities][ECL sources][10 entries][32 teams] partial Gram sums
+    double *npart = gpart + 2 * ECL * 32 * 10;              // [ECL sources][D] partial squared norms
+    double *nrm = npart + ECL * D;                     // [D] column norms (identical in every CTA)
+    double *rotcs = nrm + D;                           // [32 teams][6 rotations] (c, s) of the current round
+    int *rank = reinterpret_cast<int *>(rotcs + 32 * 12);
     const int h = blockIdx.x / ECL, tid = threadIdx.x;
     const int team = tid >> 3, l8 = tid & 7;
     const double *M = gram + (long long)h * D * D;
@@ -259,53 +327,105 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
         cluster.sync();                                // nobody overwrites npart before everyone has read it
     };
 
+    // Sweeps.  Columns are handled in 64 blocks of 2; a round pairs the blocks (tournament order, 63 rounds per
+    // sweep) and a team of 16 lanes owns one pair of blocks = 4 columns.  The team forms the 4 x 4 Gram matrix of
+    // its columns (partial over the local rows, exchanged through distributed shared memory: ONE cluster barrier
+    // per round), then runs the three stages (0,1)(2,3) / (0,2)(1,3) / (0,3)(1,2) of rotations on the Gram matrix
+    // itself -- in exact arithmetic the same rotations the column-by-column method would take -- and applies the six
+    // rotations to its rows.  Every CTA sums the partials in the same order, so all take bit-identical decisions.
+    // 4 lanes per team, 8 rows per lane: threads 0..127 move data, the rest only keep the barriers company
+    constexpr int TL = 8, RPL = ESL_ROWS / TL;
+    const int team16 = tid / TL, l16 = tid % TL;
+    const bool mover = tid < 32 * TL;
     bool converged = false;
     int sweep = 0;
     for (; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
-        refresh_norms(false);
         int big = 0;
-        for (int round = 0; round < D - 1; ++round) {
-            int p, q;
-            if (team == 0) { p = D - 1; q = round; }
-            else { p = (round + team) % (D - 1); q = (round - team + (D - 1)) % (D - 1); }
-            double *gp = Gl + p * ESL_LD + l8, *gq = Gl + q * ESL_LD + l8;
-            double a[ESL_RPL], b[ESL_RPL];
-            double part = 0.0;
+        for (int round = 0; round < D / 2 - 1; ++round) {
+            int col[4] = {0, 0, 0, 0};
+            double x[RPL][4];
+            if (mover) {
+                int bp, bq;
+                if (team16 == 0) { bp = D / 2 - 1; bq = round; }
+                else { bp = (round + team16) % (D / 2 - 1); bq = (round - team16 + (D / 2 - 1)) % (D / 2 - 1); }
+                col[0] = 2 * bp; col[1] = 2 * bp + 1; col[2] = 2 * bq; col[3] = 2 * bq + 1;
 #pragma unroll
-            for (int i = 0; i < ESL_RPL; ++i) { a[i] = gp[8 * i]; b[i] = gq[8 * i]; part = fma(a[i], b[i], part); }
-            part = team8_sum(part);
-            double *slot = gpart + (round & 1) * (ECL * 64);
-            if (l8 < ECL) gpart_remote[l8][(round & 1) * (ECL * 64) + crank * 64 + team] = part;
-            cluster.barrier_arrive();                  // release: the partial sums are visible cluster-wide ...
-            const double alpha = nrm[p], beta = nrm[q];
-            const double ab = alpha * beta, diff = beta - alpha;
-            cluster.barrier_wait();                    // ... once every CTA has arrived
-            double gam = 0.0;
+                for (int k = 0; k < 4; ++k)
 #pragma unroll
-            for (int r = 0; r < ECL; ++r) gam += slot[r * 64 + team];
-            const double g2 = gam * gam;
-            if ((alpha > null_thr || beta > null_thr) && g2 > tol2 * ab) {
-                // Rotation angle theta with tan(2 theta) = 2 gam / (beta - alpha), |theta| <= pi/4, from two
-                // reciprocal square roots (no division, no square root on the serial path):
-                //   cos(2 theta) = |diff| / hypot(diff, 2 gam),  c = sqrt((1 + cos 2theta)/2),  s = sin(2 theta)/(2c)
-                const double inv_r = rsqrt(fma(diff, diff, 4.0 * g2));
-                const double hc = fma(0.5 * fabs(diff), inv_r, 0.5);          // (1 + cos 2theta)/2 = c^2
-                const double inv_c = rsqrt(hc);
-                const double c = hc * inv_c;
-                double s = gam * inv_r * inv_c;                               // |sin 2theta| / (2c), sign of gam
-                if (diff < 0.0) s = -s;
-                const double t = s * inv_c;                                   // tan(theta)
+                    for (int i = 0; i < RPL; ++i) x[i][k] = Gl[col[k] * ESL_LD + l16 + TL * i];
+                double pg[10];                           // upper triangle of the partial Gram matrix
+                int n = 0;
 #pragma unroll
-                for (int i = 0; i < ESL_RPL; ++i) {
-                    gp[8 * i] = c * a[i] - s * b[i];
-                    gq[8 * i] = s * a[i] + c * b[i];
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = a; b < 4; ++b) {
+                        double v = 0.0;
+#pragma unroll
+                        for (int i = 0; i < RPL; ++i) v = fma(x[i][a], x[i][b], v);
+#pragma unroll
+                        for (int m = 1; m < TL; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+                        pg[n++] = v;
+                    }
+                // lane l sends all ten values to CTA l
+                if (l16 < ECL) {
+                    double *dst = gpart_remote[l16 % ECL] + (round & 1) * (ECL * 32 * 10) + crank * 320 + team16;
+#pragma unroll
+                    for (int k = 0; k < 10; ++k) dst[k * 32] = pg[k];
                 }
-                if (g2 > 1e-14 * ab) big = 1;
-                if (l8 == 0) { nrm[p] = alpha - t * gam; nrm[q] = beta + t * gam; }
+            }
+            cluster.barrier_arrive();
+            cluster.barrier_wait();
+            // the six rotations of every team are worked out once, by one lane per team (warp 0), and broadcast
+            if (tid < 32) {
+                double g[4][4];
+                const double *slot = gpart + (round & 1) * (ECL * 32 * 10) + tid;
+                int n = 0;
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = a; b < 4; ++b) {
+                        double v = 0.0;
+#pragma unroll
+                        for (int r = 0; r < ECL; ++r) v += slot[r * 320 + n * 32];
+                        g[a][b] = g[b][a] = v;
+                        ++n;
+                    }
+                double cc[6], ss[6];
+                gram_stage<0, 1, 2, 3>(g, null_thr, tol2, cc[0], ss[0], cc[1], ss[1], big);
+                gram_stage<0, 2, 1, 3>(g, null_thr, tol2, cc[2], ss[2], cc[3], ss[3], big);
+                gram_stage<0, 3, 1, 2>(g, null_thr, tol2, cc[4], ss[4], cc[5], ss[5], big);
+#pragma unroll
+                for (int k = 0; k < 6; ++k) {
+                    rotcs[tid * 12 + 2 * k] = cc[k];
+                    rotcs[tid * 12 + 2 * k + 1] = ss[k];
+                }
+            }
+            __syncthreads();
+            double c[6], sn[6];
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+                c[k] = rotcs[(mover ? team16 : 0) * 12 + 2 * k];
+                sn[k] = rotcs[(mover ? team16 : 0) * 12 + 2 * k + 1];
+            }
+            constexpr int RP[6] = {0, 2, 0, 1, 0, 1}, RQ[6] = {1, 3, 2, 3, 3, 2};
+            if (mover) {
+#pragma unroll
+                for (int row = 0; row < RPL; ++row) {
+#pragma unroll
+                    for (int k = 0; k < 6; ++k) {
+                        const double xp_ = x[row][RP[k]], xq_ = x[row][RQ[k]];
+                        x[row][RP[k]] = c[k] * xp_ - sn[k] * xq_;
+                        x[row][RQ[k]] = sn[k] * xp_ + c[k] * xq_;
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+#pragma unroll
+                    for (int i = 0; i < RPL; ++i) Gl[col[k] * ESL_LD + l16 + TL * i] = x[i][k];
             }
             __syncthreads();                           // this round's rotations are visible to the next round's reads
         }
-        converged = (__syncthreads_or(big) == 0);      // identical in every CTA: same gam, alpha, beta everywhere
+        converged = (__syncthreads_or(big) == 0);      // identical in every CTA: same Gram matrices everywhere
     }
     if (tid == 0 && crank == 0) {
         sweeps_out[h] = sweep;
@@ -468,7 +588,7 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
 
 int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * EIG_LD + D * ESL_LD + 2 * ECL * 64 + ECL * D + D) + sizeof(int) * D;
+    const size_t smem = sizeof(double) * (D * EIG_LD + D * ESL_LD + 2 * ECL * 32 * 10 + ECL * D + D + 32 * 12) + sizeof(int) * D;
     SQUAT_CUDA(cudaFuncSetAttribute(eig_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     eig_cluster_kernel<<<s->n_kv_heads * ECL, ECT, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
     squat_count_launch();
