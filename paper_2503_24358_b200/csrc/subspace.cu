@@ -152,42 +152,41 @@ __global__ void gram_reduce_kernel(const double *__restrict__ partial, int chunk
 constexpr int EIG_LD = D + 2;       // padded column stride (doubles) of the full matrix
 constexpr int EIG_MAX_SWEEPS = 40;
 
-// Eigen-decomposition of M: Cholesky M + shift I = L L^T, then one-sided (Hestenes) Jacobi on the columns of L
-// (cyclic tournament order, 64 disjoint column pairs per round, cached squared norms, rotations skipped below
-// 1e-14 relative).  L has the square root of M's condition number and L^T L is much closer to diagonal than
-// M^2, which cuts the sweeps (14 -> 10 on the 4096-token workload).  The shift (1e-12 of the trace) keeps
-// the factorisation defined for rank-deficient M and is subtracted from the eigenvalues at the end;
-// eigenvectors are unaffected by it.  Jacobi converges quadratically, so a sweep in which every pair starts
-// below 1e-7 relative leaves them below ~1e-14: that sweep is the last.
+// Eigen-decomposition of M: Cholesky M + shift I = L L^T, then one-sided (Hestenes) Jacobi on the columns of L.
+// L has the square root of M's condition number and L^T L is much closer to diagonal than M^2, which cuts the
+// sweeps (14 -> 10 on the 4096-token workload).  The shift (1e-12 of the trace) keeps the factorisation defined
+// for rank-deficient M and is subtracted from the eigenvalues at the end; eigenvectors are unaffected by it.
+// Rotations are skipped below 1e-14 relative; a sweep that applied none above that level is the last.
 //
-// The rows of L are split over a cluster of 4 CTAs (4 SMs per head instead of 1; a
-// 32-head layer then occupies 128 of the 148 SMs).  Column rotations act on every row independently, so each
-// CTA rotates its own 32-row slice; only the dot product of a column pair needs all rows: every CTA writes its
-// partial sums into the shared memory of all four (distributed shared memory), one hardware cluster barrier
-// per round, and then all four CTAs add the partials in the same order -- every CTA takes bit-identical
-// rotation decisions, so they stay in step without further communication.  The Cholesky factorisation is
-// done redundantly by each CTA on a full copy (it is a small part of the time).
+// One head is worked on by a cluster of 4 CTAs (4 SMs per head instead of 1; a 32-head layer then occupies 128
+// of the 148 SMs).  The 128 columns form 8 blocks of 16, and every CTA holds two blocks with ALL their rows, so a
+// rotation of two columns held by the same CTA needs no communication at all: one warp owns the pair (4 rows
+// per lane), the dot product is a warp reduction, and rounds inside a CTA are separated by a CTA barrier only.
+// A sweep is
+//   one intra phase   15 rounds that pair the columns inside each held block (8 + 8 pairs per round), then
+//   7 block rounds    of 16 rounds each that pair every column of one held block with every column of the other;
+//                     after each block round the blocks move on to their next holder (round-robin tournament of
+//                     the 8 blocks: position 0 stays, positions 1..7 rotate; CTA c holds positions c and 7 - c).
+// So the CTAs talk 7 times per sweep instead of once per round.  A block moves as ONE bulk copy from the sender's
+// shared memory into the receiver's spare buffer and completes a transaction barrier there; a cluster barrier
+// before the copies makes sure every spare buffer is free.  The squared column norms ride along with the block:
+// they are refreshed from the data at the start of a sweep and updated by each rotation in between
+// (alpha' = alpha - t gamma, beta' = beta + t gamma), so a round reduces one dot product, not three.
+// The Cholesky factorisation is done redundantly by each CTA on a full copy (it is a small part of the time).
 namespace cg = cooperative_groups;
 constexpr int ECL = 4;                       // CTAs per cluster
-constexpr int ECT = 512;                     // threads per CTA: 64 column pairs x 8 lanes
-constexpr int ESL_ROWS = D / ECL;            // rows per CTA (32)
-constexpr int ESL_LD = ESL_ROWS + 2;         // padded column stride of the slice
-constexpr int ESL_RPL = ESL_ROWS / 8;        // rows per lane (4)
+constexpr int ECT = 512;                     // threads per CTA: 16 warps = 16 column pairs per round
+constexpr int BW = 16;                       // columns per block
+constexpr int BLD = D + 2;                   // column stride inside a block buffer (doubles)
+constexpr int BLK_DOUBLES = BW * BLD + BW;   // 16 columns and their 16 squared norms
+constexpr unsigned BLK_BYTES = BLK_DOUBLES * (unsigned)sizeof(double);
+static_assert(D / BW == 2 * ECL, "two blocks per CTA");
+static_assert(BLK_BYTES % 16 == 0 && (D * EIG_LD * sizeof(double)) % 16 == 0, "bulk copies move 16-byte units");
 
-__device__ __forceinline__ double team8_sum(double v)
+__device__ __forceinline__ double warp_sum(double v)
 {
-    v += __shfl_xor_sync(0xffffffffu, v, 1);
-    v += __shfl_xor_sync(0xffffffffu, v, 2);
-    v += __shfl_xor_sync(0xffffffffu, v, 4);
-    return v;
-}
-
-__device__ __forceinline__ double team16_sum(double v)
-{
-    v += __shfl_xor_sync(0xffffffffu, v, 1);
-    v += __shfl_xor_sync(0xffffffffu, v, 2);
-    v += __shfl_xor_sync(0xffffffffu, v, 4);
-    v += __shfl_xor_sync(0xffffffffu, v, 8);
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
     return v;
 }
 
@@ -201,52 +200,76 @@ __device__ __forceinline__ double rsqrt_nr(double x)
     return fma(y * r, fma(0.375, r, 0.5), y);
 }
 
-// One stage of the Jacobi method on the 4 x 4 Gram matrix g of a 4-column set: the two rotations (P,Q) and (R,S) act
-// on disjoint planes, so both are decided from the current g and applied together, free of branches (the two
-// dependency chains interleave).  A rotation turns col P into c colP - s colQ and col Q into s colP + c colQ with the
-// angle that makes them orthogonal (tan 2theta = 2 g_PQ / (g_QQ - g_PP), |theta| <= pi/4), from two reciprocal
-// square roots.  A pair already orthogonal to 1e-14 relative, or numerically null twice over, keeps c = 1, s = 0.
-struct RotParams { double c, s, t; bool act; };
-
-__device__ __forceinline__ RotParams rot_params(double alpha, double beta, double gam, double null_thr, double tol2, int &big)
+// Shared-memory addresses, transaction barriers and the bulk copy between the CTAs of a cluster.
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned peer_u32(unsigned addr, int cta)
 {
-    RotParams p;
-    const double g2 = gam * gam, ab = alpha * beta;
-    p.act = (alpha > null_thr || beta > null_thr) && g2 > tol2 * ab;
-    const double diff = beta - alpha;
-    const double rr = fma(diff, diff, 4.0 * g2);
-    const double inv_r = rsqrt_nr(p.act ? rr : 1.0);
-    const double hc = fma(0.5 * fabs(diff), inv_r, 0.5);              // (1 + cos 2theta)/2 = c^2, in [1/2, 1]
-    const double inv_c = rsqrt_nr(p.act ? hc : 1.0);
-    const double sm = gam * inv_r * inv_c;
-    p.c = p.act ? hc * inv_c : 1.0;
-    p.s = p.act ? (diff < 0.0 ? -sm : sm) : 0.0;
-    p.t = p.s * inv_c;                                                // tan(theta)
-    if (p.act && g2 > 1e-14 * ab) big = 1;
-    return p;
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
+    return r;
+}
+__device__ __forceinline__ void mbar_init(unsigned bar, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Waits for the phase of the given parity; gives up after a bounded number of polls (returns false).
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity)
+{
+    for (int it = 0; it < (1 << 18); ++it) {
+        unsigned done;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// bytes from this CTA's shared memory to a peer's, completing `bytes` of the PEER's barrier when they have landed
+__device__ __forceinline__ void bulk_copy_to_peer(unsigned dst_peer, unsigned src, unsigned bytes, unsigned bar_peer)
+{
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_peer), "r"(src), "r"(bytes), "r"(bar_peer) : "memory");
 }
 
-template <int P, int Q, int R, int S>
-__device__ __forceinline__ void gram_stage(double (&g)[4][4], double null_thr, double tol2,
-                                           double &c1, double &s1, double &c2, double &s2, int &big)
+// One Jacobi rotation of the column pair (P, Q), by one warp: lane l owns rows l, l + 32, l + 64, l + 96.
+// alpha, beta are the (cached) squared norms, gamma = P . Q is reduced here.  New P = c P - s Q, new Q = s P + c Q
+// with the angle that makes them orthogonal (tan 2theta = 2 gamma / (beta - alpha), |theta| <= pi/4), from two
+// reciprocal square roots.  A pair already orthogonal to 1e-14 relative, or numerically null twice over, is left
+// alone.  Returns 1 when the pair was rotated from above the convergence level.
+__device__ __forceinline__ int rotate_pair(double *P, double *Q, double *nP, double *nQ, double null_thr, int lane)
 {
-    const RotParams a = rot_params(g[P][P], g[Q][Q], g[P][Q], null_thr, tol2, big);
-    const RotParams b = rot_params(g[R][R], g[S][S], g[R][S], null_thr, tol2, big);
-    const double gpq = g[P][Q], grs = g[R][S];
-    g[P][P] -= a.t * gpq;
-    g[Q][Q] += a.t * gpq;
-    g[R][R] -= b.t * grs;
-    g[S][S] += b.t * grs;
-    g[P][Q] = g[Q][P] = a.act ? 0.0 : gpq;
-    g[R][S] = g[S][R] = b.act ? 0.0 : grs;
-    // the 2 x 2 block between the planes: rotate its (P,Q) index by a, then its (R,S) index by b
-    const double pr = a.c * g[P][R] - a.s * g[Q][R], qr = a.s * g[P][R] + a.c * g[Q][R];
-    const double ps = a.c * g[P][S] - a.s * g[Q][S], qs = a.s * g[P][S] + a.c * g[Q][S];
-    g[P][R] = g[R][P] = b.c * pr - b.s * ps;
-    g[P][S] = g[S][P] = b.s * pr + b.c * ps;
-    g[Q][R] = g[R][Q] = b.c * qr - b.s * qs;
-    g[Q][S] = g[S][Q] = b.s * qr + b.c * qs;
-    c1 = a.c; s1 = a.s; c2 = b.c; s2 = b.s;
+    double xp[4], xq[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { xp[i] = P[lane + 32 * i]; xq[i] = Q[lane + 32 * i]; }
+    const double alpha = *nP, beta = *nQ;
+    double gam = 0.0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) gam = fma(xp[i], xq[i], gam);
+    gam = warp_sum(gam);
+    const double g2 = gam * gam, ab = alpha * beta;
+    if (!((alpha > null_thr || beta > null_thr) && g2 > 1e-28 * ab)) return 0;      // warp-uniform
+    const double diff = beta - alpha;
+    const double inv_r = rsqrt_nr(fma(diff, diff, 4.0 * g2));
+    const double hc = fma(0.5 * fabs(diff), inv_r, 0.5);              // (1 + cos 2theta)/2 = c^2, in [1/2, 1]
+    const double inv_c = rsqrt_nr(hc);
+    const double c = hc * inv_c;
+    const double sm = gam * inv_r * inv_c;
+    const double s = diff < 0.0 ? -sm : sm;
+    const double t = s * inv_c;                                       // tan(theta)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        P[lane + 32 * i] = c * xp[i] - s * xq[i];
+        Q[lane + 32 * i] = s * xp[i] + c * xq[i];
+    }
+    if (lane == 0) {
+        *nP = alpha - t * gam;
+        *nQ = beta + t * gam;
+    }
+    return g2 > 1e-14 * ab;
 }
 
 __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluster_kernel(
@@ -257,14 +280,13 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
     const int crank = (int)cluster.block_rank();
     extern __shared__ __align__(16) double sm[];
     double *Gs = sm;                                   // full matrix for the factorisation: Gs[col * EIG_LD + row]
-    double *Gl = Gs + D * EIG_LD;                      // this CTA's row slice: Gl[col * ESL_LD + r]
-    double *gpart = Gl + D * ESL_LD;                   // [2 parities][ECL sources][10 entries][32 teams] partial Gram sums
-    double *npart = gpart + 2 * ECL * 32 * 10;              // [ECL sources][D] partial squared norms
-    double *nrm = npart + ECL * D;                     // [D] column norms (identical in every CTA)
-    double *rotcs = nrm + D;                           // [32 teams][6 rotations] (c, s) of the current round
-    int *rank = reinterpret_cast<int *>(rotcs + 32 * 12);
+    double *blk = Gs + D * EIG_LD;                     // [2 buffers][2 slots][BLK_DOUBLES]: the held blocks and the spare
+    double *nall = blk + 4 * BLK_DOUBLES;              // [ECL][32] final column norms of the whole cluster
+    double *lcol = nall + ECL * 32;                    // [D] scratch of the factorisation
+    unsigned long long *mbar = reinterpret_cast<unsigned long long *>(lcol + D);      // [2 buffers]
+    int *flags = reinterpret_cast<int *>(mbar + 2);    // [ECL] "rotated above the convergence level" per CTA
     const int h = blockIdx.x / ECL, tid = threadIdx.x;
-    const int team = tid >> 3, l8 = tid & 7;
+    const int warp = tid >> 5, lane = tid & 31;
     const double *M = gram + (long long)h * D * D;
 
     for (int idx = tid; idx < D * D; idx += ECT) {
@@ -277,7 +299,6 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
     const double shift = trace > 0.0 ? 1e-12 * trace : 1e-300;       // M + shift I = L L^T
     __syncthreads();
     if (tid < D) Gs[tid * EIG_LD + tid] += shift;
-    double *lcol = nrm;
     for (int j = 0; j < D; ++j) {
         __syncthreads();
         const double ajj = Gs[j * EIG_LD + j];
@@ -292,166 +313,131 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
         if (tid >= j && tid < D) Gs[j * EIG_LD + tid] = lcol[tid];
     }
     __syncthreads();
-    // keep rows [32 crank, 32 crank + 32) of L (lower triangular: zero above the diagonal)
-    for (int idx = tid; idx < D * ESL_ROWS; idx += ECT) {
-        const int c = idx / ESL_ROWS, r = idx % ESL_ROWS, gr = crank * ESL_ROWS + r;
-        Gl[c * ESL_LD + r] = (gr >= c) ? Gs[c * EIG_LD + gr] : 0.0;
+    // this CTA starts with the blocks at positions crank (slot 0) and 7 - crank (slot 1); L is lower triangular
+    for (int idx = tid; idx < 2 * BW * D; idx += ECT) {
+        const int r = idx % D, ci = (idx / D) % BW, slot = idx / (D * BW);
+        const int col = BW * (slot == 0 ? crank : 2 * ECL - 1 - crank) + ci;
+        blk[slot * BLK_DOUBLES + ci * BLD + r] = (r >= col) ? Gs[col * EIG_LD + r] : 0.0;
     }
     const double null_thr = 4.0 * shift;
-    const double tol2 = 1e-14 * 1e-14;
-    cluster.sync();                                    // every CTA's shared memory is set up before remote writes
-
-    double *gpart_remote[ECL], *npart_remote[ECL];
-#pragma unroll
-    for (int r = 0; r < ECL; ++r) {
-        gpart_remote[r] = cluster.map_shared_rank(gpart, r);
-        npart_remote[r] = cluster.map_shared_rank(npart, r);
+    if (tid == 0) {
+        mbar_init(smem_u32(&mbar[0]), 1);
+        mbar_init(smem_u32(&mbar[1]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    cluster.sync();                                    // every CTA's barriers exist before anybody copies
 
-    // squared norms of all columns: partial over the local rows, exchanged, summed in rank order
-    auto refresh_norms = [&](bool take_sqrt) {
-        for (int col = team; col < D; col += ECT / 8) {
+    // squared norms of the 32 held columns, from the data: warp w takes columns w and w + 16
+    auto refresh_norms = [&](double *cur) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            double *col = cur + k * BLK_DOUBLES + warp * BLD;
             double s = 0.0;
 #pragma unroll
-            for (int i = 0; i < ESL_RPL; ++i) { const double v = Gl[col * ESL_LD + l8 + 8 * i]; s = fma(v, v, s); }
-            s = team8_sum(s);
-            if (l8 < ECL) npart_remote[l8][crank * D + col] = s;
+            for (int i = 0; i < 4; ++i) { const double v = col[lane + 32 * i]; s = fma(v, v, s); }
+            s = warp_sum(s);
+            if (lane == 0) cur[k * BLK_DOUBLES + BW * BLD + warp] = s;
         }
-        cluster.sync();
-        if (tid < D) {
-            double s = 0.0;
-#pragma unroll
-            for (int r = 0; r < ECL; ++r) s += npart[r * D + tid];
-            nrm[tid] = take_sqrt ? sqrt(s) : s;
-        }
-        cluster.sync();                                // nobody overwrites npart before everyone has read it
+        __syncthreads();
     };
 
-    // Sweeps.  Columns are handled in 64 blocks of 2; a round pairs the blocks (tournament order, 63 rounds per
-    // sweep) and a team of 16 lanes owns one pair of blocks = 4 columns.  The team forms the 4 x 4 Gram matrix of
-    // its columns (partial over the local rows, exchanged through distributed shared memory: ONE cluster barrier
-    // per round), then runs the three stages (0,1)(2,3) / (0,2)(1,3) / (0,3)(1,2) of rotations on the Gram matrix
-    // itself -- in exact arithmetic the same rotations the column-by-column method would take -- and applies the six
-    // rotations to its rows.  Every CTA sums the partials in the same order, so all take bit-identical decisions.
-    // 4 lanes per team, 8 rows per lane: threads 0..127 move data, the rest only keep the barriers company
-    constexpr int TL = 8, RPL = ESL_ROWS / TL;
-    const int team16 = tid / TL, l16 = tid % TL;
-    const bool mover = tid < 32 * TL;
-    bool converged = false;
+    int cur_buf = 0, moves = 0;                         // which buffer holds the blocks; block moves so far
+    bool converged = false, failed = false;
     int sweep = 0;
-    for (; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
+    for (; sweep < EIG_MAX_SWEEPS && !converged && !failed; ++sweep) {
         int big = 0;
-        for (int round = 0; round < D / 2 - 1; ++round) {
-            int col[4] = {0, 0, 0, 0};
-            double x[RPL][4];
-            if (mover) {
-                int bp, bq;
-                if (team16 == 0) { bp = D / 2 - 1; bq = round; }
-                else { bp = (round + team16) % (D / 2 - 1); bq = (round - team16 + (D / 2 - 1)) % (D / 2 - 1); }
-                col[0] = 2 * bp; col[1] = 2 * bp + 1; col[2] = 2 * bq; col[3] = 2 * bq + 1;
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-#pragma unroll
-                    for (int i = 0; i < RPL; ++i) x[i][k] = Gl[col[k] * ESL_LD + l16 + TL * i];
-                double pg[10];                           // upper triangle of the partial Gram matrix
-                int n = 0;
-#pragma unroll
-                for (int a = 0; a < 4; ++a)
-#pragma unroll
-                    for (int b = a; b < 4; ++b) {
-                        double v = 0.0;
-#pragma unroll
-                        for (int i = 0; i < RPL; ++i) v = fma(x[i][a], x[i][b], v);
-#pragma unroll
-                        for (int m = 1; m < TL; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
-                        pg[n++] = v;
-                    }
-                // lane l sends all ten values to CTA l
-                if (l16 < ECL) {
-                    double *dst = gpart_remote[l16 % ECL] + (round & 1) * (ECL * 32 * 10) + crank * 320 + team16;
-#pragma unroll
-                    for (int k = 0; k < 10; ++k) dst[k * 32] = pg[k];
-                }
+        double *cur = blk + cur_buf * 2 * BLK_DOUBLES;
+        refresh_norms(cur);
+        // intra phase: round-robin of the 16 columns of a block; warps 0-7 on slot 0, warps 8-15 on slot 1
+        {
+            double *b = cur + (warp >> 3) * BLK_DOUBLES, *nb = b + BW * BLD;
+            const int t = warp & 7;
+            for (int round = 0; round < BW - 1; ++round) {
+                int p, q;
+                if (t == 0) { p = BW - 1; q = round; }
+                else { p = (round + t) % (BW - 1); q = (round - t + (BW - 1)) % (BW - 1); }
+                big |= rotate_pair(b + p * BLD, b + q * BLD, nb + p, nb + q, null_thr, lane);
+                __syncthreads();
             }
-            cluster.barrier_arrive();
-            cluster.barrier_wait();
-            // the six rotations of every team are worked out once, by one lane per team (warp 0), and broadcast
-            if (tid < 32) {
-                double g[4][4];
-                const double *slot = gpart + (round & 1) * (ECL * 32 * 10) + tid;
-                int n = 0;
-#pragma unroll
-                for (int a = 0; a < 4; ++a)
-#pragma unroll
-                    for (int b = a; b < 4; ++b) {
-                        double v = 0.0;
-#pragma unroll
-                        for (int r = 0; r < ECL; ++r) v += slot[r * 320 + n * 32];
-                        g[a][b] = g[b][a] = v;
-                        ++n;
-                    }
-                double cc[6], ss[6];
-                gram_stage<0, 1, 2, 3>(g, null_thr, tol2, cc[0], ss[0], cc[1], ss[1], big);
-                gram_stage<0, 2, 1, 3>(g, null_thr, tol2, cc[2], ss[2], cc[3], ss[3], big);
-                gram_stage<0, 3, 1, 2>(g, null_thr, tol2, cc[4], ss[4], cc[5], ss[5], big);
-#pragma unroll
-                for (int k = 0; k < 6; ++k) {
-                    rotcs[tid * 12 + 2 * k] = cc[k];
-                    rotcs[tid * 12 + 2 * k + 1] = ss[k];
-                }
-            }
-            __syncthreads();
-            double c[6], sn[6];
-#pragma unroll
-            for (int k = 0; k < 6; ++k) {
-                c[k] = rotcs[(mover ? team16 : 0) * 12 + 2 * k];
-                sn[k] = rotcs[(mover ? team16 : 0) * 12 + 2 * k + 1];
-            }
-            constexpr int RP[6] = {0, 2, 0, 1, 0, 1}, RQ[6] = {1, 3, 2, 3, 3, 2};
-            if (mover) {
-#pragma unroll
-                for (int row = 0; row < RPL; ++row) {
-#pragma unroll
-                    for (int k = 0; k < 6; ++k) {
-                        const double xp_ = x[row][RP[k]], xq_ = x[row][RQ[k]];
-                        x[row][RP[k]] = c[k] * xp_ - sn[k] * xq_;
-                        x[row][RQ[k]] = sn[k] * xp_ + c[k] * xq_;
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-#pragma unroll
-                    for (int i = 0; i < RPL; ++i) Gl[col[k] * ESL_LD + l16 + TL * i] = x[i][k];
-            }
-            __syncthreads();                           // this round's rotations are visible to the next round's reads
         }
-        converged = (__syncthreads_or(big) == 0);      // identical in every CTA: same Gram matrices everywhere
+        for (int br = 0; br < 2 * ECL - 1; ++br) {
+            cur = blk + cur_buf * 2 * BLK_DOUBLES;
+            double *b0 = cur, *b1 = cur + BLK_DOUBLES;
+            for (int round = 0; round < BW; ++round) {
+                const int q = (warp + round) & (BW - 1);
+                big |= rotate_pair(b0 + warp * BLD, b1 + q * BLD, b0 + BW * BLD + warp, b1 + BW * BLD + q, null_thr, lane);
+                __syncthreads();
+            }
+            // move the blocks on: position 0 stays, 1 -> 2 -> ... -> 7 -> 1.  Position p lives in CTA min(p, 7 - p),
+            // slot 0 if p < 4.  The copies are made by the copy engine: order this thread's stores before them.
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            cluster.sync();                            // everybody is done with this block round: all spares are free
+            const int nxt = cur_buf ^ 1;
+            const unsigned bar = smem_u32(&mbar[nxt]);
+            if (tid == 0 && !failed) {
+                mbar_expect_tx(bar, 2 * BLK_BYTES);
+#pragma unroll
+                for (int slot = 0; slot < 2; ++slot) {
+                    const int pos = slot == 0 ? crank : 2 * ECL - 1 - crank;
+                    const int npos = pos == 0 ? 0 : (pos == 2 * ECL - 1 ? 1 : pos + 1);
+                    const int dcta = npos < ECL ? npos : 2 * ECL - 1 - npos, dslot = npos < ECL ? 0 : 1;
+                    const unsigned src = smem_u32(blk + (cur_buf * 2 + slot) * BLK_DOUBLES);
+                    const unsigned dst = smem_u32(blk + (nxt * 2 + dslot) * BLK_DOUBLES);
+                    bulk_copy_to_peer(peer_u32(dst, dcta), src, BLK_BYTES, peer_u32(bar, dcta));
+                }
+            }
+            // after a wait has run out nothing is waited for any more, but every CTA keeps making the same
+            // sequence of barrier calls until the end of the sweep, where the failure is made known to all
+            const bool arrived = failed || mbar_wait(bar, (unsigned)(moves >> 1) & 1u);
+            failed = __syncthreads_or(!arrived) != 0 || failed;
+            cur_buf = nxt;
+            ++moves;
+        }
+        // the sweep is the last one if no CTA of the cluster rotated a pair from above the convergence level
+        big = __syncthreads_or(big);
+        if (tid < ECL) *cluster.map_shared_rank(&flags[crank], tid) = (big ? 1 : 0) | (failed ? 2 : 0);
+        cluster.sync();
+        int any = 0;
+#pragma unroll
+        for (int r = 0; r < ECL; ++r) any |= flags[r];
+        converged = (any & 1) == 0;
+        failed = (any & 2) != 0;
+        cluster.sync();                                // flags are read before the next sweep may overwrite them
     }
     if (tid == 0 && crank == 0) {
         sweeps_out[h] = sweep;
-        if (!converged) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
+        if (!converged || failed) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
     }
 
-    refresh_norms(true);                               // nrm = singular values of L = sqrt(mu + shift)
-    if (tid < D) {
-        const double mine = nrm[tid];
+    // singular values of L = sqrt(mu + shift) are the column norms; rank them over the whole cluster
+    double *cur = blk + cur_buf * 2 * BLK_DOUBLES;
+    refresh_norms(cur);
+    if (tid < 32) {
+        const double n2 = cur[(tid >> 4) * BLK_DOUBLES + BW * BLD + (tid & 15)];
+        const double nv = sqrt(n2);
+#pragma unroll
+        for (int r = 0; r < ECL; ++r) *cluster.map_shared_rank(&nall[crank * 32 + tid], r) = nv;
+    }
+    cluster.sync();
+    for (int k = 0; k < 2; ++k) {                      // warp w writes held columns w (slot 0) and w (slot 1)
+        const int id = crank * 32 + k * BW + warp;
+        const double mine = nall[id];
         int rk = 0;
-        for (int j = 0; j < D; ++j) {
-            const double o = nrm[j];
-            rk += (o > mine) || (o == mine && j < tid);
+        for (int j = lane; j < D; j += 32) {
+            const double o = nall[j];
+            rk += (o > mine) || (o == mine && j < id);
         }
-        rank[tid] = rk;
-        if (crank == 0) {
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) rk += __shfl_xor_sync(0xffffffffu, rk, m);
+        const double *col = cur + k * BLK_DOUBLES + warp * BLD;
+        const double inv = mine > 0.0 ? 1.0 / mine : 0.0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            eigvec[(long long)h * D * D + (long long)rk * D + lane + 32 * i] = col[lane + 32 * i] * inv;
+        if (lane == 0) {
             const double mu_out = mine * mine - shift;
             eigval[(long long)h * D + rk] = mu_out > 0.0 ? mu_out : 0.0;
         }
-    }
-    __syncthreads();
-    for (int idx = tid; idx < D * ESL_ROWS; idx += ECT) {
-        const int col = idx / ESL_ROWS, r = idx % ESL_ROWS;
-        const double mu = nrm[col];
-        const double v = mu > 0.0 ? Gl[col * ESL_LD + r] / mu : 0.0;
-        eigvec[(long long)h * D * D + (long long)rank[col] * D + crank * ESL_ROWS + r] = v;
     }
     cluster.sync();                                    // no CTA exits while a peer may still write into it
 }
@@ -588,7 +574,7 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
 
 int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * EIG_LD + D * ESL_LD + 2 * ECL * 32 * 10 + ECL * D + D + 32 * 12) + sizeof(int) * D;
+    const size_t smem = sizeof(double) * (D * EIG_LD + 4 * BLK_DOUBLES + ECL * 32 + D + 2) + sizeof(int) * ECL;
     SQUAT_CUDA(cudaFuncSetAttribute(eig_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     eig_cluster_kernel<<<s->n_kv_heads * ECL, ECT, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
     squat_count_launch();
