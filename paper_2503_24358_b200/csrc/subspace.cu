@@ -235,23 +235,25 @@ __device__ __forceinline__ void bulk_copy_to_peer(unsigned dst_peer, unsigned sr
                  ::"r"(dst_peer), "r"(src), "r"(bytes), "r"(bar_peer) : "memory");
 }
 
-// One Jacobi rotation of the column pair (P, Q), by one warp: lane l owns rows l, l + 32, l + 64, l + 96.
-// alpha, beta are the (cached) squared norms, gamma = P . Q is reduced here.  New P = c P - s Q, new Q = s P + c Q
-// with the angle that makes them orthogonal (tan 2theta = 2 gamma / (beta - alpha), |theta| <= pi/4), from two
-// reciprocal square roots.  A pair already orthogonal to 1e-14 relative, or numerically null twice over, is left
-// alone.  Returns 1 when the pair was rotated from above the convergence level.
-__device__ __forceinline__ int rotate_pair(double *P, double *Q, double *nP, double *nQ, double null_thr, int lane)
+__device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+
+// One Jacobi rotation of a column pair (P, Q) held in registers by a team of 16 lanes (both halves of a warp work
+// on different pairs): lane l owns rows l, l + 16, ..., l + 112.  alpha, beta are the (cached) squared norms, kept by
+// every lane; gamma = P . Q is reduced here.  New P = c P - s Q, new Q = s P + c Q with the angle that makes them
+// orthogonal (tan 2theta = 2 gamma / (beta - alpha), |theta| <= pi/4), from two reciprocal square roots.  A pair
+// already orthogonal to 1e-14 relative, or numerically null twice over, is left alone (returns 0); otherwise
+// returns 1, or 3 when the pair started above the convergence level.
+constexpr int TROWS = D / 16;                // rows per lane of a team
+__device__ __forceinline__ int rotate_regs(double (&xp)[TROWS], double (&xq)[TROWS], double &alpha, double &beta, double null_thr)
 {
-    double xp[4], xq[4];
+    double g0 = 0.0, g1 = 0.0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) { xp[i] = P[lane + 32 * i]; xq[i] = Q[lane + 32 * i]; }
-    const double alpha = *nP, beta = *nQ;
-    double gam = 0.0;
+    for (int i = 0; i < TROWS; i += 2) { g0 = fma(xp[i], xq[i], g0); g1 = fma(xp[i + 1], xq[i + 1], g1); }
+    double gam = g0 + g1;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) gam = fma(xp[i], xq[i], gam);
-    gam = warp_sum(gam);
+    for (int m = 8; m >= 1; m >>= 1) gam += __shfl_xor_sync(0xffffffffu, gam, m);
     const double g2 = gam * gam, ab = alpha * beta;
-    if (!((alpha > null_thr || beta > null_thr) && g2 > 1e-28 * ab)) return 0;      // warp-uniform
+    if (!((alpha > null_thr || beta > null_thr) && g2 > 1e-28 * ab)) return 0;      // uniform over the team
     const double diff = beta - alpha;
     const double inv_r = rsqrt_nr(fma(diff, diff, 4.0 * g2));
     const double hc = fma(0.5 * fabs(diff), inv_r, 0.5);              // (1 + cos 2theta)/2 = c^2, in [1/2, 1]
@@ -261,15 +263,14 @@ __device__ __forceinline__ int rotate_pair(double *P, double *Q, double *nP, dou
     const double s = diff < 0.0 ? -sm : sm;
     const double t = s * inv_c;                                       // tan(theta)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        P[lane + 32 * i] = c * xp[i] - s * xq[i];
-        Q[lane + 32 * i] = s * xp[i] + c * xq[i];
+    for (int i = 0; i < TROWS; ++i) {
+        const double p = xp[i], q = xq[i];
+        xp[i] = c * p - s * q;
+        xq[i] = s * p + c * q;
     }
-    if (lane == 0) {
-        *nP = alpha - t * gam;
-        *nQ = beta + t * gam;
-    }
-    return g2 > 1e-14 * ab;
+    alpha -= t * gam;
+    beta += t * gam;
+    return g2 > 1e-14 * ab ? 3 : 1;
 }
 
 __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluster_kernel(
@@ -348,25 +349,58 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
         int big = 0;
         double *cur = blk + cur_buf * 2 * BLK_DOUBLES;
         refresh_norms(cur);
-        // intra phase: round-robin of the 16 columns of a block; warps 0-7 on slot 0, warps 8-15 on slot 1
-        {
-            double *b = cur + (warp >> 3) * BLK_DOUBLES, *nb = b + BW * BLD;
-            const int t = warp & 7;
+        // Pairs are worked on by 16 teams of 16 lanes (warps 0-7); they keep in step through a barrier of their own.
+        const int team = tid >> 4, tl = tid & 15;
+        constexpr int TEAM_THREADS = 16 * 16;
+        // intra phase: round-robin of the 16 columns of a block; teams 0-7 on slot 0, teams 8-15 on slot 1
+        if (tid < TEAM_THREADS) {
+            double *b = cur + (team >> 3) * BLK_DOUBLES, *nb = b + BW * BLD;
+            const int t = team & 7;
             for (int round = 0; round < BW - 1; ++round) {
                 int p, q;
                 if (t == 0) { p = BW - 1; q = round; }
                 else { p = (round + t) % (BW - 1); q = (round - t + (BW - 1)) % (BW - 1); }
-                big |= rotate_pair(b + p * BLD, b + q * BLD, nb + p, nb + q, null_thr, lane);
-                __syncthreads();
+                double xp[TROWS], xq[TROWS];
+#pragma unroll
+                for (int i = 0; i < TROWS; ++i) { xp[i] = b[p * BLD + tl + 16 * i]; xq[i] = b[q * BLD + tl + 16 * i]; }
+                double alpha = nb[p], beta = nb[q];
+                const int did = rotate_regs(xp, xq, alpha, beta, null_thr);
+                if (did) {
+#pragma unroll
+                    for (int i = 0; i < TROWS; ++i) { b[p * BLD + tl + 16 * i] = xp[i]; b[q * BLD + tl + 16 * i] = xq[i]; }
+                    if (tl == 0) { nb[p] = alpha; nb[q] = beta; }
+                }
+                big |= did >> 1;
+                named_bar_sync(1, TEAM_THREADS);
             }
         }
+        __syncthreads();
         for (int br = 0; br < 2 * ECL - 1; ++br) {
             cur = blk + cur_buf * 2 * BLK_DOUBLES;
-            double *b0 = cur, *b1 = cur + BLK_DOUBLES;
-            for (int round = 0; round < BW; ++round) {
-                const int q = (warp + round) & (BW - 1);
-                big |= rotate_pair(b0 + warp * BLD, b1 + q * BLD, b0 + BW * BLD + warp, b1 + BW * BLD + q, null_thr, lane);
-                __syncthreads();
+            // block round: team t keeps column t of slot 0 in registers and meets column (t + round) mod 16 of slot 1
+            if (tid < TEAM_THREADS) {
+                double *b0 = cur, *b1 = cur + BLK_DOUBLES, *n0 = b0 + BW * BLD, *n1 = b1 + BW * BLD;
+                double xa[TROWS], xb[TROWS];
+#pragma unroll
+                for (int i = 0; i < TROWS; ++i) xa[i] = b0[team * BLD + tl + 16 * i];
+                double alpha = n0[team];
+                for (int round = 0; round < BW; ++round) {
+                    const int q = (team + round) & (BW - 1);
+#pragma unroll
+                    for (int i = 0; i < TROWS; ++i) xb[i] = b1[q * BLD + tl + 16 * i];
+                    double beta = n1[q];
+                    const int did = rotate_regs(xa, xb, alpha, beta, null_thr);
+                    if (did) {
+#pragma unroll
+                        for (int i = 0; i < TROWS; ++i) b1[q * BLD + tl + 16 * i] = xb[i];
+                        if (tl == 0) n1[q] = beta;
+                    }
+                    big |= did >> 1;
+                    named_bar_sync(1, TEAM_THREADS);
+                }
+#pragma unroll
+                for (int i = 0; i < TROWS; ++i) b0[team * BLD + tl + 16 * i] = xa[i];
+                if (tl == 0) n0[team] = alpha;
             }
             // move the blocks on: position 0 stays, 1 -> 2 -> ... -> 7 -> 1.  Position p lives in CTA min(p, 7 - p),
             // slot 0 if p < 4.  The copies are made by the copy engine: order this thread's stores before them.
