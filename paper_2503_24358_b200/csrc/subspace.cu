@@ -149,7 +149,6 @@ __global__ void gram_reduce_kernel(const double *__restrict__ partial, int chunk
 }
 
 // ------------------------------------------------------------------------------------- eigen
-constexpr int EIG_LD = D + 2;       // padded column stride (doubles) of the full matrix
 constexpr int EIG_MAX_SWEEPS = 40;
 
 // Eigen-decomposition of M: Cholesky M + shift I = L L^T, then one-sided (Hestenes) Jacobi on the columns of L.
@@ -181,7 +180,7 @@ constexpr int BLD = D + 2;                   // column stride inside a block buf
 constexpr int BLK_DOUBLES = BW * BLD + BW;   // 16 columns and their 16 squared norms
 constexpr unsigned BLK_BYTES = BLK_DOUBLES * (unsigned)sizeof(double);
 static_assert(D / BW == 2 * ECL, "two blocks per CTA");
-static_assert(BLK_BYTES % 16 == 0 && (D * EIG_LD * sizeof(double)) % 16 == 0, "bulk copies move 16-byte units");
+static_assert(BLK_BYTES % 16 == 0, "bulk copies move 16-byte units");
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -243,7 +242,8 @@ __device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile
 // orthogonal (tan 2theta = 2 gamma / (beta - alpha), |theta| <= pi/4), from two reciprocal square roots.  A pair
 // already orthogonal to 1e-14 relative, or numerically null twice over, is left alone (returns 0); otherwise
 // returns 1, or 3 when the pair started above the convergence level.
-constexpr int TROWS = D / 16;                // rows per lane of a team
+constexpr int TLN = 16;                      // lanes per team
+constexpr int TROWS = D / TLN;               // rows per lane of a team
 __device__ __forceinline__ int rotate_regs(double (&xp)[TROWS], double (&xq)[TROWS], double &alpha, double &beta, double null_thr)
 {
     double g0 = 0.0, g1 = 0.0;
@@ -251,7 +251,7 @@ __device__ __forceinline__ int rotate_regs(double (&xp)[TROWS], double (&xq)[TRO
     for (int i = 0; i < TROWS; i += 2) { g0 = fma(xp[i], xq[i], g0); g1 = fma(xp[i + 1], xq[i + 1], g1); }
     double gam = g0 + g1;
 #pragma unroll
-    for (int m = 8; m >= 1; m >>= 1) gam += __shfl_xor_sync(0xffffffffu, gam, m);
+    for (int m = TLN / 2; m >= 1; m >>= 1) gam += __shfl_xor_sync(0xffffffffu, gam, m);
     const double g2 = gam * gam, ab = alpha * beta;
     if (!((alpha > null_thr || beta > null_thr) && g2 > 1e-28 * ab)) return 0;      // uniform over the team
     const double diff = beta - alpha;
@@ -280,46 +280,80 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
     extern __shared__ __align__(16) double sm[];
-    double *Gs = sm;                                   // full matrix for the factorisation: Gs[col * EIG_LD + row]
-    double *blk = Gs + D * EIG_LD;                     // [2 buffers][2 slots][BLK_DOUBLES]: the held blocks and the spare
+    double *blk = sm;                                  // [2 buffers][2 slots][BLK_DOUBLES]: the held blocks and the spare
     double *nall = blk + 4 * BLK_DOUBLES;              // [ECL][32] final column norms of the whole cluster
-    double *lcol = nall + ECL * 32;                    // [D] scratch of the factorisation
-    unsigned long long *mbar = reinterpret_cast<unsigned long long *>(lcol + D);      // [2 buffers]
+    double *lcol = nall + ECL * 32;                    // [2][D] column of L being eliminated (double-buffered)
+    double *red = lcol + 2 * D;                        // [16] per-warp partial sums
+    unsigned long long *mbar = reinterpret_cast<unsigned long long *>(red + 16);      // [2 buffers]
     int *flags = reinterpret_cast<int *>(mbar + 2);    // [ECL] "rotated above the convergence level" per CTA
     const int h = blockIdx.x / ECL, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const double *M = gram + (long long)h * D * D;
 
-    for (int idx = tid; idx < D * D; idx += ECT) {
-        const int r = idx / D, c = idx % D;
-        Gs[c * EIG_LD + r] = M[idx];
-    }
+    // Cholesky factorisation M + shift I = L L^T with the matrix in REGISTERS: thread (lane, warp) owns the
+    // elements (row lane + 32 i, column warp + 16 k), i < 4, k < 8; only those on or below the diagonal are used.
+    // Step j: the warp that owns column j gets the pivot by a shuffle, scales its column and publishes it in shared
+    // memory; after ONE barrier (the column buffer alternates) every thread subtracts the rank-1 term from its
+    // elements.  Columns of the two blocks this CTA starts with go straight into the block buffers:
+    // positions crank (slot 0) and 7 - crank (slot 1).
+    double a[4][8];
+    double tr = 0.0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = lane + 32 * i, c = warp + 16 * k;
+            a[i][k] = M[c * D + r];                    // M is symmetric: read along the contiguous direction
+            if (r == c) tr += a[i][k];
+        }
+    tr = warp_sum(tr);
+    if (lane == 0) red[warp] = tr;
     __syncthreads();
     double trace = 0.0;
-    for (int i = 0; i < D; ++i) trace += Gs[i * EIG_LD + i];
+#pragma unroll
+    for (int w = 0; w < 16; ++w) trace += red[w];
     const double shift = trace > 0.0 ? 1e-12 * trace : 1e-300;       // M + shift I = L L^T
-    __syncthreads();
-    if (tid < D) Gs[tid * EIG_LD + tid] += shift;
-    for (int j = 0; j < D; ++j) {
-        __syncthreads();
-        const double ajj = Gs[j * EIG_LD + j];
-        const double ljj = sqrt(ajj > 0.0 ? ajj : shift);
-        if (tid >= j && tid < D) lcol[tid] = (tid == j) ? ljj : Gs[j * EIG_LD + tid] / ljj;
-        __syncthreads();
-        // trailing update of the lower triangle (row >= col); 2-D thread grid, no index division
-        for (int c = j + 1 + (tid >> 5); c < D; c += ECT / 32) {
-            const double lc = lcol[c];
-            for (int r = c + (tid & 31); r < D; r += 32) Gs[c * EIG_LD + r] = fma(-lcol[r], lc, Gs[c * EIG_LD + r]);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (lane + 32 * i == warp + 16 * k) a[i][k] += shift;
+#pragma unroll
+    for (int kj = 0; kj < 8; ++kj) {
+        const int slot = kj == crank ? 0 : (kj == 2 * ECL - 1 - crank ? 1 : -1);
+#pragma unroll 1
+        for (int wj = 0; wj < 16; ++wj) {
+            const int j = 16 * kj + wj;
+            double *lc = lcol + (j & 1) * D;
+            if (warp == wj) {
+                double piv = __shfl_sync(0xffffffffu, a[kj >> 1][kj], j & 31);
+                piv = piv > 0.0 ? piv : shift;
+                const double inv = rsqrt_nr(piv);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = lane + 32 * i;
+                    const double l = r > j ? a[i][kj] * inv : (r == j ? piv * inv : 0.0);
+                    lc[r] = l;
+                    if (slot >= 0) blk[slot * BLK_DOUBLES + wj * BLD + r] = l;
+                }
+            }
+            __syncthreads();
+            double lr[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) lr[i] = lc[lane + 32 * i];
+#pragma unroll
+            for (int k = kj; k < 8; ++k) {
+                const int c = warp + 16 * k;
+                if (c > j) {                           // warp-uniform
+                    const double lcc = lc[c];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (32 * i + 31 >= 16 * k) a[i][k] = fma(-lr[i], lcc, a[i][k]);
+                }
+            }
         }
-        if (tid >= j && tid < D) Gs[j * EIG_LD + tid] = lcol[tid];
     }
     __syncthreads();
-    // this CTA starts with the blocks at positions crank (slot 0) and 7 - crank (slot 1); L is lower triangular
-    for (int idx = tid; idx < 2 * BW * D; idx += ECT) {
-        const int r = idx % D, ci = (idx / D) % BW, slot = idx / (D * BW);
-        const int col = BW * (slot == 0 ? crank : 2 * ECL - 1 - crank) + ci;
-        blk[slot * BLK_DOUBLES + ci * BLD + r] = (r >= col) ? Gs[col * EIG_LD + r] : 0.0;
-    }
     const double null_thr = 4.0 * shift;
     if (tid == 0) {
         mbar_init(smem_u32(&mbar[0]), 1);
@@ -350,8 +384,8 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
         double *cur = blk + cur_buf * 2 * BLK_DOUBLES;
         refresh_norms(cur);
         // Pairs are worked on by 16 teams of 16 lanes (warps 0-7); they keep in step through a barrier of their own.
-        const int team = tid >> 4, tl = tid & 15;
-        constexpr int TEAM_THREADS = 16 * 16;
+        const int team = tid / TLN, tl = tid % TLN;
+        constexpr int TEAM_THREADS = 16 * TLN;
         // intra phase: round-robin of the 16 columns of a block; teams 0-7 on slot 0, teams 8-15 on slot 1
         if (tid < TEAM_THREADS) {
             double *b = cur + (team >> 3) * BLK_DOUBLES, *nb = b + BW * BLD;
@@ -362,12 +396,12 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
                 else { p = (round + t) % (BW - 1); q = (round - t + (BW - 1)) % (BW - 1); }
                 double xp[TROWS], xq[TROWS];
 #pragma unroll
-                for (int i = 0; i < TROWS; ++i) { xp[i] = b[p * BLD + tl + 16 * i]; xq[i] = b[q * BLD + tl + 16 * i]; }
+                for (int i = 0; i < TROWS; ++i) { xp[i] = b[p * BLD + tl + TLN * i]; xq[i] = b[q * BLD + tl + TLN * i]; }
                 double alpha = nb[p], beta = nb[q];
                 const int did = rotate_regs(xp, xq, alpha, beta, null_thr);
                 if (did) {
 #pragma unroll
-                    for (int i = 0; i < TROWS; ++i) { b[p * BLD + tl + 16 * i] = xp[i]; b[q * BLD + tl + 16 * i] = xq[i]; }
+                    for (int i = 0; i < TROWS; ++i) { b[p * BLD + tl + TLN * i] = xp[i]; b[q * BLD + tl + TLN * i] = xq[i]; }
                     if (tl == 0) { nb[p] = alpha; nb[q] = beta; }
                 }
                 big |= did >> 1;
@@ -382,24 +416,24 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
                 double *b0 = cur, *b1 = cur + BLK_DOUBLES, *n0 = b0 + BW * BLD, *n1 = b1 + BW * BLD;
                 double xa[TROWS], xb[TROWS];
 #pragma unroll
-                for (int i = 0; i < TROWS; ++i) xa[i] = b0[team * BLD + tl + 16 * i];
+                for (int i = 0; i < TROWS; ++i) xa[i] = b0[team * BLD + tl + TLN * i];
                 double alpha = n0[team];
                 for (int round = 0; round < BW; ++round) {
                     const int q = (team + round) & (BW - 1);
 #pragma unroll
-                    for (int i = 0; i < TROWS; ++i) xb[i] = b1[q * BLD + tl + 16 * i];
+                    for (int i = 0; i < TROWS; ++i) xb[i] = b1[q * BLD + tl + TLN * i];
                     double beta = n1[q];
                     const int did = rotate_regs(xa, xb, alpha, beta, null_thr);
                     if (did) {
 #pragma unroll
-                        for (int i = 0; i < TROWS; ++i) b1[q * BLD + tl + 16 * i] = xb[i];
+                        for (int i = 0; i < TROWS; ++i) b1[q * BLD + tl + TLN * i] = xb[i];
                         if (tl == 0) n1[q] = beta;
                     }
                     big |= did >> 1;
                     named_bar_sync(1, TEAM_THREADS);
                 }
 #pragma unroll
-                for (int i = 0; i < TROWS; ++i) b0[team * BLD + tl + 16 * i] = xa[i];
+                for (int i = 0; i < TROWS; ++i) b0[team * BLD + tl + TLN * i] = xa[i];
                 if (tl == 0) n0[team] = alpha;
             }
             // move the blocks on: position 0 stays, 1 -> 2 -> ... -> 7 -> 1.  Position p lives in CTA min(p, 7 - p),
@@ -608,7 +642,7 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
 
 int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * EIG_LD + 4 * BLK_DOUBLES + ECL * 32 + D + 2) + sizeof(int) * ECL;
+    const size_t smem = sizeof(double) * (4 * BLK_DOUBLES + ECL * 32 + 2 * D + 16 + 2) + sizeof(int) * ECL;
     SQUAT_CUDA(cudaFuncSetAttribute(eig_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     eig_cluster_kernel<<<s->n_kv_heads * ECL, ECT, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
     squat_count_launch();
