@@ -20,6 +20,8 @@
 // downstream; products of bf16 inputs are exact in fp64 and everything stays fp64 until W is
 // rounded to float32 at the very end.
 #include <cooperative_groups.h>
+#include <type_traits>
+#include <utility>
 #include "squat_internal.cuh"
 
 namespace {
@@ -27,58 +29,101 @@ namespace {
 constexpr int D = SQUAT_D;
 
 // ------------------------------------------------------------------------------------- Gram
-constexpr int GRAM_THREADS = 160;   // 136 upper-triangular 8x8 tiles of the 16x16 tile grid, 5 warps
-constexpr int GRAM_ROWS = 32;       // rows staged in shared memory per step
+// M = Qc^T Qc on the fp64 tensor-core path (mma.sync m8n8k4, fp64 operands and accumulators: products of bf16 or
+// fp32 inputs are exact in fp64).  M is symmetric: of the 16 x 16 grid of 8 x 8 tiles only the 136 tiles on or above
+// the diagonal are computed, 17 per warp, 8 warps per CTA.  The A fragment of tile row i (A[m][k] = Q[token k][8 i + m])
+// and the B fragment of tile column i (B[k][n] = Q[token k][8 i + n]) are the same register, so a warp loads one
+// fragment per 8-channel group and 4-token step and feeds it to every tile that touches the group.
+constexpr int GRAM_THREADS = 256;
+constexpr int GRAM_ROWS = 32;                  // token rows staged in shared memory per step
+constexpr int GRAM_LDR = D + 4;                // row stride (doubles): 4 tokens x 8 channels of a fragment hit 32 distinct words
+constexpr int GRAM_TILES_PER_WARP = 17;
+constexpr int GRAM_CTAS_PER_SM = 2;
+
+// u-th tile of the upper triangle, row by row: (ti, tj), ti <= tj
+template <int U>
+struct GramTile {
+    static constexpr int row()
+    {
+        int u = U, ti = 0, len = 16;
+        while (u >= len) { u -= len; --len; ++ti; }
+        return ti;
+    }
+    static constexpr int ti = row();
+    static constexpr int tj = ti + (U - (ti * 16 - ti * (ti - 1) / 2));
+};
+
+__device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+
+template <int W, int... N>
+__device__ __forceinline__ void gram_warp_step(double (&acc)[GRAM_TILES_PER_WARP][2], const double (&F)[16],
+                                               std::integer_sequence<int, N...>)
+{
+    (dmma_m8n8k4(acc[N][0], acc[N][1], F[GramTile<GRAM_TILES_PER_WARP * W + N>::ti], F[GramTile<GRAM_TILES_PER_WARP * W + N>::tj]), ...);
+}
+
+template <int W, int... N>
+__device__ __forceinline__ void gram_warp_store(const double (&acc)[GRAM_TILES_PER_WARP][2], double *out, int lane,
+                                                std::integer_sequence<int, N...>)
+{
+    // C fragment: thread holds row lane / 4, columns 2 (lane % 4) and 2 (lane % 4) + 1 of the tile
+    ((*reinterpret_cast<double2 *>(out + (GramTile<GRAM_TILES_PER_WARP * W + N>::ti * 8 + (lane >> 2)) * D +
+                                   GramTile<GRAM_TILES_PER_WARP * W + N>::tj * 8 + 2 * (lane & 3)) = make_double2(acc[N][0], acc[N][1])), ...);
+}
+
+template <bool BF16, int W>
+__device__ __forceinline__ void gram_warp_body(const double *rows, double (&acc)[GRAM_TILES_PER_WARP][2], int lane)
+{
+    const double *base = rows + (lane & 3) * GRAM_LDR + (lane >> 2);
+#pragma unroll 2
+    for (int k0 = 0; k0 < GRAM_ROWS; k0 += 4) {
+        double F[16];
+#pragma unroll
+        for (int g = 0; g < 16; ++g) F[g] = base[k0 * GRAM_LDR + g * 8];
+        gram_warp_step<W>(acc, F, std::make_integer_sequence<int, GRAM_TILES_PER_WARP>{});
+    }
+}
 
 template <bool BF16>
-__global__ void __launch_bounds__(GRAM_THREADS) gram_kernel(
+__global__ void __launch_bounds__(GRAM_THREADS, GRAM_CTAS_PER_SM) gram_kernel(
     const void *__restrict__ q, int n_tokens, int q_per_kv, long long stride_h, long long stride_t,
     int rows_per_chunk, double *__restrict__ partial /* [chunks, H, D, D] */)
 {
-    __shared__ __align__(16) double rows[GRAM_ROWS][D];
+    __shared__ __align__(16) double rows[GRAM_ROWS * GRAM_LDR];
     const int h = blockIdx.y, chunk = blockIdx.x, H = gridDim.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long N = (long long)n_tokens * q_per_kv;
     const long long row_lo = (long long)chunk * rows_per_chunk;
     long long row_hi = row_lo + rows_per_chunk;
     if (row_hi > N) row_hi = N;
 
-    // tile of this thread: (ti <= tj) in the 16 x 16 grid of 8 x 8 tiles
-    int ti = 0, tj = 0;
-    {
-        int t = threadIdx.x, rowlen = 16;
-        while (t >= rowlen && ti < 15) { t -= rowlen; --rowlen; ++ti; }
-        tj = ti + t;
-    }
-    const bool active = threadIdx.x < 136;
-    double acc[8][8];
+    double acc[GRAM_TILES_PER_WARP][2];
 #pragma unroll
-    for (int a = 0; a < 8; ++a)
-#pragma unroll
-        for (int b = 0; b < 8; ++b) acc[a][b] = 0.0;
+    for (int n = 0; n < GRAM_TILES_PER_WARP; ++n) acc[n][0] = acc[n][1] = 0.0;
 
-    // Each thread stages up to 4 pieces of 8 elements per step (32 rows x 16 pieces over 160 threads).  The
-    // global loads of step s+1 are issued before the arithmetic of step s, so their latency is hidden.
-    constexpr int NPIECE = (GRAM_ROWS * (D / 8) + GRAM_THREADS - 1) / GRAM_THREADS;
-    uint4 pre[NPIECE][BF16 ? 1 : 2];
+    // Staging: a thread moves pairs of neighbouring channels (4 bytes of bf16, 8 of fp32), so that a warp's
+    // 16-byte stores of the converted pairs fall on consecutive words.  The global loads of step s + 1 are
+    // issued before the arithmetic of step s, so their latency is hidden.
+    constexpr int NPAIR = GRAM_ROWS * (D / 2) / GRAM_THREADS;          // 16
+    using raw_t = typename std::conditional<BF16, uint32_t, uint2>::type;
+    raw_t pre[NPAIR];
     auto fetch = [&](long long r0) {
 #pragma unroll
-        for (int it = 0; it < NPIECE; ++it) {
+        for (int it = 0; it < NPAIR; ++it) {
             const int idx = threadIdx.x + it * GRAM_THREADS;
-            const int rr = idx / (D / 8), c8 = idx % (D / 8);
+            const int rr = idx / (D / 2), c2 = idx % (D / 2);
             const long long n = r0 + rr;
-            if (idx < GRAM_ROWS * (D / 8) && n < row_hi) {
+            pre[it] = raw_t{};
+            if (n < row_hi) {
                 const long long hq = (long long)h * q_per_kv + n / n_tokens;
                 const long long t = n % n_tokens;
-                const long long off = hq * stride_h + t * stride_t + c8 * 8;
-                if (BF16) {
-                    pre[it][0] = ldg128(reinterpret_cast<const __nv_bfloat16 *>(q) + off);
-                } else {
-                    pre[it][0] = ldg128(reinterpret_cast<const float *>(q) + off);
-                    pre[it][BF16 ? 0 : 1] = ldg128(reinterpret_cast<const float *>(q) + off + 4);
-                }
-            } else {
-                pre[it][0] = make_uint4(0, 0, 0, 0);
-                pre[it][BF16 ? 0 : 1] = make_uint4(0, 0, 0, 0);
+                const long long off = hq * stride_h + t * stride_t + c2 * 2;
+                if constexpr (BF16) pre[it] = __ldg(reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(q) + off));
+                else pre[it] = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const float *>(q) + off));
             }
         }
     };
@@ -86,52 +131,38 @@ __global__ void __launch_bounds__(GRAM_THREADS) gram_kernel(
     for (long long r0 = row_lo; r0 < row_hi; r0 += GRAM_ROWS) {
         __syncthreads();
 #pragma unroll
-        for (int it = 0; it < NPIECE; ++it) {
+        for (int it = 0; it < NPAIR; ++it) {
             const int idx = threadIdx.x + it * GRAM_THREADS;
-            if (idx >= GRAM_ROWS * (D / 8)) continue;
-            const int rr = idx / (D / 8), c8 = idx % (D / 8);
-            double v[8];
-            if (BF16) {
-                const uint32_t w[4] = {pre[it][0].x, pre[it][0].y, pre[it][0].z, pre[it][0].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    v[2 * k] = (double)bf16lo_to_f32(w[k]);
-                    v[2 * k + 1] = (double)bf16hi_to_f32(w[k]);
-                }
-            } else {
-                const uint4 a = pre[it][0], b = pre[it][BF16 ? 0 : 1];
-                v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y); v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
-                v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y); v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) rows[rr][c8 * 8 + k] = v[k];
+            const int rr = idx / (D / 2), c2 = idx % (D / 2);
+            double2 v;
+            if constexpr (BF16) { v.x = (double)bf16lo_to_f32(pre[it]); v.y = (double)bf16hi_to_f32(pre[it]); }
+            else { v.x = (double)__uint_as_float(pre[it].x); v.y = (double)__uint_as_float(pre[it].y); }
+            *reinterpret_cast<double2 *>(&rows[rr * GRAM_LDR + c2 * 2]) = v;
         }
         __syncthreads();
         if (r0 + GRAM_ROWS < row_hi) fetch(r0 + GRAM_ROWS);
-        if (active) {
-#pragma unroll 4
-            for (int rr = 0; rr < GRAM_ROWS; ++rr) {
-                double a[8], b[8];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const double2 va = *reinterpret_cast<const double2 *>(&rows[rr][ti * 8 + 2 * k]);
-                    const double2 vb = *reinterpret_cast<const double2 *>(&rows[rr][tj * 8 + 2 * k]);
-                    a[2 * k] = va.x; a[2 * k + 1] = va.y;
-                    b[2 * k] = vb.x; b[2 * k + 1] = vb.y;
-                }
-#pragma unroll
-                for (int x = 0; x < 8; ++x)
-#pragma unroll
-                    for (int y = 0; y < 8; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
-            }
+        switch (warp) {
+        case 0: gram_warp_body<BF16, 0>(rows, acc, lane); break;
+        case 1: gram_warp_body<BF16, 1>(rows, acc, lane); break;
+        case 2: gram_warp_body<BF16, 2>(rows, acc, lane); break;
+        case 3: gram_warp_body<BF16, 3>(rows, acc, lane); break;
+        case 4: gram_warp_body<BF16, 4>(rows, acc, lane); break;
+        case 5: gram_warp_body<BF16, 5>(rows, acc, lane); break;
+        case 6: gram_warp_body<BF16, 6>(rows, acc, lane); break;
+        default: gram_warp_body<BF16, 7>(rows, acc, lane); break;
         }
     }
-    if (active) {
-        double *out = partial + ((long long)chunk * H + h) * D * D;
-#pragma unroll
-        for (int x = 0; x < 8; ++x)
-#pragma unroll
-            for (int y = 0; y < 8; ++y) out[(ti * 8 + x) * D + tj * 8 + y] = acc[x][y];
+    double *out = partial + ((long long)chunk * H + h) * D * D;
+    constexpr auto seq = std::make_integer_sequence<int, GRAM_TILES_PER_WARP>{};
+    switch (warp) {
+    case 0: gram_warp_store<0>(acc, out, lane, seq); break;
+    case 1: gram_warp_store<1>(acc, out, lane, seq); break;
+    case 2: gram_warp_store<2>(acc, out, lane, seq); break;
+    case 3: gram_warp_store<3>(acc, out, lane, seq); break;
+    case 4: gram_warp_store<4>(acc, out, lane, seq); break;
+    case 5: gram_warp_store<5>(acc, out, lane, seq); break;
+    case 6: gram_warp_store<6>(acc, out, lane, seq); break;
+    default: gram_warp_store<7>(acc, out, lane, seq); break;
     }
 }
 
@@ -179,6 +210,7 @@ constexpr int BW = 16;                       // columns per block
 constexpr int BLD = D + 2;                   // column stride inside a block buffer (doubles)
 constexpr int BLK_DOUBLES = BW * BLD + BW;   // 16 columns and their 16 squared norms
 constexpr unsigned BLK_BYTES = BLK_DOUBLES * (unsigned)sizeof(double);
+static_assert(GRAM_TILES_PER_WARP * (GRAM_THREADS / 32) == 136, "the warps share the upper triangle evenly");
 static_assert(D / BW == 2 * ECL, "two blocks per CTA");
 static_assert(BLK_BYTES % 16 == 0, "bulk copies move 16-byte units");
 
