@@ -552,9 +552,8 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
 {
     extern __shared__ __align__(16) double sm[];
     double *A = sm;                         // A[row * ASM_LD + col]
-    double *colv = sm + D * ASM_LD;         // column j before scaling
-    double *lcol = colv + D;                // column j of L
-    double *coef = lcol + D;                // s_i / (1 + s_i)
+    double *colv = sm + D * ASM_LD;         // [2 parities][l, v][D]: column j of L and of the matrix, as published
+    double *coef = colv + 4 * D;            // s_i / (1 + s_i)
     const int h = blockIdx.x, tid = threadIdx.x;
     const double *V = eigvec + (long long)h * D * D;
 
@@ -565,62 +564,97 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
         coef[tid] = (tid < rank_r) ? s / (1.0 + s) : 0.0;
     }
     __syncthreads();
-    // P_inv = I - sum_{i<r} coef_i v_i v_i^T, register-tiled: thread (ta, tb) owns rows 4 ta .. 4 ta + 3 and columns
-    // 8 tb .. 8 tb + 7; the eigenvectors are staged 32 at a time in shared memory behind A
+    // The matrix lives in REGISTERS from here to the end of the factorisation: thread (lane, warp) owns the elements
+    // (row lane + 32 i, column warp + 16 k), i < 4, k < 8; only those on or below the diagonal are used.
+    const int warp = tid >> 5, lane = tid & 31;
+    double a[4][8];
+    // P_inv = I - sum_{i<r} coef_i v_i v_i^T; the eigenvectors are staged 32 at a time in shared memory
     {
         double *U = coef + D;                           // [32][D] staged eigenvectors
-        const int ta = tid >> 4, tb = tid & 15;         // 32 x 16 tiles
-        double acc[4][8];
 #pragma unroll
-        for (int x = 0; x < 4; ++x)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int y = 0; y < 8; ++y) acc[x][y] = (4 * ta + x == 8 * tb + y) ? 1.0 : 0.0;
+            for (int k = 0; k < 8; ++k) a[i][k] = (lane + 32 * i == warp + 16 * k) ? 1.0 : 0.0;
         for (int i0 = 0; i0 < rank_r; i0 += 32) {
             const int ni = rank_r - i0 < 32 ? rank_r - i0 : 32;
             __syncthreads();
             for (int idx = tid; idx < ni * D; idx += ASM_THREADS) U[idx] = V[(long long)i0 * D + idx];
             __syncthreads();
-            for (int i = 0; i < ni; ++i) {
-                const double cf = -coef[i0 + i];
-                double a[4], b[8];
+            for (int e = 0; e < ni; ++e) {
+                const double cf = -coef[i0 + e];
+                double vr[4], vc[8];
 #pragma unroll
-                for (int x = 0; x < 4; x += 2) {
-                    const double2 v = *reinterpret_cast<const double2 *>(U + i * D + 4 * ta + x);
-                    a[x] = cf * v.x; a[x + 1] = cf * v.y;
-                }
+                for (int i = 0; i < 4; ++i) vr[i] = cf * U[e * D + lane + 32 * i];
 #pragma unroll
-                for (int y = 0; y < 8; y += 2) {
-                    const double2 v = *reinterpret_cast<const double2 *>(U + i * D + 8 * tb + y);
-                    b[y] = v.x; b[y + 1] = v.y;
-                }
+                for (int k = 0; k < 8; ++k) vc[k] = U[e * D + warp + 16 * k];
 #pragma unroll
-                for (int x = 0; x < 4; ++x)
+                for (int k = 0; k < 8; ++k)
 #pragma unroll
-                    for (int y = 0; y < 8; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
+                    for (int i = 0; i < 4; ++i)
+                        if (32 * i + 31 >= 16 * k) a[i][k] = fma(vr[i], vc[k], a[i][k]);
             }
         }
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-#pragma unroll
-            for (int y = 0; y < 8; ++y) A[(4 * ta + x) * ASM_LD + 8 * tb + y] = acc[x][y];
     }
     __syncthreads();
-    // in-place LDL^T (right-looking): afterwards the strict lower triangle of A holds L
-    for (int j = 0; j < D - 1; ++j) {
-        if (tid > j && tid < D) {
-            const double v = A[tid * ASM_LD + j];
-            colv[tid] = v;
-            lcol[tid] = v / A[j * ASM_LD + j];
+    // LDL^T (right-looking), afterwards the strict lower triangle holds L.  Step j: the warp that owns column j gets
+    // the pivot d_j by a shuffle and publishes v = column j and l = v / d_j in shared memory; after ONE barrier (the
+    // buffers alternate) every thread subtracts l_r v_c from its elements.
+    {
+        double *pub = colv;                             // [2 parities][l, v][D], overlays colv, lcol and more
+#pragma unroll
+        for (int kj = 0; kj < 8; ++kj) {
+#pragma unroll 1
+            for (int wj = 0; wj < 16; ++wj) {
+                const int j = 16 * kj + wj;
+                double *lp = pub + (j & 1) * 2 * D, *vp = lp + D;
+                if (warp == wj) {
+                    const double d = __shfl_sync(0xffffffffu, a[kj >> 1][kj], j & 31);
+                    const double inv = 1.0 / d;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = lane + 32 * i;
+                        const double v = a[i][kj], l = v * inv;
+                        if (r > j) { lp[r] = l; vp[r] = v; a[i][kj] = l; }
+                    }
+                }
+                __syncthreads();
+                double lr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) lr[i] = lp[lane + 32 * i];     // rows <= j hold stale values: only feed unused elements
+#pragma unroll
+                for (int k = kj; k < 8; ++k) {
+                    const int c = warp + 16 * k;
+                    if (c > j) {                        // warp-uniform
+                        const double vc = vp[c];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (32 * i + 31 >= 16 * k) a[i][k] = fma(-lr[i], vc, a[i][k]);
+                    }
+                }
+            }
         }
-        __syncthreads();
-        // trailing update (full square, both triangles kept); 2-D thread grid, no index division
-        for (int i = j + 1 + (tid >> 5); i < D; i += ASM_THREADS / 32) {
-            const double li = lcol[i];
-            for (int k = j + 1 + (tid & 31); k < D; k += 32) A[i * ASM_LD + k] = fma(-li, colv[k], A[i * ASM_LD + k]);
-        }
-        if (tid > j && tid < D) A[tid * ASM_LD + j] = lcol[tid];
-        __syncthreads();
     }
+    float *out = Wt + (long long)h * D * D;
+    if (g == 1) {
+        // Wt[j][j'] = W[j'][j] = L[j'][j] below the diagonal, zero on and above it: straight from the registers
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = lane + 32 * i, c = warp + 16 * k;
+                out[c * D + r] = (r > c) ? (float)a[i][k] : 0.0f;
+            }
+        return;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = lane + 32 * i, c = warp + 16 * k;
+            if (r > c) A[r * ASM_LD + c] = a[i][k];
+        }
+    __syncthreads();
     // g > 1: block column t becomes L[rest, blk] * inverse(unit-lower diagonal block)
     if (g > 1) {
         const int T = D / g;
@@ -638,7 +672,6 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
         __syncthreads();
     }
     // Wt[j][j'] = W[j'][j]: zero on and above the block diagonal
-    float *out = Wt + (long long)h * D * D;
     for (int idx = tid; idx < D * D; idx += ASM_THREADS) {
         const int j = idx / D, jp = idx % D;
         const int blk_end = (j / g + 1) * g;
@@ -684,7 +717,7 @@ int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 
 int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * ASM_LD + 3 * D + 32 * D);
+    const size_t smem = sizeof(double) * (D * ASM_LD + 5 * D + 32 * D);
     SQUAT_CUDA(cudaFuncSetAttribute(assemble_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt);
     squat_count_launch();
