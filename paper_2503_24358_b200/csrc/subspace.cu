@@ -231,41 +231,6 @@ __device__ __forceinline__ double rsqrt_nr(double x)
     return fma(y * r, fma(0.375, r, 0.5), y);
 }
 
-// Shared-memory addresses, transaction barriers and the bulk copy between the CTAs of a cluster.
-__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned peer_u32(unsigned addr, int cta)
-{
-    unsigned r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
-    return r;
-}
-__device__ __forceinline__ void mbar_init(unsigned bar, int count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Waits for the phase of the given parity; gives up after a bounded number of polls (returns false).
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity)
-{
-    for (int it = 0; it < (1 << 18); ++it) {
-        unsigned done;
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-// bytes from this CTA's shared memory to a peer's, completing `bytes` of the PEER's barrier when they have landed
-__device__ __forceinline__ void bulk_copy_to_peer(unsigned dst_peer, unsigned src, unsigned bytes, unsigned bar_peer)
-{
-    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst_peer), "r"(src), "r"(bytes), "r"(bar_peer) : "memory");
-}
-
 __device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
 // One Jacobi rotation of a column pair (P, Q) held in registers by a team of 16 lanes (both halves of a warp work
@@ -275,7 +240,21 @@ __device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile
 // already orthogonal to 1e-14 relative, or numerically null twice over, is left alone (returns 0); otherwise
 // returns 1, or 3 when the pair started above the convergence level.
 constexpr int TLN = 16;                      // lanes per team
-constexpr int TROWS = D / TLN;               // rows per lane of a team
+constexpr int TROWS = D / TLN;               // rows per lane of a team: 2 tl + 32 i and 2 tl + 1 + 32 i, i < TROWS / 2
+__device__ __forceinline__ void load_col(double (&x)[TROWS], const double *col, int tl)
+{
+#pragma unroll
+    for (int i = 0; i < TROWS / 2; ++i) {
+        const double2 v = *reinterpret_cast<const double2 *>(col + 2 * tl + 2 * TLN * i);
+        x[2 * i] = v.x;
+        x[2 * i + 1] = v.y;
+    }
+}
+__device__ __forceinline__ void store_col(double *col, const double (&x)[TROWS], int tl)
+{
+#pragma unroll
+    for (int i = 0; i < TROWS / 2; ++i) *reinterpret_cast<double2 *>(col + 2 * tl + 2 * TLN * i) = make_double2(x[2 * i], x[2 * i + 1]);
+}
 __device__ __forceinline__ int rotate_regs(double (&xp)[TROWS], double (&xq)[TROWS], double &alpha, double &beta, double null_thr)
 {
     double g0 = 0.0, g1 = 0.0;
@@ -316,8 +295,7 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
     double *nall = blk + 4 * BLK_DOUBLES;              // [ECL][32] final column norms of the whole cluster
     double *lcol = nall + ECL * 32;                    // [2][D] column of L being eliminated (double-buffered)
     double *red = lcol + 2 * D;                        // [16] per-warp partial sums
-    unsigned long long *mbar = reinterpret_cast<unsigned long long *>(red + 16);      // [2 buffers]
-    int *flags = reinterpret_cast<int *>(mbar + 2);    // [ECL] "rotated above the convergence level" per CTA
+    int *flags = reinterpret_cast<int *>(red + 16);    // [ECL] "rotated above the convergence level" per CTA
     const int h = blockIdx.x / ECL, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const double *M = gram + (long long)h * D * D;
@@ -387,12 +365,7 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
     }
     __syncthreads();
     const double null_thr = 4.0 * shift;
-    if (tid == 0) {
-        mbar_init(smem_u32(&mbar[0]), 1);
-        mbar_init(smem_u32(&mbar[1]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    cluster.sync();                                    // every CTA's barriers exist before anybody copies
+    cluster.sync();                                    // every CTA of the cluster is running before anybody writes into it
 
     // squared norms of the 32 held columns, from the data: warp w takes columns w and w + 16
     auto refresh_norms = [&](double *cur) {
@@ -408,10 +381,10 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
         __syncthreads();
     };
 
-    int cur_buf = 0, moves = 0;                         // which buffer holds the blocks; block moves so far
-    bool converged = false, failed = false;
+    int cur_buf = 0;                                   // which buffer holds the blocks
+    bool converged = false;
     int sweep = 0;
-    for (; sweep < EIG_MAX_SWEEPS && !converged && !failed; ++sweep) {
+    for (; sweep < EIG_MAX_SWEEPS && !converged; ++sweep) {
         int big = 0;
         double *cur = blk + cur_buf * 2 * BLK_DOUBLES;
         refresh_norms(cur);
@@ -427,13 +400,13 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
                 if (t == 0) { p = BW - 1; q = round; }
                 else { p = (round + t) % (BW - 1); q = (round - t + (BW - 1)) % (BW - 1); }
                 double xp[TROWS], xq[TROWS];
-#pragma unroll
-                for (int i = 0; i < TROWS; ++i) { xp[i] = b[p * BLD + tl + TLN * i]; xq[i] = b[q * BLD + tl + TLN * i]; }
+                load_col(xp, b + p * BLD, tl);
+                load_col(xq, b + q * BLD, tl);
                 double alpha = nb[p], beta = nb[q];
                 const int did = rotate_regs(xp, xq, alpha, beta, null_thr);
                 if (did) {
-#pragma unroll
-                    for (int i = 0; i < TROWS; ++i) { b[p * BLD + tl + TLN * i] = xp[i]; b[q * BLD + tl + TLN * i] = xq[i]; }
+                    store_col(b + p * BLD, xp, tl);
+                    store_col(b + q * BLD, xq, tl);
                     if (tl == 0) { nb[p] = alpha; nb[q] = beta; }
                 }
                 big |= did >> 1;
@@ -447,66 +420,52 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
             if (tid < TEAM_THREADS) {
                 double *b0 = cur, *b1 = cur + BLK_DOUBLES, *n0 = b0 + BW * BLD, *n1 = b1 + BW * BLD;
                 double xa[TROWS], xb[TROWS];
-#pragma unroll
-                for (int i = 0; i < TROWS; ++i) xa[i] = b0[team * BLD + tl + TLN * i];
-                double alpha = n0[team];
+                load_col(xa, b0 + team * BLD, tl);
+                double alpha = n0[team], beta = 0.0;
                 for (int round = 0; round < BW; ++round) {
                     const int q = (team + round) & (BW - 1);
-#pragma unroll
-                    for (int i = 0; i < TROWS; ++i) xb[i] = b1[q * BLD + tl + TLN * i];
-                    double beta = n1[q];
+                    load_col(xb, b1 + q * BLD, tl);
+                    beta = n1[q];
                     const int did = rotate_regs(xa, xb, alpha, beta, null_thr);
-                    if (did) {
-#pragma unroll
-                        for (int i = 0; i < TROWS; ++i) b1[q * BLD + tl + TLN * i] = xb[i];
+                    if (did && round < BW - 1) {
+                        store_col(b1 + q * BLD, xb, tl);
                         if (tl == 0) n1[q] = beta;
                     }
                     big |= did >> 1;
                     named_bar_sync(1, TEAM_THREADS);
                 }
-#pragma unroll
-                for (int i = 0; i < TROWS; ++i) b0[team * BLD + tl + TLN * i] = xa[i];
-                if (tl == 0) n0[team] = alpha;
-            }
-            // move the blocks on: position 0 stays, 1 -> 2 -> ... -> 7 -> 1.  Position p lives in CTA min(p, 7 - p),
-            // slot 0 if p < 4.  The copies are made by the copy engine: order this thread's stores before them.
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            cluster.sync();                            // everybody is done with this block round: all spares are free
-            const int nxt = cur_buf ^ 1;
-            const unsigned bar = smem_u32(&mbar[nxt]);
-            if (tid == 0 && !failed) {
-                mbar_expect_tx(bar, 2 * BLK_BYTES);
-#pragma unroll
-                for (int slot = 0; slot < 2; ++slot) {
+                // Move the blocks on: position 0 stays, 1 -> 2 -> ... -> 7 -> 1; position p lives in CTA min(p, 7 - p),
+                // slot 0 if p < 4.  After the last round every column sits in some team's registers (column `team` of
+                // slot 0 and column team + 15 mod 16 of slot 1), so the teams write them straight into the spare
+                // buffer of the next holder.  That buffer is free: its owner left it when it began this block round.
+                auto next_home = [&](int slot) {
                     const int pos = slot == 0 ? crank : 2 * ECL - 1 - crank;
                     const int npos = pos == 0 ? 0 : (pos == 2 * ECL - 1 ? 1 : pos + 1);
                     const int dcta = npos < ECL ? npos : 2 * ECL - 1 - npos, dslot = npos < ECL ? 0 : 1;
-                    const unsigned src = smem_u32(blk + (cur_buf * 2 + slot) * BLK_DOUBLES);
-                    const unsigned dst = smem_u32(blk + (nxt * 2 + dslot) * BLK_DOUBLES);
-                    bulk_copy_to_peer(peer_u32(dst, dcta), src, BLK_BYTES, peer_u32(bar, dcta));
-                }
+                    return cluster.map_shared_rank(blk + ((cur_buf ^ 1) * 2 + dslot) * BLK_DOUBLES, dcta);
+                };
+                double *d0 = next_home(0), *d1 = next_home(1);
+                const int ql = (team + BW - 1) & (BW - 1);
+                store_col(d0 + team * BLD, xa, tl);
+                store_col(d1 + ql * BLD, xb, tl);
+                if (tl == 0) { d0[BW * BLD + team] = alpha; d1[BW * BLD + ql] = beta; }
             }
-            // after a wait has run out nothing is waited for any more, but every CTA keeps making the same
-            // sequence of barrier calls until the end of the sweep, where the failure is made known to all
-            const bool arrived = failed || mbar_wait(bar, (unsigned)(moves >> 1) & 1u);
-            failed = __syncthreads_or(!arrived) != 0 || failed;
-            cur_buf = nxt;
-            ++moves;
+            if (br == 2 * ECL - 2) {
+                // the sweep is the last one if no CTA of the cluster rotated a pair from above the convergence level
+                big = __syncthreads_or(big);
+                if (tid < ECL) *cluster.map_shared_rank(&flags[crank], tid) = big ? 1 : 0;
+            }
+            cluster.sync();                            // blocks (and flags) have arrived; nobody is behind by a block round
+            cur_buf ^= 1;
         }
-        // the sweep is the last one if no CTA of the cluster rotated a pair from above the convergence level
-        big = __syncthreads_or(big);
-        if (tid < ECL) *cluster.map_shared_rank(&flags[crank], tid) = (big ? 1 : 0) | (failed ? 2 : 0);
-        cluster.sync();
         int any = 0;
 #pragma unroll
-        for (int r = 0; r < ECL; ++r) any |= flags[r];
-        converged = (any & 1) == 0;
-        failed = (any & 2) != 0;
-        cluster.sync();                                // flags are read before the next sweep may overwrite them
+        for (int r = 0; r < ECL; ++r) any |= flags[r];  // rewritten only after seven more cluster barriers
+        converged = any == 0;
     }
     if (tid == 0 && crank == 0) {
         sweeps_out[h] = sweep;
-        if (!converged || failed) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
+        if (!converged) atomicOr(status, SQUAT_FLAG_NO_CONVERGE);
     }
 
     // singular values of L = sqrt(mu + shift) are the column norms; rank them over the whole cluster
@@ -707,7 +666,7 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
 
 int squat_launch_eig(squat_subspace *s, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (4 * BLK_DOUBLES + ECL * 32 + 2 * D + 16 + 2) + sizeof(int) * ECL;
+    const size_t smem = sizeof(double) * (4 * BLK_DOUBLES + ECL * 32 + 2 * D + 16) + sizeof(int) * ECL;
     SQUAT_CUDA(cudaFuncSetAttribute(eig_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     eig_cluster_kernel<<<s->n_kv_heads * ECL, ECT, smem, st>>>(s->gram, s->eigval, s->eigvec, s->eig_sweeps, s->status);
     squat_count_launch();
