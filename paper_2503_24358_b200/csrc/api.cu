@@ -128,6 +128,10 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
 int squat_subspace_destroy(squat_subspace *s)
 {
     if (!s) return SQUAT_OK;
+    if (s->side_ready) {
+        for (int i = 0; i < 2; ++i) cudaStreamDestroy(s->side[i]);
+        for (int i = 0; i < 5; ++i) cudaEventDestroy(s->ev[i]);
+    }
     cudaError_t e = cudaFree(s->Wt);     // Wt is the base of the single allocation
     delete s;
     return e == cudaSuccess ? SQUAT_OK : squat_cuda_fail(e);
@@ -338,27 +342,46 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
     const size_t es = elem_size(dtype);
     const size_t toks = (size_t)batch * n_kv_heads * n_tokens;
     const long long T = n_tokens, d = head_dim;
+    // Copies and kernels overlap: q goes up first (the subspace build needs it), k and v follow on a side stream
+    // while the build runs; the key outputs go down on a second side stream while v is still coming up and the
+    // values are quantized.  Everything is ordered after the work already in `stream` and joined back into it.
+    if (!s->side_ready) {
+        for (int i = 0; i < 2; ++i) SQUAT_CUDA(cudaStreamCreateWithFlags(&s->side[i], cudaStreamNonBlocking));
+        for (int i = 0; i < 5; ++i) SQUAT_CUDA(cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming));
+        s->side_ready = true;
+    }
+    cudaEvent_t ev_q = s->ev[0], ev_k = s->ev[1], ev_v = s->ev[2], ev_keys = s->ev[3], ev_kout = s->ev[4];
     SQUAT_CUDA(cudaMemcpyAsync(w + L.q, q_host, (size_t)n_q_heads * T * d * es, cudaMemcpyHostToDevice, st));
-    SQUAT_CUDA(cudaMemcpyAsync(w + L.k, k_host, toks * d * es, cudaMemcpyHostToDevice, st));
-    SQUAT_CUDA(cudaMemcpyAsync(w + L.v, v_host, toks * d * es, cudaMemcpyHostToDevice, st));
+    SQUAT_CUDA(cudaEventRecord(ev_q, st));
+    SQUAT_CUDA(cudaStreamWaitEvent(s->side[0], ev_q, 0));
+    SQUAT_CUDA(cudaMemcpyAsync(w + L.k, k_host, toks * d * es, cudaMemcpyHostToDevice, s->side[0]));
+    SQUAT_CUDA(cudaEventRecord(ev_k, s->side[0]));
+    SQUAT_CUDA(cudaMemcpyAsync(w + L.v, v_host, toks * d * es, cudaMemcpyHostToDevice, s->side[0]));
+    SQUAT_CUDA(cudaEventRecord(ev_v, s->side[0]));
     int rc = squat_build_subspace(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g, stream);
     if (rc != SQUAT_OK) return rc;
+    SQUAT_CUDA(cudaStreamWaitEvent(st, ev_k, 0));
     rc = squat_quantize_keys(s, w + L.k, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
                              T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.kc),
                              reinterpret_cast<float *>(w + L.ks), reinterpret_cast<float *>(w + L.kz),
                              (long long)n_kv_heads * T, T, stream);
     if (rc != SQUAT_OK) return rc;
+    SQUAT_CUDA(cudaEventRecord(ev_keys, st));
+    SQUAT_CUDA(cudaStreamWaitEvent(s->side[1], ev_keys, 0));
+    SQUAT_CUDA(cudaMemcpyAsync(k_codes_host, w + L.kc, toks * d * bits / 8, cudaMemcpyDeviceToHost, s->side[1]));
+    SQUAT_CUDA(cudaMemcpyAsync(k_scales_host, w + L.ks, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, s->side[1]));
+    SQUAT_CUDA(cudaMemcpyAsync(k_zeros_host, w + L.kz, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, s->side[1]));
+    SQUAT_CUDA(cudaEventRecord(ev_kout, s->side[1]));
+    SQUAT_CUDA(cudaStreamWaitEvent(st, ev_v, 0));
     rc = squat_quantize_values(w + L.v, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
                                T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.vc),
                                reinterpret_cast<float *>(w + L.vs), reinterpret_cast<float *>(w + L.vz),
                                (long long)n_kv_heads * T, T, stream);
     if (rc != SQUAT_OK) return rc;
-    SQUAT_CUDA(cudaMemcpyAsync(k_codes_host, w + L.kc, toks * d * bits / 8, cudaMemcpyDeviceToHost, st));
-    SQUAT_CUDA(cudaMemcpyAsync(k_scales_host, w + L.ks, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, st));
-    SQUAT_CUDA(cudaMemcpyAsync(k_zeros_host, w + L.kz, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, st));
     SQUAT_CUDA(cudaMemcpyAsync(v_codes_host, w + L.vc, toks * d * bits / 8, cudaMemcpyDeviceToHost, st));
     SQUAT_CUDA(cudaMemcpyAsync(v_scales_host, w + L.vs, toks * (d / group_size) * sizeof(float), cudaMemcpyDeviceToHost, st));
     SQUAT_CUDA(cudaMemcpyAsync(v_zeros_host, w + L.vz, toks * (d / group_size) * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaStreamWaitEvent(st, ev_kout, 0));
     SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;
 }

@@ -20,6 +20,10 @@ struct squat_subspace {
     double *eigvec;        // [H, d, d], row i = eigenvector i
     int *eig_sweeps;       // [H] sweeps of the last eigen-decomposition
     unsigned *status;      // device status word of this device
+    // host path only (created on its first call): two side streams and the events that order them
+    cudaStream_t side[2];
+    cudaEvent_t ev[5];
+    bool side_ready;
 };
 
 // ---- host-side helpers (api.cu) ------------------------------------------------------
