@@ -66,15 +66,63 @@ def bytes_per_vector(d, bits, G, elem_bytes):
 
 # --------------------------------------------------------------------------- clocks sampling
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons while the timed region runs: NVML polled every 2 ms from a thread
+    (read-only queries), or, where the NVML binding is missing, nvidia-smi at its 100 ms cadence."""
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, gpu_index):
-        self.gpu_index, self.proc, self.lines = gpu_index, None, []
+    def __init__(self, gpu_index, pci_bus_id=None):
+        self.gpu_index, self.pci_bus_id = gpu_index, pci_bus_id
+        self.proc, self.lines = None, []
+        self.nvml, self.handle, self.thread, self.stop_flag = None, None, None, threading.Event()
+        self.sm, self.mx, self.reasons = [], [], set()
+
+    def _nvml_open(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            if self.pci_bus_id:
+                try:
+                    self.handle = pynvml.nvmlDeviceGetHandleByPciBusId(self.pci_bus_id.encode())
+                except pynvml.NVMLError:
+                    self.handle = None
+            if self.handle is None:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(self.gpu_index)
+            self.nvml = pynvml
+            return True
+        except Exception:
+            self.nvml = None
+            return False
+
+    def _nvml_poll(self):
+        n = self.nvml
+        masks = {"hw_slowdown": n.nvmlClocksEventReasonHwSlowdown if hasattr(n, "nvmlClocksEventReasonHwSlowdown") else 0x8,
+                 "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        get_reasons = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or n.nvmlDeviceGetCurrentClocksThrottleReasons
+        try:
+            mx = n.nvmlDeviceGetMaxClockInfo(self.handle, n.NVML_CLOCK_SM)
+        except n.NVMLError:
+            mx = None
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
+                if mx:
+                    self.mx.append(float(mx))
+                r = int(get_reasons(self.handle))
+                for name, bit in masks.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except n.NVMLError:
+                pass
+            time.sleep(0.002)
 
     def start(self):
+        if self._nvml_open():
+            self.thread = threading.Thread(target=self._nvml_poll, daemon=True)
+            self.thread.start()
+            return
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                                           "-i", str(self.gpu_index), "-lms", "100"], stdout=subprocess.PIPE,
@@ -88,6 +136,15 @@ class ClockSampler:
             self.lines.append(line.strip())
 
     def stop(self):
+        if self.thread is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=1)
+            try:
+                self.nvml.nvmlShutdown()
+            except Exception:
+                pass
+            return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": max(self.mx) if self.mx else None,
+                    "samples": len(self.sm), "source": "nvml", "reasons": sorted(self.reasons)}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
@@ -97,7 +154,6 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
@@ -106,11 +162,11 @@ class ClockSampler:
                 sm.append(float(f[1])); mx.append(float(f[2]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[5:9]):
+            for name, val in zip(self.NAMES, f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "source": "nvidia-smi", "reasons": sorted(reasons)}
 
 
 # --------------------------------------------------------------------------- distributed glue
@@ -262,7 +318,11 @@ def run_gpu(args, cfg):
         step()
     torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
+    props = torch.cuda.get_device_properties(local_rank)
+    bus = None
+    if all(hasattr(props, a) for a in ("pci_domain_id", "pci_bus_id", "pci_device_id")):
+        bus = "%08x:%02x:%02x.0" % (props.pci_domain_id, props.pci_bus_id, props.pci_device_id)
+    sampler = ClockSampler(local_rank, bus)
     if rank == 0:
         sampler.start()
     if world > 1:
@@ -377,7 +437,7 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="workload index (default 1: Llama-2-7B-shaped layer)")
     ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
