@@ -96,6 +96,59 @@ def test_subspace_fewer_tokens_than_channels():
     s.close()
 
 
+def _build_from_queries(q64, n_kv_heads, rank_r, lam, g=1, dtype=torch.float32):
+    """q64 [Hq, T, d] float64 -> (handle, exported matrices); the GPU gets the values rounded to dtype."""
+    q = torch.from_numpy(np.ascontiguousarray(q64)).to(dtype).cuda()
+    s = sq.Subspace(n_kv_heads, D)
+    sq.squat_build_subspace(s, q, rank_r, lam, g)
+    return s, sq.squat_subspace_export(s, ("W", "gram", "eigval", "eigvec")), q.double().cpu().numpy()
+
+
+def test_subspace_zero_queries_give_zero_update():
+    # M = 0: every eigenvalue is 0, P = I, nothing is fed back; no NaN may come out of the factorisations
+    s, out, _ = _build_from_queries(np.zeros((2, 64, D)), 2, 16, 1e-3)
+    assert np.all(out["gram"] == 0.0) and np.abs(out["eigval"]).max() <= 1e-290
+    assert np.all(np.isfinite(out["eigvec"])) and np.all(out["W"] == 0.0)
+    assert sq.squat_get_device_status(clear=True) & sq.FLAG_NO_CONVERGE == 0
+    s.close()
+
+
+def test_subspace_rank_one_queries_single_head():
+    # all query rows are multiples of one direction u: one eigenvalue |a|^2 |u|^2, the rest 0.  With
+    # s = lambda mu_0, P_inv = I - s/(1+s) u u^T / |u|^2, whose LDL^T factor the oracle also gives.
+    rng = np.random.default_rng(5)
+    u = rng.standard_normal(D)
+    a = rng.standard_normal(200)
+    q64 = np.outer(a, u)[None]                                    # one query head, one KV head
+    s, out, q_used = _build_from_queries(q64, 1, 8, 0.05)
+    Qc = q_used[0]
+    M = oracle.gram(Qc)
+    assert np.abs(out["gram"][0] - M).max() <= 1e-12 * np.abs(M).max()
+    mu0 = np.trace(M)
+    assert abs(out["eigval"][0][0] - mu0) <= 1e-10 * mu0 and np.abs(out["eigval"][0][1:]).max() <= 1e-9 * mu0
+    v0 = out["eigvec"][0][0]
+    assert abs(abs(v0 @ M @ v0) - mu0) <= 1e-9 * mu0              # first eigenvector spans the direction (float32-rounded u)
+    m = oracle.build_W(Qc, 8, 0.05, 1)
+    assert np.abs(out["W"][0].astype(np.float64) - m["W"]).max() <= W_TOL
+    # closed form of the same thing: P_inv = I - s/(1+s) v v^T, unit lower LDL^T factor L, W = L - I
+    sv = 0.05 * mu0
+    P_inv = np.eye(D) - sv / (1 + sv) * np.outer(v0, v0)
+    Lc = np.linalg.cholesky(P_inv)
+    L_unit = Lc / np.diag(Lc)
+    assert np.abs(out["W"][0].astype(np.float64) - (L_unit - np.eye(D))).max() <= 2e-7
+    s.close()
+
+
+def test_subspace_many_heads_more_than_one_wave():
+    # 40 KV heads = 160 CTAs of the eigensolver on 148 SMs: clusters run in two waves; heads must not mix
+    cfg = si.get_config(0).with_(n_kv_heads=40, n_q_heads=40, n_tokens=96)
+    s, out = _build(cfg, rank_r=8)
+    for h in (0, 17, 36, 37, 39):
+        _check_head(cfg, h, out, rank_r=8)
+    assert sq.squat_get_device_status(clear=True) & sq.FLAG_NO_CONVERGE == 0
+    s.close()
+
+
 def test_subspace_strided_queries_and_argument_errors():
     cfg = si.get_config(1).with_(n_kv_heads=2, n_q_heads=4, n_tokens=256)
     q_np = si.gen_queries(cfg)
