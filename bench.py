@@ -343,7 +343,7 @@ def run_gpu(args, cfg):
     step_ms = [e[0].elapsed_time(e[4]) for e in events]
     stage_ms = {n: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in events) for i, n in enumerate(stage_names)}
     local_ms = sum(step_ms)
-    vec_per_step = cfg.key_vectors()
+    vec_per_step = B * H * T               # what one step really quantizes: the prompt pass of the workload
     total_ms, total_units = aggregate_over_ranks(local_ms, vec_per_step * args.steps, dev)
     flags = sq.squat_get_device_status(clear=True)
 
