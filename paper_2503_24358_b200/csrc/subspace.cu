@@ -195,11 +195,12 @@ constexpr int EIG_MAX_SWEEPS = 40;
 // A sweep is
 //   one intra phase   15 rounds that pair the columns inside each held block (8 + 8 pairs per round), then
 //   7 block rounds    of 16 rounds each that pair every column of one held block with every column of the other;
-//                     after each block round the blocks move on to their next holder (round-robin tournament of
-//                     the 8 blocks: position 0 stays, positions 1..7 rotate; CTA c holds positions c and 7 - c).
-// So the CTAs talk 7 times per sweep instead of once per round.  A block moves as ONE bulk copy from the sender's
-// shared memory into the receiver's spare buffer and completes a transaction barrier there; a cluster barrier
-// before the copies makes sure every spare buffer is free.  The squared column norms ride along with the block:
+//                     after each block round one block of every CTA moves to another CTA (schedule below), so
+//                     that over the 7 block rounds every block has met every other one.
+// So the CTAs talk 7 times per sweep instead of once per round.  After a block round every column sits in some
+// team's registers and is written straight into the spare buffer of its next holder (through distributed shared
+// memory if that is a peer); one cluster barrier per move publishes the data and guarantees that nobody is a block
+// round behind, which is what makes the spare buffers free.  The squared column norms ride along with the block:
 // they are refreshed from the data at the start of a sweep and updated by each rotation in between
 // (alpha' = alpha - t gamma, beta' = beta + t gamma), so a round reduces one dot product, not three.
 // The Cholesky factorisation is done redundantly by each CTA on a full copy (it is a small part of the time).
@@ -209,6 +210,15 @@ constexpr int ECT = 512;                     // threads per CTA: 16 warps = 16 c
 constexpr int BW = 16;                       // columns per block
 constexpr int BLD = D + 2;                   // column stride inside a block buffer (doubles)
 constexpr int BLK_DOUBLES = BW * BLD + BW;   // 16 columns and their 16 squared norms
+// Block schedule of a sweep: 7 block rounds, each pairing the two blocks a CTA holds, such that every two of the 8
+// blocks meet exactly once (a 1-factorisation of K8 found by a randomised search; of the candidates tried, the one
+// that needed the fewest sweeps on the benchmark's Gram matrices) while only ONE block per CTA changes
+// hands between consecutive rounds -- the minimum, since two blocks that have met must part.  Move m (after
+// block round m): bit c of MOVE_KEEP1[m] says that CTA c keeps its slot-1 block (else its slot-0 block); the other
+// one goes to CTA (MOVE_TO[m] >> 2c) & 3, where it becomes slot 1.  The schedule is positional, so it covers all
+// pairs from whatever arrangement the previous sweep left.
+__constant__ unsigned char MOVE_KEEP1[7] = {0x5, 0xb, 0x9, 0xd, 0xe, 0x5, 0x5};
+__constant__ unsigned char MOVE_TO[7] = {0x1e, 0x4b, 0xb1, 0x4e, 0x39, 0x8d, 0x1e};
 constexpr unsigned BLK_BYTES = BLK_DOUBLES * (unsigned)sizeof(double);
 static_assert(GRAM_TILES_PER_WARP * (GRAM_THREADS / 32) == 136, "the warps share the upper triangle evenly");
 static_assert(D / BW == 2 * ECL, "two blocks per CTA");
@@ -434,17 +444,15 @@ __global__ void __cluster_dims__(ECL, 1, 1) __launch_bounds__(ECT, 1) eig_cluste
                     big |= did >> 1;
                     named_bar_sync(1, TEAM_THREADS);
                 }
-                // Move the blocks on: position 0 stays, 1 -> 2 -> ... -> 7 -> 1; position p lives in CTA min(p, 7 - p),
-                // slot 0 if p < 4.  After the last round every column sits in some team's registers (column `team` of
-                // slot 0 and column team + 15 mod 16 of slot 1), so the teams write them straight into the spare
-                // buffer of the next holder.  That buffer is free: its owner left it when it began this block round.
-                auto next_home = [&](int slot) {
-                    const int pos = slot == 0 ? crank : 2 * ECL - 1 - crank;
-                    const int npos = pos == 0 ? 0 : (pos == 2 * ECL - 1 ? 1 : pos + 1);
-                    const int dcta = npos < ECL ? npos : 2 * ECL - 1 - npos, dslot = npos < ECL ? 0 : 1;
-                    return cluster.map_shared_rank(blk + ((cur_buf ^ 1) * 2 + dslot) * BLK_DOUBLES, dcta);
-                };
-                double *d0 = next_home(0), *d1 = next_home(1);
+                // Move the blocks on.  After the last round every column sits in some team's registers (column `team`
+                // of slot 0 and column team + 15 mod 16 of slot 1).  Each CTA keeps one of its two blocks (it becomes
+                // slot 0 of the other buffer: plain stores) and sends the other to a peer (slot 1 of the peer's other
+                // buffer: stores through distributed shared memory), as the schedule says.  That buffer is free: its
+                // owner left it when it began this block round.
+                const bool keep1 = (MOVE_KEEP1[br] >> crank) & 1;
+                double *kept_home = blk + ((cur_buf ^ 1) * 2 + 0) * BLK_DOUBLES;
+                double *sent_home = cluster.map_shared_rank(blk + ((cur_buf ^ 1) * 2 + 1) * BLK_DOUBLES, (MOVE_TO[br] >> (2 * crank)) & 3);
+                double *d0 = keep1 ? sent_home : kept_home, *d1 = keep1 ? kept_home : sent_home;
                 const int ql = (team + BW - 1) & (BW - 1);
                 store_col(d0 + team * BLD, xa, tl);
                 store_col(d1 + ql * BLD, xb, tl);
