@@ -185,6 +185,31 @@ def unpack(packed, d, bits):
     return codes
 
 
+def attention_decode(q, K, V):
+    """One decode step over cached rows K, V [n, d] for the query vectors q [nq, d] (Section 2)."""
+    q = np.ascontiguousarray(np.atleast_2d(q), dtype=np.float64)
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    nq, d = q.shape
+    n = K.shape[0]
+    out = np.empty((nq, d), dtype=np.float64)
+    _check(_load().sqo_attention_decode(_p(q, _D), nq, _p(K, _D), _p(V, _D), ctypes.c_long(n), d, _p(out, _D)),
+           "attention_decode")
+    return out
+
+
+def decode_attention_over_cache(q, k_codes, k_scale, k_zero, v_codes, v_scale, v_zero, G, k_res=None, v_res=None):
+    """What a decode step computes for one (batch, KV head): the quantized part of the cache is
+    dequantized (codes [n, d] unpacked), the residual buffer's full-precision rows are appended, then
+    attention_decode.  Marshalling only: every number comes from the C functions."""
+    Kd = dequant_keys(k_codes, k_scale, k_zero, G)
+    Vd = dequant_values(v_codes, v_scale, v_zero, G)
+    if k_res is not None and len(k_res):
+        Kd = np.concatenate([Kd, np.asarray(k_res, dtype=np.float64)], axis=0)
+        Vd = np.concatenate([Vd, np.asarray(v_res, dtype=np.float64)], axis=0)
+    return attention_decode(q, Kd, Vd)
+
+
 def kv_cache_bytes(batch, seq_len, layers, heads, head_dim, bytes_per_param):
     return int(_load().sqo_kv_cache_bytes(batch, seq_len, layers, heads, head_dim, bytes_per_param))
 

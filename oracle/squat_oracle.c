@@ -20,14 +20,18 @@
  *   sqo_dequant_keys / sqo_dequant_values          Section 2, deq(.)
  *   sqo_pack / sqo_unpack                          cache layout (the paper gives none; ours)
  *   sqo_kv_cache_bytes                             Appendix B, memory formula
+ *   sqo_attention_decode                           Section 2 "(Masked) Attention mechanism": one decode step,
+ *                                                  softmax(q K^T / sqrt(d)) V over the cached tokens (the
+ *                                                  score vector w^deq of the proof of Theorem 1)
  *
  * Pins (tests, CPU only): the chain of Lemma 4 against direct inverses; B_t H_t against a
  * generic KKT solve of Eq. (2) and against the LDL^T factor of P_inv; lambda = 0 / r = 0
  * against ordinary round-to-nearest; the invariant delta^T P delta = e^T D^-1 e; idempotence;
  * chunking invariance; exhaustive search on tiny problems; the subspace against a library
  * SVD; the value path against a library float32 computation; the memory formula against
- * the worked example printed in Appendix B.  The paper prints no input/output pair for the
- * quantizer itself.
+ * the worked example printed in Appendix B; the decode-step attention against a loop-by-loop
+ * restatement, its closed forms (zero query = mean of the values, one dominant score) and the
+ * bound of Theorem 1.  The paper prints no input/output pair for the quantizer itself.
  *
  * Readings of the paper where it is silent (same list as the design notes):
  *   - rounding is round-half-to-even;
@@ -491,4 +495,39 @@ long long sqo_kv_cache_bytes(long long batch, long long seq_len, long long layer
                              long long head_dim, long long bytes_per_param)
 {
     return 2LL * batch * seq_len * layers * heads * head_dim * bytes_per_param;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* One decode step of attention (Section 2): for each of the nq query vectors (the query heads
+ * that share this KV head), w_i = <q, k_i> / sqrt(d) over the n cached tokens, p = softmax(w),
+ * out = sum_i p_i v_i.  K and V are what a reader of the cache sees: dequantized rows followed
+ * by the full-precision rows of the residual buffer.  The largest score is subtracted before
+ * exponentiation; that leaves softmax unchanged and keeps exp() in range. */
+int sqo_attention_decode(const double *q, int nq, const double *K, const double *V, long n, int d, double *out)
+{
+    if (!q || !K || !V || !out || nq <= 0 || n <= 0 || d <= 0) return SQO_ERR_ARG;
+    double *w = (double *)malloc((size_t)n * sizeof(double));
+    if (!w) return SQO_ERR_ALLOC;
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    for (int h = 0; h < nq; ++h) {
+        double wmax = -INFINITY;
+        for (long i = 0; i < n; ++i) {
+            double s = 0.0;
+            for (int j = 0; j < d; ++j) s += q[h * d + j] * K[i * d + j];
+            w[i] = s * inv_sqrt_d;
+            if (w[i] > wmax) wmax = w[i];
+        }
+        double denom = 0.0;
+        for (long i = 0; i < n; ++i) {
+            w[i] = exp(w[i] - wmax);
+            denom += w[i];
+        }
+        for (int j = 0; j < d; ++j) {
+            double s = 0.0;
+            for (long i = 0; i < n; ++i) s += w[i] * V[i * d + j];
+            out[h * d + j] = s / denom;
+        }
+    }
+    free(w);
+    return SQO_OK;
 }
