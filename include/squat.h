@@ -152,6 +152,38 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Reader of the cache -- one decode step of attention over the packed cache (Section 2, "(Masked) Attention
+ * mechanism": softmax(q K^T / sqrt(d)) V for the newest token; the score vector w^deq of the proof of
+ * Theorem 1; the most recent tokens come from the full-precision residual buffer of Algorithm 1).  This is
+ * the step that follows the write path; the cache is read in its packed form, never dequantized to memory.
+ *
+ *   out[b][hq] = sum_i p_i v_i,   p = softmax_i( softmax_scale * <q[b][hq], k_i> ),
+ *   i over the n_tokens dequantized rows of KV head hq / (n_q_heads / n_kv_heads) (GQA rule of Appendix C),
+ *   then the n_res rows of the residual buffer.
+ *
+ * q            [batch, n_q_heads, d] device, dense, dtype q_dtype.
+ * k_codes .. v_zeros   the cache as squat_quantize_keys / squat_quantize_values wrote it (device); token 0
+ *              of (b, h) sits at token index b * cache_stride_b + h * cache_stride_h, strides in tokens and
+ *              multiples of group_size, so a cache longer than n_tokens can be read.  n_tokens is the number
+ *              of quantized tokens per (b, h): a multiple of group_size, may be 0.
+ * k_res, v_res [batch, n_kv_heads, n_res, d] device, dense, dtype res_dtype: the residual buffer;
+ *              n_res <= SQUAT_ATTN_MAX_RESIDUAL, may be 0 (then both may be NULL).  n_tokens + n_res >= 1.
+ * softmax_scale  multiplies the scores; 0 selects the paper's 1 / sqrt(d).
+ * out          [batch, n_q_heads, d] float32 device.
+ * workspace    device, caller-owned, 256-byte aligned, at least squat_decode_attention_workspace_bytes(...);
+ *              holds the per-chunk partial results, no state is kept between calls.
+ * All arithmetic is float32.  Returns a status code; nothing is launched on an argument error.
+ */
+#define SQUAT_ATTN_MAX_RESIDUAL 128
+size_t squat_decode_attention_workspace_bytes(int batch, int n_q_heads, int n_tokens);
+int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                           const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
+                           const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                           int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                           int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                           float softmax_scale, float *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Gram matrices of the stacked prompt queries without any allocation.  (The paper has no counterpart:
  * this entry exists for callers that must not allocate.)
  *

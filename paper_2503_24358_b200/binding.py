@@ -22,6 +22,7 @@ EXPORTED_SYMBOLS = (
     "squat_subspace_import", "squat_subspace_eig_sweeps", "squat_quantize_keys", "squat_quantize_values", "squat_dequantize",
     "squat_write_path_workspace_bytes", "squat_write_path_host", "squat_get_device_status",
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
+    "squat_decode_attention_workspace_bytes", "squat_decode_attention",
 )
 
 _lib = None
@@ -60,6 +61,10 @@ def _load():
         lib.squat_write_path_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, dbl, i, i, i,
                                               vp, vp, vp, vp, vp, vp, vp, c.c_size_t, vp]
         lib.squat_gram_static.argtypes = [vp, i, i, i, i, i, ll, ll, vp, vp]
+        lib.squat_decode_attention_workspace_bytes.argtypes = [i, i, i]
+        lib.squat_decode_attention_workspace_bytes.restype = c.c_size_t
+        lib.squat_decode_attention.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, ll, ll, i, i, vp, vp, i, i,
+                                               c.c_float, vp, vp, c.c_size_t, vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
         lib.squat_status_string.argtypes = [i]
@@ -239,6 +244,36 @@ def squat_gram_static(q: torch.Tensor, n_kv_heads: int, gram_out: torch.Tensor, 
     _check(_load().squat_gram_static(_dev(q, "q"), _dtype_code(q), q.shape[0], n_kv_heads, q.shape[1], q.shape[2],
                                      q.stride(0), q.stride(1), _dev(gram_out, "gram_out"), _stream(stream)),
            "squat_gram_static")
+
+
+def squat_decode_attention_workspace_bytes(batch: int, n_q_heads: int, n_tokens: int) -> int:
+    return int(_load().squat_decode_attention_workspace_bytes(batch, n_q_heads, n_tokens))
+
+
+def squat_decode_attention(q: torch.Tensor, k_codes, k_scales, k_zeros, v_codes, v_scales, v_zeros, n_kv_heads: int,
+                           n_tokens: int, bits: int, group_size: int, out: torch.Tensor, workspace: torch.Tensor,
+                           k_res: torch.Tensor = None, v_res: torch.Tensor = None, softmax_scale: float = 0.0,
+                           cache_stride_b: int = None, cache_stride_h: int = None, stream=None):
+    """One decode step of attention over the packed cache.  q [B, Hq, d]; the cache tensors as the write path
+    produced them; k_res / v_res [B, H, R, d] the full-precision residual buffer (optional); out [B, Hq, d]
+    float32; workspace a CUDA uint8 tensor of squat_decode_attention_workspace_bytes(...)."""
+    if q.dim() != 3 or not q.is_contiguous() or not out.is_contiguous() or out.dtype != torch.float32:
+        raise ValueError("q must be contiguous [batch, n_q_heads, d]; out contiguous float32")
+    B, Hq, d = q.shape
+    csh = n_tokens if cache_stride_h is None else cache_stride_h
+    csb = n_kv_heads * csh if cache_stride_b is None else cache_stride_b
+    n_res = 0 if k_res is None else k_res.shape[2]
+    if n_res and (not k_res.is_contiguous() or not v_res.is_contiguous() or k_res.dtype != v_res.dtype):
+        raise ValueError("k_res and v_res must be contiguous [batch, n_kv_heads, n_res, d] of one dtype")
+    opt = lambda t, n: _dev(t, n) if t is not None and t.numel() else None
+    _check(_load().squat_decode_attention(_dev(q, "q"), _dtype_code(q), B, Hq, n_kv_heads, d, opt(k_codes, "k_codes"),
+                                          opt(k_scales, "k_scales"), opt(k_zeros, "k_zeros"), opt(v_codes, "v_codes"),
+                                          opt(v_scales, "v_scales"), opt(v_zeros, "v_zeros"), n_tokens, csb, csh, bits,
+                                          group_size, opt(k_res, "k_res"), opt(v_res, "v_res"),
+                                          _dtype_code(k_res) if n_res else SQUAT_F32, n_res, float(softmax_scale),
+                                          _dev(out, "out"), _dev(workspace, "workspace"),
+                                          workspace.numel() * workspace.element_size(), _stream(stream)),
+           "squat_decode_attention")
 
 
 def squat_get_device_status(clear: bool = True, stream=None) -> int:

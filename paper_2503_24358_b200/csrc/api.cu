@@ -272,6 +272,45 @@ int squat_dequantize(int kind, const unsigned char *codes, const float *scales, 
                                 in_stride_b, in_stride_h, out, out_dtype, static_cast<cudaStream_t>(stream));
 }
 
+size_t squat_decode_attention_workspace_bytes(int batch, int n_q_heads, int n_tokens)
+{
+    if (batch <= 0 || n_q_heads <= 0 || n_tokens < 0) return 0;
+    return (squat_attention_workspace_floats(batch, n_q_heads, n_tokens) * sizeof(float) + 255) / 256 * 256 + 256;
+}
+
+int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                           const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
+                           const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                           int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                           int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                           float softmax_scale, float *out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!valid_dtype(q_dtype) || batch < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_tokens < 0 || n_res < 0)
+        return SQUAT_ERR_INVALID_ARG;
+    if (batch == 0) return SQUAT_OK;
+    if (!q || !out || !workspace || !aligned16(q) || !aligned16(out)) return SQUAT_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQUAT_ERR_INVALID_ARG;
+    if (head_dim != D || n_q_heads % n_kv_heads != 0) return SQUAT_ERR_SHAPE;
+    if (bits != 2 && bits != 4) return SQUAT_ERR_UNSUPPORTED;
+    if (group_size != 32 && group_size != 64 && group_size != 128) return SQUAT_ERR_UNSUPPORTED;
+    if (n_res > SQUAT_ATTN_MAX_RESIDUAL) return SQUAT_ERR_UNSUPPORTED;
+    if (n_tokens + n_res < 1) return SQUAT_ERR_SHAPE;
+    if (n_tokens % group_size || cache_stride_b % group_size || cache_stride_h % group_size || cache_stride_b < 0 ||
+        cache_stride_h < 0)
+        return SQUAT_ERR_SHAPE;
+    if (n_tokens > 0 && (!k_codes || !k_scales || !k_zeros || !v_codes || !v_scales || !v_zeros)) return SQUAT_ERR_INVALID_ARG;
+    if (n_tokens > 0 && (!aligned16(k_codes) || !aligned16(k_scales) || !aligned16(k_zeros) || !aligned16(v_codes) ||
+                         !aligned16(v_scales) || !aligned16(v_zeros)))
+        return SQUAT_ERR_INVALID_ARG;
+    if (n_res > 0 && (!k_res || !v_res || !valid_dtype(res_dtype))) return SQUAT_ERR_INVALID_ARG;
+    if (workspace_bytes < squat_decode_attention_workspace_bytes(batch, n_q_heads, n_tokens)) return SQUAT_ERR_INVALID_ARG;
+    const float scale = softmax_scale != 0.0f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    return squat_launch_decode_attention(q, q_dtype, batch, n_q_heads, n_kv_heads, n_tokens, k_codes, k_scales, k_zeros,
+                                         v_codes, v_scales, v_zeros, cache_stride_b, cache_stride_h, bits, group_size,
+                                         k_res, v_res, res_dtype, n_res, scale, out, static_cast<float *>(workspace),
+                                         static_cast<cudaStream_t>(stream));
+}
+
 int squat_get_device_status(void *stream, unsigned *flags, int clear)
 {
     if (!flags) return SQUAT_ERR_INVALID_ARG;

@@ -1,0 +1,338 @@
+// Reader of the packed cache: one decode step of attention (Section 2, "(Masked) Attention mechanism";
+// the score vector w^deq = <q, deq(k_i)> / sqrt(d) of the proof of Theorem 1; the most recent tokens come
+// from the full-precision residual buffer of Algorithm 1).
+//
+//   out_hq = softmax_i( s <q_hq, k_i> ) . v_i ,   k_i, v_i = dequantized cache rows, then the residual rows
+//
+// The cache is never dequantized to memory.  Per-channel key metadata folds into the query: for the G tokens
+// that share (scale_c, zero_c),  <q, deq(k_t)> = sum_c (q_c scale_c) code_tc + sum_c q_c zero_c, so a group
+// costs one scaled copy of the query and each token one dot product with its 128 codes.  Per-token value
+// metadata folds into the weight: p_t deq(v_t)_c = (p_t scale_tg) code_tc + p_t zero_tg.  Codes become floats
+// without a conversion: the code bits are shifted under the top of a float's mantissa, giving 1 + code / 2^bits
+// exactly (two integer instructions); the "1 +" is taken out again through one constant per group.
+//
+// attn_partial_kernel   grid (token chunks of 1024 x query-head passes, KV heads, batch).  Key phase: a warp takes
+//                       32 tokens (lane = token, its codes are 2 or 4 128-bit loads), scores go to shared
+//                       memory.  Then the chunk's maximum and exp().  Value phase: a warp reads 128 bytes of
+//                       codes per step (lane = one 32-bit word of one of 4 or 2 tokens) and accumulates
+//                       weight x code for its channels.  Writes (unnormalised sum, max, denominator) per chunk.
+// attn_combine_kernel   grid (query heads, batch): adds the residual buffer's tokens (plain fp32 dot products)
+//                       and merges the chunks with the usual max / denominator rescaling.
+//
+// Bound: HBM (bits/8 + metadata bytes per cached element); the unpacking arithmetic is close behind.
+#include "squat_internal.cuh"
+
+namespace {
+
+constexpr int D = SQUAT_D;
+constexpr int AT_THREADS = 256;
+constexpr int AT_WARPS = AT_THREADS / 32;
+constexpr int AT_CHUNK = 1024;            // tokens per CTA
+constexpr int AT_VTOK = AT_CHUNK / AT_WARPS;   // tokens per warp in the value phase
+
+struct AttnParams {
+    const void *q;             // [B, Hq, D]
+    int q_bf16;
+    int B, Hq, H, T;           // T: quantized tokens per (batch, head)
+    const unsigned char *kc, *vc;
+    const float *ks, *kz, *vs, *vz;
+    long long csb, csh;        // cache strides in tokens
+    int G;
+    const void *k_res, *v_res; // [B, H, R, D]
+    int res_bf16, R;
+    float scale;
+    float *part;               // [B, Hq, nchunk, D]
+    float *ml;                 // [B, Hq, nchunk, 2]
+    int nchunk;
+    float *out;                // [B, Hq, D]
+};
+
+// 1 + code / 2^BITS as a float, for the code at position i of a 32-bit word (low bits first)
+template <int BITS>
+__device__ __forceinline__ float code_as_float(uint32_t w, int i)
+{
+    constexpr int TOP = 23 - BITS;                              // the code's low bit lands here
+    constexpr uint32_t MASK = ((1u << BITS) - 1u) << TOP;
+    const int pos = BITS * i;
+    const uint32_t sh = pos <= TOP ? (w << (TOP - pos)) : (w >> (pos - TOP));
+    return __uint_as_float((sh & MASK) | 0x3F800000u);
+}
+
+__device__ __forceinline__ float warp_sum_f(float v)
+{
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    return v;
+}
+__device__ __forceinline__ float warp_max_f(float v)
+{
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, m));
+    return v;
+}
+
+__device__ __forceinline__ float load_elem(const void *p, long long idx, int bf16)
+{
+    if (bf16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(p)[idx]);
+    return reinterpret_cast<const float *>(p)[idx];
+}
+
+template <int BITS, int NQ>
+__global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnParams p)
+{
+    constexpr int WPT = D * BITS / 32;                          // 32-bit words per token: 8 or 16
+    constexpr int CPW = 32 / BITS;                              // codes per word: 16 or 8
+    constexpr float LV = float(1 << BITS);
+    extern __shared__ __align__(16) float sm[];
+    float *qsm = sm;                                            // [NQ][D]      q * softmax scale
+    float *qs = qsm + NQ * D;                                   // [warps][NQ][D] query x key scale x 2^BITS of the warp's group
+    float *sc = qs + AT_WARPS * NQ * D;                         // [NQ][AT_CHUNK] scores, then weights
+    float *red = sc + NQ * AT_CHUNK;                            // [NQ][warps] and [NQ] scratch of the reductions
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chunk = blockIdx.x % p.nchunk, qpass = blockIdx.x / p.nchunk;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int qpk = p.Hq / p.H;
+    const int hq0 = h * qpk + qpass * NQ;
+    const int nq_here = min(NQ, qpk - qpass * NQ);
+    const int t0 = chunk * AT_CHUNK, t1 = min(p.T, t0 + AT_CHUNK);
+    const long long ctok0 = (long long)b * p.csb + (long long)h * p.csh;
+
+    for (int i = tid; i < NQ * D; i += AT_THREADS) {
+        const int qi = i / D, c = i % D;
+        qsm[i] = qi < nq_here ? p.scale * load_elem(p.q, ((long long)b * p.Hq + hq0 + qi) * D + c, p.q_bf16) : 0.0f;
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- key phase: scores
+    float *qsw = qs + warp * NQ * D;
+    for (int blk = t0 + 32 * warp; blk < t1; blk += 32 * AT_WARPS) {
+        const long long mrow = (ctok0 / p.G + blk / p.G) * D;
+        const float4 s4 = __ldg(reinterpret_cast<const float4 *>(p.ks + mrow) + lane);
+        const float4 z4 = __ldg(reinterpret_cast<const float4 *>(p.kz + mrow) + lane);
+        float k0[NQ];
+        __syncwarp();
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) {
+            const float4 qv = *reinterpret_cast<const float4 *>(qsm + qi * D + 4 * lane);
+            const float4 v = make_float4(qv.x * s4.x * LV, qv.y * s4.y * LV, qv.z * s4.z * LV, qv.w * s4.w * LV);
+            *reinterpret_cast<float4 *>(qsw + qi * D + 4 * lane) = v;
+            const float zs = qv.x * z4.x + qv.y * z4.y + qv.z * z4.z + qv.w * z4.w;
+            k0[qi] = warp_sum_f(zs - (v.x + v.y + v.z + v.w));  // sum_c q_c zero_c - sum_c qs'_c  (takes the "1 +" out)
+        }
+        __syncwarp();
+        const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
+        float acc[NQ];
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) acc[qi] = 0.0f;
+#pragma unroll
+        for (int v4 = 0; v4 < WPT / 4; ++v4) {
+            const uint4 cw = __ldg(cp + v4);
+            const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+            for (int wi = 0; wi < 4; ++wi)
+#pragma unroll
+                for (int i4 = 0; i4 < CPW / 4; ++i4) {
+                    const int ch = (v4 * 4 + wi) * CPW + 4 * i4;
+                    const float f0 = code_as_float<BITS>(w4[wi], 4 * i4), f1 = code_as_float<BITS>(w4[wi], 4 * i4 + 1),
+                                f2 = code_as_float<BITS>(w4[wi], 4 * i4 + 2), f3 = code_as_float<BITS>(w4[wi], 4 * i4 + 3);
+#pragma unroll
+                    for (int qi = 0; qi < NQ; ++qi) {
+                        const float4 qq = *reinterpret_cast<const float4 *>(qsw + qi * D + ch);
+                        acc[qi] = fmaf(f0, qq.x, acc[qi]);
+                        acc[qi] = fmaf(f1, qq.y, acc[qi]);
+                        acc[qi] = fmaf(f2, qq.z, acc[qi]);
+                        acc[qi] = fmaf(f3, qq.w, acc[qi]);
+                    }
+                }
+        }
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) sc[qi * AT_CHUNK + blk - t0 + lane] = acc[qi] + k0[qi];
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- chunk maximum, weights, denominator
+    const int nt = t1 - t0;
+    float mx[NQ], den[NQ];
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        float m = -INFINITY;
+        for (int i = tid; i < nt; i += AT_THREADS) m = fmaxf(m, sc[qi * AT_CHUNK + i]);
+        m = warp_max_f(m);
+        if (lane == 0) red[qi * AT_WARPS + warp] = m;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        float m = red[qi * AT_WARPS];
+#pragma unroll
+        for (int w = 1; w < AT_WARPS; ++w) m = fmaxf(m, red[qi * AT_WARPS + w]);
+        mx[qi] = m;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        float s = 0.0f;
+        for (int i = tid; i < nt; i += AT_THREADS) {
+            const float e = expf(sc[qi * AT_CHUNK + i] - mx[qi]);
+            sc[qi * AT_CHUNK + i] = e;
+            s += e;
+        }
+        s = warp_sum_f(s);
+        if (lane == 0) red[qi * AT_WARPS + warp] = s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < AT_WARPS; ++w) s += red[qi * AT_WARPS + w];
+        den[qi] = s;
+    }
+
+    // ---------------------------------------------------------------- value phase: sum_t weight_t deq(v_t)
+    constexpr int TPI = 32 / WPT;                               // tokens per warp step: 4 or 2
+    const int ts = lane / WPT, j = lane % WPT;
+    const int ng = D / p.G, gidx = (j * CPW) / p.G;
+    float accv[NQ][CPW], corr[NQ];
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        corr[qi] = 0.0f;
+#pragma unroll
+        for (int i = 0; i < CPW; ++i) accv[qi][i] = 0.0f;
+    }
+    const int vbase = t0 + warp * AT_VTOK;
+    const int vend = min(t1, vbase + AT_VTOK);
+    for (int tk = vbase + ts; tk < vend; tk += TPI) {
+        const long long ct = ctok0 + tk;
+        const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(p.vc) + ct * WPT + j);
+        const float vsc = __ldg(p.vs + ct * ng + gidx) * LV, vzr = __ldg(p.vz + ct * ng + gidx);
+        float a[NQ];
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) {
+            const float pw = sc[qi * AT_CHUNK + tk - t0];
+            a[qi] = pw * vsc;
+            corr[qi] += pw * vzr - a[qi];
+        }
+#pragma unroll
+        for (int i = 0; i < CPW; ++i) {
+            const float f = code_as_float<BITS>(w, i);
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) accv[qi][i] = fmaf(f, a[qi], accv[qi][i]);
+        }
+    }
+    // add the group constant, fold the token classes of the warp, then the warps
+    __syncthreads();                                            // everybody is done reading sc: reuse it as [warps][NQ][D]
+    float *part_sm = sc;
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi)
+#pragma unroll
+        for (int i = 0; i < CPW; ++i) {
+            float v = accv[qi][i] + corr[qi];
+#pragma unroll
+            for (int m = WPT; m < 32; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+            if (ts == 0) part_sm[(warp * NQ + qi) * D + j * CPW + i] = v;
+        }
+    __syncthreads();
+    for (int i = tid; i < NQ * D; i += AT_THREADS) {
+        const int qi = i / D, c = i % D;
+        if (qi >= nq_here) continue;
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < AT_WARPS; ++w) s += part_sm[(w * NQ + qi) * D + c];
+        p.part[(((long long)b * p.Hq + hq0 + qi) * p.nchunk + chunk) * D + c] = s;
+    }
+    if (tid < nq_here) {
+        float *ml = p.ml + (((long long)b * p.Hq + hq0 + tid) * p.nchunk + chunk) * 2;
+        ml[0] = mx[tid];
+        ml[1] = den[tid];
+    }
+}
+
+// One CTA per (batch, query head), thread = channel: the residual buffer's tokens, then the merge.
+__global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
+{
+    __shared__ float qv[D];
+    __shared__ float w[SQUAT_ATTN_MAX_RESIDUAL];
+    __shared__ float red[4];
+    const int hq = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+    const int h = hq / (p.Hq / p.H);
+    qv[c] = p.scale * load_elem(p.q, ((long long)b * p.Hq + hq) * D + c, p.q_bf16);
+    __syncthreads();
+    const long long rbase = ((long long)b * p.H + h) * p.R * D;
+    float m = -INFINITY;
+    if (c < p.R) {
+        float s = 0.0f;
+        for (int j = 0; j < D; ++j) s = fmaf(qv[j], load_elem(p.k_res, rbase + (long long)c * D + j, p.res_bf16), s);
+        w[c] = s;
+        m = s;
+    }
+    const float *ml = p.ml + ((long long)b * p.Hq + hq) * p.nchunk * 2;
+    for (int s = c; s < p.nchunk; s += D) m = fmaxf(m, ml[2 * s]);
+    m = warp_max_f(m);
+    if ((c & 31) == 0) red[c >> 5] = m;
+    __syncthreads();
+    m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    __syncthreads();
+    if (c < p.R) w[c] = expf(w[c] - m);
+    __syncthreads();
+    float acc = 0.0f, den = 0.0f;
+    for (int t = 0; t < p.R; ++t) {
+        acc = fmaf(w[t], load_elem(p.v_res, rbase + (long long)t * D + c, p.res_bf16), acc);
+        den += w[t];
+    }
+    const float *part = p.part + ((long long)b * p.Hq + hq) * p.nchunk * D;
+    for (int s = 0; s < p.nchunk; ++s) {
+        const float f = expf(ml[2 * s] - m);
+        acc = fmaf(f, part[(long long)s * D + c], acc);
+        den = fmaf(f, ml[2 * s + 1], den);
+    }
+    p.out[((long long)b * p.Hq + hq) * D + c] = acc / den;
+}
+
+template <int BITS, int NQ>
+int launch_partial(const AttnParams &p, int qpasses, cudaStream_t st)
+{
+    const size_t smem = sizeof(float) * (NQ * D + AT_WARPS * NQ * D + NQ * AT_CHUNK + NQ * AT_WARPS + 8);
+    SQUAT_CUDA(cudaFuncSetAttribute(attn_partial_kernel<BITS, NQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attn_partial_kernel<BITS, NQ><<<dim3(p.nchunk * qpasses, p.H, p.B), AT_THREADS, smem, st>>>(p);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}
+
+}  // namespace
+
+size_t squat_attention_workspace_floats(int batch, int n_q_heads, int n_tokens)
+{
+    const long long nchunk = (n_tokens + AT_CHUNK - 1) / AT_CHUNK;
+    return (size_t)batch * n_q_heads * nchunk * (D + 2);
+}
+
+int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq, int H, int T,
+                                  const unsigned char *kc, const float *ks, const float *kz,
+                                  const unsigned char *vc, const float *vs, const float *vz,
+                                  long long csb, long long csh, int bits, int G,
+                                  const void *k_res, const void *v_res, int res_dtype, int R,
+                                  float scale, float *out, float *workspace, cudaStream_t st)
+{
+    AttnParams p;
+    p.q = q; p.q_bf16 = q_dtype == SQUAT_BF16; p.B = batch; p.Hq = Hq; p.H = H; p.T = T;
+    p.kc = kc; p.vc = vc; p.ks = ks; p.kz = kz; p.vs = vs; p.vz = vz; p.csb = csb; p.csh = csh; p.G = G;
+    p.k_res = k_res; p.v_res = v_res; p.res_bf16 = res_dtype == SQUAT_BF16; p.R = R;
+    p.scale = scale; p.out = out;
+    p.nchunk = (T + AT_CHUNK - 1) / AT_CHUNK;
+    p.part = workspace;
+    p.ml = workspace + (size_t)batch * Hq * p.nchunk * D;
+    const int qpk = Hq / H;
+    if (p.nchunk > 0) {
+        int rc;
+        if (qpk == 1) rc = bits == 2 ? launch_partial<2, 1>(p, 1, st) : launch_partial<4, 1>(p, 1, st);
+        else if (qpk == 2) rc = bits == 2 ? launch_partial<2, 2>(p, 1, st) : launch_partial<4, 2>(p, 1, st);
+        else rc = bits == 2 ? launch_partial<2, 4>(p, (qpk + 3) / 4, st) : launch_partial<4, 4>(p, (qpk + 3) / 4, st);
+        if (rc != SQUAT_OK) return rc;
+    }
+    attn_combine_kernel<<<dim3(Hq, batch), D, 0, st>>>(p);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}

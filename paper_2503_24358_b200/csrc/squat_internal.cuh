@@ -47,6 +47,13 @@ int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T,
                               long long sb, long long sh, long long st_, int bits, int G,
                               unsigned char *codes, float *scales, float *zeros,
                               long long osb, long long osh, unsigned *status, cudaStream_t st);
+size_t squat_attention_workspace_floats(int batch, int n_q_heads, int n_tokens);
+int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq, int H, int T,
+                                  const unsigned char *kc, const float *ks, const float *kz,
+                                  const unsigned char *vc, const float *vs, const float *vz,
+                                  long long csb, long long csh, int bits, int G,
+                                  const void *k_res, const void *v_res, int res_dtype, int R,
+                                  float scale, float *out, float *workspace, cudaStream_t st);
 int squat_launch_dequant(int kind, const unsigned char *codes, const float *scales, const float *zeros,
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
                          void *out, int out_dtype, cudaStream_t st);
