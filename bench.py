@@ -352,9 +352,13 @@ def run_gpu(args, cfg):
     if not args.no_e2e:
         e2e = run_e2e(args, cfg, sq, s, (q_np, k_np, v_np), (kc, ks, kz, vc, vs, vz), to_dev, flush, tdt, dev,
                       vec_per_step)
+    # ---- the reader that follows the write path (not part of a step): one decode step of attention -----
+    reader = None
+    if rank == 0 and not args.no_reader:
+        reader = run_reader(cfg, sq, (kc, ks, kz, vc, vs, vz), flush, tdt, dev)
     if rank == 0:
         report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches,
-               wall, flags, clocks)
+               wall, flags, clocks, reader)
     s.close()
     if world > 1:
         dist.destroy_process_group()
@@ -387,8 +391,43 @@ def run_e2e(args, cfg, sq, s, host_np, dev_outs, to_dev, flush, tdt, dev, vec_pe
             "api": "squat_write_path_host (pinned host buffers; build + keys + values)"}
 
 
+def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10):
+    """One decode step of attention over the cache the step has just written (plus a full residual buffer of
+    random full-precision rows): time per call and the bytes it has to read, against the copy bandwidth."""
+    import torch
+    B, H, T, d, bits, G = cfg.batch, cfg.n_kv_heads, cfg.n_tokens, cfg.head_dim, cfg.bits, cfg.group_size
+    Hq, R = cfg.n_q_heads, (cfg.residual or 32)
+    gen = torch.Generator(device=dev).manual_seed(1234)
+    q = torch.randn(B, Hq, d, generator=gen, device=dev).to(tdt)
+    k_res = torch.randn(B, H, R, d, generator=gen, device=dev).to(tdt)
+    v_res = torch.randn(B, H, R, d, generator=gen, device=dev).to(tdt)
+    out = torch.empty((B, Hq, d), dtype=torch.float32, device=dev)
+    ws = torch.empty(sq.squat_decode_attention_workspace_bytes(B, Hq, T), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    call = lambda: sq.squat_decode_attention(q, *cache, H, T, bits, G, out, ws, k_res, v_res)
+    for _ in range(3):
+        flush.zero_()
+        call()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for a, b in ev:
+        flush.zero_()
+        a.record(stream)
+        call()
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+    elem = 4 if cfg.dtype == "f32" else 2
+    toks = B * H * T
+    nbytes = toks * (2 * d * bits // 8 + 8 * d // G + 8 * d // G) + 2 * B * H * R * d * elem + B * Hq * d * (elem + 4)
+    peaks = measured_peaks()
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"what": "squat_decode_attention: softmax(q K^T / sqrt(d)) V over the packed cache + residual buffer",
+            "ms_per_call": ms, "cached_tokens": toks, "n_q_heads": Hq, "residual_tokens": R, "bytes_per_call": nbytes,
+            "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "cached_tokens_per_s": toks / (ms * 1e-3)}
+
+
 def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches, wall,
-           flags, clocks):
+           flags, clocks, reader=None):
     d, bits, G = cfg.head_dim, cfg.bits, cfg.group_size
     if rank_is_zero():
         peaks = measured_peaks()
@@ -430,6 +469,7 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
             "gpu_launches": int(launches), "wall_s_timed_region": wall, "device_status_flags": int(flags),
             "clocks": clocks,
             "cpu_baseline": cpu_baseline(cfg) if (world == 1 and not args.no_cpu_baseline) else None,
+            "reader_decode_attention": reader,
         }
         print(json.dumps(line))
 
@@ -437,6 +477,7 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--no-reader", action="store_true", help="skip the decode-attention leg that follows the step")
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="workload index (default 1: Llama-2-7B-shaped layer)")

@@ -11,7 +11,7 @@
 // without a conversion: the code bits are shifted under the top of a float's mantissa, giving 1 + code / 2^bits
 // exactly (two integer instructions); the "1 +" is taken out again through one constant per group.
 //
-// attn_partial_kernel   grid (token chunks of 1024 x query-head passes, KV heads, batch).  Key phase: a warp takes
+// attn_partial_kernel   grid (token chunks of 256..1024 x query-head passes, KV heads, batch).  Key phase: a warp takes
 //                       32 tokens (lane = token, its codes are 2 or 4 128-bit loads), scores go to shared
 //                       memory.  Then the chunk's maximum and exp().  Value phase: a warp reads 128 bytes of
 //                       codes per step (lane = one 32-bit word of one of 4 or 2 tokens) and accumulates
@@ -27,8 +27,7 @@ namespace {
 constexpr int D = SQUAT_D;
 constexpr int AT_THREADS = 256;
 constexpr int AT_WARPS = AT_THREADS / 32;
-constexpr int AT_CHUNK = 1024;            // tokens per CTA
-constexpr int AT_VTOK = AT_CHUNK / AT_WARPS;   // tokens per warp in the value phase
+constexpr int AT_CHUNK = 1024;            // most tokens per CTA (the launcher takes 256, 512 or 1024: enough CTAs to fill the GPU)
 
 struct AttnParams {
     const void *q;             // [B, Hq, D]
@@ -43,7 +42,7 @@ struct AttnParams {
     float scale;
     float *part;               // [B, Hq, nchunk, D]
     float *ml;                 // [B, Hq, nchunk, 2]
-    int nchunk;
+    int nchunk, chunk;         // chunk: tokens per CTA, a multiple of 256
     float *out;                // [B, Hq, D]
 };
 
@@ -94,7 +93,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnPara
     const int qpk = p.Hq / p.H;
     const int hq0 = h * qpk + qpass * NQ;
     const int nq_here = min(NQ, qpk - qpass * NQ);
-    const int t0 = chunk * AT_CHUNK, t1 = min(p.T, t0 + AT_CHUNK);
+    const int t0 = chunk * p.chunk, t1 = min(p.T, t0 + p.chunk);
     const long long ctok0 = (long long)b * p.csb + (long long)h * p.csh;
 
     for (int i = tid; i < NQ * D; i += AT_THREADS) {
@@ -121,9 +120,9 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnPara
         }
         __syncwarp();
         const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
-        float acc[NQ];
+        float acc[NQ][4];                                      // four partial sums per query head: independent FMA chains
 #pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) acc[qi] = 0.0f;
+        for (int qi = 0; qi < NQ; ++qi) acc[qi][0] = acc[qi][1] = acc[qi][2] = acc[qi][3] = 0.0f;
 #pragma unroll
         for (int v4 = 0; v4 < WPT / 4; ++v4) {
             const uint4 cw = __ldg(cp + v4);
@@ -138,15 +137,16 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnPara
 #pragma unroll
                     for (int qi = 0; qi < NQ; ++qi) {
                         const float4 qq = *reinterpret_cast<const float4 *>(qsw + qi * D + ch);
-                        acc[qi] = fmaf(f0, qq.x, acc[qi]);
-                        acc[qi] = fmaf(f1, qq.y, acc[qi]);
-                        acc[qi] = fmaf(f2, qq.z, acc[qi]);
-                        acc[qi] = fmaf(f3, qq.w, acc[qi]);
+                        acc[qi][0] = fmaf(f0, qq.x, acc[qi][0]);
+                        acc[qi][1] = fmaf(f1, qq.y, acc[qi][1]);
+                        acc[qi][2] = fmaf(f2, qq.z, acc[qi][2]);
+                        acc[qi][3] = fmaf(f3, qq.w, acc[qi][3]);
                     }
                 }
         }
 #pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) sc[qi * AT_CHUNK + blk - t0 + lane] = acc[qi] + k0[qi];
+        for (int qi = 0; qi < NQ; ++qi)
+            sc[qi * AT_CHUNK + blk - t0 + lane] = ((acc[qi][0] + acc[qi][1]) + (acc[qi][2] + acc[qi][3])) + k0[qi];
     }
     __syncthreads();
 
@@ -200,12 +200,12 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnPara
 #pragma unroll
         for (int i = 0; i < CPW; ++i) accv[qi][i] = 0.0f;
     }
-    const int vbase = t0 + warp * AT_VTOK;
-    const int vend = min(t1, vbase + AT_VTOK);
-    for (int tk = vbase + ts; tk < vend; tk += TPI) {
-        const long long ct = ctok0 + tk;
-        const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(p.vc) + ct * WPT + j);
-        const float vsc = __ldg(p.vs + ct * ng + gidx) * LV, vzr = __ldg(p.vz + ct * ng + gidx);
+    const int vtok = p.chunk / AT_WARPS;
+    const int vbase = t0 + warp * vtok;
+    const int vend = min(t1, vbase + vtok);
+    const uint32_t *vcw = reinterpret_cast<const uint32_t *>(p.vc);
+    auto vstep = [&](int tk, uint32_t w, float vs_raw, float vzr) {
+        const float vsc = vs_raw * LV;
         float a[NQ];
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi) {
@@ -219,6 +219,19 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnPara
 #pragma unroll
             for (int qi = 0; qi < NQ; ++qi) accv[qi][i] = fmaf(f, a[qi], accv[qi][i]);
         }
+    };
+    int tk = vbase + ts;
+    for (; tk + TPI < vend; tk += 2 * TPI) {                    // two steps' loads in flight before either is used
+        const long long c0 = ctok0 + tk, c1 = c0 + TPI;
+        const uint32_t w0 = __ldg(vcw + c0 * WPT + j), w1 = __ldg(vcw + c1 * WPT + j);
+        const float s0 = __ldg(p.vs + c0 * ng + gidx), z0 = __ldg(p.vz + c0 * ng + gidx);
+        const float s1 = __ldg(p.vs + c1 * ng + gidx), z1 = __ldg(p.vz + c1 * ng + gidx);
+        vstep(tk, w0, s0, z0);
+        vstep(tk + TPI, w1, s1, z1);
+    }
+    if (tk < vend) {
+        const long long c0 = ctok0 + tk;
+        vstep(tk, __ldg(vcw + c0 * WPT + j), __ldg(p.vs + c0 * ng + gidx), __ldg(p.vz + c0 * ng + gidx));
     }
     // add the group constant, fold the token classes of the warp, then the warps
     __syncthreads();                                            // everybody is done reading sc: reuse it as [warps][NQ][D]
@@ -304,7 +317,7 @@ int launch_partial(const AttnParams &p, int qpasses, cudaStream_t st)
 
 size_t squat_attention_workspace_floats(int batch, int n_q_heads, int n_tokens)
 {
-    const long long nchunk = (n_tokens + AT_CHUNK - 1) / AT_CHUNK;
+    const long long nchunk = (n_tokens + 255) / 256;             // the smallest chunk the launcher may choose
     return (size_t)batch * n_q_heads * nchunk * (D + 2);
 }
 
@@ -320,7 +333,12 @@ int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq,
     p.kc = kc; p.vc = vc; p.ks = ks; p.kz = kz; p.vs = vs; p.vz = vz; p.csb = csb; p.csh = csh; p.G = G;
     p.k_res = k_res; p.v_res = v_res; p.res_bf16 = res_dtype == SQUAT_BF16; p.R = R;
     p.scale = scale; p.out = out;
-    p.nchunk = (T + AT_CHUNK - 1) / AT_CHUNK;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p.chunk = AT_CHUNK;                                          // smaller chunks while that leaves fewer than ~4 CTAs per SM
+    while (p.chunk > 256 && (long long)batch * H * ((T + p.chunk - 1) / p.chunk) < 4LL * sms) p.chunk /= 2;
+    p.nchunk = (T + p.chunk - 1) / p.chunk;
     p.part = workspace;
     p.ml = workspace + (size_t)batch * Hq * p.nchunk * D;
     const int qpk = Hq / H;
