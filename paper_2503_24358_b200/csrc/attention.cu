@@ -77,7 +77,7 @@ __device__ __forceinline__ float load_elem(const void *p, long long idx, int bf1
 }
 
 template <int BITS, int NQ>
-__global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(const AttnParams p)
+__global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? 3 : 1) attn_partial_kernel(const AttnParams p)
 {
     constexpr int WPT = D * BITS / 32;                          // 32-bit words per token: 8 or 16
     constexpr int CPW = 32 / BITS;                              // codes per word: 16 or 8
