@@ -111,45 +111,45 @@ struct KeyParams {
     int exact_blocks;         // leading 32-channel blocks that no earlier channel corrects (see sweep_block)
 };
 
-// One lane's share of a 32-token x 32-channel block in the trailing-update layout: 4 tokens x 8 channels.
+// One lane's share of a 32-token x 32-channel block in the trailing-update layout: 8 tokens x 4 channels
+// (tokens 8 tr .. 8 tr + 7, channels 4 cr .. 4 cr + 3 with tr = lane >> 3, cr = lane & 7).  The shape is chosen
+// for the shared-memory pipe: 8 consecutive lanes share their token rows, so the two 16-byte reads of the
+// error rows cost 2.5 cycles each instead of 4, and only the one read of W^T has 8 different addresses.
 template <bool BF16>
 struct RawTile {
-    uint4 v[BF16 ? 4 : 8];      // per token: 8 channels = 16 B (bf16) or 32 B (f32)
+    uint2 v[BF16 ? 8 : 16];     // per token: 4 channels = 8 B (bf16) or 16 B (f32)
 };
 
 template <bool BF16>
 __device__ __forceinline__ void load_tile(RawTile<BF16> &r, const void *row0, long long st, int chan)
 {
-    // row0: first of the lane's 4 consecutive tokens; st: token stride in elements; chan: first channel
+    // row0: first of the lane's 8 consecutive tokens; st: token stride in elements; chan: first channel
     if (BF16) {
         const __nv_bfloat16 *p = reinterpret_cast<const __nv_bfloat16 *>(row0) + chan;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) r.v[i] = ldg128(p + i * st);
+        for (int i = 0; i < 8; ++i) r.v[i] = __ldg(reinterpret_cast<const uint2 *>(p + i * st));
     } else {
         const float *p = reinterpret_cast<const float *>(row0) + chan;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            r.v[2 * i] = ldg128(p + i * st);
-            r.v[2 * i + 1] = ldg128(p + i * st + 4);
+        for (int i = 0; i < 8; ++i) {
+            const uint4 t = ldg128(p + i * st);
+            r.v[2 * i] = make_uint2(t.x, t.y);
+            r.v[2 * i + 1] = make_uint2(t.z, t.w);
         }
     }
 }
 
 template <bool BF16>
-__device__ __forceinline__ void unpack_tile(const RawTile<BF16> &r, u64 (&acc)[4][4])
+__device__ __forceinline__ void unpack_tile(const RawTile<BF16> &r, u64 (&acc)[8][2])
 {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 8; ++i) {
         if (BF16) {
             acc[i][0] = pack2(bf16lo_to_f32(r.v[i].x), bf16hi_to_f32(r.v[i].x));
             acc[i][1] = pack2(bf16lo_to_f32(r.v[i].y), bf16hi_to_f32(r.v[i].y));
-            acc[i][2] = pack2(bf16lo_to_f32(r.v[i].z), bf16hi_to_f32(r.v[i].z));
-            acc[i][3] = pack2(bf16lo_to_f32(r.v[i].w), bf16hi_to_f32(r.v[i].w));
         } else {
             acc[i][0] = pack2(__uint_as_float(r.v[2 * i].x), __uint_as_float(r.v[2 * i].y));
-            acc[i][1] = pack2(__uint_as_float(r.v[2 * i].z), __uint_as_float(r.v[2 * i].w));
-            acc[i][2] = pack2(__uint_as_float(r.v[2 * i + 1].x), __uint_as_float(r.v[2 * i + 1].y));
-            acc[i][3] = pack2(__uint_as_float(r.v[2 * i + 1].z), __uint_as_float(r.v[2 * i + 1].w));
+            acc[i][1] = pack2(__uint_as_float(r.v[2 * i + 1].x), __uint_as_float(r.v[2 * i + 1].y));
         }
     }
 }
@@ -281,14 +281,14 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                 float *zr_out = p.zeros + (out_tok0 / G + grp) * D;
                 unsigned char *cp = p.codes + (out_tok0 + tok) * (D * BITS / 8);
 
-                // trailing-update layout: this lane owns tokens 4 tr .. 4 tr + 3 and channels 8 cr .. 8 cr + 7 of a block
-                const int tr = lane >> 2, cr = lane & 3;
+                // trailing-update layout: this lane owns tokens 8 tr .. 8 tr + 7 and channels 4 cr .. 4 cr + 3 of a block
+                const int tr = lane >> 3, cr = lane & 7;
                 const long long row0_off = (long long)b * p.sb + (long long)h * p.sh +
-                                           (long long)(grp * G + wteam * 32 + 4 * tr) * p.st;
+                                           (long long)(grp * G + wteam * 32 + 8 * tr) * p.st;
                 const void *row0 = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row0_off)
                                         : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row0_off);
                 RawTile<BF16> raw;
-                load_tile<BF16>(raw, row0, p.st, 8 * cr);
+                load_tile<BF16>(raw, row0, p.st, 4 * cr);
 
                 for (int blk = 0; blk < NBLK; ++blk) {
                     const float *panel = Wp + (blk * (blk + 1) / 2) * (BLK * BLK);
@@ -297,35 +297,34 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                     {
                         // ---- left-looking update from all earlier channels, as a register-tiled product:
                         //      acc[token][channel pair] = k + sum_j e_j[token] * W^T[j][channel]
-                        u64 acc[4][4];
+                        u64 acc[8][2];
                         unpack_tile<BF16>(raw, acc);
-                        if (blk + 1 < NBLK) load_tile<BF16>(raw, row0, p.st, (blk + 1) * BLK + 8 * cr);   // prefetch
-                        const float *e_ptr = Ew - lane + 4 * tr;          // E[j][4 tr .. 4 tr + 3]
-                        const float *w_ptr = panel + 8 * cr;              // W^T[j][8 cr .. 8 cr + 7]
+                        if (blk + 1 < NBLK) load_tile<BF16>(raw, row0, p.st, (blk + 1) * BLK + 4 * cr);   // prefetch
+                        const float *e_ptr = Ew - lane + 8 * tr;          // E[j][8 tr .. 8 tr + 7]
+                        const float *w_ptr = panel + 4 * cr;              // W^T[j][4 cr .. 4 cr + 3]
                         // software-pipelined over j: the operands of the next 2 steps are loaded while the current 2
                         // steps' 32 packed FMAs issue (warps issue in order, so the loads must be hoisted by hand)
                         constexpr int PF = 2;
-                        float4 ea[PF], eb[PF];
-                        ulonglong2 wa[PF][2], wb[PF][2];
-                        auto loadn = [&](float4 (&ev)[PF], ulonglong2 (&wv)[PF][2], int j0) {
+                        float4 ea[PF][2], eb[PF][2];
+                        ulonglong2 wa[PF], wb[PF];
+                        auto loadn = [&](float4 (&ev)[PF][2], ulonglong2 (&wv)[PF], int j0) {
 #pragma unroll
                             for (int u = 0; u < PF; ++u) {
-                                ev[u] = *reinterpret_cast<const float4 *>(e_ptr + (j0 + u) * 32);
-                                wv[u][0] = *reinterpret_cast<const ulonglong2 *>(w_ptr + (j0 + u) * BLK);
-                                wv[u][1] = *reinterpret_cast<const ulonglong2 *>(w_ptr + (j0 + u) * BLK + 4);
+                                ev[u][0] = *reinterpret_cast<const float4 *>(e_ptr + (j0 + u) * 32);
+                                ev[u][1] = *reinterpret_cast<const float4 *>(e_ptr + (j0 + u) * 32 + 4);
+                                wv[u] = *reinterpret_cast<const ulonglong2 *>(w_ptr + (j0 + u) * BLK);
                             }
                         };
-                        auto fman = [&](const float4 (&ev)[PF], const ulonglong2 (&wv)[PF][2]) {
+                        auto fman = [&](const float4 (&ev)[PF][2], const ulonglong2 (&wv)[PF]) {
 #pragma unroll
                             for (int u = 0; u < PF; ++u) {
-                                const float e[4] = {ev[u].x, ev[u].y, ev[u].z, ev[u].w};
+                                const float e[8] = {ev[u][0].x, ev[u][0].y, ev[u][0].z, ev[u][0].w,
+                                                    ev[u][1].x, ev[u][1].y, ev[u][1].z, ev[u][1].w};
 #pragma unroll
-                                for (int i = 0; i < 4; ++i) {
+                                for (int i = 0; i < 8; ++i) {
                                     const u64 ee = pack2(e[i], e[i]);
-                                    acc[i][0] = ffma2(ee, wv[u][0].x, acc[i][0]);
-                                    acc[i][1] = ffma2(ee, wv[u][0].y, acc[i][1]);
-                                    acc[i][2] = ffma2(ee, wv[u][1].x, acc[i][2]);
-                                    acc[i][3] = ffma2(ee, wv[u][1].y, acc[i][3]);
+                                    acc[i][0] = ffma2(ee, wv[u].x, acc[i][0]);
+                                    acc[i][1] = ffma2(ee, wv[u].y, acc[i][1]);
                                 }
                             }
                         };
@@ -341,18 +340,14 @@ __global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyPar
                         }
                         // ---- transpose to one token per lane through a 4 KB staging tile (the error rows this
                         //      block is about to fill; for the last block, rows 0..31, which nothing reads any more).
-                        //      16-byte chunks are swizzled with the token index so the row reads are conflict-free.
+                        //      16-byte chunks are swizzled with the token index: 8 consecutive lanes write one token's
+                        //      8 chunks (one 128-byte row), 8 consecutive tokens read 8 different chunks.
                         float *stage = Ew - lane + ((blk + 1 < NBLK) ? nprev * 32 : 0);
                         __syncwarp();
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int tok = 4 * tr + i;
-#pragma unroll
-                            for (int v = 0; v < 2; ++v) {
-                                const int phys = (2 * cr + v) ^ (tok & 7);
-                                *reinterpret_cast<ulonglong2 *>(stage + tok * 32 + 4 * phys) =
-                                    make_ulonglong2(acc[i][2 * v], acc[i][2 * v + 1]);
-                            }
+                        for (int i = 0; i < 8; ++i) {
+                            const int tok = 8 * tr + i;
+                            *reinterpret_cast<ulonglong2 *>(stage + tok * 32 + 4 * (cr ^ i)) = make_ulonglong2(acc[i][0], acc[i][1]);
                         }
                         __syncwarp();
 #pragma unroll
