@@ -8,10 +8,10 @@
 //
 //   left-looking trailing update (runtime loop, tiny code):
 //       x_blk[tok][c] = k[tok][c] + sum_{j < block start} e_j[tok] * W[c][j]
-//     a (32 tokens x J) x (J x 32 channels) product, register-tiled: each lane owns 4 tokens x 8
-//     channels, reads 4 errors (one LDS.128 of the [channel][token] error store) and 8 entries of
-//     W^T (two LDS.128) per j and issues 16 packed fma.rn.f32x2 -- 6 shared-memory wavefronts per
-//     j instead of 17 with one token per lane, which would make shared memory the bound.  The tile
+//     a (32 tokens x J) x (J x 32 channels) product, register-tiled: each lane owns 8 tokens x 4
+//     channels, reads 8 errors (two LDS.128 of the [channel][token] error store) and 4 entries of
+//     W^T (one LDS.128) per j and issues 16 packed fma.rn.f32x2 -- 3 shared-memory reads per j
+//     instead of 17 with one token per lane, which would make shared memory the bound.  The tile
 //     is then transposed through shared memory to one token per lane for the sequential part.
 //   in-block triangle (32 channels, unrolled so every register index is static; the same code
 //   serves all 4 blocks):
@@ -50,17 +50,11 @@ __device__ __forceinline__ u64 pack2(float lo, float hi)
 }
 __device__ __forceinline__ float lo_of(u64 v)
 {
-    float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-    (void)hi;
-    return lo;
+    return __uint_as_float((unsigned)(v & 0xffffffffull));
 }
 __device__ __forceinline__ float hi_of(u64 v)
 {
-    float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-    (void)lo;
-    return hi;
+    return __uint_as_float((unsigned)(v >> 32));
 }
 __device__ __forceinline__ u64 ffma2(u64 a, u64 b, u64 c)
 {
