@@ -302,7 +302,8 @@ int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads,
     if (n_tokens > 0 && (!aligned16(k_codes) || !aligned16(k_scales) || !aligned16(k_zeros) || !aligned16(v_codes) ||
                          !aligned16(v_scales) || !aligned16(v_zeros)))
         return SQUAT_ERR_INVALID_ARG;
-    if (n_res > 0 && (!k_res || !v_res || !valid_dtype(res_dtype))) return SQUAT_ERR_INVALID_ARG;
+    if (n_res > 0 && (!k_res || !v_res || !valid_dtype(res_dtype) || !aligned16(k_res) || !aligned16(v_res)))
+        return SQUAT_ERR_INVALID_ARG;
     if (workspace_bytes < squat_decode_attention_workspace_bytes(batch, n_q_heads, n_tokens)) return SQUAT_ERR_INVALID_ARG;
     const float scale = softmax_scale != 0.0f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
     return squat_launch_decode_attention(q, q_dtype, batch, n_q_heads, n_kv_heads, n_tokens, k_codes, k_scales, k_zeros,

@@ -272,13 +272,26 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
     qv[c] = p.scale * load_elem(p.q, ((long long)b * p.Hq + hq) * D + c, p.q_bf16);
     __syncthreads();
     const long long rbase = ((long long)b * p.H + h) * p.R * D;
-    float m = -INFINITY;
-    if (c < p.R) {
-        float s = 0.0f;
-        for (int j = 0; j < D; ++j) s = fmaf(qv[j], load_elem(p.k_res, rbase + (long long)c * D + j, p.res_bf16), s);
-        w[c] = s;
-        m = s;
+    // scores of the residual rows: warp w takes rows w, w + 4, ...; a lane takes 4 neighbouring channels (one 8- or
+    // 16-byte load), so a row is read as one contiguous piece
+    {
+        const int warp = c >> 5, lane = c & 31;
+        const float4 q4 = *reinterpret_cast<const float4 *>(qv + 4 * lane);
+#pragma unroll 4
+        for (int t = warp; t < p.R; t += D / 32) {
+            float4 k4;
+            if (p.res_bf16) {
+                const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(p.k_res) + rbase + (long long)t * D) + lane);
+                k4 = make_float4(bf16lo_to_f32(raw.x), bf16hi_to_f32(raw.x), bf16lo_to_f32(raw.y), bf16hi_to_f32(raw.y));
+            } else {
+                k4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.k_res) + rbase + (long long)t * D) + lane);
+            }
+            const float s = warp_sum_f(fmaf(q4.x, k4.x, fmaf(q4.y, k4.y, fmaf(q4.z, k4.z, q4.w * k4.w))));
+            if (lane == 0) w[t] = s;
+        }
     }
+    __syncthreads();
+    float m = c < p.R ? w[c] : -INFINITY;
     const float *ml = p.ml + ((long long)b * p.Hq + hq) * p.nchunk * 2;
     for (int s = c; s < p.nchunk; s += D) m = fmaxf(m, ml[2 * s]);
     m = warp_max_f(m);
@@ -289,6 +302,7 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
     if (c < p.R) w[c] = expf(w[c] - m);
     __syncthreads();
     float acc = 0.0f, den = 0.0f;
+#pragma unroll 8
     for (int t = 0; t < p.R; ++t) {
         acc = fmaf(w[t], load_elem(p.v_res, rbase + (long long)t * D + c, p.res_bf16), acc);
         den += w[t];
