@@ -59,6 +59,12 @@ def key_flops_per_vector(d, g):
     return 2 * sum(g * (d - t * g) for t in range(1, T))
 
 
+def reader_bytes_per_cached_token(d, bits, G):
+    """What one decode step has to read per cached token: key and value codes, key metadata (fp32 scale and zero
+    per channel, shared by G tokens), value metadata (fp32 scale and zero per group of G channels)."""
+    return 2 * d * bits // 8 + 8 * d // G + 8 * d // G
+
+
 def bytes_per_vector(d, bits, G, elem_bytes):
     """Algorithmic HBM bytes per key (or value) vector: read the vector, write codes + fp32 scale/zero."""
     return d * elem_bytes + d * bits // 8 + 8 * d // G
@@ -418,7 +424,7 @@ def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10):
     ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
     elem = 4 if cfg.dtype == "f32" else 2
     toks = B * H * T
-    nbytes = toks * (2 * d * bits // 8 + 8 * d // G + 8 * d // G) + 2 * B * H * R * d * elem + B * Hq * d * (elem + 4)
+    nbytes = toks * reader_bytes_per_cached_token(d, bits, G) + 2 * B * H * R * d * elem + B * Hq * d * (elem + 4)
     peaks = measured_peaks()
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"what": "squat_decode_attention: softmax(q K^T / sqrt(d)) V over the packed cache + residual buffer",
