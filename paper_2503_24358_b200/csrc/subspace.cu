@@ -190,8 +190,9 @@ constexpr int EIG_MAX_SWEEPS = 40;
 //
 // One head is worked on by a cluster of 4 CTAs (4 SMs per head instead of 1; a 32-head layer then occupies 128
 // of the 148 SMs).  The 128 columns form 8 blocks of 16, and every CTA holds two blocks with ALL their rows, so a
-// rotation of two columns held by the same CTA needs no communication at all: one warp owns the pair (4 rows
-// per lane), the dot product is a warp reduction, and rounds inside a CTA are separated by a CTA barrier only.
+// rotation of two columns held by the same CTA needs no communication at all: a team of 16 lanes owns the pair
+// (8 rows per lane), the dot product is a 4-step shuffle reduction, and rounds inside a CTA are separated by a
+// barrier among the 8 working warps only.
 // A sweep is
 //   one intra phase   15 rounds that pair the columns inside each held block (8 + 8 pairs per round), then
 //   7 block rounds    of 16 rounds each that pair every column of one held block with every column of the other;
