@@ -248,7 +248,7 @@ int grid_for(long long n_threads, int block)
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     long long blocks = (n_threads + block - 1) / block;
-    const long long cap = (long long)sms * 8;           // a multiple of the SM count; grid-stride covers the rest
+    const long long cap = (long long)sms * 32;          // a multiple of the SM count; grid-stride covers the rest
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     return (int)blocks;
