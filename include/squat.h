@@ -47,6 +47,7 @@ typedef enum { SQUAT_KEYS = 0, SQUAT_VALUES = 1 } squat_kind;
 #define SQUAT_FLAG_NONFINITE   1u   /* a scale came out NaN/Inf: non-finite input                  */
 #define SQUAT_FLAG_ZERO_RANGE  2u   /* some group had max == min (scale 0, all codes 0)            */
 #define SQUAT_FLAG_NO_CONVERGE 4u   /* eigensolver hit its sweep limit for some head               */
+#define SQUAT_FLAG_DEVICE_TIMEOUT 8u /* a bounded wait inside a kernel ran out; outputs are invalid     */
 
 /* Opaque per-layer state: the update matrices of every KV head (shared by all samples of a
  * batch, Appendix C) plus the scratch the subspace build needs.  Owns device memory. */

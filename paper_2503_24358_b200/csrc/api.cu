@@ -105,6 +105,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     size_t off = 0;
     auto carve = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
     const size_t o_wt = carve(hdd * sizeof(float));
+    const size_t o_img = carve(hdd * sizeof(float));
     const size_t o_gram = carve(hdd * sizeof(double));
     const size_t o_part = carve(hdd * sizeof(double) * s->gram_chunks_cap);
     const size_t o_val = carve((size_t)n_kv_heads * D * sizeof(double));
@@ -114,6 +115,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     if (cudaMalloc(&base, off) != cudaSuccess) { cudaGetLastError(); delete s; return SQUAT_ERR_ALLOC; }
     if (cudaMemset(base, 0, off) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
     s->Wt = reinterpret_cast<float *>(base + o_wt);
+    s->Wimg = reinterpret_cast<float *>(base + o_img);
     s->gram = reinterpret_cast<double *>(base + o_gram);
     s->gram_partial = reinterpret_cast<double *>(base + o_part);
     s->eigval = reinterpret_cast<double *>(base + o_val);
@@ -212,6 +214,8 @@ int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
     const int exact = (uncorrected + 31) / 32;
     s->exact_blocks = exact;
     SQUAT_CUDA(cudaMemcpyAsync(s->Wt, wt.data(), hdd * sizeof(float), cudaMemcpyHostToDevice, st));
+    int rc = squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, st);
+    if (rc != SQUAT_OK) return rc;
     SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;
 }
@@ -231,7 +235,7 @@ int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int b
     if (n_tokens % group_size != 0 || out_stride_b % group_size != 0 || out_stride_h % group_size != 0)
         return SQUAT_ERR_SHAPE;
     if (batch == 0 || n_tokens == 0) return SQUAT_OK;
-    return squat_launch_quant_keys(s->Wt, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
+    return squat_launch_quant_keys(s->Wimg, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
                                    group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status, s->exact_blocks,
                                    static_cast<cudaStream_t>(stream));
 }

@@ -4,29 +4,36 @@
 //
 // Mapping.  A group is G consecutive tokens of one (batch, head); its channels must be visited in
 // order, and each channel's grid needs min/max over the group's tokens.  So: lane = token, one warp
-// (G = 32) or a team of G/32 warps per group.  The 128 channels are processed in 4 blocks of 32:
+// (G = 32) or a team of G/32 warps per group.  The 128 channels are processed in 4 blocks of 32.
 //
-//   left-looking trailing update (runtime loop, tiny code):
-//       x_blk[tok][c] = k[tok][c] + sum_{j < block start} e_j[tok] * W[c][j]
-//     a (32 tokens x J) x (J x 32 channels) product, register-tiled: each lane owns 8 tokens x 4
-//     channels, reads 8 errors (two LDS.128 of the [channel][token] error store) and 4 entries of
-//     W^T (one LDS.128) per j and issues 16 packed fma.rn.f32x2 -- 3 shared-memory reads per j
-//     instead of 17 with one token per lane, which would make shared memory the bound.  The tile
-//     is then transposed through shared memory to one token per lane for the sequential part.
-//   in-block triangle (32 channels, unrolled so every register index is static; the same code
-//   serves all 4 blocks):
+//   sequential sweep of a block (CUDA cores; 32 channels, unrolled so every register index is static):
 //       m, M  = warp min / max (redux.sync on f32)         -> scale = (M-m)/L, zero = m
 //       c     = rint((x_j - m)/scale), decided exactly through the remainder c*scale - (x_j - m)
 //       e     = fma(c, scale, -(x_j - m))                   (= deq(qtz(x_j)) - x_j)
-//       x_j' += e * W[j'][j]  for the later channels j' of the block; e goes to shared memory.
+//       x_j' += e * W[j'][j]  for the later channels j' of the block (the diagonal 32 x 32 block of W^T,
+//       read from shared memory as broadcast 16-byte loads, applied with packed fma.rn.f32x2)
 //
-// The update matrix of the CTA's current head is kept in shared memory as 4 column panels
-// (panel b = W^T[0 .. 32b+31][32b .. 32b+31], 40 KB in all: only the lower triangle is ever read).
-// CTAs are persistent: each takes a contiguous range of groups ordered head-major, so W is
-// reloaded only when the range crosses a head.  14 warps per SM x 2 rounds cover the 27.7 groups
-// per SM of the 32-head x 4096-token workload.
+//   update of the later blocks (tcgen05 tensor cores): three quarters of the multiply-adds are the
+//   dense contractions (tokens x 32 errors) x (32 x later channels).  A tile is 128 tokens' worth of
+//   groups worked by 4 warps: row m of the tile = lane (m % 32) of the warp with warp % 4 == m / 32 =
+//   tensor-memory lane m.  Tensor memory holds, per tile, the fp32 accumulator D[128 x 96] of the
+//   corrections to channels 32 .. 127.  After the sweep of block b each warp writes its errors to
+//   shared memory as the tile's A operand (K-major 8 x 16-byte core matrices): the raw fp32 words
+//   serve as E_hi (the tensor core reads the top 19 bits of a word: tf32 by truncation) and
+//   E_lo = e - trunc(e) is exact in fp32.  The last of the tile's 4 warps to get there issues
+//        D[:, 32 b .. 95] (+)= E_lo * Whi_b + E_hi * Wlo_b + E_hi * Whi_b     (12 MMAs of 128 x (96 - 32 b) x 8)
+//   with W^T's off-diagonal panels split into tf32 hi / lo the same way (small terms first within a
+//   block: the accumulator truncates on every add) and commits them to the tile's mbarrier; nobody
+//   waits at a CTA or tile barrier.  Before the next sweep each warp waits for that phase (bounded),
+//   reads its 32 columns of D with tcgen05.ld -- one token per lane, no transpose -- and adds the keys.
 //
-// Work per key vector: 8128 fp32 FMA (dense triangle, g = 1) -> bound by the FP32 pipes, not HBM.
+// Per head the CTA stages 64 KB in shared memory: the four diagonal blocks (fp32) and the three
+// hi / lo panels, copied as they are from the image that pack_w_kernel writes when the update
+// matrices are built or imported.  CTAs are persistent over rounds (= 4 consecutive tiles of one head,
+// one per tile slot), taken in contiguous ranges so that a head is staged once per CTA that touches it.
+//
+// Work per key vector: 8128 fp32 multiply-adds (dense triangle, g = 1): 2032 on the CUDA cores
+// (sweeps), 6096 x 3 tf32 products on the tensor cores.
 #include "squat_internal.cuh"
 
 namespace {
@@ -34,11 +41,23 @@ namespace {
 constexpr int D = SQUAT_D;
 constexpr int BLK = 32;                   // channels per block
 constexpr int NBLK = D / BLK;             // 4
-constexpr int PANEL_FLOATS = BLK * BLK * (NBLK * (NBLK + 1) / 2);   // 10 blocks of 32 x 32
-constexpr int E_ROWS = D - BLK;           // errors of the last block are never read
 constexpr float kMagic = 12582912.0f;     // 1.5 * 2^23
-constexpr int KEY_WARPS = 14;
-constexpr int KEY_THREADS = KEY_WARPS * 32;
+
+constexpr int TC_SLOTS = 4;                          // 128-token tiles in flight per CTA
+constexpr int TC_WARPS = TC_SLOTS * 4;
+constexpr int TC_THREADS = TC_WARPS * 32;
+constexpr int TC_COLS_PER_TILE = 128;                // 96 used: channels 32 .. 127
+constexpr int TC_TMEM_COLS = 512;
+static_assert(TC_SLOTS * TC_COLS_PER_TILE <= TC_TMEM_COLS, "tensor memory has 512 columns");
+constexpr int TC_E_FLOATS = 128 * BLK;               // one tile's E_hi (or E_lo): 128 rows x 32 channels
+constexpr int TC_DIAG_FLOATS = NBLK * BLK * BLK;     // four 32 x 32 diagonal blocks of W^T
+constexpr int TC_PANEL_FLOATS = BLK * (3 * BLK + 2 * BLK + BLK);     // panels of source blocks 0..2: (96 - 32 b) x 32
+constexpr int TC_IMG_FLOATS = TC_DIAG_FLOATS + 2 * TC_PANEL_FLOATS;  // = d * d: diag | hi panels | lo panels
+static_assert(TC_IMG_FLOATS == D * D, "the staged image of W has the size of W");
+constexpr unsigned TC_A_LBO = 128 * 16, TC_SBO = 128;                 // bytes
+__host__ __device__ constexpr int tc_panel_off(int b) { return b == 0 ? 0 : (b == 1 ? 3 * BLK * BLK : 5 * BLK * BLK); }
+// instruction descriptor: fp32 accumulator, tf32 A and B, both K-major, N = n, M = 128
+__host__ __device__ constexpr unsigned tc_idesc(int n) { return (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(n >> 3) << 17) | ((128u >> 4) << 24); }
 
 typedef unsigned long long u64;
 
@@ -91,8 +110,59 @@ __device__ __forceinline__ float div_by_levels(float rng)
     return __fmaf_rn(r, invL, q);
 }
 
+// ---- tcgen05 / tensor-memory helpers (5th-generation tensor cores) -------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void *ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
+__device__ __forceinline__ unsigned tf32_of(float x)             // round to nearest tf32 (10 mantissa bits)
+{
+    unsigned r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+// 32 consecutive columns of the warp's lanes into registers (lane l gets row l)
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// shared-memory matrix descriptor, no swizzle, K-major: 8 x 16-byte core matrices, lbo bytes between the two
+// halves of a K step, sbo bytes between groups of 8 rows
+__device__ __forceinline__ u64 umma_desc(unsigned addr, unsigned lbo, unsigned sbo)
+{
+    return (u64)((addr & 0x3FFFF) >> 4) | ((u64)(lbo >> 4) << 16) | ((u64)(sbo >> 4) << 32) | (1ull << 46);
+}
+// D[128 x N] (+)= A[128 x 8] * B[N x 8]^T, tf32 operands from shared memory, fp32 accumulation in tensor memory
+__device__ __forceinline__ void umma_tf32_ss(unsigned d_taddr, u64 a_desc, u64 b_desc, unsigned idesc, unsigned accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_taddr), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned mbar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
+}
+// Bounded wait for a phase of an mbarrier: false when the limit ran out (the caller records it and moves on).
+__device__ __forceinline__ bool mbar_wait(unsigned mbar, unsigned parity)
+{
+    for (int it = 0; it < (1 << 22); ++it) {
+        unsigned done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(mbar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
 struct KeyParams {
-    const float *Wt;          // [H, D, D] transposed update matrices: Wt[j][j'] = W[j'][j]
+    const float *Wimg;        // [H, d * d] staged images of the update matrices (pack_w_kernel)
     const void *k;
     long long sb, sh, st;     // element strides of k
     unsigned char *codes;
@@ -100,57 +170,47 @@ struct KeyParams {
     long long osb, osh;       // output strides in tokens
     int B, H, T;
     int groups_per_bh;        // T / G
-    long long total_groups;   // H * B * groups_per_bh, ordered (h, b, grp)
     unsigned *status;
     int exact_blocks;         // leading 32-channel blocks that no earlier channel corrects (see sweep_block)
 };
 
-// One lane's share of a 32-token x 32-channel block in the trailing-update layout: 8 tokens x 4 channels
-// (tokens 8 tr .. 8 tr + 7, channels 4 cr .. 4 cr + 3 with tr = lane >> 3, cr = lane & 7).  The shape is chosen
-// for the shared-memory pipe: 8 consecutive lanes share their token rows, so the two 16-byte reads of the
-// error rows cost 2.5 cycles each instead of 4, and only the one read of W^T has 8 different addresses.
 template <bool BF16>
-struct RawTile {
-    uint2 v[BF16 ? 8 : 16];     // per token: 4 channels = 8 B (bf16) or 16 B (f32)
+struct RawRow {
+    uint4 v[BF16 ? 4 : 8];      // 32 channels of one token
 };
-
 template <bool BF16>
-__device__ __forceinline__ void load_tile(RawTile<BF16> &r, const void *row0, long long st, int chan)
+__device__ __forceinline__ void load_row(RawRow<BF16> &r, const void *row, int chan)
 {
-    // row0: first of the lane's 8 consecutive tokens; st: token stride in elements; chan: first channel
     if (BF16) {
-        const __nv_bfloat16 *p = reinterpret_cast<const __nv_bfloat16 *>(row0) + chan;
+        const uint4 *q = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(row) + chan);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) r.v[i] = __ldg(reinterpret_cast<const uint2 *>(p + i * st));
+        for (int i = 0; i < 4; ++i) r.v[i] = __ldg(q + i);
     } else {
-        const float *p = reinterpret_cast<const float *>(row0) + chan;
+        const uint4 *q = reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(row) + chan);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint4 t = ldg128(p + i * st);
-            r.v[2 * i] = make_uint2(t.x, t.y);
-            r.v[2 * i + 1] = make_uint2(t.z, t.w);
-        }
+        for (int i = 0; i < 8; ++i) r.v[i] = __ldg(q + i);
     }
 }
-
+// channel pair q (channels 2q, 2q + 1) of the row as two floats
 template <bool BF16>
-__device__ __forceinline__ void unpack_tile(const RawTile<BF16> &r, u64 (&acc)[8][2])
+__device__ __forceinline__ float2 row_pair(const RawRow<BF16> &r, int q)
 {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        if (BF16) {
-            acc[i][0] = pack2(bf16lo_to_f32(r.v[i].x), bf16hi_to_f32(r.v[i].x));
-            acc[i][1] = pack2(bf16lo_to_f32(r.v[i].y), bf16hi_to_f32(r.v[i].y));
-        } else {
-            acc[i][0] = pack2(__uint_as_float(r.v[2 * i].x), __uint_as_float(r.v[2 * i].y));
-            acc[i][1] = pack2(__uint_as_float(r.v[2 * i + 1].x), __uint_as_float(r.v[2 * i + 1].y));
-        }
+    if (BF16) {
+        const uint4 &t = r.v[q >> 2];
+        const unsigned w = (q & 3) == 0 ? t.x : (q & 3) == 1 ? t.y : (q & 3) == 2 ? t.z : t.w;
+        return make_float2(bf16lo_to_f32(w), bf16hi_to_f32(w));
+    } else {
+        const uint4 &t = r.v[q >> 1];
+        return (q & 1) ? make_float2(__uint_as_float(t.z), __uint_as_float(t.w))
+                       : make_float2(__uint_as_float(t.x), __uint_as_float(t.y));
     }
 }
 
 // The sequential part: the 32 channels of one block, one token per lane, values in xp (16 packed pairs).
 // For every channel: grid from the warp (team) min / max, rounding decision, error e; e is pushed onto the
-// later channels of the block through the diagonal 32 x 32 block of W^T and stored for the later blocks.
+// later channels of the block through the diagonal 32 x 32 block of W^T and written, 4 channels at a time, to
+// this lane's row of the tile's A operands (e_hi, e_lo: 4 floats per 4-channel chunk, chunks TC_A_LBO bytes
+// apart) for the tensor-core update of the later blocks.
 //
 // Rounding decision.  t = (x - m) / scale is formed as (x - m) * L * rcp(M - m) with the hardware reciprocal,
 // so c0 = rint(t) can be off by one when t is within ~1e-6 of a rounding midpoint.  Channels that earlier
@@ -161,22 +221,23 @@ __device__ __forceinline__ void unpack_tile(const RawTile<BF16> &r, u64 (&acc)[8
 // +-scale/2: that settles the rounding exactly as real arithmetic on the stored float32 scale would, ties
 // going to the even code (the threshold of an odd c0 is one ulp lower, so "remainder == scale/2" moves it).
 template <int BITS, int NW, bool EXACT>
-__device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, float *Eblk, bool store_e,
-                                            int lane, int team, int wteam, float2 *red, float2 *park,
+__device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, float *e_hi, float *e_lo, bool store_e,
+                                            int lane, int bar_id, int wteam, float2 *red, float2 *park,
                                             uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
 {
     constexpr float L = float((1 << BITS) - 1);
     constexpr int PER_ACC = 16 / BITS;              // codes accumulated exactly in one float (16 bits of mantissa)
     float cacc[BLK / PER_ACC];
+    float eh[4], el[4];
 #pragma unroll
     for (int jj = 0; jj < BLK; ++jj) {
         const float xj = (jj & 1) ? hi_of(xp[jj >> 1]) : lo_of(xp[jj >> 1]);
         float m = warp_min(xj);
         float Mx = warp_max(xj);
         if (NW > 1) {
-            float2 *slot = red + (team * 2 + (jj & 1)) * NW;
+            float2 *slot = red + (jj & 1) * NW;             // [parity][warp of the team]
             if (lane == 0) slot[wteam] = make_float2(m, Mx);
-            team_barrier(1 + team, 32 * NW);
+            team_barrier(bar_id, 32 * NW);
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
                 const float2 o = slot[w];
@@ -203,7 +264,14 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         if (jj % PER_ACC == 0) cacc[jj / PER_ACC] = c;
         else cacc[jj / PER_ACC] = __fmaf_rn(c, float(1 << ((jj % PER_ACC) * BITS)), cacc[jj / PER_ACC]);
         park[jj] = make_float2(scale, m);               // same value from every lane; lane jj picks it up below
-        if (store_e) Eblk[jj * 32] = e;
+        // tf32 split by truncation: the tensor core reads only the top 19 bits of each word, so e itself serves
+        // as E_hi = trunc(e), and E_lo = e - trunc(e) is exact in fp32
+        eh[jj & 3] = e;
+        el[jj & 3] = __fsub_rn(e, __uint_as_float(__float_as_uint(e) & 0xffffe000u));
+        if ((jj & 3) == 3 && store_e) {
+            *reinterpret_cast<float4 *>(e_hi + (jj >> 2) * (TC_A_LBO / 4)) = make_float4(eh[0], eh[1], eh[2], eh[3]);
+            *reinterpret_cast<float4 *>(e_lo + (jj >> 2) * (TC_A_LBO / 4)) = make_float4(el[0], el[1], el[2], el[3]);
+        }
         const u64 ee = pack2(e, e);
         const float *wrow = diag + jj * BLK;
 #pragma unroll
@@ -223,162 +291,253 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         cw[w] = (uint32_t)__float2int_rn(cacc[2 * w]) | ((uint32_t)__float2int_rn(cacc[2 * w + 1]) << 16);
 }
 
+// Where one warp's 32 tokens of a round live.
+struct TileRows {
+    bool valid;               // the warp's slot has a tile in this round
+    bool active;              // ... and the warp's group exists (a head's last tile may be ragged: its spare warps redo the
+                              // last group and store nothing)
+    int tok, grp;
+    long long out_tok0;
+    const void *row;          // this lane's key vector
+};
+
 template <int BITS, int NW, bool BF16>
-__global__ void __launch_bounds__(KEY_THREADS, 1) quant_keys_kernel(const KeyParams p)
+__global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyParams p)
 {
     constexpr int G = 32 * NW;
-    constexpr int NTEAMS = KEY_WARPS / NW;
+    constexpr int GPT = 4 / NW;                          // groups per tile
+    constexpr int NTEAMS = TC_SLOTS * GPT;               // teams of NW warps
     constexpr int WORDS_PER_BLK = BLK * BITS / 32;       // 2 (2-bit) or 4 (4-bit)
-    extern __shared__ __align__(16) float smem[];
-    float *Wp = smem;                                    // 4 column panels, PANEL_FLOATS
-    float *Eall = smem + PANEL_FLOATS;                   // [KEY_WARPS][E_ROWS][32]
-    float2 *red = reinterpret_cast<float2 *>(Eall + KEY_WARPS * E_ROWS * 32);   // [NTEAMS][2][NW]
-    float2 *park = red + NTEAMS * 2 * NW + (threadIdx.x >> 5) * BLK;             // [KEY_WARPS][BLK] (scale, zero) of a block
+    extern __shared__ __align__(128) float smem[];
+    float *Eall = smem;                                  // [TC_SLOTS][hi, lo][TC_E_FLOATS]
+    float *diag_all = Eall + TC_SLOTS * 2 * TC_E_FLOATS; // [NBLK][32][32], then the hi panels, then the lo panels
+    float *Bhi = diag_all + TC_DIAG_FLOATS;              // panels of source blocks 0, 1, 2
+    float *Blo = Bhi + TC_PANEL_FLOATS;
+    float2 *red_all = reinterpret_cast<float2 *>(Blo + TC_PANEL_FLOATS);         // [NTEAMS][2][NW]
+    float2 *park = red_all + NTEAMS * 2 * NW + (threadIdx.x >> 5) * BLK;         // [TC_WARPS][BLK] (scale, zero) of a block
+    u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW + TC_WARPS * BLK);   // [TC_SLOTS]
+    // [0] tensor-memory base, [1] a bounded wait ran out, [2 + slot] arrivals of the slot's warps
+    volatile unsigned *shared_words = reinterpret_cast<volatile unsigned *>(mbar + TC_SLOTS);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int team = warp / NW;
-    const int wteam = warp % NW;
-    float *Ew = Eall + warp * (E_ROWS * 32) + lane;      // this lane's column of the warp's error store
+    const int slot = warp >> 2;                          // tile slot of this warp
+    const int wq = warp & 3;                             // its quarter of the tile = its tensor-memory lanes
+    const int team = slot * GPT + wq / NW;
+    const int wteam = wq % NW;
+    float2 *red = red_all + team * (2 * NW);
 
-    const long long lo = p.total_groups * blockIdx.x / gridDim.x;
-    const long long hi = p.total_groups * (blockIdx.x + 1) / gridDim.x;
-    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
-
-    long long pos = lo;
-    while (pos < hi) {
-        const int h = (int)(pos / groups_per_head);
-        long long seg_end = (long long)(h + 1) * groups_per_head;
-        if (seg_end > hi) seg_end = hi;
-
-        __syncthreads();                                 // everyone is done with the previous head's W
-        {
-            // panel cb holds rows j = 0 .. 32 cb + 31 of W^T restricted to columns 32 cb .. 32 cb + 31
-            const float *src = p.Wt + (long long)h * D * D;
-            for (int i = threadIdx.x; i < PANEL_FLOATS / 4; i += KEY_THREADS) {
-                int f = i * 4, cb = 0;
-                while (f >= BLK * BLK * (cb + 1)) { f -= BLK * BLK * (cb + 1); ++cb; }
-                const int j = f / BLK, c = f % BLK;
-                reinterpret_cast<float4 *>(Wp)[i] = __ldg(reinterpret_cast<const float4 *>(src + j * D + cb * BLK + c));
-            }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<unsigned *>(shared_words))), "r"((unsigned)TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 32) {
+#pragma unroll
+        for (int t = 0; t < TC_SLOTS; ++t) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(mbar + t)), "r"(1) : "memory");
+            shared_words[2 + t] = 0;
         }
-        __syncthreads();
+        shared_words[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = shared_words[0];
+    const unsigned t_tile = tmem_base + slot * TC_COLS_PER_TILE;               // lane field 0: the MMAs' accumulator
+    const unsigned t_mine = t_tile + ((unsigned)(wq * 32) << 16);              // this warp's 32 lanes
+    float *e_hi = Eall + slot * 2 * TC_E_FLOATS + (wq * 32 + lane) * 4;        // this lane's row of the tile's A operands
+    float *e_lo = e_hi + TC_E_FLOATS;
+    const unsigned a_hi = smem_u32(Eall + slot * 2 * TC_E_FLOATS), a_lo = a_hi + TC_E_FLOATS * 4;
+    const unsigned my_mbar = smem_u32(mbar + slot);
+    unsigned phase = 0;
 
-        if (team < NTEAMS) {
-            for (long long gi = pos + team; gi < seg_end; gi += NTEAMS) {
-                const long long in_head = gi - (long long)h * groups_per_head;
-                const int b = (int)(in_head / p.groups_per_bh);
-                const int grp = (int)(in_head % p.groups_per_bh);
-                const int tok = grp * G + wteam * 32 + lane;
-                const long long out_tok0 = (long long)b * p.osb + (long long)h * p.osh;
-                float *sc_out = p.scales + (out_tok0 / G + grp) * D;
-                float *zr_out = p.zeros + (out_tok0 / G + grp) * D;
-                unsigned char *cp = p.codes + (out_tok0 + tok) * (D * BITS / 8);
+    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
+    const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
+    // Work unit of a CTA: a round = TC_SLOTS consecutive tiles of one head, one per slot.  CTAs take contiguous
+    // ranges of rounds, so a head's update matrix is staged once per CTA that touches the head and no CTA's
+    // slots are split unevenly by a head boundary.
+    const long long rounds_per_head = (tiles_per_head + TC_SLOTS - 1) / TC_SLOTS;
+    const long long total_rounds = rounds_per_head * p.H;
+    const long long lo = total_rounds * blockIdx.x / gridDim.x;
+    const long long hi = total_rounds * (blockIdx.x + 1) / gridDim.x;
 
-                // trailing-update layout: this lane owns tokens 8 tr .. 8 tr + 7 and channels 4 cr .. 4 cr + 3 of a block
-                const int tr = lane >> 3, cr = lane & 7;
-                const long long row0_off = (long long)b * p.sb + (long long)h * p.sh +
-                                           (long long)(grp * G + wteam * 32 + 8 * tr) * p.st;
-                const void *row0 = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row0_off)
-                                        : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row0_off);
-                RawTile<BF16> raw;
-                load_tile<BF16>(raw, row0, p.st, 4 * cr);
+    auto locate = [&](long long rnd, TileRows &t) {
+        const int h = (int)(rnd / rounds_per_head);
+        const long long ti = (rnd - (long long)h * rounds_per_head) * TC_SLOTS + slot;   // tile within the head
+        t.valid = ti < tiles_per_head;
+        const long long g_raw = ti * GPT + wq / NW;
+        t.active = t.valid && g_raw < groups_per_head;
+        const long long in_head = g_raw < groups_per_head ? g_raw : groups_per_head - 1;
+        const int b = (int)(in_head / p.groups_per_bh);
+        t.grp = (int)(in_head % p.groups_per_bh);
+        t.tok = t.grp * G + wteam * 32 + lane;
+        t.out_tok0 = (long long)b * p.osb + (long long)h * p.osh;
+        const long long row_off = (long long)b * p.sb + (long long)h * p.sh + (long long)t.tok * p.st;
+        t.row = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row_off)
+                     : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row_off);
+    };
 
-                for (int blk = 0; blk < NBLK; ++blk) {
-                    const float *panel = Wp + (blk * (blk + 1) / 2) * (BLK * BLK);
-                    const int nprev = blk * BLK;
-                    u64 xp[BLK / 2];
-                    {
-                        // ---- left-looking update from all earlier channels, as a register-tiled product:
-                        //      acc[token][channel pair] = k + sum_j e_j[token] * W^T[j][channel]
-                        u64 acc[8][2];
-                        unpack_tile<BF16>(raw, acc);
-                        if (blk + 1 < NBLK) load_tile<BF16>(raw, row0, p.st, (blk + 1) * BLK + 4 * cr);   // prefetch
-                        const float *e_ptr = Ew - lane + 8 * tr;          // E[j][8 tr .. 8 tr + 7]
-                        const float *w_ptr = panel + 4 * cr;              // W^T[j][4 cr .. 4 cr + 3]
-                        // software-pipelined over j: the operands of the next 2 steps are loaded while the current 2
-                        // steps' 32 packed FMAs issue (warps issue in order, so the loads must be hoisted by hand)
-                        constexpr int PF = 2;
-                        float4 ea[PF][2], eb[PF][2];
-                        ulonglong2 wa[PF], wb[PF];
-                        auto loadn = [&](float4 (&ev)[PF][2], ulonglong2 (&wv)[PF], int j0) {
+    TileRows cur, nxt;
+    RawRow<BF16> raw;
+    cur.valid = false;
+    if (lo < hi) {
+        locate(lo, cur);
+        if (cur.valid) load_row<BF16>(raw, cur.row, 0);  // in flight while the first head is staged
+    }
+    int cur_head = -1;
+    for (long long rnd = lo; rnd < hi; ++rnd) {
+        const int h = (int)(rnd / rounds_per_head);
+        if (h != cur_head) {
+            cur_head = h;
+            __syncthreads();                             // every MMA that read the previous head's panels has been waited for
+            const float4 *src = reinterpret_cast<const float4 *>(p.Wimg + (long long)h * TC_IMG_FLOATS);
+            float4 *dst = reinterpret_cast<float4 *>(diag_all);
+            constexpr int PER_THREAD = TC_IMG_FLOATS / 4 / TC_THREADS;     // 8
+            float4 t[PER_THREAD];
 #pragma unroll
-                            for (int u = 0; u < PF; ++u) {
-                                ev[u][0] = *reinterpret_cast<const float4 *>(e_ptr + (j0 + u) * 32);
-                                ev[u][1] = *reinterpret_cast<const float4 *>(e_ptr + (j0 + u) * 32 + 4);
-                                wv[u] = *reinterpret_cast<const ulonglong2 *>(w_ptr + (j0 + u) * BLK);
-                            }
-                        };
-                        auto fman = [&](const float4 (&ev)[PF][2], const ulonglong2 (&wv)[PF]) {
+            for (int i = 0; i < PER_THREAD; ++i) t[i] = __ldg(src + i * TC_THREADS + threadIdx.x);
 #pragma unroll
-                            for (int u = 0; u < PF; ++u) {
-                                const float e[8] = {ev[u][0].x, ev[u][0].y, ev[u][0].z, ev[u][0].w,
-                                                    ev[u][1].x, ev[u][1].y, ev[u][1].z, ev[u][1].w};
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const u64 ee = pack2(e[i], e[i]);
-                                    acc[i][0] = ffma2(ee, wv[u].x, acc[i][0]);
-                                    acc[i][1] = ffma2(ee, wv[u].y, acc[i][1]);
-                                }
-                            }
-                        };
-                        if (nprev > 0) {
-                            loadn(ea, wa, 0);
+            for (int i = 0; i < PER_THREAD; ++i) dst[i * TC_THREADS + threadIdx.x] = t[i];
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor core reads the panels through the async proxy
+            __syncthreads();
+        }
+        nxt.valid = false;
+        if (rnd + 1 < hi) locate(rnd + 1, nxt);
+
+        if (cur.valid) {
 #pragma unroll 1
-                            for (int j = 0; j < nprev; j += 2 * PF) {        // nprev is a multiple of 32
-                                loadn(eb, wb, j + PF);
-                                fman(ea, wa);
-                                loadn(ea, wa, (j + 2 * PF < nprev) ? j + 2 * PF : j);   // last reload: redundant, in range
-                                fman(eb, wb);
-                            }
-                        }
-                        // ---- transpose to one token per lane through a 4 KB staging tile (the error rows this
-                        //      block is about to fill; for the last block, rows 0..31, which nothing reads any more).
-                        //      16-byte chunks are swizzled with the token index: 8 consecutive lanes write one token's
-                        //      8 chunks (one 128-byte row), 8 consecutive tokens read 8 different chunks.
-                        float *stage = Ew - lane + ((blk + 1 < NBLK) ? nprev * 32 : 0);
-                        __syncwarp();
+            for (int blk = 0; blk < NBLK; ++blk) {
+                u64 xp[BLK / 2];
+                if (blk == 0) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int tok = 8 * tr + i;
-                            *reinterpret_cast<ulonglong2 *>(stage + tok * 32 + 4 * (cr ^ i)) = make_ulonglong2(acc[i][0], acc[i][1]);
-                        }
-                        __syncwarp();
-#pragma unroll
-                        for (int q = 0; q < BLK / 4; ++q) {
-                            const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(stage + lane * 32 + 4 * (q ^ (lane & 7)));
-                            xp[2 * q] = v.x;
-                            xp[2 * q + 1] = v.y;
-                        }
-                        __syncwarp();
+                    for (int q = 0; q < BLK / 2; ++q) {
+                        const float2 kv = row_pair<BF16>(raw, q);
+                        xp[q] = pack2(kv.x, kv.y);
                     }
+                } else {
+                    // the MMAs that complete this block's corrections were committed after the previous sweep
+                    if (!shared_words[1] && !mbar_wait(my_mbar, phase)) {
+                        shared_words[1] = 1;
+                        atomicOr(p.status, SQUAT_FLAG_DEVICE_TIMEOUT);
+                    }
+                    phase ^= 1;
+                    tc_fence_after();
+                    unsigned dv[32];
+                    tmem_ld32(t_mine + (blk - 1) * BLK, dv);
+#pragma unroll
+                    for (int q = 0; q < BLK / 2; ++q) {
+                        const float2 kv = row_pair<BF16>(raw, q);
+                        xp[q] = pack2(__fadd_rn(kv.x, __uint_as_float(dv[2 * q])), __fadd_rn(kv.y, __uint_as_float(dv[2 * q + 1])));
+                    }
+                }
+                const bool more = blk + 1 < NBLK;
+                // prefetch: the next block of this tile, or the first block of the next round's tile
+                if (more) load_row<BF16>(raw, cur.row, (blk + 1) * BLK);
+                else if (nxt.valid) load_row<BF16>(raw, nxt.row, 0);
 
-                    // ---- sequential sweep over the block's 32 channels ------------------------
-                    const float *diag = panel + nprev * BLK;
-                    float *Eblk = Ew + nprev * 32;
-                    uint32_t cw[WORDS_PER_BLK];
-                    float my_scale = 0.0f, my_zero = 0.0f;
-                    if (blk < p.exact_blocks)
-                        sweep_block<BITS, NW, true>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, park, cw, my_scale, my_zero);
-                    else
-                        sweep_block<BITS, NW, false>(xp, diag, Eblk, blk + 1 < NBLK, lane, team, wteam, red, park, cw, my_scale, my_zero);
+                const float *diag = diag_all + blk * BLK * BLK;
+                uint32_t cw[WORDS_PER_BLK];
+                float my_scale = 0.0f, my_zero = 0.0f;
+                if (blk < p.exact_blocks)
+                    sweep_block<BITS, NW, true>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, park, cw, my_scale, my_zero);
+                else
+                    sweep_block<BITS, NW, false>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, park, cw, my_scale, my_zero);
 
-                    // ---- this block's outputs -----------------------------------------------
+                if (more) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the error rows, for the tensor core
+                    tc_fence_before();
+                    __threadfence_block();
+                    __syncwarp();
+                    // the last of the slot's four warps to get here issues the MMAs; nobody waits at a barrier
+                    bool last = false;
+                    if (lane == 0) last = (atomicAdd(const_cast<unsigned *>(shared_words) + 2 + slot, 1u) & 3u) == 3u;
+                    if (last) {
+                        __threadfence_block();
+                        tc_fence_after();
+                        const int nb = 3 * BLK - blk * BLK;        // channels still to come: 96, 64, 32
+                        const unsigned idesc = tc_idesc(nb);
+                        const unsigned b_lbo = 16u * nb;
+                        const unsigned bhi = smem_u32(Bhi + tc_panel_off(blk)), blo = smem_u32(Blo + tc_panel_off(blk));
+                        const unsigned d = t_tile + blk * BLK;
+#pragma unroll
+                        for (int term = 0; term < 3; ++term) {
+                            const unsigned a = term == 0 ? a_lo : a_hi;
+                            const unsigned bb = term == 1 ? blo : bhi;
+#pragma unroll
+                            for (int ks = 0; ks < BLK / 8; ++ks)
+                                umma_tf32_ss(d, umma_desc(a + ks * 2 * TC_A_LBO, TC_A_LBO, TC_SBO),
+                                             umma_desc(bb + ks * 2 * b_lbo, b_lbo, TC_SBO), idesc, (blk | term | ks) != 0);
+                        }
+                        umma_commit(my_mbar);
+                    }
+                    __syncwarp();
+                }
+
+                if (cur.active) {
+                    unsigned char *cp = p.codes + (cur.out_tok0 + cur.tok) * (D * BITS / 8) + blk * (BLK * BITS / 8);
                     if (WORDS_PER_BLK == 2)
-                        *reinterpret_cast<uint2 *>(cp + blk * (BLK * BITS / 8)) = make_uint2(cw[0], cw[1]);
+                        *reinterpret_cast<uint2 *>(cp) = make_uint2(cw[0], cw[1]);
                     else
-                        *reinterpret_cast<uint4 *>(cp + blk * (BLK * BITS / 8)) =
-                            make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
+                        *reinterpret_cast<uint4 *>(cp) = make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
                     if (wteam == 0) {
-                        sc_out[blk * BLK + lane] = my_scale;
-                        zr_out[blk * BLK + lane] = my_zero;
+                        const long long o = (cur.out_tok0 / G + cur.grp) * D + blk * BLK + lane;
+                        p.scales[o] = my_scale;
+                        p.zeros[o] = my_zero;
                         if (!(my_scale > 0.0f && my_scale < __int_as_float(0x7f800000)))
                             atomicOr(p.status, my_scale == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
                     }
                 }
             }
+        } else if (nxt.valid) {
+            load_row<BF16>(raw, nxt.row, 0);
         }
-        pos = seg_end;
+        cur = nxt;
+    }
+
+    // Every committed batch has been waited for unless a wait ran out; then commit once more per slot and give the
+    // tensor core a bounded time to drain before the columns are handed back.
+    if (shared_words[1] && wq == 0 && lane == 0) {
+        umma_commit(my_mbar);
+        mbar_wait(my_mbar, phase);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)TC_TMEM_COLS) : "memory");
+}
+
+// Writes, per head, the 64 KB image of the update matrix that the key kernel stages in shared memory:
+//   [0, 4096)        the four diagonal 32 x 32 blocks of W^T, row-major: block b, row jj, column c = W^T[32 b + jj][32 b + c]
+//   [4096, 10240)    hi panels of source blocks b = 0, 1, 2: B_b(n, k) = W[32 (b + 1) + n][32 b + k] = W^T[32 b + k][32 (b + 1) + n],
+//                    n < 96 - 32 b, k < 32, rounded to tf32, K-major in 8 x 16-byte core matrices:
+//                    float index (k / 4) * 4 N + 4 n + k % 4 with N = 96 - 32 b
+//   [10240, 16384)   lo panels: tf32(W - hi), same layout
+// One CTA per head; each thread takes (panel, 4-k chunk, channel n): four coalesced row reads, one 16-byte store.
+__global__ void __launch_bounds__(256) pack_w_kernel(const float *__restrict__ Wt, float *__restrict__ Wimg)
+{
+    const float *src = Wt + (long long)blockIdx.x * D * D;
+    float *img = Wimg + (long long)blockIdx.x * TC_IMG_FLOATS;
+    for (int i = threadIdx.x; i < TC_DIAG_FLOATS / 4; i += blockDim.x) {
+        const int b = i / (BLK * BLK / 4), r = i % (BLK * BLK / 4), jj = r / (BLK / 4), c4 = r % (BLK / 4);
+        reinterpret_cast<float4 *>(img)[i] = __ldg(reinterpret_cast<const float4 *>(src + (b * BLK + jj) * D + b * BLK + 4 * c4));
+    }
+    float *Bhi = img + TC_DIAG_FLOATS, *Blo = Bhi + TC_PANEL_FLOATS;
+    for (int i = threadIdx.x; i < TC_PANEL_FLOATS / 4; i += blockDim.x) {
+        const int f = 4 * i;                                 // first float of the 16-byte unit
+        const int b = f < tc_panel_off(1) ? 0 : (f < tc_panel_off(2) ? 1 : 2);
+        const int nb = 3 * BLK - b * BLK;
+        const int r = (f - tc_panel_off(b)) / 4;             // unit within the panel: kc * nb + n
+        const int kc = r / nb, n = r % nb;
+        const float *g = src + (b * BLK + 4 * kc) * D + (b + 1) * BLK + n;
+        const float w0 = __ldg(g), w1 = __ldg(g + D), w2 = __ldg(g + 2 * D), w3 = __ldg(g + 3 * D);
+        const float4 whi = make_float4(__uint_as_float(tf32_of(w0)), __uint_as_float(tf32_of(w1)),
+                                       __uint_as_float(tf32_of(w2)), __uint_as_float(tf32_of(w3)));
+        reinterpret_cast<float4 *>(Bhi)[i] = whi;
+        reinterpret_cast<float4 *>(Blo)[i] =
+            make_float4(__uint_as_float(tf32_of(__fsub_rn(w0, whi.x))), __uint_as_float(tf32_of(__fsub_rn(w1, whi.y))),
+                        __uint_as_float(tf32_of(__fsub_rn(w2, whi.z))), __uint_as_float(tf32_of(__fsub_rn(w3, whi.w))));
     }
 }
 
@@ -388,16 +547,22 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    constexpr int NTEAMS = KEY_WARPS / NW;
-    const size_t smem = sizeof(float) * (PANEL_FLOATS + KEY_WARPS * E_ROWS * 32) + sizeof(float2) * (NTEAMS * 2 * NW + KEY_WARPS * BLK);
-    long long want = (p.total_groups + NTEAMS - 1) / NTEAMS;
+    constexpr int GPT = 4 / NW;
+    constexpr int NTEAMS = TC_SLOTS * GPT;
+    // 193 KB: well over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
+    // never share an SM
+    const size_t smem = sizeof(float) * (TC_SLOTS * 2 * TC_E_FLOATS + TC_IMG_FLOATS) +
+                        sizeof(float2) * (NTEAMS * 2 * NW + TC_WARPS * BLK) + sizeof(u64) * TC_SLOTS + 4 * (2 + TC_SLOTS) + 8;
+    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
+    const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
+    const long long want = ((tiles_per_head + TC_SLOTS - 1) / TC_SLOTS) * p.H;      // rounds
     const int grid = (int)(want < sms ? want : sms);
     if (dtype == SQUAT_BF16) {
         SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quant_keys_kernel<BITS, NW, true><<<grid, KEY_THREADS, smem, st>>>(p);
+        quant_keys_kernel<BITS, NW, true><<<grid, TC_THREADS, smem, st>>>(p);
     } else {
         SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quant_keys_kernel<BITS, NW, false><<<grid, KEY_THREADS, smem, st>>>(p);
+        quant_keys_kernel<BITS, NW, false><<<grid, TC_THREADS, smem, st>>>(p);
     }
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
@@ -406,19 +571,26 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
 
 }  // namespace
 
-int squat_launch_quant_keys(const float *Wt, const void *k, int dtype, int batch, int H, int T,
+int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaStream_t st)
+{
+    pack_w_kernel<<<H, 256, 0, st>>>(Wt, Wimg);
+    squat_count_launch();
+    SQUAT_LAUNCH_CHECK();
+    return SQUAT_OK;
+}
+
+int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
                             unsigned char *codes, float *scales, float *zeros,
                             long long osb, long long osh, unsigned *status, int exact_blocks, cudaStream_t st)
 {
     KeyParams p;
-    p.Wt = Wt; p.k = k; p.sb = sb; p.sh = sh; p.st = st_;
+    p.Wimg = Wimg; p.k = k; p.sb = sb; p.sh = sh; p.st = st_;
     p.codes = codes; p.scales = scales; p.zeros = zeros; p.osb = osb; p.osh = osh;
     p.B = batch; p.H = H; p.T = T; p.groups_per_bh = T / G;
-    p.total_groups = (long long)H * batch * (T / G);
     p.status = status;
     p.exact_blocks = exact_blocks;
-    if (p.total_groups == 0) return SQUAT_OK;
+    if ((long long)H * batch * (T / G) == 0) return SQUAT_OK;
     if (bits == 2) {
         if (G == 32) return launch_keys<2, 1>(p, dtype, st);
         if (G == 64) return launch_keys<2, 2>(p, dtype, st);

@@ -14,6 +14,7 @@ struct squat_subspace {
     int gram_chunks_cap;   // capacity (in row chunks per head) of gram_partial
     int exact_blocks;      // leading 32-channel blocks of W that receive no correction (4 when W = 0)
     float *Wt;             // [H, d, d] float32, Wt[h][j][j'] = W[j'][j]  (row j = update vector of channel j)
+    float *Wimg;           // [H, d * d] the same matrices as the key kernel stages them in shared memory (see keys.cu)
     double *gram;          // [H, d, d] Gram matrices
     double *gram_partial;  // [chunks, H, d, d] per-chunk partial Gram matrices (deterministic reduction)
     double *eigval;        // [H, d] descending
@@ -39,7 +40,8 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
 int squat_launch_eig(squat_subspace *s, cudaStream_t st);
 int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st);
 
-int squat_launch_quant_keys(const float *Wt, const void *k, int dtype, int batch, int H, int T,
+int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaStream_t st);
+int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
                             unsigned char *codes, float *scales, float *zeros,
                             long long osb, long long osh, unsigned *status, int exact_blocks, cudaStream_t st);

@@ -690,7 +690,7 @@ int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int bloc
     assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
-    return SQUAT_OK;
+    return squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, st);
 }
 
 // ------------------------------------------------------------------------- allocation-free Gram entry
