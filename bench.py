@@ -41,15 +41,15 @@ ALU_PEAK_TFLOPS = SM_COUNT * FMA_LANES * 2 * SM_MAX_GHZ / 1e3
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the key kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists for that workload).
-NCU_KEY_KERNEL_TRAFFIC_BYTES = {1: 34_950_912, 2: 325_360_640}    # profiles/quant_keys_kernel_config1.md, streaming_kernels_config2.md
+NCU_KEY_KERNEL_TRAFFIC_BYTES = {1: 36_055_040, 2: 325_360_640}    # profiles/quant_keys_kernel_config1.md, streaming_kernels_config2.md
 
 
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return {"hbm_gbs": d["hbm_gbs"], "source": "measured"}
-    return {"hbm_gbs": 6650.0, "source": "fallback"}
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d.get("bf16_tflops", 1590.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
 
 
 # --------------------------------------------------------------------------- algorithmic counts
@@ -57,6 +57,14 @@ def key_flops_per_vector(d, g):
     """2 x FMAs of the dense block-triangular update (Eq. (3) / Eq. (update_block))."""
     T = d // g
     return 2 * sum(g * (d - t * g) for t in range(1, T))
+
+
+def key_fma_split(d, g, blk=32):
+    """The same multiply-adds split by where the key kernel runs them: (inside a 32-channel block: FP32 pipes,
+    across blocks: tensor cores).  W[j'][j] is non-zero iff j' lies in a later g-block than j."""
+    alu = sum(1 for j in range(d) for jp in range(j + 1, d) if jp // g > j // g and jp // blk == j // blk)
+    tensor = sum(1 for j in range(d) for jp in range(j + 1, d) if jp // g > j // g and jp // blk != j // blk)
+    return alu, tensor
 
 
 def reader_bytes_per_cached_token(d, bits, G):
@@ -450,6 +458,18 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
             roof = {"bound": "hbm", "achieved": kbytes / (key_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "peak_source": peaks["source"]}
         roof["frac"] = roof["achieved"] / roof["peak"]
+        # the strict reading for a kernel that runs its cross-block updates on the tensor cores: the slowest of the
+        # in-block FP32 work at the FP32 peak, three tf32 products per cross-block multiply-add at the tf32 peak
+        # (half the measured bf16 peak: the nominal ratio), and the bytes at the HBM copy bandwidth
+        alu_fma, tensor_fma = key_fma_split(d, cfg.block_g)
+        tf32_peak = 0.5 * peaks["bf16_tflops"]
+        t_alu = 2 * alu_fma * vec_per_step / (ALU_PEAK_TFLOPS * 1e12) * 1e6
+        t_tensor = 3 * 2 * tensor_fma * vec_per_step / (tf32_peak * 1e12) * 1e6
+        floor_us = max(t_alu, t_tensor, hbm_time_ms * 1e3)
+        roof["pipes"] = {"fp32_fma_per_vector": alu_fma, "tensor_fma_per_vector": tensor_fma, "tf32_products_per_fma": 3,
+                         "tf32_peak_tflops": tf32_peak, "fp32_floor_us": t_alu, "tensor_floor_us": t_tensor,
+                         "hbm_floor_us": hbm_time_ms * 1e3, "floor_us": floor_us,
+                         "frac_of_floor": floor_us / (key_ms * 1e3)}
         roof["traffic"] = NCU_KEY_KERNEL_TRAFFIC_BYTES.get(cfg.index)
         roof["kernel"] = "quant_keys_kernel"
         roof["ms_per_launch"] = key_ms

@@ -47,7 +47,8 @@ typedef enum { SQUAT_KEYS = 0, SQUAT_VALUES = 1 } squat_kind;
 #define SQUAT_FLAG_NONFINITE   1u   /* a scale came out NaN/Inf: non-finite input                  */
 #define SQUAT_FLAG_ZERO_RANGE  2u   /* some group had max == min (scale 0, all codes 0)            */
 #define SQUAT_FLAG_NO_CONVERGE 4u   /* eigensolver hit its sweep limit for some head               */
-#define SQUAT_FLAG_DEVICE_TIMEOUT 8u /* a bounded wait inside a kernel ran out; outputs are invalid     */
+#define SQUAT_FLAG_DEVICE_TIMEOUT 8u /* a bounded wait on the tensor core inside squat_quantize_keys ran
+                                       * out: that call's outputs are invalid (the kernel still ends)  */
 
 /* Opaque per-layer state: the update matrices of every KV head (shared by all samples of a
  * batch, Appendix C) plus the scratch the subspace build needs.  Owns device memory. */
@@ -107,6 +108,11 @@ int squat_subspace_eig_sweeps(const squat_subspace *s, void *stream, int *sweeps
  * (corrected) values, round half to even, push each token's error on its later channels
  * through W.  Splitting n_tokens at multiples of G over several calls gives identical bytes.
  * bits in {2, 4}; group_size in {32, 64, 128}; d = 128; n_kv_heads must match the handle.
+ * The updates that cross 32-channel blocks are computed on the tensor cores as three tf32
+ * products per multiply-add (operands split hi + lo), accumulated in fp32; the result agrees
+ * with fp32 arithmetic to a few 1e-7 of sum |e W|.  Every wait on the tensor core is bounded; if
+ * one runs out the kernel still ends, SQUAT_FLAG_DEVICE_TIMEOUT is set in the device status word
+ * and the outputs of that call are invalid.
  */
 int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
                         int n_tokens, int head_dim, long long stride_b, long long stride_h,

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libsquat.so")
 
 SQUAT_F32, SQUAT_BF16 = 0, 1
 SQUAT_KEYS, SQUAT_VALUES = 0, 1
-FLAG_NONFINITE, FLAG_ZERO_RANGE, FLAG_NO_CONVERGE = 1, 2, 4
+FLAG_NONFINITE, FLAG_ZERO_RANGE, FLAG_NO_CONVERGE, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
 
 EXPORTED_SYMBOLS = (
     "squat_subspace_create", "squat_subspace_destroy", "squat_build_subspace", "squat_subspace_export",

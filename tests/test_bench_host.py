@@ -42,6 +42,9 @@ def test_algorithmic_counts():
     assert bench.key_flops_per_vector(128, 1) == 2 * 8128
     assert bench.key_flops_per_vector(128, 32) == 2 * 6144
     assert bench.key_flops_per_vector(128, 64) == 2 * 4096
+    assert bench.key_fma_split(128, 1) == (4 * 496, 8128 - 4 * 496)      # four 32 x 32 triangles stay on the FP32 pipes
+    assert sum(bench.key_fma_split(128, 32)) == 6144 and bench.key_fma_split(128, 32)[0] == 0
+    assert sum(bench.key_fma_split(128, 64)) == 4096
     assert bench.bytes_per_vector(128, 2, 32, 2) == 320
     assert bench.bytes_per_vector(128, 4, 128, 2) == 328
     assert abs(bench.ALU_PEAK_TFLOPS - 74.45) < 0.01

@@ -80,6 +80,25 @@ def test_keys_variants_bf16(bits, G, r, g):
     _compare_all_units(cfg, k_np, W32, mats, bits, G, got, min_raw=0.99)
 
 
+@pytest.mark.parametrize("G,T,B,H", [
+    (32, 160, 1, 2),     # 5 groups per head: the second 128-token tile has one group, its other three warps idle along
+    (32, 96, 3, 3),      # 9 groups per head across 3 batch entries: tiles mix batch entries, the last one is ragged
+    (64, 192, 1, 2),     # 3 groups of 64: tile 1 holds one team and a spare one
+    (128, 128, 5, 1),    # 5 groups of 128 = 5 tiles: two rounds, the second with one tile slot in use
+    (32, 32, 1, 5),      # one group per head: every tile ragged, every round a new head
+])
+def test_keys_ragged_tiles_and_rounds(G, T, B, H):
+    # the kernel works in tiles of 128 tokens (4 warps) and rounds of 4 tiles of one head
+    bits = 2
+    cfg = si.get_config(1).with_(batch=B, n_kv_heads=H, n_q_heads=H, n_tokens=T)
+    W32, mats = _oracle_W32(cfg, range(H), n_tokens=max(T, 256))
+    k_np = si.gen_keys(cfg)
+    sq.squat_get_device_status(clear=True)
+    got = _run_keys(cfg, k_np, W32, bits, G)
+    assert not (sq.squat_get_device_status(clear=True) & sq.FLAG_DEVICE_TIMEOUT)
+    _compare_all_units(cfg, k_np, W32, mats, bits, G, got, min_raw=0.99)
+
+
 def test_keys_zero_update_reduces_to_round_to_nearest():
     # r = 0 / lambda = 0: W = 0 and the kernel must reproduce plain per-channel round-to-nearest
     # (Section 3.3).  Scales and zeros are bit-exact against the binary32 computation; codes may differ
