@@ -222,7 +222,7 @@ __device__ __forceinline__ float2 row_pair(const RawRow<BF16> &r, int q)
 // going to the even code (the threshold of an odd c0 is one ulp lower, so "remainder == scale/2" moves it).
 template <int BITS, int NW, bool EXACT>
 __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, float *e_hi, float *e_lo, bool store_e,
-                                            int lane, int bar_id, int wteam, float2 *red, float2 *park,
+                                            int lane, int bar_id, int wteam, float2 *red,
                                             uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
 {
     constexpr float L = float((1 << BITS) - 1);
@@ -263,7 +263,10 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         // pack the code arithmetically: sum of c * 2^(BITS k) is exact in float32 up to 16 bits
         if (jj % PER_ACC == 0) cacc[jj / PER_ACC] = c;
         else cacc[jj / PER_ACC] = __fmaf_rn(c, float(1 << ((jj % PER_ACC) * BITS)), cacc[jj / PER_ACC]);
-        park[jj] = make_float2(scale, m);               // same value from every lane; lane jj picks it up below
+        if (lane == jj) {                               // lane jj keeps channel jj's grid for the store after the sweep
+            my_scale = scale;
+            my_zero = m;
+        }
         // tf32 split by truncation: the tensor core reads only the top 19 bits of each word, so e itself serves
         // as E_hi = trunc(e), and E_lo = e - trunc(e) is exact in fp32
         eh[jj & 3] = e;
@@ -281,11 +284,6 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
             xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
         }
     }
-    __syncwarp();
-    const float2 sz = park[lane];
-    my_scale = sz.x;
-    my_zero = sz.y;
-    __syncwarp();
 #pragma unroll
     for (int w = 0; w < BLK * BITS / 32; ++w)
         cw[w] = (uint32_t)__float2int_rn(cacc[2 * w]) | ((uint32_t)__float2int_rn(cacc[2 * w + 1]) << 16);
@@ -314,8 +312,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     float *Bhi = diag_all + TC_DIAG_FLOATS;              // panels of source blocks 0, 1, 2
     float *Blo = Bhi + TC_PANEL_FLOATS;
     float2 *red_all = reinterpret_cast<float2 *>(Blo + TC_PANEL_FLOATS);         // [NTEAMS][2][NW]
-    float2 *park = red_all + NTEAMS * 2 * NW + (threadIdx.x >> 5) * BLK;         // [TC_WARPS][BLK] (scale, zero) of a block
-    u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW + TC_WARPS * BLK);   // [TC_SLOTS]
+    u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW);              // [TC_SLOTS]
     // [0] tensor-memory base, [1] a bounded wait ran out, [2 + slot] arrivals of the slot's warps
     volatile unsigned *shared_words = reinterpret_cast<volatile unsigned *>(mbar + TC_SLOTS);
 
@@ -441,9 +438,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 uint32_t cw[WORDS_PER_BLK];
                 float my_scale = 0.0f, my_zero = 0.0f;
                 if (blk < p.exact_blocks)
-                    sweep_block<BITS, NW, true>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, park, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, true>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
                 else
-                    sweep_block<BITS, NW, false>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, park, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, false>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
 
                 if (more) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the error rows, for the tensor core
@@ -552,7 +549,7 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     // 193 KB: well over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
     // never share an SM
     const size_t smem = sizeof(float) * (TC_SLOTS * 2 * TC_E_FLOATS + TC_IMG_FLOATS) +
-                        sizeof(float2) * (NTEAMS * 2 * NW + TC_WARPS * BLK) + sizeof(u64) * TC_SLOTS + 4 * (2 + TC_SLOTS) + 8;
+                        sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * TC_SLOTS + 4 * (2 + TC_SLOTS) + 8;
     const long long groups_per_head = (long long)p.B * p.groups_per_bh;
     const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
     const long long want = ((tiles_per_head + TC_SLOTS - 1) / TC_SLOTS) * p.H;      // rounds
