@@ -46,7 +46,8 @@ constexpr float kMagic = 12582912.0f;     // 1.5 * 2^23
 constexpr int TC_SLOTS = 4;                          // 128-token tiles in flight per CTA
 constexpr int TC_WARPS = TC_SLOTS * 4;
 constexpr int TC_THREADS = TC_WARPS * 32;
-constexpr int TC_COLS_PER_TILE = 128;                // 96 used: channels 32 .. 127
+constexpr int TC_COLS_PER_TILE = 128;                // [0, 96) D: corrections of channels 32 .. 127; [96, 128) E_hi of the block just swept
+constexpr int TC_EHI_COL = 96;
 constexpr int TC_TMEM_COLS = 512;
 static_assert(TC_SLOTS * TC_COLS_PER_TILE <= TC_TMEM_COLS, "tensor memory has 512 columns");
 constexpr int TC_E_FLOATS = 128 * BLK;               // one tile's E_hi (or E_lo): 128 rows x 32 channels
@@ -145,6 +146,19 @@ __device__ __forceinline__ void umma_tf32_ss(unsigned d_taddr, u64 a_desc, u64 b
                  " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
                  ::"r"(d_taddr), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// the same with A from tensor memory (rows = lanes, 8 consecutive 32-bit columns)
+__device__ __forceinline__ void umma_tf32_ts(unsigned d_taddr, unsigned a_taddr, u64 b_desc, unsigned idesc, unsigned accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d_taddr), "r"(a_taddr), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 4 consecutive 32-bit columns of the warp's 32 tensor-memory lanes: lane l writes its own row
+__device__ __forceinline__ void tmem_st4(unsigned taddr, float a, float b, float c, float d)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(taddr), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)), "r"(__float_as_uint(d)) : "memory");
+}
 __device__ __forceinline__ void umma_commit(unsigned mbar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
@@ -221,7 +235,7 @@ __device__ __forceinline__ float2 row_pair(const RawRow<BF16> &r, int q)
 // +-scale/2: that settles the rounding exactly as real arithmetic on the stored float32 scale would, ties
 // going to the even code (the threshold of an odd c0 is one ulp lower, so "remainder == scale/2" moves it).
 template <int BITS, int NW, bool EXACT>
-__device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, float *e_hi, float *e_lo, bool store_e,
+__device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, unsigned e_hi_taddr, float *e_lo, bool store_e,
                                             int lane, int bar_id, int wteam, float2 *red,
                                             uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
 {
@@ -272,7 +286,7 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         eh[jj & 3] = e;
         el[jj & 3] = __fsub_rn(e, __uint_as_float(__float_as_uint(e) & 0xffffe000u));
         if ((jj & 3) == 3 && store_e) {
-            *reinterpret_cast<float4 *>(e_hi + (jj >> 2) * (TC_A_LBO / 4)) = make_float4(eh[0], eh[1], eh[2], eh[3]);
+            tmem_st4(e_hi_taddr + (jj - 3), eh[0], eh[1], eh[2], eh[3]);
             *reinterpret_cast<float4 *>(e_lo + (jj >> 2) * (TC_A_LBO / 4)) = make_float4(el[0], el[1], el[2], el[3]);
         }
         const u64 ee = pack2(e, e);
@@ -307,8 +321,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     constexpr int NTEAMS = TC_SLOTS * GPT;               // teams of NW warps
     constexpr int WORDS_PER_BLK = BLK * BITS / 32;       // 2 (2-bit) or 4 (4-bit)
     extern __shared__ __align__(128) float smem[];
-    float *Eall = smem;                                  // [TC_SLOTS][hi, lo][TC_E_FLOATS]
-    float *diag_all = Eall + TC_SLOTS * 2 * TC_E_FLOATS; // [NBLK][32][32], then the hi panels, then the lo panels
+    float *Eall = smem;                                  // [TC_SLOTS][TC_E_FLOATS]: the tiles' E_lo operands
+    float *diag_all = Eall + TC_SLOTS * TC_E_FLOATS; // [NBLK][32][32], then the hi panels, then the lo panels
     float *Bhi = diag_all + TC_DIAG_FLOATS;              // panels of source blocks 0, 1, 2
     float *Blo = Bhi + TC_PANEL_FLOATS;
     float2 *red_all = reinterpret_cast<float2 *>(Blo + TC_PANEL_FLOATS);         // [NTEAMS][2][NW]
@@ -344,9 +358,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     const unsigned tmem_base = shared_words[0];
     const unsigned t_tile = tmem_base + slot * TC_COLS_PER_TILE;               // lane field 0: the MMAs' accumulator
     const unsigned t_mine = t_tile + ((unsigned)(wq * 32) << 16);              // this warp's 32 lanes
-    float *e_hi = Eall + slot * 2 * TC_E_FLOATS + (wq * 32 + lane) * 4;        // this lane's row of the tile's A operands
-    float *e_lo = e_hi + TC_E_FLOATS;
-    const unsigned a_hi = smem_u32(Eall + slot * 2 * TC_E_FLOATS), a_lo = a_hi + TC_E_FLOATS * 4;
+    float *e_lo = Eall + slot * TC_E_FLOATS + (wq * 32 + lane) * 4;            // this lane's row of the tile's E_lo operand
+    const unsigned a_lo = smem_u32(Eall + slot * TC_E_FLOATS);
     const unsigned my_mbar = smem_u32(mbar + slot);
     unsigned phase = 0;
 
@@ -438,12 +451,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 uint32_t cw[WORDS_PER_BLK];
                 float my_scale = 0.0f, my_zero = 0.0f;
                 if (blk < p.exact_blocks)
-                    sweep_block<BITS, NW, true>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, true>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
                 else
-                    sweep_block<BITS, NW, false>(xp, diag, e_hi, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, false>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
 
                 if (more) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the error rows, for the tensor core
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");   // E_hi is in tensor memory
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // E_lo rows, for the tensor core
                     tc_fence_before();
                     __threadfence_block();
                     __syncwarp();
@@ -459,14 +473,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                         const unsigned bhi = smem_u32(Bhi + tc_panel_off(blk)), blo = smem_u32(Blo + tc_panel_off(blk));
                         const unsigned d = t_tile + blk * BLK;
 #pragma unroll
-                        for (int term = 0; term < 3; ++term) {
-                            const unsigned a = term == 0 ? a_lo : a_hi;
-                            const unsigned bb = term == 1 ? blo : bhi;
+                        for (int ks = 0; ks < BLK / 8; ++ks)         // E_lo (shared memory) x Whi
+                            umma_tf32_ss(d, umma_desc(a_lo + ks * 2 * TC_A_LBO, TC_A_LBO, TC_SBO),
+                                         umma_desc(bhi + ks * 2 * b_lbo, b_lbo, TC_SBO), idesc, (blk | ks) != 0);
 #pragma unroll
-                            for (int ks = 0; ks < BLK / 8; ++ks)
-                                umma_tf32_ss(d, umma_desc(a + ks * 2 * TC_A_LBO, TC_A_LBO, TC_SBO),
-                                             umma_desc(bb + ks * 2 * b_lbo, b_lbo, TC_SBO), idesc, (blk | term | ks) != 0);
-                        }
+                        for (int ks = 0; ks < BLK / 8; ++ks)         // E_hi (tensor memory) x Wlo
+                            umma_tf32_ts(d, t_tile + TC_EHI_COL + 8 * ks, umma_desc(blo + ks * 2 * b_lbo, b_lbo, TC_SBO), idesc, 1u);
+#pragma unroll
+                        for (int ks = 0; ks < BLK / 8; ++ks)         // E_hi x Whi
+                            umma_tf32_ts(d, t_tile + TC_EHI_COL + 8 * ks, umma_desc(bhi + ks * 2 * b_lbo, b_lbo, TC_SBO), idesc, 1u);
                         umma_commit(my_mbar);
                     }
                     __syncwarp();
@@ -546,9 +561,9 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     constexpr int GPT = 4 / NW;
     constexpr int NTEAMS = TC_SLOTS * GPT;
-    // 193 KB: well over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
+    // 129 KB: over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
     // never share an SM
-    const size_t smem = sizeof(float) * (TC_SLOTS * 2 * TC_E_FLOATS + TC_IMG_FLOATS) +
+    const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + TC_IMG_FLOATS) +
                         sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * TC_SLOTS + 4 * (2 + TC_SLOTS) + 8;
     const long long groups_per_head = (long long)p.B * p.groups_per_bh;
     const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
