@@ -291,8 +291,15 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         }
         const u64 ee = pack2(e, e);
         const float *wrow = diag + jj * BLK;
+        // later channels of the block, 4 per 16-byte broadcast read; where only the upper half of the first chunk
+        // is still to come, an 8-byte read does (a broadcast read is charged by its width)
+        if ((jj + 1) % 4 >= 2) {
+            const int q = (jj + 1) / 4;
+            const u64 wy = *reinterpret_cast<const u64 *>(wrow + 4 * q + 2);
+            xp[2 * q + 1] = ffma2(ee, wy, xp[2 * q + 1]);
+        }
 #pragma unroll
-        for (int q = (jj + 1) / 4; q < BLK / 4; ++q) {
+        for (int q = ((jj + 1) % 4 >= 2 ? (jj + 1) / 4 + 1 : (jj + 1) / 4); q < BLK / 4; ++q) {
             const ulonglong2 wv = *reinterpret_cast<const ulonglong2 *>(wrow + 4 * q);
             if (2 * q >= (jj + 1) / 2) xp[2 * q] = ffma2(ee, wv.x, xp[2 * q]);
             xp[2 * q + 1] = ffma2(ee, wv.y, xp[2 * q + 1]);
