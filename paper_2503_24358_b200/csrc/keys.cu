@@ -175,6 +175,19 @@ __device__ __forceinline__ bool mbar_wait(unsigned mbar, unsigned parity)
     return false;
 }
 
+// Starts the copy of one head's 64 KB image into shared memory on the bulk-copy engine (no multicast); the bytes are
+// counted on `mbar`, whose current phase completes when all of them have landed.
+__device__ __forceinline__ void stage_image_async(float *dst, const float *src, unsigned mbar)
+{
+    constexpr unsigned BYTES = TC_IMG_FLOATS * 4, PIECE = 16384;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // earlier reads of the old image, before the engine's writes
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(BYTES) : "memory");
+#pragma unroll
+    for (unsigned o = 0; o < BYTES; o += PIECE)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(dst) + o), "l"(reinterpret_cast<const char *>(src) + o), "r"(PIECE), "r"(mbar) : "memory");
+}
+
 struct KeyParams {
     const float *Wimg;        // [H, d * d] staged images of the update matrices (pack_w_kernel)
     const void *k;
@@ -333,9 +346,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     float *Bhi = diag_all + TC_DIAG_FLOATS;              // panels of source blocks 0, 1, 2
     float *Blo = Bhi + TC_PANEL_FLOATS;
     float2 *red_all = reinterpret_cast<float2 *>(Blo + TC_PANEL_FLOATS);         // [NTEAMS][2][NW]
-    u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW);              // [TC_SLOTS]
+    u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW);              // [TC_SLOTS] MMAs done, [1] image staged
     // [0] tensor-memory base, [1] a bounded wait ran out, [2 + slot] arrivals of the slot's warps
-    volatile unsigned *shared_words = reinterpret_cast<volatile unsigned *>(mbar + TC_SLOTS);
+    volatile unsigned *shared_words = reinterpret_cast<volatile unsigned *>(mbar + TC_SLOTS + 1);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -345,19 +358,34 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     const int wteam = wq % NW;
     float2 *red = red_all + team * (2 * NW);
 
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(const_cast<unsigned *>(shared_words))), "r"((unsigned)TC_TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
+    const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
+    // Work unit of a CTA: a round = TC_SLOTS consecutive tiles of one head, one per slot.  CTAs take contiguous
+    // ranges of rounds, so a head's update matrix is staged once per CTA that touches the head and no CTA's
+    // slots are split unevenly by a head boundary.
+    const long long rounds_per_head = (tiles_per_head + TC_SLOTS - 1) / TC_SLOTS;
+    const long long total_rounds = rounds_per_head * p.H;
+    const long long lo = total_rounds * blockIdx.x / gridDim.x;
+    const long long hi = total_rounds * (blockIdx.x + 1) / gridDim.x;
+    const unsigned img_mbar = smem_u32(mbar + TC_SLOTS);
+    unsigned img_phase = 0;
+
     if (threadIdx.x == 32) {
 #pragma unroll
         for (int t = 0; t < TC_SLOTS; ++t) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(mbar + t)), "r"(1) : "memory");
             shared_words[2 + t] = 0;
         }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(img_mbar), "r"(1) : "memory");
         shared_words[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // the first head's image is on its way while the rest of the set-up runs
+        if (lo < hi) stage_image_async(diag_all, p.Wimg + (lo / rounds_per_head) * TC_IMG_FLOATS, img_mbar);
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<unsigned *>(shared_words))), "r"((unsigned)TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
@@ -369,16 +397,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     const unsigned a_lo = smem_u32(Eall + slot * TC_E_FLOATS);
     const unsigned my_mbar = smem_u32(mbar + slot);
     unsigned phase = 0;
-
-    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
-    const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
-    // Work unit of a CTA: a round = TC_SLOTS consecutive tiles of one head, one per slot.  CTAs take contiguous
-    // ranges of rounds, so a head's update matrix is staged once per CTA that touches the head and no CTA's
-    // slots are split unevenly by a head boundary.
-    const long long rounds_per_head = (tiles_per_head + TC_SLOTS - 1) / TC_SLOTS;
-    const long long total_rounds = rounds_per_head * p.H;
-    const long long lo = total_rounds * blockIdx.x / gridDim.x;
-    const long long hi = total_rounds * (blockIdx.x + 1) / gridDim.x;
 
     auto locate = [&](long long rnd, TileRows &t) {
         const int h = (int)(rnd / rounds_per_head);
@@ -407,18 +425,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     for (long long rnd = lo; rnd < hi; ++rnd) {
         const int h = (int)(rnd / rounds_per_head);
         if (h != cur_head) {
+            if (cur_head >= 0) {
+                __syncthreads();                         // every read of the previous head's image, by a lane or by an MMA, is over
+                if (threadIdx.x == 32) stage_image_async(diag_all, p.Wimg + (long long)h * TC_IMG_FLOATS, img_mbar);
+            }
             cur_head = h;
-            __syncthreads();                             // every MMA that read the previous head's panels has been waited for
-            const float4 *src = reinterpret_cast<const float4 *>(p.Wimg + (long long)h * TC_IMG_FLOATS);
-            float4 *dst = reinterpret_cast<float4 *>(diag_all);
-            constexpr int PER_THREAD = TC_IMG_FLOATS / 4 / TC_THREADS;     // 8
-            float4 t[PER_THREAD];
-#pragma unroll
-            for (int i = 0; i < PER_THREAD; ++i) t[i] = __ldg(src + i * TC_THREADS + threadIdx.x);
-#pragma unroll
-            for (int i = 0; i < PER_THREAD; ++i) dst[i * TC_THREADS + threadIdx.x] = t[i];
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor core reads the panels through the async proxy
-            __syncthreads();
+            if (!shared_words[1] && !mbar_wait(img_mbar, img_phase)) {   // bounded, like every wait here
+                shared_words[1] = 1;
+                atomicOr(p.status, SQUAT_FLAG_DEVICE_TIMEOUT);
+            }
+            img_phase ^= 1;
         }
         nxt.valid = false;
         if (rnd + 1 < hi) locate(rnd + 1, nxt);
@@ -571,7 +587,7 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     // 129 KB: over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
     // never share an SM
     const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + TC_IMG_FLOATS) +
-                        sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * TC_SLOTS + 4 * (2 + TC_SLOTS) + 8;
+                        sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * (TC_SLOTS + 1) + 4 * (2 + TC_SLOTS) + 8;
     const long long groups_per_head = (long long)p.B * p.groups_per_bh;
     const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
     const long long want = ((tiles_per_head + TC_SLOTS - 1) / TC_SLOTS) * p.H;      // rounds
