@@ -328,7 +328,7 @@ struct TileRows {
     bool valid;               // the warp's slot has a tile in this round
     bool active;              // ... and the warp's group exists (a head's last tile may be ragged: its spare warps redo the
                               // last group and store nothing)
-    int tok, grp;
+    int head, tok, grp;
     long long out_tok0;
     const void *row;          // this lane's key vector
 };
@@ -342,10 +342,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     constexpr int WORDS_PER_BLK = BLK * BITS / 32;       // 2 (2-bit) or 4 (4-bit)
     extern __shared__ __align__(128) float smem[];
     float *Eall = smem;                                  // [TC_SLOTS][TC_E_FLOATS]: the tiles' E_lo operands
-    float *diag_all = Eall + TC_SLOTS * TC_E_FLOATS; // [NBLK][32][32], then the hi panels, then the lo panels
-    float *Bhi = diag_all + TC_DIAG_FLOATS;              // panels of source blocks 0, 1, 2
-    float *Blo = Bhi + TC_PANEL_FLOATS;
-    float2 *red_all = reinterpret_cast<float2 *>(Blo + TC_PANEL_FLOATS);         // [NTEAMS][2][NW]
+    float *images = Eall + TC_SLOTS * TC_E_FLOATS;       // [2][TC_IMG_FLOATS]: head h's image lives in buffer h & 1
+    float2 *red_all = reinterpret_cast<float2 *>(images + 2 * TC_IMG_FLOATS);    // [NTEAMS][2][NW]
     u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW);              // [TC_SLOTS] MMAs done, [1] image staged
     // [0] tensor-memory base, [1] a bounded wait ran out, [2 + slot] arrivals of the slot's warps
     volatile unsigned *shared_words = reinterpret_cast<volatile unsigned *>(mbar + TC_SLOTS + 1);
@@ -360,13 +358,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
 
     const long long groups_per_head = (long long)p.B * p.groups_per_bh;
     const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
-    // Work unit of a CTA: a round = TC_SLOTS consecutive tiles of one head, one per slot.  CTAs take contiguous
-    // ranges of rounds, so a head's update matrix is staged once per CTA that touches the head and no CTA's
-    // slots are split unevenly by a head boundary.
-    const long long rounds_per_head = (tiles_per_head + TC_SLOTS - 1) / TC_SLOTS;
-    const long long total_rounds = rounds_per_head * p.H;
-    const long long lo = total_rounds * blockIdx.x / gridDim.x;
-    const long long hi = total_rounds * (blockIdx.x + 1) / gridDim.x;
+    // A CTA takes a contiguous range of tiles (head-major order) and works it in rounds of up to TC_SLOTS tiles, one per
+    // slot, sized as evenly as its range allows (7 tiles = 4 + 3, not 4 + 4 elsewhere).  Two images fit in shared memory,
+    // so a round may run across one head boundary.
+    const long long total_tiles = tiles_per_head * p.H;
+    const long long t_lo = total_tiles * blockIdx.x / gridDim.x;
+    const long long t_hi = total_tiles * (blockIdx.x + 1) / gridDim.x;
+    auto round_size = [&](long long start) {
+        const long long left = t_hi - start;
+        if (left <= 0) return 0;
+        const long long rounds_left = (left + TC_SLOTS - 1) / TC_SLOTS;
+        long long n = (left + rounds_left - 1) / rounds_left;
+        const long long two_heads_end = (start / tiles_per_head + 2) * tiles_per_head;
+        if (start + n > two_heads_end) n = two_heads_end - start;
+        return (int)n;
+    };
     const unsigned img_mbar = smem_u32(mbar + TC_SLOTS);
     unsigned img_phase = 0;
 
@@ -380,7 +386,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
         shared_words[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         // the first head's image is on its way while the rest of the set-up runs
-        if (lo < hi) stage_image_async(diag_all, p.Wimg + (lo / rounds_per_head) * TC_IMG_FLOATS, img_mbar);
+        if (t_lo < t_hi) {
+            const long long h0 = t_lo / tiles_per_head;
+            stage_image_async(images + (h0 & 1) * TC_IMG_FLOATS, p.Wimg + h0 * TC_IMG_FLOATS, img_mbar);
+        }
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -398,10 +407,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     const unsigned my_mbar = smem_u32(mbar + slot);
     unsigned phase = 0;
 
-    auto locate = [&](long long rnd, TileRows &t) {
-        const int h = (int)(rnd / rounds_per_head);
-        const long long ti = (rnd - (long long)h * rounds_per_head) * TC_SLOTS + slot;   // tile within the head
-        t.valid = ti < tiles_per_head;
+    auto locate = [&](long long tile, bool valid, TileRows &t) {
+        const int h = (int)(tile / tiles_per_head);
+        const long long ti = tile - (long long)h * tiles_per_head;                        // tile within the head
+        t.valid = valid;
+        t.head = h;
         const long long g_raw = ti * GPT + wq / NW;
         t.active = t.valid && g_raw < groups_per_head;
         const long long in_head = g_raw < groups_per_head ? g_raw : groups_per_head - 1;
@@ -416,29 +426,42 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
 
     TileRows cur, nxt;
     RawRow<BF16> raw;
+    long long start = t_lo;
+    int n_round = round_size(start);
     cur.valid = false;
-    if (lo < hi) {
-        locate(lo, cur);
-        if (cur.valid) load_row<BF16>(raw, cur.row, 0);  // in flight while the first head is staged
+    cur.head = 0;
+    if (slot < n_round) {
+        locate(start + slot, true, cur);
+        load_row<BF16>(raw, cur.row, 0);                 // in flight while the first head is staged
     }
-    int cur_head = -1;
-    for (long long rnd = lo; rnd < hi; ++rnd) {
-        const int h = (int)(rnd / rounds_per_head);
-        if (h != cur_head) {
-            if (cur_head >= 0) {
-                __syncthreads();                         // every read of the previous head's image, by a lane or by an MMA, is over
-                if (threadIdx.x == 32) stage_image_async(diag_all, p.Wimg + (long long)h * TC_IMG_FLOATS, img_mbar);
+    int resident[2] = {-1, -1};                          // heads whose images the two buffers hold
+    int pending = t_lo < t_hi ? (int)(t_lo / tiles_per_head) : -1;     // head whose copy was started at kernel entry
+    while (start < t_hi) {
+        // images of the (at most two) heads of this round
+        const int h_first = (int)(start / tiles_per_head), h_last = (int)((start + n_round - 1) / tiles_per_head);
+        for (int hh = h_first; hh <= h_last; ++hh) {
+            if (resident[hh & 1] == hh) continue;
+            if (pending != hh) {
+                __syncthreads();                         // every read of the buffer's old image, by a lane or by an MMA, is over
+                if (threadIdx.x == 32)
+                    stage_image_async(images + (hh & 1) * TC_IMG_FLOATS, p.Wimg + (long long)hh * TC_IMG_FLOATS, img_mbar);
             }
-            cur_head = h;
+            pending = -1;
             if (!shared_words[1] && !mbar_wait(img_mbar, img_phase)) {   // bounded, like every wait here
                 shared_words[1] = 1;
                 atomicOr(p.status, SQUAT_FLAG_DEVICE_TIMEOUT);
             }
             img_phase ^= 1;
+            resident[hh & 1] = hh;
         }
+        const long long next_start = start + n_round;
+        const int n_next = round_size(next_start);
         nxt.valid = false;
-        if (rnd + 1 < hi) locate(rnd + 1, nxt);
+        nxt.head = 0;
+        if (slot < n_next) locate(next_start + slot, true, nxt);
 
+        const float *img = images + (cur.head & 1) * TC_IMG_FLOATS;       // diagonal blocks | hi panels | lo panels
+        const float *Bhi = img + TC_DIAG_FLOATS, *Blo = Bhi + TC_PANEL_FLOATS;
         if (cur.valid) {
 #pragma unroll 1
             for (int blk = 0; blk < NBLK; ++blk) {
@@ -470,7 +493,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 if (more) load_row<BF16>(raw, cur.row, (blk + 1) * BLK);
                 else if (nxt.valid) load_row<BF16>(raw, nxt.row, 0);
 
-                const float *diag = diag_all + blk * BLK * BLK;
+                const float *diag = img + blk * BLK * BLK;
                 uint32_t cw[WORDS_PER_BLK];
                 float my_scale = 0.0f, my_zero = 0.0f;
                 if (blk < p.exact_blocks)
@@ -529,6 +552,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
             load_row<BF16>(raw, nxt.row, 0);
         }
         cur = nxt;
+        start = next_start;
+        n_round = n_next;
     }
 
     // Every committed batch has been waited for unless a wait ran out; then commit once more per slot and give the
@@ -584,13 +609,13 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     constexpr int GPT = 4 / NW;
     constexpr int NTEAMS = TC_SLOTS * GPT;
-    // 129 KB: over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
+    // 193 KB: well over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
     // never share an SM
-    const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + TC_IMG_FLOATS) +
+    const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + 2 * TC_IMG_FLOATS) +
                         sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * (TC_SLOTS + 1) + 4 * (2 + TC_SLOTS) + 8;
     const long long groups_per_head = (long long)p.B * p.groups_per_bh;
     const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
-    const long long want = ((tiles_per_head + TC_SLOTS - 1) / TC_SLOTS) * p.H;      // rounds
+    const long long want = tiles_per_head * p.H;                                    // one tile per CTA at least
     const int grid = (int)(want < sms ? want : sms);
     if (dtype == SQUAT_BF16) {
         SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
