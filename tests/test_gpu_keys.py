@@ -86,9 +86,11 @@ def test_keys_variants_bf16(bits, G, r, g):
     (64, 192, 1, 2),     # 3 groups of 64: tile 1 holds one team and a spare one
     (128, 128, 5, 1),    # 5 groups of 128 = 5 tiles: two rounds, the second with one tile slot in use
     (32, 32, 1, 5),      # one group per head: every tile ragged, every round a new head
+    (32, 160, 4, 40),    # 200 tiles of 40 heads on 148 CTAs: some CTAs' rounds run across a head boundary (two images staged)
+    (32, 64, 1, 170),    # 170 one-tile heads: a CTA's two tiles belong to different heads
 ])
 def test_keys_ragged_tiles_and_rounds(G, T, B, H):
-    # the kernel works in tiles of 128 tokens (4 warps) and rounds of 4 tiles of one head
+    # the kernel works in tiles of 128 tokens (4 warps) and rounds of up to 4 tiles that may span two heads
     bits = 2
     cfg = si.get_config(1).with_(batch=B, n_kv_heads=H, n_q_heads=H, n_tokens=T)
     W32, mats = _oracle_W32(cfg, range(H), n_tokens=max(T, 256))
