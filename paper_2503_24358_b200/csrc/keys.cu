@@ -197,6 +197,9 @@ struct KeyParams {
     long long osb, osh;       // output strides in tokens
     int B, H, T;
     int groups_per_bh;        // T / G
+    int groups_per_head;      // B * T / G
+    int tiles_per_head;       // 128-token tiles per head (the last one may be ragged)
+    int total_tiles;          // H * tiles_per_head
     unsigned *status;
     int exact_blocks;         // leading 32-channel blocks that no earlier channel corrects (see sweep_block)
 };
@@ -323,14 +326,14 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         cw[w] = (uint32_t)__float2int_rn(cacc[2 * w]) | ((uint32_t)__float2int_rn(cacc[2 * w + 1]) << 16);
 }
 
-// Where one warp's 32 tokens of a round live.
+// Where one warp's 32 tokens of a round come from and go to.
 struct TileRows {
-    bool valid;               // the warp's slot has a tile in this round
-    bool active;              // ... and the warp's group exists (a head's last tile may be ragged: its spare warps redo the
-                              // last group and store nothing)
-    int head, tok, grp;
-    long long out_tok0;
+    bool active;              // the warp's group exists (a head's last tile may be ragged: its spare warps redo the last
+                              // group and store nothing)
+    int head;
     const void *row;          // this lane's key vector
+    unsigned char *codes;     // this lane's code row
+    long long meta;           // offset of the group's scales / zeros (lane = channel within a block)
 };
 
 template <int BITS, int NW, bool BF16>
@@ -356,22 +359,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     const int wteam = wq % NW;
     float2 *red = red_all + team * (2 * NW);
 
-    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
-    const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
     // A CTA takes a contiguous range of tiles (head-major order) and works it in rounds of up to TC_SLOTS tiles, one per
     // slot, sized as evenly as its range allows (7 tiles = 4 + 3, not 4 + 4 elsewhere).  Two images fit in shared memory,
-    // so a round may run across one head boundary.
-    const long long total_tiles = tiles_per_head * p.H;
-    const long long t_lo = total_tiles * blockIdx.x / gridDim.x;
-    const long long t_hi = total_tiles * (blockIdx.x + 1) / gridDim.x;
-    auto round_size = [&](long long start) {
-        const long long left = t_hi - start;
+    // so a round may run across one head boundary.  (All of this in 32-bit integers and recomputed rather than kept:
+    // the sweeps need every register.)
+    const int t_lo = (int)((long long)p.total_tiles * blockIdx.x / gridDim.x);
+    const int t_hi = (int)((long long)p.total_tiles * (blockIdx.x + 1) / gridDim.x);
+    auto round_size = [&](int start) {
+        const int left = t_hi - start;
         if (left <= 0) return 0;
-        const long long rounds_left = (left + TC_SLOTS - 1) / TC_SLOTS;
-        long long n = (left + rounds_left - 1) / rounds_left;
-        const long long two_heads_end = (start / tiles_per_head + 2) * tiles_per_head;
-        if (start + n > two_heads_end) n = two_heads_end - start;
-        return (int)n;
+        const int rounds_left = (left + TC_SLOTS - 1) / TC_SLOTS;
+        int n = (left + rounds_left - 1) / rounds_left;
+        const int two_heads_end = (start / p.tiles_per_head + 2) * p.tiles_per_head;
+        if (n > two_heads_end - start) n = two_heads_end - start;
+        return n;
     };
     const unsigned img_mbar = smem_u32(mbar + TC_SLOTS);
     unsigned img_phase = 0;
@@ -387,8 +388,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         // the first head's image is on its way while the rest of the set-up runs
         if (t_lo < t_hi) {
-            const long long h0 = t_lo / tiles_per_head;
-            stage_image_async(images + (h0 & 1) * TC_IMG_FLOATS, p.Wimg + h0 * TC_IMG_FLOATS, img_mbar);
+            const int h0 = t_lo / p.tiles_per_head;
+            stage_image_async(images + (h0 & 1) * TC_IMG_FLOATS, p.Wimg + (long long)h0 * TC_IMG_FLOATS, img_mbar);
         }
     }
     if (warp == 0) {
@@ -407,62 +408,64 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     const unsigned my_mbar = smem_u32(mbar + slot);
     unsigned phase = 0;
 
-    auto locate = [&](long long tile, bool valid, TileRows &t) {
-        const int h = (int)(tile / tiles_per_head);
-        const long long ti = tile - (long long)h * tiles_per_head;                        // tile within the head
-        t.valid = valid;
+    auto locate = [&](int tile, TileRows &t) {
+        const int h = tile / p.tiles_per_head;
+        const int g_raw = (tile - h * p.tiles_per_head) * GPT + wq / NW;                  // group within the head
         t.head = h;
-        const long long g_raw = ti * GPT + wq / NW;
-        t.active = t.valid && g_raw < groups_per_head;
-        const long long in_head = g_raw < groups_per_head ? g_raw : groups_per_head - 1;
-        const int b = (int)(in_head / p.groups_per_bh);
-        t.grp = (int)(in_head % p.groups_per_bh);
-        t.tok = t.grp * G + wteam * 32 + lane;
-        t.out_tok0 = (long long)b * p.osb + (long long)h * p.osh;
-        const long long row_off = (long long)b * p.sb + (long long)h * p.sh + (long long)t.tok * p.st;
+        t.active = g_raw < p.groups_per_head;
+        const int in_head = t.active ? g_raw : p.groups_per_head - 1;
+        const int b = in_head / p.groups_per_bh;
+        const int grp = in_head - b * p.groups_per_bh;
+        const int tok = grp * G + wteam * 32 + lane;
+        const long long out_tok0 = (long long)b * p.osb + (long long)h * p.osh;
+        t.codes = p.codes + (out_tok0 + tok) * (D * BITS / 8);
+        t.meta = (out_tok0 / G + grp) * D + lane;
+        const long long row_off = (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st;
         t.row = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.k) + row_off)
                      : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row_off);
     };
 
-    TileRows cur, nxt;
     RawRow<BF16> raw;
-    long long start = t_lo;
-    int n_round = round_size(start);
-    cur.valid = false;
-    cur.head = 0;
-    if (slot < n_round) {
-        locate(start + slot, true, cur);
-        load_row<BF16>(raw, cur.row, 0);                 // in flight while the first head is staged
+    int start = t_lo;
+    if (slot < round_size(start)) {
+        TileRows first;
+        locate(start + slot, first);
+        load_row<BF16>(raw, first.row, 0);               // in flight while the first head is staged
     }
-    int resident[2] = {-1, -1};                          // heads whose images the two buffers hold
-    int pending = t_lo < t_hi ? (int)(t_lo / tiles_per_head) : -1;     // head whose copy was started at kernel entry
+    int max_staged = -1;     // heads come in increasing order: the buffers hold max_staged and, earlier, max_staged - 1
     while (start < t_hi) {
+        const int n_round = round_size(start);
         // images of the (at most two) heads of this round
-        const int h_first = (int)(start / tiles_per_head), h_last = (int)((start + n_round - 1) / tiles_per_head);
+        const int h_first = start / p.tiles_per_head, h_last = (start + n_round - 1) / p.tiles_per_head;
         for (int hh = h_first; hh <= h_last; ++hh) {
-            if (resident[hh & 1] == hh) continue;
-            if (pending != hh) {
+            if (hh <= max_staged) continue;
+            if (max_staged >= 0) {                       // (the very first copy was started at kernel entry)
                 __syncthreads();                         // every read of the buffer's old image, by a lane or by an MMA, is over
                 if (threadIdx.x == 32)
                     stage_image_async(images + (hh & 1) * TC_IMG_FLOATS, p.Wimg + (long long)hh * TC_IMG_FLOATS, img_mbar);
             }
-            pending = -1;
             if (!shared_words[1] && !mbar_wait(img_mbar, img_phase)) {   // bounded, like every wait here
                 shared_words[1] = 1;
                 atomicOr(p.status, SQUAT_FLAG_DEVICE_TIMEOUT);
             }
             img_phase ^= 1;
-            resident[hh & 1] = hh;
+            max_staged = hh;
         }
-        const long long next_start = start + n_round;
-        const int n_next = round_size(next_start);
-        nxt.valid = false;
-        nxt.head = 0;
-        if (slot < n_next) locate(next_start + slot, true, nxt);
+        const bool valid = slot < n_round;
+        const bool nxt_valid = slot < round_size(start + n_round);
+        const void *nxt_row = nullptr;
+        if (nxt_valid) {
+            TileRows nxt;
+            locate(start + n_round + slot, nxt);
+            nxt_row = nxt.row;
+        }
+        TileRows cur;
+        cur.head = 0;
+        if (valid) locate(start + slot, cur);
 
         const float *img = images + (cur.head & 1) * TC_IMG_FLOATS;       // diagonal blocks | hi panels | lo panels
         const float *Bhi = img + TC_DIAG_FLOATS, *Blo = Bhi + TC_PANEL_FLOATS;
-        if (cur.valid) {
+        if (valid) {
 #pragma unroll 1
             for (int blk = 0; blk < NBLK; ++blk) {
                 u64 xp[BLK / 2];
@@ -491,7 +494,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 const bool more = blk + 1 < NBLK;
                 // prefetch: the next block of this tile, or the first block of the next round's tile
                 if (more) load_row<BF16>(raw, cur.row, (blk + 1) * BLK);
-                else if (nxt.valid) load_row<BF16>(raw, nxt.row, 0);
+                else if (nxt_valid) load_row<BF16>(raw, nxt_row, 0);
 
                 const float *diag = img + blk * BLK * BLK;
                 uint32_t cw[WORDS_PER_BLK];
@@ -534,26 +537,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 }
 
                 if (cur.active) {
-                    unsigned char *cp = p.codes + (cur.out_tok0 + cur.tok) * (D * BITS / 8) + blk * (BLK * BITS / 8);
+                    unsigned char *cp = cur.codes + blk * (BLK * BITS / 8);
                     if (WORDS_PER_BLK == 2)
                         *reinterpret_cast<uint2 *>(cp) = make_uint2(cw[0], cw[1]);
                     else
                         *reinterpret_cast<uint4 *>(cp) = make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
                     if (wteam == 0) {
-                        const long long o = (cur.out_tok0 / G + cur.grp) * D + blk * BLK + lane;
-                        p.scales[o] = my_scale;
-                        p.zeros[o] = my_zero;
+                        p.scales[cur.meta + blk * BLK] = my_scale;
+                        p.zeros[cur.meta + blk * BLK] = my_zero;
                         if (!(my_scale > 0.0f && my_scale < __int_as_float(0x7f800000)))
                             atomicOr(p.status, my_scale == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
                     }
                 }
             }
-        } else if (nxt.valid) {
-            load_row<BF16>(raw, nxt.row, 0);
+        } else if (nxt_valid) {
+            load_row<BF16>(raw, nxt_row, 0);
         }
-        cur = nxt;
-        start = next_start;
-        n_round = n_next;
+        start += n_round;
     }
 
     // Every committed batch has been waited for unless a wait ran out; then commit once more per slot and give the
@@ -602,8 +602,15 @@ __global__ void __launch_bounds__(256) pack_w_kernel(const float *__restrict__ W
 }
 
 template <int BITS, int NW>
-int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
+int launch_keys(KeyParams p, int dtype, cudaStream_t st)
 {
+    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
+    const long long tiles_per_head = (groups_per_head + 4 / NW - 1) / (4 / NW);
+    if (tiles_per_head * p.H > 0x7fffffffLL) return SQUAT_ERR_UNSUPPORTED;          // the kernel counts tiles in 32 bits
+    p.groups_per_head = (int)groups_per_head;
+    p.tiles_per_head = (int)tiles_per_head;
+    p.total_tiles = (int)(tiles_per_head * p.H);
+
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -613,10 +620,7 @@ int launch_keys(const KeyParams &p, int dtype, cudaStream_t st)
     // never share an SM
     const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + 2 * TC_IMG_FLOATS) +
                         sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * (TC_SLOTS + 1) + 4 * (2 + TC_SLOTS) + 8;
-    const long long groups_per_head = (long long)p.B * p.groups_per_bh;
-    const long long tiles_per_head = (groups_per_head + GPT - 1) / GPT;
-    const long long want = tiles_per_head * p.H;                                    // one tile per CTA at least
-    const int grid = (int)(want < sms ? want : sms);
+    const int grid = p.total_tiles < sms ? p.total_tiles : sms;                     // one tile per CTA at least
     if (dtype == SQUAT_BF16) {
         SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         quant_keys_kernel<BITS, NW, true><<<grid, TC_THREADS, smem, st>>>(p);
