@@ -17,20 +17,21 @@
 //   dense contractions (tokens x 32 errors) x (32 x later channels).  A tile is 128 tokens' worth of
 //   groups worked by 4 warps: row m of the tile = lane (m % 32) of the warp with warp % 4 == m / 32 =
 //   tensor-memory lane m.  Tensor memory holds, per tile, the fp32 accumulator D[128 x 96] of the
-//   corrections to channels 32 .. 127.  After the sweep of block b each warp writes its errors to
-//   shared memory as the tile's A operand (K-major 8 x 16-byte core matrices): the raw fp32 words
-//   serve as E_hi (the tensor core reads the top 19 bits of a word: tf32 by truncation) and
-//   E_lo = e - trunc(e) is exact in fp32.  The last of the tile's 4 warps to get there issues
+//   corrections to channels 32 .. 127 and, in the tile's other 32 columns, E_hi of the block just swept:
+//   the raw fp32 errors (the tensor core reads the top 19 bits of a word: tf32 by truncation).
+//   E_lo = e - trunc(e), exact in fp32, goes to shared memory as an A operand (K-major 8 x 16-byte core
+//   matrices).  After the sweep of block b the last of the tile's 4 warps to get there issues
 //        D[:, 32 b .. 95] (+)= E_lo * Whi_b + E_hi * Wlo_b + E_hi * Whi_b     (12 MMAs of 128 x (96 - 32 b) x 8)
-//   with W^T's off-diagonal panels split into tf32 hi / lo the same way (small terms first within a
-//   block: the accumulator truncates on every add) and commits them to the tile's mbarrier; nobody
-//   waits at a CTA or tile barrier.  Before the next sweep each warp waits for that phase (bounded),
-//   reads its 32 columns of D with tcgen05.ld -- one token per lane, no transpose -- and adds the keys.
+//   with W^T's off-diagonal panels split into tf32 hi / lo (small terms first within a block: the
+//   accumulator truncates on every add) and commits them to the tile's mbarrier; nobody waits at a CTA
+//   or tile barrier.  Before the next sweep each warp waits for that phase (bounded), reads its 32
+//   columns of D with tcgen05.ld -- one token per lane, no transpose -- and adds the keys.
 //
-// Per head the CTA stages 64 KB in shared memory: the four diagonal blocks (fp32) and the three
-// hi / lo panels, copied as they are from the image that pack_w_kernel writes when the update
-// matrices are built or imported.  CTAs are persistent over rounds (= 4 consecutive tiles of one head,
-// one per tile slot), taken in contiguous ranges so that a head is staged once per CTA that touches it.
+// Per head the kernel needs 64 KB in shared memory: the four diagonal blocks (fp32) and the three
+// hi / lo panels, copied as they are (cp.async.bulk, counted on an mbarrier) from the image that
+// pack_w_kernel writes when the update matrices are built or imported.  Two images fit (head h in buffer
+// h & 1).  CTAs are persistent: each takes a contiguous range of tiles and works it in rounds of up to 4
+// tiles, one per tile slot, sized as evenly as the range allows; a round may cross one head boundary.
 //
 // Work per key vector: 8128 fp32 multiply-adds (dense triangle, g = 1): 2032 on the CUDA cores
 // (sweeps), 6096 x 3 tf32 products on the tensor cores.
