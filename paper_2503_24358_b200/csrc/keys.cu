@@ -176,7 +176,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned mbar, unsigned parity)
     return false;
 }
 
-// Starts the copy of one head's 64 KB image into shared memory on the bulk-copy engine (no multicast); the bytes are
+// Starts the copy of one head's 64 KB image into shared memory on the bulk-copy engine (one CTA, one destination); the bytes are
 // counted on `mbar`, whose current phase completes when all of them have landed.
 __device__ __forceinline__ void stage_image_async(float *dst, const float *src, unsigned mbar)
 {
