@@ -53,10 +53,13 @@ def measured_peaks():
 
 
 # --------------------------------------------------------------------------- algorithmic counts
-def key_flops_per_vector(d, g):
-    """2 x FMAs of the dense block-triangular update (Eq. (3) / Eq. (update_block))."""
+def key_flops_per_vector(d, g, r=None):
+    """2 x FMAs of the update per key vector: the dense block-triangular form (Eq. (3) / Eq. (update_block)) or, if
+    cheaper, the rank-r form of the same update (2 r d FMAs) -- the algorithmic count is the smaller of the two,
+    whichever of them a kernel runs."""
     T = d // g
-    return 2 * sum(g * (d - t * g) for t in range(1, T))
+    tri = sum(g * (d - t * g) for t in range(1, T))
+    return 2 * (tri if r is None else min(tri, 2 * r * d))
 
 
 def key_fma_split(d, g, blk=32):
@@ -447,7 +450,7 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
         peaks = measured_peaks()
         elem = 4 if cfg.dtype == "f32" else 2
         key_ms = stage_ms["quantize_keys"]
-        flops = key_flops_per_vector(d, cfg.block_g) * vec_per_step
+        flops = key_flops_per_vector(d, cfg.block_g, cfg.rank_r) * vec_per_step
         kbytes = bytes_per_vector(d, bits, G, elem) * vec_per_step
         alu_time_ms = flops / (ALU_PEAK_TFLOPS * 1e12) * 1e3
         hbm_time_ms = kbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
@@ -507,11 +510,17 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="workload index (default 1: Llama-2-7B-shaped layer)")
+    ap.add_argument("--bits", type=int, default=None, choices=[2, 4], help="override the workload's code width")
+    ap.add_argument("--rank", type=int, default=None, help="override the workload's subspace rank r")
+    ap.add_argument("--group-size", type=int, default=None, choices=[32, 64, 128], help="override the workload's group size G")
     ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     args = ap.parse_args()
     cfg = si.get_config(args.config)
+    over = {k: v for k, v in (("bits", args.bits), ("rank_r", args.rank), ("group_size", args.group_size)) if v is not None}
+    if over:                                             # one point of a workload's (bits, r, G) sweep
+        cfg = cfg.with_(**over)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

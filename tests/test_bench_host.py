@@ -42,6 +42,8 @@ def test_algorithmic_counts():
     assert bench.key_flops_per_vector(128, 1) == 2 * 8128
     assert bench.key_flops_per_vector(128, 32) == 2 * 6144
     assert bench.key_flops_per_vector(128, 64) == 2 * 4096
+    assert bench.key_flops_per_vector(128, 1, 32) == 2 * 8128          # r = 32: the triangle (8128) beats 2 r d = 8192
+    assert bench.key_flops_per_vector(128, 1, 8) == 2 * 2048           # r = 8: the rank-r form is the cheaper count
     assert bench.key_fma_split(128, 1) == (4 * 496, 8128 - 4 * 496)      # four 32 x 32 triangles stay on the FP32 pipes
     assert sum(bench.key_fma_split(128, 32)) == 6144 and bench.key_fma_split(128, 32)[0] == 0
     assert sum(bench.key_fma_split(128, 64)) == 4096
