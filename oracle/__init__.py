@@ -210,6 +210,32 @@ def decode_attention_over_cache(q, k_codes, k_scale, k_zero, v_codes, v_scale, v
     return attention_decode(q, Kd, Vd)
 
 
+def rope_rows(X, pos, base=10000.0):
+    """Rotary position embedding of the rows X [n, d] at integer positions pos [n] (Section 4, the variant
+    that stores keys before the embedding); returns a new array."""
+    X = np.array(X, dtype=np.float64, order="C", copy=True)
+    n, d = X.shape
+    pos = np.ascontiguousarray(pos, dtype=np.int64)
+    assert pos.shape == (n,)
+    posl = (ctypes.c_long * n)(*[int(v) for v in pos])
+    _check(_load().sqo_rope_rows(_p(X, _D), ctypes.c_long(n), d, posl, ctypes.c_double(base)), "rope_rows")
+    return X
+
+
+def decode_attention_over_pre_rope_cache(q, k_codes, k_scale, k_zero, v_codes, v_scale, v_zero, G, first_pos,
+                                         k_res=None, v_res=None, base=10000.0):
+    """decode_attention_over_cache for a cache whose keys were quantized BEFORE the rotary embedding: cached
+    token t (and then the residual rows) sits at position first_pos + t; its dequantized key row is rotated
+    there, the query comes already rotated at its own position.  Marshalling only."""
+    Kd = dequant_keys(k_codes, k_scale, k_zero, G) if len(k_codes) else np.zeros((0, np.asarray(q).shape[-1]))
+    Vd = dequant_values(v_codes, v_scale, v_zero, G) if len(v_codes) else np.zeros_like(Kd)
+    if k_res is not None and len(k_res):
+        Kd = np.concatenate([Kd, np.asarray(k_res, dtype=np.float64)], axis=0)
+        Vd = np.concatenate([Vd, np.asarray(v_res, dtype=np.float64)], axis=0)
+    Kr = rope_rows(Kd, first_pos + np.arange(Kd.shape[0]), base)
+    return attention_decode(q, Kr, Vd)
+
+
 def kv_cache_bytes(batch, seq_len, layers, heads, head_dim, bytes_per_param):
     return int(_load().sqo_kv_cache_bytes(batch, seq_len, layers, heads, head_dim, bytes_per_param))
 

@@ -23,6 +23,10 @@
  *   sqo_attention_decode                           Section 2 "(Masked) Attention mechanism": one decode step,
  *                                                  softmax(q K^T / sqrt(d)) V over the cached tokens (the
  *                                                  score vector w^deq of the proof of Theorem 1)
+ *   sqo_rope_rows                                  Section 4, the variant that stores keys before the rotary
+ *                                                  position embedding: the embedding a reader applies to
+ *                                                  the dequantized rows (rotation of the channel pairs
+ *                                                  (i, i + d/2) by pos * base^(-2i/d))
  *
  * Pins (tests, CPU only): the chain of Lemma 4 against direct inverses; B_t H_t against a
  * generic KKT solve of Eq. (2) and against the LDL^T factor of P_inv; lambda = 0 / r = 0
@@ -31,7 +35,9 @@
  * SVD; the value path against a library float32 computation; the memory formula against
  * the worked example printed in Appendix B; the decode-step attention against a loop-by-loop
  * restatement, its closed forms (zero query = mean of the values, one dominant score) and the
- * bound of Theorem 1.  The paper prints no input/output pair for the quantizer itself.
+ * bound of Theorem 1; the rotary embedding against explicit 2 x 2 rotation matrices, position 0,
+ * norms, and the relative-position property of the scores.  The paper prints no input/output
+ * pair for the quantizer itself.
  *
  * Readings of the paper where it is silent (same list as the design notes):
  *   - rounding is round-half-to-even;
@@ -41,7 +47,10 @@
  *   - the value fed back is the one a reader of the cache reconstructs, i.e. computed from
  *     the stored float32 scale and zero-point;
  *   - scale and zero-point are stored as float32;
- *   - channels are visited in natural order.
+ *   - channels are visited in natural order;
+ *   - the rotary embedding (the paper only names it) pairs channel i with channel i + d/2 and
+ *     uses the angles pos * base^(-2i/d), i < d/2: the convention of the Llama family the
+ *     paper evaluates.
  */
 #include <math.h>
 #include <stdint.h>
@@ -529,5 +538,29 @@ int sqo_attention_decode(const double *q, int nq, const double *K, const double 
         }
     }
     free(w);
+    return SQO_OK;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Rotary position embedding of n rows X [n, d] (d even), in place: for row t at position
+ * pos[t] and every i < d/2, with angle a = pos[t] * base^(-2 i / d),
+ *     (x_i, x_{i + d/2})  <-  (x_i cos a - x_{i + d/2} sin a,  x_i sin a + x_{i + d/2} cos a).
+ * The variant of Section 4 that quantizes keys before the embedding stores un-rotated rows; a
+ * reader applies this to each dequantized (and each residual) key row at that row's position
+ * before the scores of sqo_attention_decode are formed. */
+int sqo_rope_rows(double *X, long n, int d, const long *pos, double base)
+{
+    if (!X || !pos || n < 0 || d <= 0 || (d & 1) || !(base > 0.0)) return SQO_ERR_ARG;
+    const int half = d / 2;
+    for (long t = 0; t < n; ++t) {
+        for (int i = 0; i < half; ++i) {
+            const double theta = pow(base, -2.0 * (double)i / (double)d);
+            const double a = (double)pos[t] * theta;
+            const double c = cos(a), sn = sin(a);
+            const double x0 = X[t * d + i], x1 = X[t * d + i + half];
+            X[t * d + i] = x0 * c - x1 * sn;
+            X[t * d + i + half] = x0 * sn + x1 * c;
+        }
+    }
     return SQO_OK;
 }
