@@ -191,6 +191,36 @@ int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads,
                            float softmax_scale, float *out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same decode step over a cache whose keys were quantized BEFORE the rotary position embedding (Section 4:
+ * the variant of the method that "quantizes and stores the KV cache before applying RoPE" and applies the
+ * embedding on the fly after dequantization).  The write path is the one above, fed with un-rotated keys and a
+ * subspace built from un-rotated queries; the cost of the embedding moves to this reader.
+ *
+ *   k_i  =  rope( deq(cached row i),  first_pos + i ),   then the residual rows at the positions that follow;
+ *   rope(x, P): every channel pair (c, c + d/2), c < d/2, turns by the angle P * base^(-2c/d)
+ *               (x_c, x_{c+d/2}) <- (x_c cos - x_{c+d/2} sin, x_c sin + x_{c+d/2} cos)
+ *   -- the pairing and angles of the Llama family the paper evaluates; the paper itself only names the embedding.
+ *   q comes already rotated at its own position; values are not rotated.
+ *
+ * rope_table   device, 16-byte aligned, squat_rope_table_floats(table_positions) floats as filled (on the host, in
+ *              float64, then rounded) by squat_rope_table_fill(base, d, table_positions, .) and copied by the
+ *              caller: (cos, sin) of 32 a theta_c for a < ceil(table_positions / 32), then of l theta_c for l < 32.
+ *              Must cover every position used: first_pos + n_tokens + n_res <= table_positions.
+ * first_pos    position of cached token 0 of every (b, h); >= 0 and a multiple of 32.
+ * Everything else as for squat_decode_attention.  Errors: the same, plus SQUAT_ERR_SHAPE for a first_pos that is
+ * not a multiple of 32 or a table that is too short.
+ */
+size_t squat_rope_table_floats(int n_positions);
+int squat_rope_table_fill(double base, int head_dim, int n_positions, float *table_host);
+int squat_decode_attention_pre_rope(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                                    const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
+                                    const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                                    int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                                    int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                                    float softmax_scale, const float *rope_table, int table_positions,
+                                    long long first_pos, float *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Gram matrices of the stacked prompt queries without any allocation.  (The paper has no counterpart:
  * this entry exists for callers that must not allocate.)
  *

@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = (
     "squat_write_path_workspace_bytes", "squat_write_path_host", "squat_get_device_status",
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
+    "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
 )
 
 _lib = None
@@ -274,6 +275,47 @@ def squat_decode_attention(q: torch.Tensor, k_codes, k_scales, k_zeros, v_codes,
                                           _dev(out, "out"), _dev(workspace, "workspace"),
                                           workspace.numel() * workspace.element_size(), _stream(stream)),
            "squat_decode_attention")
+
+
+def squat_rope_table(n_positions: int, base: float = 10000.0, head_dim: int = 128) -> torch.Tensor:
+    """The rotary tables squat_decode_attention_pre_rope reads, as a CPU float32 tensor (the caller moves it to the
+    device): filled by the library on the host in float64."""
+    lib = _load()
+    lib.squat_rope_table_floats.restype = ctypes.c_size_t
+    n = int(lib.squat_rope_table_floats(int(n_positions)))
+    t = torch.empty(n, dtype=torch.float32)
+    _check(lib.squat_rope_table_fill(ctypes.c_double(base), int(head_dim), int(n_positions),
+                                     ctypes.c_void_p(t.data_ptr())), "squat_rope_table_fill")
+    return t
+
+
+def squat_decode_attention_pre_rope(q: torch.Tensor, k_codes, k_scales, k_zeros, v_codes, v_scales, v_zeros,
+                                    n_kv_heads: int, n_tokens: int, bits: int, group_size: int, out: torch.Tensor,
+                                    workspace: torch.Tensor, rope_table: torch.Tensor, table_positions: int,
+                                    first_pos: int = 0, k_res: torch.Tensor = None, v_res: torch.Tensor = None,
+                                    softmax_scale: float = 0.0, cache_stride_b: int = None, cache_stride_h: int = None,
+                                    stream=None):
+    """squat_decode_attention over a cache whose keys (and residual keys) were stored before the rotary position
+    embedding: cached token t sits at position first_pos + t.  rope_table: squat_rope_table(table_positions) on the
+    device."""
+    if q.dim() != 3 or not q.is_contiguous() or not out.is_contiguous() or out.dtype != torch.float32:
+        raise ValueError("q must be contiguous [batch, n_q_heads, d]; out contiguous float32")
+    if rope_table.dtype != torch.float32 or not rope_table.is_contiguous():
+        raise ValueError("rope_table must be a contiguous float32 tensor")
+    B, Hq, d = q.shape
+    csh = n_tokens if cache_stride_h is None else cache_stride_h
+    csb = n_kv_heads * csh if cache_stride_b is None else cache_stride_b
+    n_res = 0 if k_res is None else k_res.shape[2]
+    if n_res and (not k_res.is_contiguous() or not v_res.is_contiguous() or k_res.dtype != v_res.dtype):
+        raise ValueError("k_res and v_res must be contiguous [batch, n_kv_heads, n_res, d] of one dtype")
+    opt = lambda t, n: _dev(t, n) if t is not None and t.numel() else None
+    _check(_load().squat_decode_attention_pre_rope(
+        _dev(q, "q"), _dtype_code(q), B, Hq, n_kv_heads, d, opt(k_codes, "k_codes"), opt(k_scales, "k_scales"),
+        opt(k_zeros, "k_zeros"), opt(v_codes, "v_codes"), opt(v_scales, "v_scales"), opt(v_zeros, "v_zeros"), n_tokens,
+        ctypes.c_longlong(csb), ctypes.c_longlong(csh), bits, group_size, opt(k_res, "k_res"), opt(v_res, "v_res"),
+        _dtype_code(k_res) if n_res else SQUAT_F32, n_res, ctypes.c_float(softmax_scale), _dev(rope_table, "rope_table"),
+        int(table_positions), ctypes.c_longlong(first_pos), _dev(out, "out"), _dev(workspace, "workspace"),
+        ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)), "squat_decode_attention_pre_rope")
 
 
 def squat_get_device_status(clear: bool = True, stream=None) -> int:

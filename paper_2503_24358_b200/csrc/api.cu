@@ -282,12 +282,14 @@ size_t squat_decode_attention_workspace_bytes(int batch, int n_q_heads, int n_to
     return (squat_attention_workspace_floats(batch, n_q_heads, n_tokens) * sizeof(float) + 255) / 256 * 256 + 256;
 }
 
-int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
-                           const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
-                           const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
-                           int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
-                           int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
-                           float softmax_scale, float *out, void *workspace, size_t workspace_bytes, void *stream)
+namespace {
+int decode_attention_impl(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                          const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
+                          const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                          int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                          int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                          float softmax_scale, float *out, void *workspace, size_t workspace_bytes,
+                          const float *rope_table, int rope_blocks, long long first_pos, void *stream)
 {
     if (!valid_dtype(q_dtype) || batch < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_tokens < 0 || n_res < 0)
         return SQUAT_ERR_INVALID_ARG;
@@ -313,7 +315,63 @@ int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads,
     return squat_launch_decode_attention(q, q_dtype, batch, n_q_heads, n_kv_heads, n_tokens, k_codes, k_scales, k_zeros,
                                          v_codes, v_scales, v_zeros, cache_stride_b, cache_stride_h, bits, group_size,
                                          k_res, v_res, res_dtype, n_res, scale, out, static_cast<float *>(workspace),
-                                         static_cast<cudaStream_t>(stream));
+                                         rope_table, rope_blocks, first_pos, static_cast<cudaStream_t>(stream));
+}
+}  // namespace
+
+int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                           const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
+                           const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                           int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                           int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                           float softmax_scale, float *out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return decode_attention_impl(q, q_dtype, batch, n_q_heads, n_kv_heads, head_dim, k_codes, k_scales, k_zeros, v_codes,
+                                 v_scales, v_zeros, n_tokens, cache_stride_b, cache_stride_h, bits, group_size, k_res, v_res,
+                                 res_dtype, n_res, softmax_scale, out, workspace, workspace_bytes, nullptr, 0, 0, stream);
+}
+
+size_t squat_rope_table_floats(int n_positions)
+{
+    if (n_positions <= 0) return 0;
+    return ((size_t)(n_positions + 31) / 32 + 32) * 64 * 2;
+}
+
+int squat_rope_table_fill(double base, int head_dim, int n_positions, float *table_host)
+{
+    if (!table_host || n_positions <= 0 || !(base > 0.0)) return SQUAT_ERR_INVALID_ARG;
+    if (head_dim != D) return SQUAT_ERR_UNSUPPORTED;
+    const int nb = (n_positions + 31) / 32, half = D / 2;
+    for (int part = 0; part < 2; ++part) {
+        const int rows = part == 0 ? nb : 32;
+        float *t = table_host + (part == 0 ? 0 : (size_t)nb * half * 2);
+        for (int r = 0; r < rows; ++r)
+            for (int i = 0; i < half; ++i) {
+                const double pos = part == 0 ? 32.0 * r : (double)r;
+                const double a = pos * std::pow(base, -2.0 * i / (double)D);
+                t[((size_t)r * half + i) * 2] = (float)std::cos(a);
+                t[((size_t)r * half + i) * 2 + 1] = (float)std::sin(a);
+            }
+    }
+    return SQUAT_OK;
+}
+
+int squat_decode_attention_pre_rope(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                                    const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
+                                    const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                                    int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                                    int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                                    float softmax_scale, const float *rope_table, int table_positions,
+                                    long long first_pos, float *out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!rope_table || table_positions <= 0 || first_pos < 0 || n_tokens < 0 || n_res < 0) return SQUAT_ERR_INVALID_ARG;
+    if (!aligned16(rope_table)) return SQUAT_ERR_INVALID_ARG;
+    if (first_pos % 32 != 0) return SQUAT_ERR_SHAPE;
+    if (first_pos + n_tokens + n_res > table_positions) return SQUAT_ERR_SHAPE;
+    return decode_attention_impl(q, q_dtype, batch, n_q_heads, n_kv_heads, head_dim, k_codes, k_scales, k_zeros, v_codes,
+                                 v_scales, v_zeros, n_tokens, cache_stride_b, cache_stride_h, bits, group_size, k_res, v_res,
+                                 res_dtype, n_res, softmax_scale, out, workspace, workspace_bytes, rope_table,
+                                 (table_positions + 31) / 32, first_pos, stream);
 }
 
 int squat_get_device_status(void *stream, unsigned *flags, int clear)

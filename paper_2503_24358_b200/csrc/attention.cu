@@ -20,6 +20,15 @@
 //                       and merges the chunks with the usual max / denominator rescaling.
 //
 // Bound: HBM (bits/8 + metadata bytes per cached element); the unpacking arithmetic is close behind.
+//
+// Keys stored BEFORE the rotary position embedding (Section 4, the "pre" variant): the reader applies the
+// embedding on the fly.  Token t of the cache sits at position P = first_pos + t; channel pair (i, i + 64) of its
+// dequantized key turns by the angle P * base^(-2i/128).  With P = 32 a + l the turn is the product of a block
+// turn (32 a theta_i: the same for the 32 tokens of a warp step, so it is applied to the query instead, with the
+// opposite sign) and a lane turn (l theta_i: a table in shared memory, one entry per lane and pair).  Cosines and
+// sines come from two tables the host fills in float64 (squat_rope_table_fill); the kernel only multiplies.  The
+// key metadata cannot be folded into the query on this path: each pair is dequantized (one FMA per element),
+// turned (4) and multiplied with the block-turned query of every head (2 per head).
 #include "squat_internal.cuh"
 
 namespace {
@@ -44,6 +53,9 @@ struct AttnParams {
     float *ml;                 // [B, Hq, nchunk, 2]
     int nchunk, chunk;         // chunk: tokens per CTA, a multiple of 256
     float *out;                // [B, Hq, D]
+    // rotary tables (pre-embedding key storage only): cos/sin of (32 a theta_i) [blocks][64] and of (l theta_i) [32][64]
+    const float2 *rope_a, *rope_b;
+    long long first_pos;       // position of cached token 0; a multiple of 32
 };
 
 // 1 + code / 2^BITS as a float, for the code at position i of a 32-bit word (low bits first)
@@ -76,8 +88,8 @@ __device__ __forceinline__ float load_elem(const void *p, long long idx, int bf1
     return reinterpret_cast<const float *>(p)[idx];
 }
 
-template <int BITS, int NQ>
-__global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? 3 : 1) attn_partial_kernel(const AttnParams p)
+template <int BITS, int NQ, bool ROPE>
+__global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : 1) attn_partial_kernel(const AttnParams p)
 {
     constexpr int WPT = D * BITS / 32;                          // 32-bit words per token: 8 or 16
     constexpr int CPW = 32 / BITS;                              // codes per word: 16 or 8
@@ -87,6 +99,8 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? 3 : 1) attn_partial_kern
     float *qs = qsm + NQ * D;                                   // [warps][NQ][D] query x key scale x 2^BITS of the warp's group
     float *sc = qs + AT_WARPS * NQ * D;                         // [NQ][AT_CHUNK] scores, then weights
     float *red = sc + NQ * AT_CHUNK;                            // [NQ][warps] and [NQ] scratch of the reductions
+    float2 *lane_turn = reinterpret_cast<float2 *>(red + NQ * AT_WARPS + 8);   // ROPE: [64][32] cos/sin of (lane theta_i)
+    float4 *sz_all = reinterpret_cast<float4 *>(lane_turn + 64 * 32);           // ROPE: [warps][64] (S_i, Z_i, S_{i+64}, Z_{i+64})
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunk = blockIdx.x % p.nchunk, qpass = blockIdx.x / p.nchunk;
     const int h = blockIdx.y, b = blockIdx.z;
@@ -100,12 +114,64 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? 3 : 1) attn_partial_kern
         const int qi = i / D, c = i % D;
         qsm[i] = qi < nq_here ? p.scale * load_elem(p.q, ((long long)b * p.Hq + hq0 + qi) * D + c, p.q_bf16) : 0.0f;
     }
+    if (ROPE) {
+        for (int i = tid; i < 64 * 32; i += AT_THREADS) lane_turn[i] = __ldg(p.rope_b + (i & 31) * 64 + (i >> 5));   // [pair][lane]
+    }
     __syncthreads();
 
     // ---------------------------------------------------------------- key phase: scores
     float *qsw = qs + warp * NQ * D;
     for (int blk = t0 + 32 * warp; blk < t1; blk += 32 * AT_WARPS) {
         const long long mrow = (ctok0 / p.G + blk / p.G) * D;
+        if (ROPE) {
+            // ---- keys stored before the rotary embedding
+            const long long a_blk = (p.first_pos + blk) >> 5;          // block turn: the same for the warp's 32 tokens
+            float2 *qb = reinterpret_cast<float2 *>(qsw);              // [NQ][64]: the heads' queries turned back by the block turn
+            float4 *sz = sz_all + warp * 64;
+            __syncwarp();
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int i = lane + 32 * hh;
+                const float2 cs = __ldg(p.rope_a + a_blk * 64 + i);
+#pragma unroll
+                for (int qi = 0; qi < NQ; ++qi) {
+                    const float q0 = qsm[qi * D + i], q1 = qsm[qi * D + i + 64];
+                    qb[qi * 64 + i] = make_float2(fmaf(q0, cs.x, q1 * cs.y), fmaf(q1, cs.x, -q0 * cs.y));
+                }
+                const float s0 = __ldg(p.ks + mrow + i) * LV, s1 = __ldg(p.ks + mrow + i + 64) * LV;
+                sz[i] = make_float4(s0, __ldg(p.kz + mrow + i) - s0, s1, __ldg(p.kz + mrow + i + 64) - s1);
+            }
+            __syncwarp();
+            const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
+            uint32_t wd[WPT];
+#pragma unroll
+            for (int v4 = 0; v4 < WPT / 4; ++v4) {
+                const uint4 cw = __ldg(cp + v4);
+                wd[4 * v4] = cw.x; wd[4 * v4 + 1] = cw.y; wd[4 * v4 + 2] = cw.z; wd[4 * v4 + 3] = cw.w;
+            }
+            float acc[NQ][2];
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) acc[qi][0] = acc[qi][1] = 0.0f;
+#pragma unroll
+            for (int wi = 0; wi < WPT / 2; ++wi)
+#pragma unroll
+                for (int pos = 0; pos < CPW; ++pos) {
+                    const int i = wi * CPW + pos;                       // pair (i, i + 64): same code position, WPT / 2 words apart
+                    const float4 m4 = sz[i];
+                    const float k0 = fmaf(code_as_float<BITS>(wd[wi], pos), m4.x, m4.y);
+                    const float k1 = fmaf(code_as_float<BITS>(wd[wi + WPT / 2], pos), m4.z, m4.w);
+                    const float2 cs = lane_turn[i * 32 + lane];
+                    const float r0 = fmaf(k0, cs.x, -k1 * cs.y), r1 = fmaf(k0, cs.y, k1 * cs.x);
+#pragma unroll
+                    for (int qi = 0; qi < NQ; ++qi) {
+                        const float2 qq = qb[qi * 64 + i];
+                        acc[qi][pos & 1] = fmaf(r1, qq.y, fmaf(r0, qq.x, acc[qi][pos & 1]));
+                    }
+                }
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) sc[qi * AT_CHUNK + blk - t0 + lane] = acc[qi][0] + acc[qi][1];
+            continue;
+        }
         const float4 s4 = __ldg(reinterpret_cast<const float4 *>(p.ks + mrow) + lane);
         const float4 z4 = __ldg(reinterpret_cast<const float4 *>(p.kz + mrow) + lane);
         float k0[NQ];
@@ -286,6 +352,24 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
             } else {
                 k4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.k_res) + rbase + (long long)t * D) + lane);
             }
+            if (p.rope_a) {
+                // residual rows are stored before the rotary embedding too: turn row t at position first_pos + T + t.
+                // Lane l < 16 holds channels 4 l .. 4 l + 3, lane l + 16 their partners 64 channels up.
+                const long long pos = p.first_pos + p.T + t;
+                const float4 o4 = make_float4(__shfl_xor_sync(0xffffffffu, k4.x, 16), __shfl_xor_sync(0xffffffffu, k4.y, 16),
+                                              __shfl_xor_sync(0xffffffffu, k4.z, 16), __shfl_xor_sync(0xffffffffu, k4.w, 16));
+                const float sign = lane < 16 ? -1.0f : 1.0f;
+                const float own[4] = {k4.x, k4.y, k4.z, k4.w}, oth[4] = {o4.x, o4.y, o4.z, o4.w};
+                float rot[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = 4 * (lane & 15) + e;
+                    const float2 ca = __ldg(p.rope_a + (pos >> 5) * 64 + i), cb = __ldg(p.rope_b + (pos & 31) * 64 + i);
+                    const float cc = fmaf(ca.x, cb.x, -ca.y * cb.y), ss = fmaf(ca.y, cb.x, ca.x * cb.y);
+                    rot[e] = fmaf(own[e], cc, sign * oth[e] * ss);
+                }
+                k4 = make_float4(rot[0], rot[1], rot[2], rot[3]);
+            }
             const float s = warp_sum_f(fmaf(q4.x, k4.x, fmaf(q4.y, k4.y, fmaf(q4.z, k4.z, q4.w * k4.w))));
             if (lane == 0) w[t] = s;
         }
@@ -316,15 +400,21 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
     p.out[((long long)b * p.Hq + hq) * D + c] = acc / den;
 }
 
-template <int BITS, int NQ>
-int launch_partial(const AttnParams &p, int qpasses, cudaStream_t st)
+template <int BITS, int NQ, bool ROPE>
+int launch_partial_r(const AttnParams &p, int qpasses, cudaStream_t st)
 {
-    const size_t smem = sizeof(float) * (NQ * D + AT_WARPS * NQ * D + NQ * AT_CHUNK + NQ * AT_WARPS + 8);
-    SQUAT_CUDA(cudaFuncSetAttribute(attn_partial_kernel<BITS, NQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_partial_kernel<BITS, NQ><<<dim3(p.nchunk * qpasses, p.H, p.B), AT_THREADS, smem, st>>>(p);
+    const size_t smem = sizeof(float) * (NQ * D + AT_WARPS * NQ * D + NQ * AT_CHUNK + NQ * AT_WARPS + 8) +
+                        (ROPE ? sizeof(float2) * 64 * 32 + sizeof(float4) * AT_WARPS * 64 : 0);
+    SQUAT_CUDA(cudaFuncSetAttribute(attn_partial_kernel<BITS, NQ, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attn_partial_kernel<BITS, NQ, ROPE><<<dim3(p.nchunk * qpasses, p.H, p.B), AT_THREADS, smem, st>>>(p);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
+}
+template <int BITS, int NQ>
+int launch_partial(const AttnParams &p, int qpasses, cudaStream_t st)
+{
+    return p.rope_a ? launch_partial_r<BITS, NQ, true>(p, qpasses, st) : launch_partial_r<BITS, NQ, false>(p, qpasses, st);
 }
 
 }  // namespace
@@ -340,9 +430,13 @@ int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq,
                                   const unsigned char *vc, const float *vs, const float *vz,
                                   long long csb, long long csh, int bits, int G,
                                   const void *k_res, const void *v_res, int res_dtype, int R,
-                                  float scale, float *out, float *workspace, cudaStream_t st)
+                                  float scale, float *out, float *workspace,
+                                  const float *rope_table, int rope_blocks, long long first_pos, cudaStream_t st)
 {
     AttnParams p;
+    p.rope_a = reinterpret_cast<const float2 *>(rope_table);                     // NULL: keys were stored after the embedding
+    p.rope_b = p.rope_a ? p.rope_a + (size_t)rope_blocks * 64 : nullptr;
+    p.first_pos = first_pos;
     p.q = q; p.q_bf16 = q_dtype == SQUAT_BF16; p.B = batch; p.Hq = Hq; p.H = H; p.T = T;
     p.kc = kc; p.vc = vc; p.ks = ks; p.kz = kz; p.vs = vs; p.vz = vz; p.csb = csb; p.csh = csh; p.G = G;
     p.k_res = k_res; p.v_res = v_res; p.res_bf16 = res_dtype == SQUAT_BF16; p.R = R;

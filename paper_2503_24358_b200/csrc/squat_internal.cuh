@@ -55,7 +55,8 @@ int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq,
                                   const unsigned char *vc, const float *vs, const float *vz,
                                   long long csb, long long csh, int bits, int G,
                                   const void *k_res, const void *v_res, int res_dtype, int R,
-                                  float scale, float *out, float *workspace, cudaStream_t st);
+                                  float scale, float *out, float *workspace,
+                                  const float *rope_table, int rope_blocks, long long first_pos, cudaStream_t st);
 int squat_launch_dequant(int kind, const unsigned char *codes, const float *scales, const float *zeros,
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
                          void *out, int out_dtype, cudaStream_t st);

@@ -84,3 +84,18 @@ def test_package_does_not_import_the_oracle():
     for f in os.listdir(os.path.join(ROOT, "oracle")):
         if f.endswith((".py", ".c", ".h")):
             assert "paper_2503_24358_b200" not in open(os.path.join(ROOT, "oracle", f)).read(), f
+
+
+def test_rope_table_is_cos_sin_of_block_and_lane_angles():
+    # host-side function of the library (no GPU): (cos, sin) of 32 a theta_i for every block a of 32 positions, then of
+    # l theta_i for l < 32, theta_i = base^(-2 i / 128) -- checked against math.cos / math.sin
+    import math
+    import paper_2503_24358_b200 as sq
+    for base, npos in ((10000.0, 100), (500000.0, 33)):
+        t = sq.squat_rope_table(npos, base).numpy().reshape(-1, 64, 2)
+        nb = (npos + 31) // 32
+        assert t.shape[0] == nb + 32
+        for row, pos in [(a, 32 * a) for a in range(nb)] + [(nb + l, l) for l in range(32)]:
+            for i in (0, 1, 31, 63):
+                ang = pos * base ** (-2.0 * i / 128)
+                assert abs(t[row, i, 0] - math.cos(ang)) <= 6e-8 and abs(t[row, i, 1] - math.sin(ang)) <= 6e-8

@@ -175,3 +175,89 @@ def test_attention_argument_errors():
     big = torch.zeros(B, H, 129, D).cuda()
     with pytest.raises(sq.SquatError):                       # residual buffer beyond the supported length
         sq.squat_decode_attention(q, *cache, H, T, bits, G, out, ws, big, big)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Keys stored before the rotary position embedding (Section 4, the "pre" variant): the reader turns every
+# dequantized key row at its position.  Oracle: dequantize, rope_rows at first_pos + t, attention in float64.
+
+def _run_pre(q, cache, H, T, bits, G, first_pos, table_positions, k_res=None, v_res=None, base=10000.0):
+    B, Hq, _ = q.shape
+    out = torch.empty((B, Hq, D), dtype=torch.float32, device="cuda")
+    ws = torch.empty(sq.squat_decode_attention_workspace_bytes(B, Hq, T), dtype=torch.uint8, device="cuda")
+    table = sq.squat_rope_table(table_positions, base).cuda()
+    sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, table_positions, first_pos, k_res, v_res)
+    torch.cuda.synchronize()
+    return out.cpu().numpy().astype(np.float64)
+
+
+def _check_pre(out, q_used, units, H, G, first_pos, k_res=None, v_res=None, T=None, base=10000.0):
+    B, Hq, _ = q_used.shape
+    qpk = Hq // H
+    worst = 0.0
+    for b in range(B):
+        for h in range(H):
+            kq, vq = units[b, h]
+            n = kq["codes"].shape[0] if T is None else T
+            ref = oracle.decode_attention_over_pre_rope_cache(
+                q_used[b, h * qpk:(h + 1) * qpk], kq["codes"][:n], kq["scale"][:n // G], kq["zero"][:n // G],
+                vq["codes"][:n], vq["scale"][:n], vq["zero"][:n], G, first_pos,
+                None if k_res is None else k_res[b, h], None if v_res is None else v_res[b, h], base)
+            worst = max(worst, np.abs(out[b, h * qpk:(h + 1) * qpk] - ref).max())
+    assert worst <= ATOL, worst
+    return worst
+
+
+@pytest.mark.parametrize("bits,G,qpk,T,R,first_pos,res_dtype", [
+    (2, 32, 1, 256, 0, 0, torch.float32),          # MHA, cache from position 0, no residual buffer
+    (2, 32, 4, 2112, 32, 4096, torch.bfloat16),    # GQA 4:1, 3 chunks with a ragged one, positions 4096 .. 6239
+    (4, 64, 2, 1088, 128, 32, torch.float32),      # 4-bit codes, full residual buffer
+    (2, 128, 8, 128, 5, 8064, torch.float32),      # two passes over the cache (8 query heads per KV head)
+    (4, 32, 3, 96, 1, 0, torch.bfloat16),
+])
+def test_pre_rope_reader_matches_the_oracle(bits, G, qpk, T, R, first_pos, res_dtype):
+    B, H = 2, 2
+    cache, units = _oracle_cache(40 + bits + G + qpk, B, H, T, bits, G)
+    g = torch.Generator().manual_seed(T + R + first_pos)
+    q = torch.randn(B, H * qpk, D, generator=g).to(torch.bfloat16).cuda()
+    k_res = v_res = None
+    if R:
+        k_res = torch.randn(B, H, R, D, generator=g).to(res_dtype).cuda()
+        v_res = torch.randn(B, H, R, D, generator=g).to(res_dtype).cuda()
+    out = _run_pre(q, cache, H, T, bits, G, first_pos, first_pos + T + R, k_res, v_res)
+    kr = None if k_res is None else k_res.double().cpu().numpy()
+    vr = None if v_res is None else v_res.double().cpu().numpy()
+    print("max err", _check_pre(out, q.double().cpu().numpy(), units, H, G, first_pos, kr, vr))
+
+
+def test_pre_rope_reader_special_cases():
+    B, H, T, bits, G = 1, 2, 512, 2, 32
+    cache, units = _oracle_cache(7, B, H, T, bits, G)
+    g = torch.Generator().manual_seed(11)
+    q = torch.randn(B, H, D, generator=g).cuda()
+    k_res, v_res = torch.randn(B, H, 16, D, generator=g).cuda(), torch.randn(B, H, 16, D, generator=g).cuda()
+    kr, vr = k_res.double().cpu().numpy(), v_res.double().cpu().numpy()
+    qn = q.double().cpu().numpy()
+    # another base (Llama-3.1 uses 500000)
+    out = _run_pre(q, cache, H, T, bits, G, 64, 1024, k_res, v_res, base=500000.0)
+    _check_pre(out, qn, units, H, G, 64, kr, vr, base=500000.0)
+    # only the residual buffer, at positions 96 ..
+    out = _run_pre(q, cache, H, 0, bits, G, 96, 256, k_res, v_res)
+    _check_pre(out, qn, units, H, G, 96, kr, vr, T=0)
+    # a prefix of a longer cache
+    out = torch.empty((B, H, D), dtype=torch.float32, device="cuda")
+    ws = torch.empty(sq.squat_decode_attention_workspace_bytes(B, H, 192), dtype=torch.uint8, device="cuda")
+    table = sq.squat_rope_table(1024).cuda()
+    sq.squat_decode_attention_pre_rope(q, *cache, H, 192, bits, G, out, ws, table, 1024, 0, k_res, v_res,
+                                       cache_stride_b=H * T, cache_stride_h=T)
+    torch.cuda.synchronize()
+    _check_pre(out.cpu().numpy().astype(np.float64), qn, units, H, G, 0, kr, vr, T=192)
+    # the embedding matters: read as if the keys had been stored after it, the result differs
+    plain = _run(q, cache, H, T, bits, G, k_res, v_res)
+    pre = _run_pre(q, cache, H, T, bits, G, 0, 1024, k_res, v_res)
+    assert np.abs(plain - pre).max() > 1e-3
+    # argument errors: first_pos not a multiple of 32, table too short
+    with pytest.raises(sq.SquatError):
+        sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, 1024, 8, k_res, v_res)
+    with pytest.raises(sq.SquatError):
+        sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, 1024, 512, k_res, v_res)
