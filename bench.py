@@ -421,18 +421,24 @@ def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10):
     out = torch.empty((B, Hq, d), dtype=torch.float32, device=dev)
     ws = torch.empty(sq.squat_decode_attention_workspace_bytes(B, Hq, T), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
-    call = lambda: sq.squat_decode_attention(q, *cache, H, T, bits, G, out, ws, k_res, v_res)
-    for _ in range(3):
-        flush.zero_()
-        call()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
-    for a, b in ev:
-        flush.zero_()
-        a.record(stream)
-        call()
-        b.record(stream)
-    torch.cuda.synchronize()
-    ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+    def timed(call):
+        for _ in range(3):
+            flush.zero_()
+            call()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        for a, b in ev:
+            flush.zero_()
+            a.record(stream)
+            call()
+            b.record(stream)
+        torch.cuda.synchronize()
+        return statistics.mean(a.elapsed_time(b) for a, b in ev)
+
+    ms = timed(lambda: sq.squat_decode_attention(q, *cache, H, T, bits, G, out, ws, k_res, v_res))
+    # the same step when the keys were stored before the rotary embedding (the cache's bytes are read as un-rotated
+    # keys at positions 0 .. T + R - 1; timing only, the parity tests cover the arithmetic)
+    table = sq.squat_rope_table(T + R).to(dev)
+    ms_pre = timed(lambda: sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, T + R, 0, k_res, v_res))
     elem = 4 if cfg.dtype == "f32" else 2
     toks = B * H * T
     nbytes = toks * reader_bytes_per_cached_token(d, bits, G) + 2 * B * H * R * d * elem + B * Hq * d * (elem + 4)
@@ -440,7 +446,11 @@ def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10):
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"what": "squat_decode_attention: softmax(q K^T / sqrt(d)) V over the packed cache + residual buffer",
             "ms_per_call": ms, "cached_tokens": toks, "n_q_heads": Hq, "residual_tokens": R, "bytes_per_call": nbytes,
-            "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "cached_tokens_per_s": toks / (ms * 1e-3)}
+            "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "cached_tokens_per_s": toks / (ms * 1e-3),
+            "pre_rope": {"what": "squat_decode_attention_pre_rope: the same step with the rotary embedding applied to "
+                                 "the dequantized keys on the fly", "ms_per_call": ms_pre,
+                         "hbm_gbs": nbytes / (ms_pre * 1e-3) / 1e9, "hbm_frac": nbytes / (ms_pre * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "slowdown": ms_pre / ms}}
 
 
 def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches, wall,
