@@ -81,6 +81,18 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
                          long long stride_h, long long stride_t, int rank_r, double lambda,
                          int block_g, void *stream);
 
+/*
+ * The same build from Gram matrices the caller already has (Section 3.2: the subspace depends on the prompt's
+ * queries only through M_h = Qc^T Qc, a sum over tokens).  This is the entry for a prompt whose tokens are spread
+ * over several GPUs: every rank forms the Gram matrices of its own tokens (squat_gram_static), the ranks add them
+ * up (one all-reduce of n_kv_heads * d * d float64), and every rank calls this with the sum.
+ *   gram   [n_kv_heads, d, d] float64, device, 16-byte aligned, symmetric; copied into the handle.
+ * rank_r, lambda, block_g and the result as for squat_build_subspace (rank_r is not checked against a token
+ * count here: the caller knows how many rows went into the sum).
+ */
+int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
+                                   void *stream);
+
 /* Test / checkpoint hooks.  Both synchronise `stream`.  Host pointers; any may be NULL.
  *   W_host      [n_kv_heads, d, d] float32, row j' column j, block strictly lower triangular.
  *   gram_host   [n_kv_heads, d, d] float64 Gram matrices of the last build.

@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
+    "squat_build_subspace_from_gram",
 )
 
 _lib = None
@@ -245,6 +246,47 @@ def squat_gram_static(q: torch.Tensor, n_kv_heads: int, gram_out: torch.Tensor, 
     _check(_load().squat_gram_static(_dev(q, "q"), _dtype_code(q), q.shape[0], n_kv_heads, q.shape[1], q.shape[2],
                                      q.stride(0), q.stride(1), _dev(gram_out, "gram_out"), _stream(stream)),
            "squat_gram_static")
+
+
+def squat_build_subspace_from_gram(s: "Subspace", gram: torch.Tensor, rank_r: int, lam: float, block_g: int = 1, stream=None):
+    """Eigen-decomposition and update matrices from Gram matrices [n_kv_heads, d, d] (float64, CUDA) the caller has
+    summed over the prompt's tokens, e.g. across the ranks that hold them."""
+    if gram.dtype != torch.float64 or not gram.is_contiguous():
+        raise ValueError("gram must be a contiguous float64 tensor")
+    _check(_load().squat_build_subspace_from_gram(s.handle, _dev(gram, "gram"), int(rank_r), ctypes.c_double(lam),
+                                                  int(block_g), _stream(stream)), "squat_build_subspace_from_gram")
+
+
+def token_shard(n_tokens: int, rank: int, world: int, multiple: int = 32):
+    """[start, stop) of the prompt tokens rank `rank` of `world` holds when a prompt is spread over ranks: contiguous,
+    boundaries at multiples of `multiple` (the quantization group size, so that no group straddles two ranks), sizes as
+    even as that allows.  n_tokens must be a multiple of `multiple`."""
+    if n_tokens % multiple or not 0 <= rank < world:
+        raise ValueError("n_tokens must be a multiple of the group size and 0 <= rank < world")
+    units = n_tokens // multiple
+    lo = units * rank // world
+    hi = units * (rank + 1) // world
+    return lo * multiple, hi * multiple
+
+
+def squat_build_subspace_sharded(s: "Subspace", q_local: torch.Tensor, rank_r: int, lam: float, block_g: int = 1,
+                                 gram_buf: torch.Tensor = None, group=None, stream=None):
+    """Step 1 for a prompt whose tokens are spread over the ranks of a torch.distributed group: Gram matrices of
+    the local tokens (q_local [n_q_heads, local_tokens, d]; a rank may hold none), one all-reduce (sum) of
+    n_kv_heads * d * d float64, then the eigen-decomposition and the update matrices on every rank.  Without an
+    initialised process group this is the single-GPU build through the same two calls."""
+    import torch.distributed as dist
+    H = s.n_kv_heads
+    if gram_buf is None:
+        gram_buf = torch.empty((H, q_local.shape[2], q_local.shape[2]), dtype=torch.float64, device=q_local.device)
+    if q_local.shape[1] > 0:
+        squat_gram_static(q_local, H, gram_buf, stream)
+    else:
+        gram_buf.zero_()
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
+    squat_build_subspace_from_gram(s, gram_buf, rank_r, lam, block_g, stream)
+    return gram_buf
 
 
 def squat_decode_attention_workspace_bytes(batch: int, n_q_heads: int, n_tokens: int) -> int:

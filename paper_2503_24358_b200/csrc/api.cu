@@ -162,6 +162,22 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
     return squat_launch_assemble(s, rank_r, lambda, block_g, st);
 }
 
+int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
+                                   void *stream)
+{
+    if (!s || !gram || !aligned16(gram)) return SQUAT_ERR_INVALID_ARG;
+    if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
+    if (!(lambda >= 0.0) || !std::isfinite(lambda)) return SQUAT_ERR_INVALID_ARG;
+    if (block_g <= 0 || D % block_g != 0) return SQUAT_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (gram != s->gram)
+        SQUAT_CUDA(cudaMemcpyAsync(s->gram, gram, (size_t)s->n_kv_heads * D * D * sizeof(double), cudaMemcpyDeviceToDevice, st));
+    int rc = squat_launch_eig(s, st);
+    if (rc != SQUAT_OK) return rc;
+    s->exact_blocks = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
+    return squat_launch_assemble(s, rank_r, lambda, block_g, st);
+}
+
 int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,
                           double *eigval_host, double *eigvec_host)
 {

@@ -222,3 +222,34 @@ def test_end_to_end_config1_full():
 def test_end_to_end_block_variant():
     cfg = si.get_config(1).with_(batch=2, n_kv_heads=2, n_q_heads=2, n_tokens=512)
     _end_to_end(cfg, [(0, 0), (1, 1)], rank_r=40, g=64, bits=4, G=64, min_raw=0.99)
+
+
+def test_build_from_summed_gram_matrices_of_token_shards_equals_the_build_on_all_tokens():
+    # a prompt spread over ranks: every rank's Gram matrices (squat_gram_static on its tokens), summed, then
+    # squat_build_subspace_from_gram -- here the "ranks" are three token ranges on one GPU, one of them empty-handed
+    cfg = si.get_config(0)
+    H, T, d = cfg.n_kv_heads, cfg.n_tokens, cfg.head_dim
+    q = to_torch(si.gen_queries(cfg), cfg.dtype)                       # [Hq, T, d]
+    full = sq.Subspace(H, d)
+    sq.squat_build_subspace(full, q, cfg.rank_r, cfg.lam, cfg.block_g)
+    ex = sq.squat_subspace_export(full, ("W", "gram"))
+    W_full, G_full = ex["W"], ex["gram"]
+    total = torch.zeros((H, d, d), dtype=torch.float64, device="cuda")
+    part = torch.empty_like(total)
+    for r in range(3):
+        lo, hi = sq.token_shard(T, r, 3, cfg.group_size)
+        if hi > lo:
+            sq.squat_gram_static(q[:, lo:hi, :], H, part)
+            total += part
+    assert np.abs(total.cpu().numpy() - G_full).max() <= 1e-12 * np.abs(G_full).max()
+    sharded = sq.Subspace(H, d)
+    sq.squat_build_subspace_from_gram(sharded, total, cfg.rank_r, cfg.lam, cfg.block_g)
+    W_sh = sq.squat_subspace_export(sharded, ("W",))["W"]
+    assert np.abs(W_sh - W_full).max() <= 1e-7
+    # the helper does the same through torch.distributed when a group is up; without one it is the plain build
+    helper = sq.Subspace(H, d)
+    sq.squat_build_subspace_sharded(helper, q, cfg.rank_r, cfg.lam, cfg.block_g)
+    W_h = sq.squat_subspace_export(helper, ("W",))["W"]
+    assert np.abs(W_h - W_full).max() <= 1e-7
+    for s in (full, sharded, helper):
+        s.close()
