@@ -161,3 +161,40 @@ def test_host_buffer_entry_equals_device_calls():
             sq.squat_write_path_host(s2, *host_in, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *host_out, ws[:1024])
         s.close()
         s2.close()
+
+
+def test_write_path_captures_into_a_cuda_graph_and_replays_identically():
+    # no call of the write path allocates, synchronises or touches the host: the whole step records into a CUDA graph
+    cfg = si.get_config(0)
+    B, H, T, d, bits, G = cfg.batch, cfg.n_kv_heads, cfg.n_tokens, cfg.head_dim, cfg.bits, cfg.group_size
+    q, k, v = (to_torch(x, cfg.dtype) for x in (si.gen_queries(cfg), si.gen_keys(cfg), si.gen_values(cfg)))
+    s = sq.Subspace(H, d)
+    kc, ks, kz = alloc_key_outputs(B, H, T, d, bits, G)
+    vc, vs, vz = alloc_value_outputs(B, H, T, d, bits, G)
+    kd = torch.empty((B, H, T, d), dtype=torch.float32, device="cuda")
+
+    def step():
+        sq.squat_build_subspace(s, q, cfg.rank_r, cfg.lam, cfg.block_g)
+        sq.squat_quantize_keys(s, k, bits, G, kc, ks, kz)
+        sq.squat_quantize_values(v, bits, G, vc, vs, vz)
+        sq.squat_dequantize(sq.SQUAT_KEYS, kc, ks, kz, B, H, T, d, bits, G, kd)
+
+    step()                                              # eager: reference outputs (and one-time set-up outside the capture)
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (kc, ks, kz, vc, vs, vz, kd)]
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    for t in (kc, ks, kz, vc, vs, vz, kd):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for got, want in zip((kc, ks, kz, vc, vs, vz, kd), ref):
+        assert torch.equal(got, want)
+    assert sq.squat_get_device_status(clear=True) & sq.FLAG_DEVICE_TIMEOUT == 0
+    s.close()
