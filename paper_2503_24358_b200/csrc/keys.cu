@@ -33,8 +33,8 @@
 // h & 1).  CTAs are persistent: each takes a contiguous range of tiles and works it in rounds of up to 4
 // tiles, one per tile slot, sized as evenly as the range allows; a round may cross one head boundary.
 //
-// Work per key vector: 8128 fp32 multiply-adds (dense triangle, g = 1): 2032 on the CUDA cores
-// (sweeps), 6096 x 3 tf32 products on the tensor cores.
+// Work per key vector: 8128 fp32 multiply-adds (dense triangle, g = 1): 1984 on the CUDA cores
+// (sweeps: four triangles of 32 * 31 / 2), 6144 x 3 tf32 products on the tensor cores.
 #include "squat_internal.cuh"
 
 namespace {
