@@ -41,7 +41,7 @@ ALU_PEAK_TFLOPS = SM_COUNT * FMA_LANES * 2 * SM_MAX_GHZ / 1e3
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the key kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists for that workload).
-NCU_KEY_KERNEL_TRAFFIC_BYTES = {1: 35_726_848, 2: 325_360_640}    # profiles/quant_keys_kernel_config1.md, streaming_kernels_config2.md
+NCU_KEY_KERNEL_TRAFFIC_BYTES = {1: 35_726_848, 2: 320_994_816}    # profiles/quant_keys_kernel_config1.md, streaming_kernels_config2.md
 
 
 def measured_peaks():
