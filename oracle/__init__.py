@@ -101,8 +101,19 @@ def update_matrices(Qhat, d, lam, g=1, want_chain=False):
     return out
 
 
-def quant_keys(K, G, bits, W=None, force=None, want_tval=False):
-    """Algorithm 1 Quant on [n, d] keys. Returns dict(codes, scale, zero, Khat[, tval])."""
+def half_round(x):
+    """float32 array rounded to the nearest binary16 value (ties to even), as float32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    lib = _load()
+    lib.sqo_half_round.restype = ctypes.c_float
+    lib.sqo_half_round.argtypes = [ctypes.c_float]
+    return np.array([lib.sqo_half_round(float(v)) for v in x.ravel()], dtype=np.float32).reshape(x.shape)
+
+
+def quant_keys(K, G, bits, W=None, force=None, want_tval=False, meta16=False, force_meta=None):
+    """Algorithm 1 Quant on [n, d] keys. Returns dict(codes, scale, zero, Khat[, tval]).  meta16: scale and zero are
+    stored as binary16 (returned as float32 arrays holding those values; raw_scale / raw_zero are the float32 values
+    before that rounding); force_meta = (scale, zero) float32 arrays [n/G, d] with NaN where nothing is forced."""
     K = np.ascontiguousarray(K, dtype=np.float64)
     n, d = K.shape
     codes = np.empty((n, d), dtype=np.uint8)
@@ -116,23 +127,33 @@ def quant_keys(K, G, bits, W=None, force=None, want_tval=False):
     if force is not None:
         force = np.ascontiguousarray(force, dtype=np.int16)
         assert force.shape == (n, d)
-    _check(_load().sqo_quant_keys(_p(K, _D), ctypes.c_long(n), d, G, bits, _p(W, _D), _p(codes, _U8),
-                                  _p(scale, _F), _p(zero, _F), _p(Khat, _D), _p(tval, _D), _p(force, _I16)),
+    raw_s = np.empty_like(scale) if meta16 else None
+    raw_z = np.empty_like(zero) if meta16 else None
+    fs = fz = None
+    if force_meta is not None:
+        fs = np.ascontiguousarray(force_meta[0], dtype=np.float32)
+        fz = np.ascontiguousarray(force_meta[1], dtype=np.float32)
+        assert fs.shape == scale.shape and fz.shape == zero.shape
+    _check(_load().sqo_quant_keys_m16(_p(K, _D), ctypes.c_long(n), d, G, bits, _p(W, _D), _p(codes, _U8),
+                                      _p(scale, _F), _p(zero, _F), _p(Khat, _D), _p(tval, _D), _p(force, _I16),
+                                      1 if meta16 else 0, _p(raw_s, _F), _p(raw_z, _F), _p(fs, _F), _p(fz, _F)),
            "quant_keys")
     out = {"codes": codes, "scale": scale, "zero": zero, "Khat": Khat}
+    if meta16:
+        out["raw_scale"], out["raw_zero"] = raw_s, raw_z
     if want_tval:
         out["tval"] = tval
     return out
 
 
-def quant_values_f32(V, G, bits):
+def quant_values_f32(V, G, bits, meta16=False):
     V = np.ascontiguousarray(V, dtype=np.float32)
     n, d = V.shape
     codes = np.empty((n, d), dtype=np.uint8)
     scale = np.empty((n, d // G), dtype=np.float32)
     zero = np.empty((n, d // G), dtype=np.float32)
-    _check(_load().sqo_quant_values_f32(_p(V, _F), ctypes.c_long(n), d, G, bits, _p(codes, _U8), _p(scale, _F),
-                                        _p(zero, _F)), "quant_values_f32")
+    fn = _load().sqo_quant_values_f32_m16 if meta16 else _load().sqo_quant_values_f32
+    _check(fn(_p(V, _F), ctypes.c_long(n), d, G, bits, _p(codes, _U8), _p(scale, _F), _p(zero, _F)), "quant_values_f32")
     return {"codes": codes, "scale": scale, "zero": zero}
 
 

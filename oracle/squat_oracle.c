@@ -17,6 +17,8 @@
  *                                                  Eq. (update_block); Section 2 "Quantization"
  *   sqo_quant_values_f32 / _f64                    Section 2 "Quantization", Appendix C
  *                                                  (per-token value quantization)
+ *   sqo_quant_keys_m16, sqo_quant_values_f32_m16,  the same with scale and zero-point stored in 16 bits
+ *   sqo_half_round                                 (IEEE binary16, round to nearest even)
  *   sqo_dequant_keys / sqo_dequant_values          Section 2, deq(.)
  *   sqo_pack / sqo_unpack                          cache layout (the paper gives none; ours)
  *   sqo_kv_cache_bytes                             Appendix B, memory formula
@@ -46,7 +48,10 @@
  *     (Eq. (2) quantizes [k_{t-1}]_t; line order of Quant);
  *   - the value fed back is the one a reader of the cache reconstructs, i.e. computed from
  *     the stored float32 scale and zero-point;
- *   - scale and zero-point are stored as float32;
+ *   - scale and zero-point are stored as float32; in the 16-bit variant (the "KV size" columns of
+ *     Tables 1-2 imply 16-bit metadata) they are stored as IEEE binary16: the float32 values rounded
+ *     once more to nearest-even, and the rounding decision and the value fed back use the STORED
+ *     values, so codes are clamped to [0, L] (a rounded zero-point can lie above the minimum);
  *   - channels are visited in natural order;
  *   - the rotary embedding (the paper only names it) pairs channel i with channel i + d/2 and
  *     uses the angles pos * base^(-2i/d), i < d/2: the convention of the Llama family the
@@ -297,6 +302,25 @@ done:
 }
 
 /* ------------------------------------------------------------------------------------ */
+/* Round a float32 to the nearest IEEE binary16 value (ties to even; subnormals kept; beyond
+ * the largest finite binary16 value plus half a step: infinity), returned as a float32.
+ * Written out on the bits: the exponent decides the spacing q of binary16 numbers around x
+ * (2^(e-10) for normal results, 2^-24 below 2^-14), and x / q is rounded to an integer. */
+float sqo_half_round(float x)
+{
+    if (x != x || x == INFINITY || x == -INFINITY || x == 0.0f) return x;
+    const double ax = fabs((double)x);
+    int e;
+    (void)frexp(ax, &e);                      /* ax = f * 2^e, 0.5 <= f < 1  ->  2^(e-1) <= ax < 2^e */
+    int qexp = (e - 1) - 10;                  /* spacing 2^qexp of binary16 numbers in [2^(e-1), 2^e) */
+    if (qexp < -24) qexp = -24;               /* subnormal range: fixed spacing 2^-24 */
+    const double q = ldexp(1.0, qexp);
+    double r = nearbyint(ax / q) * q;         /* exact: ax / q is a double with few bits, round half to even */
+    if (r >= 65520.0) r = INFINITY;           /* 65504 + half a step of 32 rounds up to 2^16: overflow */
+    return (float)(x < 0.0f ? -r : r);
+}
+
+/* ------------------------------------------------------------------------------------ */
 /* Algorithm 1, function Quant, applied to n/G consecutive groups of G tokens.
  *
  * K      [n, d] keys of one (batch, head), row = token; n % G == 0.
@@ -314,9 +338,27 @@ done:
  * (Eq. (3) for g = 1; Eq. (update_block) for g > 1, where W is zero inside a block so the
  * g channels of a block are quantized before any of them is corrected by the others).
  */
+/* The general form.  meta16 != 0: scale and zero-point are stored as binary16 (sqo_half_round of the
+ * float32 values); raw_scale / raw_zero [n/G, d] (may be NULL) receive the float32 values before that
+ * rounding, for tie diagnosis; force_scale / force_zero [n/G, d] (may be NULL; NaN = not forced) replace
+ * the stored values of single (group, channel) pairs, to replay a run after a legitimate tie of the
+ * 16-bit rounding was resolved the other way. */
+int sqo_quant_keys_m16(const double *K, long n, int d, int G, int bits, const double *W,
+                       uint8_t *codes, float *scale, float *zero, double *Khat, double *tval,
+                       const int16_t *force, int meta16, float *raw_scale, float *raw_zero,
+                       const float *force_scale, const float *force_zero);
+
 int sqo_quant_keys(const double *K, long n, int d, int G, int bits, const double *W,
                    uint8_t *codes, float *scale, float *zero, double *Khat, double *tval,
                    const int16_t *force)
+{
+    return sqo_quant_keys_m16(K, n, d, G, bits, W, codes, scale, zero, Khat, tval, force, 0, NULL, NULL, NULL, NULL);
+}
+
+int sqo_quant_keys_m16(const double *K, long n, int d, int G, int bits, const double *W,
+                       uint8_t *codes, float *scale, float *zero, double *Khat, double *tval,
+                       const int16_t *force, int meta16, float *raw_scale, float *raw_zero,
+                       const float *force_scale, const float *force_zero)
 {
     if (!K || !codes || !scale || !zero || n < 0 || d <= 0 || G <= 0 || n % G != 0 || bits < 1 || bits > 8)
         return SQO_ERR_ARG;
@@ -334,8 +376,16 @@ int sqo_quant_keys(const double *K, long n, int d, int G, int bits, const double
                 if (x < m) m = x;
                 if (x > Mx) Mx = x;
             }
-            const float zf = (float)m;                       /* stored zero-point */
-            const float sf = (float)((Mx - m) / L);          /* stored scale Delta */
+            float zf = (float)m;                             /* stored zero-point */
+            float sf = (float)((Mx - m) / L);                /* stored scale Delta */
+            if (raw_zero) raw_zero[grp * d + j] = zf;
+            if (raw_scale) raw_scale[grp * d + j] = sf;
+            if (meta16) {
+                zf = sqo_half_round(zf);
+                sf = sqo_half_round(sf);
+            }
+            if (force_zero && force_zero[grp * d + j] == force_zero[grp * d + j]) zf = force_zero[grp * d + j];
+            if (force_scale && force_scale[grp * d + j] == force_scale[grp * d + j]) sf = force_scale[grp * d + j];
             zero[grp * d + j] = zf;
             scale[grp * d + j] = sf;
             for (int i = 0; i < G; ++i) {
@@ -402,6 +452,44 @@ int sqo_quant_values_f32(const float *V, long n, int d, int G, int bits,
                 float code = 0.0f;
                 if (delta > 0.0f) {
                     volatile float num = x[c] - m;
+                    volatile float t = num / delta;
+                    code = nearbyintf(t);
+                    if (code < 0.0f) code = 0.0f;
+                    if (code > L) code = L;
+                }
+                codes[i * d + q * G + c] = (uint8_t)code;
+            }
+        }
+    return SQO_OK;
+}
+
+/* The binary32 sequence with 16-bit metadata: Delta = half(Delta32), z = half(m), t = (x - z) / Delta,
+ * c = clamp(rint(t), 0, L), every operation an IEEE binary32 operation on the rounded metadata. */
+int sqo_quant_values_f32_m16(const float *V, long n, int d, int G, int bits,
+                             uint8_t *codes, float *scale, float *zero)
+{
+    if (!V || !codes || !scale || !zero || n < 0 || d <= 0 || G <= 0 || d % G != 0 || bits < 1 || bits > 8)
+        return SQO_ERR_ARG;
+    const float L = (float)((1 << bits) - 1);
+    const int ng = d / G;
+    for (long i = 0; i < n; ++i)
+        for (int q = 0; q < ng; ++q) {
+            const float *x = V + i * d + q * G;
+            float m = x[0], Mx = x[0];
+            for (int c = 1; c < G; ++c) {
+                if (x[c] < m) m = x[c];
+                if (x[c] > Mx) Mx = x[c];
+            }
+            volatile float rng = Mx - m;
+            volatile float delta32 = rng / L;
+            const float delta = sqo_half_round(delta32);
+            const float z = sqo_half_round(m);
+            scale[i * ng + q] = delta;
+            zero[i * ng + q] = z;
+            for (int c = 0; c < G; ++c) {
+                float code = 0.0f;
+                if (delta > 0.0f && delta < INFINITY) {
+                    volatile float num = x[c] - z;
                     volatile float t = num / delta;
                     code = nearbyintf(t);
                     if (code < 0.0f) code = 0.0f;
