@@ -155,6 +155,31 @@ int squat_dequantize(int kind, const unsigned char *codes, const float *scales, 
                      void *stream);
 
 /*
+ * The same steps with scale and zero-point stored in 16 bits (IEEE binary16).  The "KV size" columns of Tables 1-2
+ * (19.1-21.4 % of the FP16 cache, residual tokens included) imply this storage: 2-bit codes plus two 16-bit numbers
+ * per 32 elements are 18.75 %; with float32 metadata the cache is 25 %.  The paper says nothing more, so, as a reading:
+ * the stored values are the float32 scale and zero-point rounded once more to the nearest binary16 (ties to even),
+ * and every decision is taken against the STORED values -- t = (x - z16) / Delta16, c = clamp(rint(t), 0, L), and (for
+ * keys) the error fed back is c * Delta16 + z16 - x -- so that a reader of the cache sees exactly what the writer
+ * corrected for.  Codes are clamped because a rounded zero-point can lie above the group's minimum.  A scale that
+ * rounds to 0 (or a range of 0) gives codes 0; one beyond the binary16 range gives codes 0 and SQUAT_FLAG_NONFINITE.
+ * scales / zeros: the same shapes and strides as the float32 variants, element type binary16 (2 bytes), 16-byte
+ * aligned.  Everything else (arguments, errors) as for the functions without the suffix.
+ */
+int squat_quantize_keys_m16(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
+                            int n_tokens, int head_dim, long long stride_b, long long stride_h,
+                            long long stride_t, int bits, int group_size, unsigned char *codes,
+                            void *scales, void *zeros, long long out_stride_b, long long out_stride_h,
+                            void *stream);
+int squat_quantize_values_m16(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
+                              int head_dim, long long stride_b, long long stride_h, long long stride_t,
+                              int bits, int group_size, unsigned char *codes, void *scales, void *zeros,
+                              long long out_stride_b, long long out_stride_h, void *stream);
+int squat_dequantize_m16(int kind, const unsigned char *codes, const void *scales, const void *zeros,
+                         int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                         long long in_stride_b, long long in_stride_h, void *out, int out_dtype, void *stream);
+
+/*
  * The whole write path from HOST buffers (prefill of one layer): copies q (sample 0,
  * [n_q_heads, n_tokens, d]), k and v ([batch, n_kv_heads, n_tokens, d]), all contiguous, to the
  * device workspace, runs steps 1-3, copies codes / scales / zeros back and synchronises the

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
-    "squat_build_subspace_from_gram",
+    "squat_build_subspace_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
 )
 
 _lib = None
@@ -67,6 +67,15 @@ def _load():
         lib.squat_decode_attention_workspace_bytes.restype = c.c_size_t
         lib.squat_decode_attention.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, ll, ll, i, i, vp, vp, i, i,
                                                c.c_float, vp, vp, c.c_size_t, vp]
+        lib.squat_quantize_keys_m16.argtypes = lib.squat_quantize_keys.argtypes
+        lib.squat_quantize_values_m16.argtypes = lib.squat_quantize_values.argtypes
+        lib.squat_dequantize_m16.argtypes = lib.squat_dequantize.argtypes
+        lib.squat_build_subspace_from_gram.argtypes = [vp, vp, i, dbl, i, vp]
+        lib.squat_rope_table_floats.argtypes = [i]
+        lib.squat_rope_table_floats.restype = c.c_size_t
+        lib.squat_rope_table_fill.argtypes = [dbl, i, i, vp]
+        lib.squat_decode_attention_pre_rope.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, ll, ll, i, i, vp, vp, i, i,
+                                                        c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
         lib.squat_status_string.argtypes = [i]
@@ -174,17 +183,25 @@ def _check_bhtd(x, name):
         raise ValueError(f"{name} must be [batch, heads, tokens, head_dim] with contiguous last dim")
 
 
+def _meta16(scales: torch.Tensor, zeros: torch.Tensor) -> bool:
+    """float16 scale / zero tensors select the entry points of the 16-bit-metadata cache."""
+    if scales.dtype != zeros.dtype or scales.dtype not in (torch.float32, torch.float16):
+        raise ValueError("scales and zeros must both be float32 or both float16")
+    return scales.dtype == torch.float16
+
+
 def squat_quantize_keys(s: Subspace, k: torch.Tensor, bits: int, group_size: int, codes: torch.Tensor,
                         scales: torch.Tensor, zeros: torch.Tensor, out_stride_b: int = None,
                         out_stride_h: int = None, stream=None):
-    """k [B,H,T,d] -> codes (uint8), scales, zeros (float32), written in place.
+    """k [B,H,T,d] -> codes (uint8), scales, zeros (float32, or float16 for the 16-bit-metadata cache), written in place.
 
     out strides are in tokens; by default the outputs are dense [B,H,T,...]."""
     _check_bhtd(k, "k")
     B, H, T, d = k.shape
     osh = T if out_stride_h is None else out_stride_h
     osb = H * osh if out_stride_b is None else out_stride_b
-    _check(_load().squat_quantize_keys(s.handle, _dev(k, "k"), _dtype_code(k), B, H, T, d, k.stride(0), k.stride(1),
+    fn = _load().squat_quantize_keys_m16 if _meta16(scales, zeros) else _load().squat_quantize_keys
+    _check(fn(s.handle, _dev(k, "k"), _dtype_code(k), B, H, T, d, k.stride(0), k.stride(1),
                                        k.stride(2), bits, group_size, _dev(codes, "codes"), _dev(scales, "scales"),
                                        _dev(zeros, "zeros"), osb, osh, _stream(stream)), "squat_quantize_keys")
 
@@ -195,7 +212,8 @@ def squat_quantize_values(v: torch.Tensor, bits: int, group_size: int, codes: to
     B, H, T, d = v.shape
     osh = T if out_stride_h is None else out_stride_h
     osb = H * osh if out_stride_b is None else out_stride_b
-    _check(_load().squat_quantize_values(_dev(v, "v"), _dtype_code(v), B, H, T, d, v.stride(0), v.stride(1),
+    fn = _load().squat_quantize_values_m16 if _meta16(scales, zeros) else _load().squat_quantize_values
+    _check(fn(_dev(v, "v"), _dtype_code(v), B, H, T, d, v.stride(0), v.stride(1),
                                          v.stride(2), bits, group_size, _dev(codes, "codes"), _dev(scales, "scales"),
                                          _dev(zeros, "zeros"), osb, osh, _stream(stream)), "squat_quantize_values")
 
@@ -207,7 +225,8 @@ def squat_dequantize(kind: int, codes: torch.Tensor, scales: torch.Tensor, zeros
     isb = n_kv_heads * ish if in_stride_b is None else in_stride_b
     if not out.is_contiguous():
         raise ValueError("out must be contiguous")
-    _check(_load().squat_dequantize(kind, _dev(codes, "codes"), _dev(scales, "scales"), _dev(zeros, "zeros"), batch,
+    fn = _load().squat_dequantize_m16 if _meta16(scales, zeros) else _load().squat_dequantize
+    _check(fn(kind, _dev(codes, "codes"), _dev(scales, "scales"), _dev(zeros, "zeros"), batch,
                                     n_kv_heads, n_tokens, head_dim, bits, group_size, isb, ish, _dev(out, "out"),
                                     _dtype_code(out), _stream(stream)), "squat_dequantize")
 

@@ -236,11 +236,12 @@ int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
     return SQUAT_OK;
 }
 
-int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
-                        int n_tokens, int head_dim, long long stride_b, long long stride_h,
-                        long long stride_t, int bits, int group_size, unsigned char *codes,
-                        float *scales, float *zeros, long long out_stride_b, long long out_stride_h,
-                        void *stream)
+namespace {
+int quantize_keys_impl(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
+                       int n_tokens, int head_dim, long long stride_b, long long stride_h,
+                       long long stride_t, int bits, int group_size, unsigned char *codes,
+                       void *scales, void *zeros, long long out_stride_b, long long out_stride_h, int meta16,
+                       void *stream)
 {
     if (!s) return SQUAT_ERR_INVALID_ARG;
     int rc = check_quant_args(k, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
@@ -253,13 +254,35 @@ int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int b
     if (batch == 0 || n_tokens == 0) return SQUAT_OK;
     return squat_launch_quant_keys(s->Wimg, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
                                    group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status, s->exact_blocks,
-                                   static_cast<cudaStream_t>(stream));
+                                   meta16, static_cast<cudaStream_t>(stream));
+}
+}  // namespace
+
+int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
+                        int n_tokens, int head_dim, long long stride_b, long long stride_h,
+                        long long stride_t, int bits, int group_size, unsigned char *codes,
+                        float *scales, float *zeros, long long out_stride_b, long long out_stride_h,
+                        void *stream)
+{
+    return quantize_keys_impl(s, k, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
+                              group_size, codes, scales, zeros, out_stride_b, out_stride_h, 0, stream);
 }
 
-int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
-                          int head_dim, long long stride_b, long long stride_h, long long stride_t,
-                          int bits, int group_size, unsigned char *codes, float *scales, float *zeros,
-                          long long out_stride_b, long long out_stride_h, void *stream)
+int squat_quantize_keys_m16(const squat_subspace *s, const void *k, int dtype, int batch, int n_kv_heads,
+                            int n_tokens, int head_dim, long long stride_b, long long stride_h,
+                            long long stride_t, int bits, int group_size, unsigned char *codes,
+                            void *scales, void *zeros, long long out_stride_b, long long out_stride_h,
+                            void *stream)
+{
+    return quantize_keys_impl(s, k, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
+                              group_size, codes, scales, zeros, out_stride_b, out_stride_h, 1, stream);
+}
+
+namespace {
+int quantize_values_impl(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
+                         int head_dim, long long stride_b, long long stride_h, long long stride_t,
+                         int bits, int group_size, unsigned char *codes, void *scales, void *zeros,
+                         long long out_stride_b, long long out_stride_h, int meta16, void *stream)
 {
     int rc = check_quant_args(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
                               group_size, codes, scales, zeros, out_stride_b, out_stride_h);
@@ -269,13 +292,13 @@ int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, i
     unsigned *status = squat_status_word();
     if (!status) return SQUAT_ERR_CUDA;
     return squat_launch_quant_values(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t,
-                                     bits, group_size, codes, scales, zeros, out_stride_b, out_stride_h, status,
+                                     bits, group_size, codes, scales, zeros, out_stride_b, out_stride_h, status, meta16,
                                      static_cast<cudaStream_t>(stream));
 }
 
-int squat_dequantize(int kind, const unsigned char *codes, const float *scales, const float *zeros,
-                     int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
-                     long long in_stride_b, long long in_stride_h, void *out, int out_dtype, void *stream)
+int dequantize_impl(int kind, const unsigned char *codes, const void *scales, const void *zeros,
+                    int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                    long long in_stride_b, long long in_stride_h, void *out, int out_dtype, int meta16, void *stream)
 {
     if (!valid_dtype(out_dtype) || (kind != SQUAT_KEYS && kind != SQUAT_VALUES)) return SQUAT_ERR_INVALID_ARG;
     if (batch != 0 && n_tokens != 0 && (!codes || !scales || !zeros || !out)) return SQUAT_ERR_INVALID_ARG;
@@ -289,7 +312,42 @@ int squat_dequantize(int kind, const unsigned char *codes, const float *scales, 
         return SQUAT_ERR_SHAPE;
     if (kind == SQUAT_VALUES && head_dim % group_size) return SQUAT_ERR_SHAPE;
     return squat_launch_dequant(kind, codes, scales, zeros, batch, n_kv_heads, n_tokens, head_dim, bits, group_size,
-                                in_stride_b, in_stride_h, out, out_dtype, static_cast<cudaStream_t>(stream));
+                                in_stride_b, in_stride_h, out, out_dtype, meta16, static_cast<cudaStream_t>(stream));
+}
+}  // namespace
+
+int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
+                          int head_dim, long long stride_b, long long stride_h, long long stride_t,
+                          int bits, int group_size, unsigned char *codes, float *scales, float *zeros,
+                          long long out_stride_b, long long out_stride_h, void *stream)
+{
+    return quantize_values_impl(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
+                                group_size, codes, scales, zeros, out_stride_b, out_stride_h, 0, stream);
+}
+
+int squat_quantize_values_m16(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
+                              int head_dim, long long stride_b, long long stride_h, long long stride_t,
+                              int bits, int group_size, unsigned char *codes, void *scales, void *zeros,
+                              long long out_stride_b, long long out_stride_h, void *stream)
+{
+    return quantize_values_impl(v, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
+                                group_size, codes, scales, zeros, out_stride_b, out_stride_h, 1, stream);
+}
+
+int squat_dequantize(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+                     int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                     long long in_stride_b, long long in_stride_h, void *out, int out_dtype, void *stream)
+{
+    return dequantize_impl(kind, codes, scales, zeros, batch, n_kv_heads, n_tokens, head_dim, bits, group_size,
+                           in_stride_b, in_stride_h, out, out_dtype, 0, stream);
+}
+
+int squat_dequantize_m16(int kind, const unsigned char *codes, const void *scales, const void *zeros,
+                         int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                         long long in_stride_b, long long in_stride_h, void *out, int out_dtype, void *stream)
+{
+    return dequantize_impl(kind, codes, scales, zeros, batch, n_kv_heads, n_tokens, head_dim, bits, group_size,
+                           in_stride_b, in_stride_h, out, out_dtype, 1, stream);
 }
 
 size_t squat_decode_attention_workspace_bytes(int batch, int n_q_heads, int n_tokens)

@@ -36,6 +36,7 @@
 // Work per key vector: 8128 fp32 multiply-adds (dense triangle, g = 1): 1984 on the CUDA cores
 // (sweeps: four triangles of 32 * 31 / 2), 6144 x 3 tf32 products on the tensor cores.
 #include "squat_internal.cuh"
+#include <cuda_fp16.h>
 
 namespace {
 
@@ -194,7 +195,7 @@ struct KeyParams {
     const void *k;
     long long sb, sh, st;     // element strides of k
     unsigned char *codes;
-    float *scales, *zeros;
+    void *scales, *zeros;     // float32, or binary16 in the M16 instances
     long long osb, osh;       // output strides in tokens
     int B, H, T;
     int groups_per_bh;        // T / G
@@ -251,7 +252,11 @@ __device__ __forceinline__ float2 row_pair(const RawRow<BF16> &r, int q)
 // (EXACT) the remainder e0 = c0*scale - (x - m), which is exact next to a midpoint, is compared with
 // +-scale/2: that settles the rounding exactly as real arithmetic on the stored float32 scale would, ties
 // going to the even code (the threshold of an odd c0 is one ulp lower, so "remainder == scale/2" moves it).
-template <int BITS, int NW, bool EXACT>
+//
+// M16: scale and zero-point are stored as binary16.  The float32 values are rounded once more, and the decision
+// and the error fed back are taken against the rounded (stored) values: t = (x - z16) / s16, clamped to [0, L]
+// because z16 can lie above the group's minimum.
+template <int BITS, int NW, bool EXACT, bool M16>
 __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, unsigned e_hi_taddr, float *e_lo, bool store_e,
                                             int lane, int bar_id, int wteam, float2 *red,
                                             uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
@@ -277,12 +282,21 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
             }
         }
         const float rng = __fsub_rn(Mx, m);
-        const float dlt = __fsub_rn(xj, m);
-        const float dltL = __fmul_rn(dlt, L);
-        float rcp;
-        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(fmaxf(rng, 1e-30f)));   // constant group: dlt = 0 -> code 0
-        const float scale = div_by_levels<BITS>(rng);
-        const float y0 = __fmaf_rn(dltL, rcp, kMagic);
+        float scale = div_by_levels<BITS>(rng);
+        float rcp, y0, dlt;
+        if (M16) {
+            scale = __half2float(__float2half_rn(scale));
+            m = __half2float(__float2half_rn(m));
+            dlt = __fsub_rn(xj, m);
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(scale));
+            rcp = scale > 0.0f ? rcp : 0.0f;                                       // scale 0 (no range, or underflow): codes 0
+            y0 = __fmaf_rn(dlt, rcp, kMagic);
+        } else {
+            dlt = __fsub_rn(xj, m);
+            const float dltL = __fmul_rn(dlt, L);
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(fmaxf(rng, 1e-30f)));   // constant group: dlt = 0 -> code 0
+            y0 = __fmaf_rn(dltL, rcp, kMagic);
+        }
         float c = __fsub_rn(y0, kMagic);
         float e = __fmaf_rn(c, scale, -dlt);
         if (EXACT) {
@@ -290,6 +304,11 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
             const float adj = (e > thr) ? -1.0f : ((e < -thr) ? 1.0f : 0.0f);
             c = __fadd_rn(c, adj);
             e = __fmaf_rn(adj, scale, e);
+        }
+        if (M16) {
+            const float cc = fminf(fmaxf(c, 0.0f), L);
+            e = cc == c ? e : __fmaf_rn(cc, scale, -dlt);
+            c = cc;
         }
         // pack the code arithmetically: sum of c * 2^(BITS k) is exact in float32 up to 16 bits
         if (jj % PER_ACC == 0) cacc[jj / PER_ACC] = c;
@@ -337,7 +356,7 @@ struct TileRows {
     long long meta;           // offset of the group's scales / zeros (lane = channel within a block)
 };
 
-template <int BITS, int NW, bool BF16>
+template <int BITS, int NW, bool BF16, bool M16>
 __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyParams p)
 {
     constexpr int G = 32 * NW;
@@ -501,9 +520,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 uint32_t cw[WORDS_PER_BLK];
                 float my_scale = 0.0f, my_zero = 0.0f;
                 if (blk < p.exact_blocks)
-                    sweep_block<BITS, NW, true>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, true, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
                 else
-                    sweep_block<BITS, NW, false>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, false, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
 
                 if (more) {
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");   // E_hi is in tensor memory
@@ -544,8 +563,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                     else
                         *reinterpret_cast<uint4 *>(cp) = make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
                     if (wteam == 0) {
-                        p.scales[cur.meta + blk * BLK] = my_scale;
-                        p.zeros[cur.meta + blk * BLK] = my_zero;
+                        if (M16) {
+                            reinterpret_cast<__half *>(p.scales)[cur.meta + blk * BLK] = __float2half_rn(my_scale);   // exact
+                            reinterpret_cast<__half *>(p.zeros)[cur.meta + blk * BLK] = __float2half_rn(my_zero);
+                        } else {
+                            reinterpret_cast<float *>(p.scales)[cur.meta + blk * BLK] = my_scale;
+                            reinterpret_cast<float *>(p.zeros)[cur.meta + blk * BLK] = my_zero;
+                        }
                         if (!(my_scale > 0.0f && my_scale < __int_as_float(0x7f800000)))
                             atomicOr(p.status, my_scale == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
                     }
@@ -602,8 +626,16 @@ __global__ void __launch_bounds__(256) pack_w_kernel(const float *__restrict__ W
     }
 }
 
+template <int BITS, int NW, bool BF16, bool M16>
+int launch_keys_inst(const KeyParams &p, int grid, size_t smem, cudaStream_t st)
+{
+    SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, BF16, M16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    quant_keys_kernel<BITS, NW, BF16, M16><<<grid, TC_THREADS, smem, st>>>(p);
+    return SQUAT_OK;
+}
+
 template <int BITS, int NW>
-int launch_keys(KeyParams p, int dtype, cudaStream_t st)
+int launch_keys(KeyParams p, int dtype, int meta16, cudaStream_t st)
 {
     const long long groups_per_head = (long long)p.B * p.groups_per_bh;
     const long long tiles_per_head = (groups_per_head + 4 / NW - 1) / (4 / NW);
@@ -622,13 +654,10 @@ int launch_keys(KeyParams p, int dtype, cudaStream_t st)
     const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + 2 * TC_IMG_FLOATS) +
                         sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * (TC_SLOTS + 1) + 4 * (2 + TC_SLOTS) + 8;
     const int grid = p.total_tiles < sms ? p.total_tiles : sms;                     // one tile per CTA at least
-    if (dtype == SQUAT_BF16) {
-        SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quant_keys_kernel<BITS, NW, true><<<grid, TC_THREADS, smem, st>>>(p);
-    } else {
-        SQUAT_CUDA(cudaFuncSetAttribute(quant_keys_kernel<BITS, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quant_keys_kernel<BITS, NW, false><<<grid, TC_THREADS, smem, st>>>(p);
-    }
+    int rc;
+    if (dtype == SQUAT_BF16) rc = meta16 ? launch_keys_inst<BITS, NW, true, true>(p, grid, smem, st) : launch_keys_inst<BITS, NW, true, false>(p, grid, smem, st);
+    else rc = meta16 ? launch_keys_inst<BITS, NW, false, true>(p, grid, smem, st) : launch_keys_inst<BITS, NW, false, false>(p, grid, smem, st);
+    if (rc != SQUAT_OK) return rc;
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
@@ -646,8 +675,8 @@ int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaS
 
 int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
-                            unsigned char *codes, float *scales, float *zeros,
-                            long long osb, long long osh, unsigned *status, int exact_blocks, cudaStream_t st)
+                            unsigned char *codes, void *scales, void *zeros,
+                            long long osb, long long osh, unsigned *status, int exact_blocks, int meta16, cudaStream_t st)
 {
     KeyParams p;
     p.Wimg = Wimg; p.k = k; p.sb = sb; p.sh = sh; p.st = st_;
@@ -657,13 +686,13 @@ int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int bat
     p.exact_blocks = exact_blocks;
     if ((long long)H * batch * (T / G) == 0) return SQUAT_OK;
     if (bits == 2) {
-        if (G == 32) return launch_keys<2, 1>(p, dtype, st);
-        if (G == 64) return launch_keys<2, 2>(p, dtype, st);
-        if (G == 128) return launch_keys<2, 4>(p, dtype, st);
+        if (G == 32) return launch_keys<2, 1>(p, dtype, meta16, st);
+        if (G == 64) return launch_keys<2, 2>(p, dtype, meta16, st);
+        if (G == 128) return launch_keys<2, 4>(p, dtype, meta16, st);
     } else if (bits == 4) {
-        if (G == 32) return launch_keys<4, 1>(p, dtype, st);
-        if (G == 64) return launch_keys<4, 2>(p, dtype, st);
-        if (G == 128) return launch_keys<4, 4>(p, dtype, st);
+        if (G == 32) return launch_keys<4, 1>(p, dtype, meta16, st);
+        if (G == 64) return launch_keys<4, 2>(p, dtype, meta16, st);
+        if (G == 128) return launch_keys<4, 4>(p, dtype, meta16, st);
     }
     return SQUAT_ERR_UNSUPPORTED;
 }

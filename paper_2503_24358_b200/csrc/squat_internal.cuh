@@ -43,12 +43,12 @@ int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int bloc
 int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaStream_t st);
 int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
-                            unsigned char *codes, float *scales, float *zeros,
-                            long long osb, long long osh, unsigned *status, int exact_blocks, cudaStream_t st);
+                            unsigned char *codes, void *scales, void *zeros,
+                            long long osb, long long osh, unsigned *status, int exact_blocks, int meta16, cudaStream_t st);
 int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T, int d,
                               long long sb, long long sh, long long st_, int bits, int G,
-                              unsigned char *codes, float *scales, float *zeros,
-                              long long osb, long long osh, unsigned *status, cudaStream_t st);
+                              unsigned char *codes, void *scales, void *zeros,
+                              long long osb, long long osh, unsigned *status, int meta16, cudaStream_t st);
 size_t squat_attention_workspace_floats(int batch, int n_q_heads, int n_tokens);
 int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq, int H, int T,
                                   const unsigned char *kc, const float *ks, const float *kz,
@@ -57,9 +57,9 @@ int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq,
                                   const void *k_res, const void *v_res, int res_dtype, int R,
                                   float scale, float *out, float *workspace,
                                   const float *rope_table, int rope_blocks, long long first_pos, cudaStream_t st);
-int squat_launch_dequant(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+int squat_launch_dequant(int kind, const unsigned char *codes, const void *scales, const void *zeros,
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
-                         void *out, int out_dtype, cudaStream_t st);
+                         void *out, int out_dtype, int meta16, cudaStream_t st);
 
 // ---- small device helpers --------------------------------------------------------------
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_float(u << 16); }

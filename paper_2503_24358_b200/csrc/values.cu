@@ -10,7 +10,12 @@
 // c = clamp(rint(t), 0, L).  The fast path multiplies by RN(1/Delta) and rounds once; it can
 // differ from the sequence above only when t is within ~1e-6 of a half-integer, so any
 // element within 1e-5 of one is redone with a correctly rounded division.
+//
+// M16 instances store scale and zero-point as IEEE binary16 (the 18.75 % cache of the paper's "KV size" columns):
+// Delta = half(Delta32), z = half(m), and the decision t = (x - z) / Delta is taken against those stored values,
+// so codes are clamped (a rounded zero-point can lie above the minimum).
 #include "squat_internal.cuh"
+#include <cuda_fp16.h>
 
 namespace {
 
@@ -49,11 +54,11 @@ struct ValRaw {
     }
 };
 
-template <int G, int BITS, bool BF16>
+template <int G, int BITS, bool BF16, bool M16>
 __global__ void __launch_bounds__(256) quant_values_kernel(
     const void *__restrict__ v, long long n_units, int H, int T, int ng,
     long long sb, long long sh, long long st, unsigned char *__restrict__ codes,
-    float *__restrict__ scales, float *__restrict__ zeros, long long osb, long long osh,
+    void *__restrict__ scales, void *__restrict__ zeros, long long osb, long long osh,
     int row_bytes, unsigned *__restrict__ status)
 {
     constexpr float L = float((1 << BITS) - 1);
@@ -117,7 +122,11 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
             for (int i = 1; i < G; ++i) { m = fminf(m, raw.get(i)); Mx = fmaxf(Mx, raw.get(i)); }
         }
 
-        const float delta = __fdiv_rn(__fsub_rn(Mx, m), L);
+        float delta = __fdiv_rn(__fsub_rn(Mx, m), L);
+        if (M16) {                                         // the stored binary16 values decide
+            delta = __half2float(__float2half_rn(delta));
+            m = __half2float(__float2half_rn(m));
+        }
         const bool ok = delta > 0.0f && delta < __int_as_float(0x7f800000);
         const float rcp = ok ? __frcp_rn(delta) : 0.0f;
         if (!ok) atomicOr(status, delta == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
@@ -139,6 +148,10 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
                 float ylo, yhi, rlo, rhi;
                 unpk2(y2, ylo, yhi);
                 unpk2(res2, rlo, rhi);
+                if (M16) {                                  // rounded metadata: t may leave [0, L]
+                    ylo = fminf(fmaxf(ylo, kMagic), kMagic + L);
+                    yhi = fminf(fmaxf(yhi, kMagic), kMagic + L);
+                }
                 uint32_t cb0 = __float_as_uint(ylo) & ((1u << BITS) - 1u);
                 uint32_t cb1 = __float_as_uint(yhi) & ((1u << BITS) - 1u);
                 // next to a rounding midpoint (structural with coarse bf16 data): the exact sequence decides
@@ -163,17 +176,22 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
             for (int i = 0; i < NWORDS / 2; ++i)
                 reinterpret_cast<uint2 *>(cp)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
         }
-        scales[out_tok * ng + q] = delta;
-        zeros[out_tok * ng + q] = m;
+        if (M16) {
+            reinterpret_cast<__half *>(scales)[out_tok * ng + q] = __float2half_rn(delta);      // exact: already binary16 values
+            reinterpret_cast<__half *>(zeros)[out_tok * ng + q] = __float2half_rn(m);
+        } else {
+            reinterpret_cast<float *>(scales)[out_tok * ng + q] = delta;
+            reinterpret_cast<float *>(zeros)[out_tok * ng + q] = m;
+        }
     }
 }
 
 // One thread dequantizes 16 consecutive channels of 4 consecutive tokens (same key group, so the 16
 // scales and zeros are read once for the four).  Codes become floats through the 2^23 trick
 // (exact), then one fma each: deq(c) = fma(c, scale, zero), rounded once.
-template <int BITS, bool KEYS, bool OUT_BF16>
+template <int BITS, bool KEYS, bool OUT_BF16, bool M16>
 __global__ void __launch_bounds__(256) dequant_kernel(
-    const unsigned char *__restrict__ codes, const float *__restrict__ scales, const float *__restrict__ zeros,
+    const unsigned char *__restrict__ codes, const void *__restrict__ scales, const void *__restrict__ zeros,
     long long n_units, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
 {
     constexpr int TOK = 4;
@@ -192,12 +210,28 @@ __global__ void __launch_bounds__(256) dequant_kernel(
         float sc[16], zr[16];
         if (KEYS) {
             const long long base = (b * (isb / G) + h * (ish / G) + t0 / G) * d + c16 * 16;
+            if (M16) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 s4 = __ldg(reinterpret_cast<const float4 *>(scales + base) + i);
-                const float4 z4 = __ldg(reinterpret_cast<const float4 *>(zeros + base) + i);
-                sc[4 * i] = s4.x; sc[4 * i + 1] = s4.y; sc[4 * i + 2] = s4.z; sc[4 * i + 3] = s4.w;
-                zr[4 * i] = z4.x; zr[4 * i + 1] = z4.y; zr[4 * i + 2] = z4.z; zr[4 * i + 3] = z4.w;
+                for (int i = 0; i < 2; ++i) {
+                    const uint4 s8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(scales) + base) + i);
+                    const uint4 z8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(zeros) + base) + i);
+                    const uint32_t sw[4] = {s8.x, s8.y, s8.z, s8.w}, zw[4] = {z8.x, z8.y, z8.z, z8.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sw[k]));
+                        const float2 zf = __half22float2(*reinterpret_cast<const __half2 *>(&zw[k]));
+                        sc[8 * i + 2 * k] = sf.x; sc[8 * i + 2 * k + 1] = sf.y;
+                        zr[8 * i + 2 * k] = zf.x; zr[8 * i + 2 * k + 1] = zf.y;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float4 s4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(scales) + base) + i);
+                    const float4 z4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(zeros) + base) + i);
+                    sc[4 * i] = s4.x; sc[4 * i + 1] = s4.y; sc[4 * i + 2] = s4.z; sc[4 * i + 3] = s4.w;
+                    zr[4 * i] = z4.x; zr[4 * i + 1] = z4.y; zr[4 * i + 2] = z4.z; zr[4 * i + 3] = z4.w;
+                }
             }
         }
 #pragma unroll
@@ -211,8 +245,13 @@ __global__ void __launch_bounds__(256) dequant_kernel(
             float s1 = 0.0f, z1 = 0.0f;
             if (!KEYS) {
                 const long long mi = (in_tok0 + t) * (d / G) + (c16 * 16) / G;
-                s1 = __ldg(scales + mi);
-                z1 = __ldg(zeros + mi);
+                if (M16) {
+                    s1 = __half2float(__ldg(reinterpret_cast<const __half *>(scales) + mi));
+                    z1 = __half2float(__ldg(reinterpret_cast<const __half *>(zeros) + mi));
+                } else {
+                    s1 = __ldg(reinterpret_cast<const float *>(scales) + mi);
+                    z1 = __ldg(reinterpret_cast<const float *>(zeros) + mi);
+                }
             }
             float y[16];
 #pragma unroll
@@ -256,14 +295,14 @@ int grid_for(long long n_threads, int block)
 
 template <int G, int BITS>
 int launch_values(const void *v, int dtype, long long n_units, int H, int T, int ng, long long sb, long long sh,
-                  long long st_, unsigned char *codes, float *scales, float *zeros, long long osb, long long osh,
-                  int row_bytes, unsigned *status, cudaStream_t st)
+                  long long st_, unsigned char *codes, void *scales, void *zeros, long long osb, long long osh,
+                  int row_bytes, unsigned *status, int meta16, cudaStream_t st)
 {
     const int grid = grid_for(n_units, 256);
-    if (dtype == SQUAT_BF16)
-        quant_values_kernel<G, BITS, true><<<grid, 256, 0, st>>>(v, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status);
-    else
-        quant_values_kernel<G, BITS, false><<<grid, 256, 0, st>>>(v, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status);
+#define SQ_VK(BF, MM) quant_values_kernel<G, BITS, BF, MM><<<grid, 256, 0, st>>>(v, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status)
+    if (dtype == SQUAT_BF16) { if (meta16) SQ_VK(true, true); else SQ_VK(true, false); }
+    else { if (meta16) SQ_VK(false, true); else SQ_VK(false, false); }
+#undef SQ_VK
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
@@ -273,28 +312,29 @@ int launch_values(const void *v, int dtype, long long n_units, int H, int T, int
 
 int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T, int d,
                               long long sb, long long sh, long long st_, int bits, int G,
-                              unsigned char *codes, float *scales, float *zeros,
-                              long long osb, long long osh, unsigned *status, cudaStream_t st)
+                              unsigned char *codes, void *scales, void *zeros,
+                              long long osb, long long osh, unsigned *status, int meta16, cudaStream_t st)
 {
     const int ng = d / G;
     const long long n_units = (long long)batch * H * T * ng;
     if (n_units == 0) return SQUAT_OK;
     const int row_bytes = d * bits / 8;
-#define SQ_V(GG, BB) return launch_values<GG, BB>(v, dtype, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status, st)
+#define SQ_V(GG, BB) return launch_values<GG, BB>(v, dtype, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status, meta16, st)
     if (bits == 2) { if (G == 32) SQ_V(32, 2); if (G == 64) SQ_V(64, 2); if (G == 128) SQ_V(128, 2); }
     if (bits == 4) { if (G == 32) SQ_V(32, 4); if (G == 64) SQ_V(64, 4); if (G == 128) SQ_V(128, 4); }
 #undef SQ_V
     return SQUAT_ERR_UNSUPPORTED;
 }
 
-int squat_launch_dequant(int kind, const unsigned char *codes, const float *scales, const float *zeros,
+int squat_launch_dequant(int kind, const unsigned char *codes, const void *scales, const void *zeros,
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
-                         void *out, int out_dtype, cudaStream_t st)
+                         void *out, int out_dtype, int meta16, cudaStream_t st)
 {
     const long long n_units = (long long)batch * H * ((T + 3) / 4) * (d / 16);     // 4 tokens x 16 channels per thread
     if (n_units == 0) return SQUAT_OK;
     const int grid = grid_for(n_units, 256);
-#define SQ_D(BB, KK, OO) dequant_kernel<BB, KK, OO><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out)
+#define SQ_D(BB, KK, OO) do { if (meta16) dequant_kernel<BB, KK, OO, true><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out); \
+                               else dequant_kernel<BB, KK, OO, false><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out); } while (0)
     const bool keys = kind == SQUAT_KEYS, obf = out_dtype == SQUAT_BF16;
     if (bits == 2) {
         if (keys) { if (obf) SQ_D(2, true, true); else SQ_D(2, true, false); }

@@ -60,10 +60,15 @@ def alloc_value_outputs(B, H, T, d, bits, G, device="cuda"):
     return codes, scales, zeros
 
 
-def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=None, Qhat=None, max_replays=64):
+def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=None, Qhat=None, max_replays=64,
+                     meta16=False):
     """Compares one (batch, head) unit.  K64 [n,d] float64; gpu_codes [n,d] unpacked uint8;
     gpu_scale/zero [n/G, d] float32; gpu_deq [n,d] float32 (optional).  Returns a dict of statistics;
-    raises AssertionError with a precise message on any violation of the protocol."""
+    raises AssertionError with a precise message on any violation of the protocol.
+    meta16: the cache stores scale and zero-point as binary16 (gpu_scale / gpu_zero hold those values widened to
+    float32); see compare_key_unit_meta16."""
+    if meta16:
+        return compare_key_unit_meta16(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq, Qhat, max_replays)
     n, d = K64.shape
     base = oracle.quant_keys(K64, G, bits, W64, want_tval=True)
     raw_equal = int((base["codes"] == gpu_codes).sum())
@@ -103,6 +108,87 @@ def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=
     zr_err = np.abs(gpu_zero.astype(np.float64) - final_zero).max() / max(np.abs(final_zero).max(), 1e-30)
     stats["scale_rel_err"], stats["zero_rel_err"] = float(sc_err), float(zr_err)
     assert sc_err < 1e-4 and zr_err < 1e-4, (sc_err, zr_err)
+    if gpu_deq is not None:
+        rel = np.linalg.norm(gpu_deq.astype(np.float64) - final_khat) / np.linalg.norm(final_khat)
+        stats["deq_rel_fro"] = float(rel)
+        assert rel < 1e-3, rel
+        if Qhat is not None and Qhat.shape[0] > 0:
+            pg = np.linalg.norm((gpu_deq.astype(np.float64) - K64) @ Qhat.T)
+            po = np.linalg.norm((final_khat - K64) @ Qhat.T)
+            stats["proj_rel"] = float(abs(pg - po) / po)
+            assert abs(pg - po) <= 1e-3 * po, (pg, po)
+    return stats
+
+
+META_TIE_BAND = 1e-5     # a binary16 rounding of scale / zero counts as a tie within this fraction of the value's size
+
+
+def compare_key_unit_meta16(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=None, Qhat=None, max_replays=64):
+    """The protocol of compare_key_unit for the 16-bit-metadata cache.  Besides rounding ties of codes there are
+    rounding ties of the metadata: the float32 scale or zero-point of a (group, channel) lies so close to the middle
+    between two binary16 numbers that the float64 oracle and the float32 kernel, whose corrected values differ by
+    rounding noise, store different neighbours.  Such a pair is accepted if the kernel's value is the adjacent
+    binary16 number and the oracle's unrounded value lies within META_TIE_BAND (relative to |zero| + range) of the
+    midpoint; the kernel's stored value is then forced into the oracle and the group replayed, exactly as for codes.
+    At the end codes, scales and zero-points must be identical."""
+    n, d = K64.shape
+    L = (1 << bits) - 1
+    base = oracle.quant_keys(K64, G, bits, W64, want_tval=True, meta16=True)
+    raw_equal = int((base["codes"] == gpu_codes).sum())
+    ties = meta_ties = 0
+    final_codes, final_khat = base["codes"].copy(), base["Khat"].copy()
+    final_scale, final_zero = base["scale"].copy(), base["zero"].copy()
+    code_bad = np.nonzero(base["codes"] != gpu_codes)[0] // G
+    meta_bad = np.nonzero((base["scale"] != gpu_scale) | (base["zero"] != gpu_zero))[0]
+    for grp in np.unique(np.concatenate([code_bad, meta_bad])):
+        lo, hi = grp * G, (grp + 1) * G
+        force = -np.ones((G, d), dtype=np.int16)
+        fs = np.full((1, d), np.nan, np.float32)
+        fz = np.full((1, d), np.nan, np.float32)
+        keys = ("codes", "Khat", "tval")
+        o = {k: (v[lo:hi] if k in keys else v[grp:grp + 1]) for k, v in base.items()}
+        for _ in range(max_replays):
+            cdiff = (o["codes"] != gpu_codes[lo:hi]).any(axis=0)
+            mdiff = (o["scale"][0] != gpu_scale[grp]) | (o["zero"][0] != gpu_zero[grp])
+            if not cdiff.any() and not mdiff.any():
+                break
+            j0 = int(np.nonzero(cdiff | mdiff)[0][0])
+            if mdiff[j0]:
+                size = abs(float(o["raw_zero"][0, j0])) + L * abs(float(o["raw_scale"][0, j0]))
+                for name, store, raw, gpu in (("scale", fs, o["raw_scale"][0, j0], gpu_scale[grp, j0]),
+                                              ("zero", fz, o["raw_zero"][0, j0], gpu_zero[grp, j0])):
+                    ora = o[name][0, j0]
+                    if ora == gpu:
+                        continue
+                    h_or, h_gpu = np.float16(ora), np.float16(gpu)
+                    assert np.float32(h_gpu) == gpu, f"stored {name} is not a binary16 number: {gpu!r}"
+                    step = np.nextafter(h_or, h_gpu)
+                    mid = 0.5 * (float(ora) + float(gpu))
+                    assert step == h_gpu and abs(float(raw) - mid) <= META_TIE_BAND * size, (
+                        f"metadata mismatch that is no tie: group {grp} channel {j0} {name}: gpu {gpu!r} oracle {ora!r} "
+                        f"unrounded {float(raw)!r} midpoint {mid!r}")
+                    store[0, j0] = gpu
+                    meta_ties += 1
+            else:
+                diff = o["codes"][:, j0] != gpu_codes[lo:hi, j0]
+                for i in np.nonzero(diff)[0]:
+                    t = o["tval"][i, j0]
+                    frac = abs((t - np.floor(t)) - 0.5)
+                    cg, co = int(gpu_codes[lo + i, j0]), int(o["codes"][i, j0])
+                    assert abs(cg - co) == 1 and frac < TIE_BAND * L / 3.0, (
+                        f"non-tie mismatch: group {grp} token {i} channel {j0}: gpu {cg} oracle {co} "
+                        f"t={t!r} |frac-0.5|={frac:.3e}")
+                    force[i, j0] = cg
+                    ties += 1
+            o = oracle.quant_keys(K64[lo:hi], G, bits, W64, force=force, want_tval=True, meta16=True, force_meta=(fs, fz))
+        else:
+            raise AssertionError(f"group {grp}: replay did not converge")
+        final_codes[lo:hi], final_khat[lo:hi] = o["codes"], o["Khat"]
+        final_scale[grp], final_zero[grp] = o["scale"][0], o["zero"][0]
+    assert np.array_equal(final_codes, gpu_codes)
+    assert np.array_equal(final_scale, gpu_scale) and np.array_equal(final_zero, gpu_zero)
+    stats = {"elements": n * d, "raw_equal": raw_equal, "ties": ties, "meta_ties": meta_ties,
+             "raw_fraction": raw_equal / (n * d)}
     if gpu_deq is not None:
         rel = np.linalg.norm(gpu_deq.astype(np.float64) - final_khat) / np.linalg.norm(final_khat)
         stats["deq_rel_fro"] = float(rel)
