@@ -76,9 +76,10 @@ def reader_bytes_per_cached_token(d, bits, G):
     return 2 * d * bits // 8 + 8 * d // G + 8 * d // G
 
 
-def bytes_per_vector(d, bits, G, elem_bytes):
-    """Algorithmic HBM bytes per key (or value) vector: read the vector, write codes + fp32 scale/zero."""
-    return d * elem_bytes + d * bits // 8 + 8 * d // G
+def bytes_per_vector(d, bits, G, elem_bytes, meta_bytes=4):
+    """Algorithmic HBM bytes per key (or value) vector: read the vector, write codes + scale and zero (float32, or
+    binary16 for the 16-bit-metadata cache)."""
+    return d * elem_bytes + d * bits // 8 + 2 * meta_bytes * d // G
 
 
 # --------------------------------------------------------------------------- clocks sampling
@@ -305,10 +306,11 @@ def run_gpu(args, cfg):
     q_np, k_np, v_np = si.gen_queries(cfg), si.gen_keys(cfg), si.gen_values(cfg)
     q, k, v = to_dev(q_np), to_dev(k_np), to_dev(v_np)
     kc = torch.empty((B, H, T, d * bits // 8), dtype=torch.uint8, device=dev)
-    ks = torch.empty((B, H, T // G, d), dtype=torch.float32, device=dev)
+    mdt = torch.float16 if args.meta16 else torch.float32   # storage type of scales and zero-points
+    ks = torch.empty((B, H, T // G, d), dtype=mdt, device=dev)
     kz = torch.empty_like(ks)
     vc = torch.empty_like(kc)
-    vs = torch.empty((B, H, T, d // G), dtype=torch.float32, device=dev)
+    vs = torch.empty((B, H, T, d // G), dtype=mdt, device=dev)
     vz = torch.empty_like(vs)
     kd = torch.empty((B, H, T, d), dtype=tdt, device=dev)
     vd = torch.empty_like(kd)
@@ -366,12 +368,12 @@ def run_gpu(args, cfg):
 
     # ---- end to end from host buffers through squat_write_path_host --------------------------------
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.meta16:              # the host-buffer entry writes float32 metadata
         e2e = run_e2e(args, cfg, sq, s, (q_np, k_np, v_np), (kc, ks, kz, vc, vs, vz), to_dev, flush, tdt, dev,
                       vec_per_step)
     # ---- the reader that follows the write path (not part of a step): one decode step of attention -----
     reader = None
-    if rank == 0 and not args.no_reader:
+    if rank == 0 and not args.no_reader and not args.meta16:     # the readers take float32 metadata
         reader = run_reader(cfg, sq, (kc, ks, kz, vc, vs, vz), flush, tdt, dev)
     if rank == 0:
         report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches,
@@ -461,7 +463,8 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
         elem = 4 if cfg.dtype == "f32" else 2
         key_ms = stage_ms["quantize_keys"]
         flops = key_flops_per_vector(d, cfg.block_g, cfg.rank_r) * vec_per_step
-        kbytes = bytes_per_vector(d, bits, G, elem) * vec_per_step
+        mb = 2 if args.meta16 else 4
+        kbytes = bytes_per_vector(d, bits, G, elem, mb) * vec_per_step
         alu_time_ms = flops / (ALU_PEAK_TFLOPS * 1e12) * 1e3
         hbm_time_ms = kbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
         if alu_time_ms >= hbm_time_ms:
@@ -490,7 +493,7 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
         roof["kv_input_gbs"] = vec_per_step * d * elem / (key_ms * 1e-3) / 1e9
         roof["hbm_frac_of_" + peaks["source"]] = kbytes / (key_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]
         # the HBM-bound stages, for the record
-        vbytes = bytes_per_vector(d, bits, G, elem) * vec_per_step
+        vbytes = bytes_per_vector(d, bits, G, elem, mb) * vec_per_step
         dq_bytes = 2 * (d * bits // 8 + 8 * d // G + d * elem) * vec_per_step
         stages = {n: {"ms": stage_ms[n], "share": stage_ms[n] / statistics.mean(step_ms)} for n in stage_names}
         stages["quantize_values"]["hbm_gbs"] = vbytes / (stage_ms["quantize_values"] * 1e-3) / 1e9
@@ -501,7 +504,7 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
             "metric": METRIC, "value": total_units / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg),
+            "config": dict(workload_config(cfg), metadata="binary16" if args.meta16 else "float32"),
             "kv_ingested_gbs": 2 * vec_per_step * world * d * elem / (total_ms / args.steps * 1e-3) / 1e9,
             "roofline": roof, "stages": stages,
             "e2e": e2e,
@@ -523,6 +526,8 @@ def main():
     ap.add_argument("--bits", type=int, default=None, choices=[2, 4], help="override the workload's code width")
     ap.add_argument("--rank", type=int, default=None, help="override the workload's subspace rank r")
     ap.add_argument("--group-size", type=int, default=None, choices=[32, 64, 128], help="override the workload's group size G")
+    ap.add_argument("--meta16", action="store_true", help="store scales and zero-points as binary16 (the 18.75 %% cache); "
+                    "times the write path only")
     ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")

@@ -49,6 +49,7 @@ def test_algorithmic_counts():
     assert sum(bench.key_fma_split(128, 64)) == 4096
     assert bench.bytes_per_vector(128, 2, 32, 2) == 320
     assert bench.bytes_per_vector(128, 4, 128, 2) == 328
+    assert bench.bytes_per_vector(128, 2, 32, 2, meta_bytes=2) == 304      # binary16 scale and zero
     assert abs(bench.ALU_PEAK_TFLOPS - 74.45) < 0.01
     # the reader: 32 + 32 code bytes, 32 bytes of key metadata, 32 of value metadata per cached token at 2 bits, G = 32
     assert bench.reader_bytes_per_cached_token(128, 2, 32) == 128

@@ -118,3 +118,15 @@ def test_keys_with_16_bit_metadata_zero_update_is_round_to_nearest_on_the_stored
         o = oracle.quant_keys(K64, 32, 2, meta16=True)
         assert np.array_equal(o["scale"], sc[0, h]) and np.array_equal(o["zero"], zr[0, h])
         assert np.array_equal(o["codes"], un[0, h])
+
+
+def test_keys_with_16_bit_metadata_workload1_four_heads_full_length():
+    # 4 heads of the Llama-2-7B-shaped workload at full length (524 288 elements per head): the 99.9 % bar on the raw
+    # (pre-replay) fraction, and how many metadata ties the protocol had to resolve
+    cfg = si.get_config(1).with_(n_kv_heads=4, n_q_heads=4)
+    mats = [oracle_mats(cfg, h) for h in range(4)]
+    W32 = np.stack([m["W"] for m in mats]).astype(np.float32)
+    k_np = si.gen_keys(cfg)
+    got = _run_keys16(cfg, k_np, W32, cfg.bits, cfg.group_size)
+    tot = _compare(cfg, k_np, W32, mats, cfg.bits, cfg.group_size, got, 0.999)
+    print("workload 1 (4 heads) 16-bit metadata:", tot)
