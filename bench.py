@@ -70,10 +70,11 @@ def key_fma_split(d, g, blk=32):
     return alu, tensor
 
 
-def reader_bytes_per_cached_token(d, bits, G):
-    """What one decode step has to read per cached token: key and value codes, key metadata (fp32 scale and zero
-    per channel, shared by G tokens), value metadata (fp32 scale and zero per group of G channels)."""
-    return 2 * d * bits // 8 + 8 * d // G + 8 * d // G
+def reader_bytes_per_cached_token(d, bits, G, meta_bytes=4):
+    """What one decode step has to read per cached token: key and value codes, key metadata (scale and zero per
+    channel, shared by G tokens), value metadata (scale and zero per group of G channels); metadata float32 or
+    binary16."""
+    return 2 * d * bits // 8 + 2 * meta_bytes * d // G + 2 * meta_bytes * d // G
 
 
 def bytes_per_vector(d, bits, G, elem_bytes, meta_bytes=4):
@@ -373,8 +374,8 @@ def run_gpu(args, cfg):
                       vec_per_step)
     # ---- the reader that follows the write path (not part of a step): one decode step of attention -----
     reader = None
-    if rank == 0 and not args.no_reader and not args.meta16:     # the readers take float32 metadata
-        reader = run_reader(cfg, sq, (kc, ks, kz, vc, vs, vz), flush, tdt, dev)
+    if rank == 0 and not args.no_reader:
+        reader = run_reader(cfg, sq, (kc, ks, kz, vc, vs, vz), flush, tdt, dev, meta_bytes=2 if args.meta16 else 4)
     if rank == 0:
         report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches,
                wall, flags, clocks, reader)
@@ -410,7 +411,7 @@ def run_e2e(args, cfg, sq, s, host_np, dev_outs, to_dev, flush, tdt, dev, vec_pe
             "api": "squat_write_path_host (pinned host buffers; build + keys + values)"}
 
 
-def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10):
+def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10, meta_bytes=4):
     """One decode step of attention over the cache the step has just written (plus a full residual buffer of
     random full-precision rows): time per call and the bytes it has to read, against the copy bandwidth."""
     import torch
@@ -443,7 +444,7 @@ def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10):
     ms_pre = timed(lambda: sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, T + R, 0, k_res, v_res))
     elem = 4 if cfg.dtype == "f32" else 2
     toks = B * H * T
-    nbytes = toks * reader_bytes_per_cached_token(d, bits, G) + 2 * B * H * R * d * elem + B * Hq * d * (elem + 4)
+    nbytes = toks * reader_bytes_per_cached_token(d, bits, G, meta_bytes) + 2 * B * H * R * d * elem + B * Hq * d * (elem + 4)
     peaks = measured_peaks()
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"what": "squat_decode_attention: softmax(q K^T / sqrt(d)) V over the packed cache + residual buffer",

@@ -247,6 +247,16 @@ int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads,
  * Everything else as for squat_decode_attention.  Errors: the same, plus SQUAT_ERR_SHAPE for a first_pos that is
  * not a multiple of 32 or a table that is too short.
  */
+/* The general form of the two readers: meta16 = 1 reads a cache whose scales and zero-points are binary16 (written
+ * by the _m16 functions; the four metadata pointers then point to 2-byte elements); rope_table = NULL reads keys
+ * stored after the rotary embedding (table_positions and first_pos are then ignored).  Everything else as above. */
+int squat_decode_attention_ex(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                              const unsigned char *k_codes, const void *k_scales, const void *k_zeros,
+                              const unsigned char *v_codes, const void *v_scales, const void *v_zeros, int meta16,
+                              int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                              int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                              float softmax_scale, const float *rope_table, int table_positions, long long first_pos,
+                              float *out, void *workspace, size_t workspace_bytes, void *stream);
 size_t squat_rope_table_floats(int n_positions);
 int squat_rope_table_fill(double base, int head_dim, int n_positions, float *table_host);
 int squat_decode_attention_pre_rope(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
-    "squat_build_subspace_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
+    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
 )
 
 _lib = None
@@ -76,6 +76,8 @@ def _load():
         lib.squat_rope_table_fill.argtypes = [dbl, i, i, vp]
         lib.squat_decode_attention_pre_rope.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, ll, ll, i, i, vp, vp, i, i,
                                                         c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
+        lib.squat_decode_attention_ex.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, i, ll, ll, i, i, vp, vp, i, i,
+                                                  c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
         lib.squat_status_string.argtypes = [i]
@@ -328,6 +330,17 @@ def squat_decode_attention(q: torch.Tensor, k_codes, k_scales, k_zeros, v_codes,
     if n_res and (not k_res.is_contiguous() or not v_res.is_contiguous() or k_res.dtype != v_res.dtype):
         raise ValueError("k_res and v_res must be contiguous [batch, n_kv_heads, n_res, d] of one dtype")
     opt = lambda t, n: _dev(t, n) if t is not None and t.numel() else None
+    if k_scales is not None and k_scales.dtype == torch.float16:         # a cache with 16-bit scales and zero-points
+        for t in (k_zeros, v_scales, v_zeros):
+            if t.dtype != torch.float16:
+                raise ValueError("scales and zero-points must all be float16 or all float32")
+        _check(_load().squat_decode_attention_ex(
+            _dev(q, "q"), _dtype_code(q), B, Hq, n_kv_heads, d, opt(k_codes, "k_codes"), opt(k_scales, "k_scales"),
+            opt(k_zeros, "k_zeros"), opt(v_codes, "v_codes"), opt(v_scales, "v_scales"), opt(v_zeros, "v_zeros"), 1, n_tokens,
+            csb, csh, bits, group_size, opt(k_res, "k_res"), opt(v_res, "v_res"), _dtype_code(k_res) if n_res else SQUAT_F32,
+            n_res, float(softmax_scale), None, 0, 0, _dev(out, "out"), _dev(workspace, "workspace"),
+            workspace.numel() * workspace.element_size(), _stream(stream)), "squat_decode_attention_ex")
+        return
     _check(_load().squat_decode_attention(_dev(q, "q"), _dtype_code(q), B, Hq, n_kv_heads, d, opt(k_codes, "k_codes"),
                                           opt(k_scales, "k_scales"), opt(k_zeros, "k_zeros"), opt(v_codes, "v_codes"),
                                           opt(v_scales, "v_scales"), opt(v_zeros, "v_zeros"), n_tokens, csb, csh, bits,
@@ -370,6 +383,15 @@ def squat_decode_attention_pre_rope(q: torch.Tensor, k_codes, k_scales, k_zeros,
     if n_res and (not k_res.is_contiguous() or not v_res.is_contiguous() or k_res.dtype != v_res.dtype):
         raise ValueError("k_res and v_res must be contiguous [batch, n_kv_heads, n_res, d] of one dtype")
     opt = lambda t, n: _dev(t, n) if t is not None and t.numel() else None
+    if k_scales is not None and k_scales.dtype == torch.float16:         # a cache with 16-bit scales and zero-points
+        _check(_load().squat_decode_attention_ex(
+            _dev(q, "q"), _dtype_code(q), B, Hq, n_kv_heads, d, opt(k_codes, "k_codes"), opt(k_scales, "k_scales"),
+            opt(k_zeros, "k_zeros"), opt(v_codes, "v_codes"), opt(v_scales, "v_scales"), opt(v_zeros, "v_zeros"), 1, n_tokens,
+            csb, csh, bits, group_size, opt(k_res, "k_res"), opt(v_res, "v_res"), _dtype_code(k_res) if n_res else SQUAT_F32,
+            n_res, float(softmax_scale), _dev(rope_table, "rope_table"), int(table_positions), int(first_pos),
+            _dev(out, "out"), _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream(stream)),
+            "squat_decode_attention_ex")
+        return
     _check(_load().squat_decode_attention_pre_rope(
         _dev(q, "q"), _dtype_code(q), B, Hq, n_kv_heads, d, opt(k_codes, "k_codes"), opt(k_scales, "k_scales"),
         opt(k_zeros, "k_zeros"), opt(v_codes, "v_codes"), opt(v_scales, "v_scales"), opt(v_zeros, "v_zeros"), n_tokens,

@@ -358,12 +358,12 @@ size_t squat_decode_attention_workspace_bytes(int batch, int n_q_heads, int n_to
 
 namespace {
 int decode_attention_impl(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
-                          const unsigned char *k_codes, const float *k_scales, const float *k_zeros,
-                          const unsigned char *v_codes, const float *v_scales, const float *v_zeros,
+                          const unsigned char *k_codes, const void *k_scales, const void *k_zeros,
+                          const unsigned char *v_codes, const void *v_scales, const void *v_zeros,
                           int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
                           int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
                           float softmax_scale, float *out, void *workspace, size_t workspace_bytes,
-                          const float *rope_table, int rope_blocks, long long first_pos, void *stream)
+                          const float *rope_table, int rope_blocks, long long first_pos, int meta16, void *stream)
 {
     if (!valid_dtype(q_dtype) || batch < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_tokens < 0 || n_res < 0)
         return SQUAT_ERR_INVALID_ARG;
@@ -389,7 +389,7 @@ int decode_attention_impl(const void *q, int q_dtype, int batch, int n_q_heads, 
     return squat_launch_decode_attention(q, q_dtype, batch, n_q_heads, n_kv_heads, n_tokens, k_codes, k_scales, k_zeros,
                                          v_codes, v_scales, v_zeros, cache_stride_b, cache_stride_h, bits, group_size,
                                          k_res, v_res, res_dtype, n_res, scale, out, static_cast<float *>(workspace),
-                                         rope_table, rope_blocks, first_pos, static_cast<cudaStream_t>(stream));
+                                         rope_table, rope_blocks, first_pos, meta16, static_cast<cudaStream_t>(stream));
 }
 }  // namespace
 
@@ -402,7 +402,26 @@ int squat_decode_attention(const void *q, int q_dtype, int batch, int n_q_heads,
 {
     return decode_attention_impl(q, q_dtype, batch, n_q_heads, n_kv_heads, head_dim, k_codes, k_scales, k_zeros, v_codes,
                                  v_scales, v_zeros, n_tokens, cache_stride_b, cache_stride_h, bits, group_size, k_res, v_res,
-                                 res_dtype, n_res, softmax_scale, out, workspace, workspace_bytes, nullptr, 0, 0, stream);
+                                 res_dtype, n_res, softmax_scale, out, workspace, workspace_bytes, nullptr, 0, 0, 0, stream);
+}
+
+int squat_decode_attention_ex(const void *q, int q_dtype, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                              const unsigned char *k_codes, const void *k_scales, const void *k_zeros,
+                              const unsigned char *v_codes, const void *v_scales, const void *v_zeros, int meta16,
+                              int n_tokens, long long cache_stride_b, long long cache_stride_h, int bits,
+                              int group_size, const void *k_res, const void *v_res, int res_dtype, int n_res,
+                              float softmax_scale, const float *rope_table, int table_positions, long long first_pos,
+                              float *out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (meta16 != 0 && meta16 != 1) return SQUAT_ERR_INVALID_ARG;
+    if (rope_table) {
+        if (table_positions <= 0 || first_pos < 0 || n_tokens < 0 || n_res < 0 || !aligned16(rope_table)) return SQUAT_ERR_INVALID_ARG;
+        if (first_pos % 32 != 0 || first_pos + n_tokens + n_res > table_positions) return SQUAT_ERR_SHAPE;
+    }
+    return decode_attention_impl(q, q_dtype, batch, n_q_heads, n_kv_heads, head_dim, k_codes, k_scales, k_zeros, v_codes,
+                                 v_scales, v_zeros, n_tokens, cache_stride_b, cache_stride_h, bits, group_size, k_res, v_res,
+                                 res_dtype, n_res, softmax_scale, out, workspace, workspace_bytes, rope_table,
+                                 rope_table ? (table_positions + 31) / 32 : 0, first_pos, meta16, stream);
 }
 
 size_t squat_rope_table_floats(int n_positions)
@@ -445,7 +464,7 @@ int squat_decode_attention_pre_rope(const void *q, int q_dtype, int batch, int n
     return decode_attention_impl(q, q_dtype, batch, n_q_heads, n_kv_heads, head_dim, k_codes, k_scales, k_zeros, v_codes,
                                  v_scales, v_zeros, n_tokens, cache_stride_b, cache_stride_h, bits, group_size, k_res, v_res,
                                  res_dtype, n_res, softmax_scale, out, workspace, workspace_bytes, rope_table,
-                                 (table_positions + 31) / 32, first_pos, stream);
+                                 (table_positions + 31) / 32, first_pos, 0, stream);
 }
 
 int squat_get_device_status(void *stream, unsigned *flags, int clear)

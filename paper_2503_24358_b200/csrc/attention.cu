@@ -30,6 +30,7 @@
 // key metadata cannot be folded into the query on this path: each pair is dequantized (one FMA per element),
 // turned (4) and multiplied with the block-turned query of every head (2 per head).
 #include "squat_internal.cuh"
+#include <cuda_fp16.h>
 
 namespace {
 
@@ -43,7 +44,7 @@ struct AttnParams {
     int q_bf16;
     int B, Hq, H, T;           // T: quantized tokens per (batch, head)
     const unsigned char *kc, *vc;
-    const float *ks, *kz, *vs, *vz;
+    const void *ks, *kz, *vs, *vz;   // float32, or binary16 in the M16 instances
     long long csb, csh;        // cache strides in tokens
     int G;
     const void *k_res, *v_res; // [B, H, R, D]
@@ -56,6 +57,7 @@ struct AttnParams {
     // rotary tables (pre-embedding key storage only): cos/sin of (32 a theta_i) [blocks][64] and of (l theta_i) [32][64]
     const float2 *rope_a, *rope_b;
     long long first_pos;       // position of cached token 0; a multiple of 32
+    int meta16;                // the cache's scales and zero-points are binary16
 };
 
 // 1 + code / 2^BITS as a float, for the code at position i of a 32-bit word (low bits first)
@@ -88,7 +90,27 @@ __device__ __forceinline__ float load_elem(const void *p, long long idx, int bf1
     return reinterpret_cast<const float *>(p)[idx];
 }
 
-template <int BITS, int NQ, bool ROPE>
+// scale / zero-point element i of a metadata array stored as float32 or binary16
+template <bool M16>
+__device__ __forceinline__ float meta_at(const void *p, long long i)
+{
+    if (M16) return __half2float(__ldg(reinterpret_cast<const __half *>(p) + i));
+    return __ldg(reinterpret_cast<const float *>(p) + i);
+}
+// four consecutive elements starting at i (a multiple of 4)
+template <bool M16>
+__device__ __forceinline__ float4 meta4_at(const void *p, long long i)
+{
+    if (M16) {
+        const uint2 r = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __half *>(p) + i));
+        const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&r.x));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&r.y));
+        return make_float4(a.x, a.y, b.x, b.y);
+    }
+    return __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p) + i));
+}
+
+template <int BITS, int NQ, bool ROPE, bool M16>
 __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : 1) attn_partial_kernel(const AttnParams p)
 {
     constexpr int WPT = D * BITS / 32;                          // 32-bit words per token: 8 or 16
@@ -138,8 +160,8 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : 1) attn
                     const float q0 = qsm[qi * D + i], q1 = qsm[qi * D + i + 64];
                     qb[qi * 64 + i] = make_float2(fmaf(q0, cs.x, q1 * cs.y), fmaf(q1, cs.x, -q0 * cs.y));
                 }
-                const float s0 = __ldg(p.ks + mrow + i) * LV, s1 = __ldg(p.ks + mrow + i + 64) * LV;
-                sz[i] = make_float4(s0, __ldg(p.kz + mrow + i) - s0, s1, __ldg(p.kz + mrow + i + 64) - s1);
+                const float s0 = meta_at<M16>(p.ks, mrow + i) * LV, s1 = meta_at<M16>(p.ks, mrow + i + 64) * LV;
+                sz[i] = make_float4(s0, meta_at<M16>(p.kz, mrow + i) - s0, s1, meta_at<M16>(p.kz, mrow + i + 64) - s1);
             }
             __syncwarp();
             const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
@@ -172,8 +194,8 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : 1) attn
             for (int qi = 0; qi < NQ; ++qi) sc[qi * AT_CHUNK + blk - t0 + lane] = acc[qi][0] + acc[qi][1];
             continue;
         }
-        const float4 s4 = __ldg(reinterpret_cast<const float4 *>(p.ks + mrow) + lane);
-        const float4 z4 = __ldg(reinterpret_cast<const float4 *>(p.kz + mrow) + lane);
+        const float4 s4 = meta4_at<M16>(p.ks, mrow + 4 * lane);
+        const float4 z4 = meta4_at<M16>(p.kz, mrow + 4 * lane);
         float k0[NQ];
         __syncwarp();
 #pragma unroll
@@ -290,14 +312,14 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : 1) attn
     for (; tk + TPI < vend; tk += 2 * TPI) {                    // two steps' loads in flight before either is used
         const long long c0 = ctok0 + tk, c1 = c0 + TPI;
         const uint32_t w0 = __ldg(vcw + c0 * WPT + j), w1 = __ldg(vcw + c1 * WPT + j);
-        const float s0 = __ldg(p.vs + c0 * ng + gidx), z0 = __ldg(p.vz + c0 * ng + gidx);
-        const float s1 = __ldg(p.vs + c1 * ng + gidx), z1 = __ldg(p.vz + c1 * ng + gidx);
+        const float s0 = meta_at<M16>(p.vs, c0 * ng + gidx), z0 = meta_at<M16>(p.vz, c0 * ng + gidx);
+        const float s1 = meta_at<M16>(p.vs, c1 * ng + gidx), z1 = meta_at<M16>(p.vz, c1 * ng + gidx);
         vstep(tk, w0, s0, z0);
         vstep(tk + TPI, w1, s1, z1);
     }
     if (tk < vend) {
         const long long c0 = ctok0 + tk;
-        vstep(tk, __ldg(vcw + c0 * WPT + j), __ldg(p.vs + c0 * ng + gidx), __ldg(p.vz + c0 * ng + gidx));
+        vstep(tk, __ldg(vcw + c0 * WPT + j), meta_at<M16>(p.vs, c0 * ng + gidx), meta_at<M16>(p.vz, c0 * ng + gidx));
     }
     // add the group constant, fold the token classes of the warp, then the warps
     __syncthreads();                                            // everybody is done reading sc: reuse it as [warps][NQ][D]
@@ -400,13 +422,13 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
     p.out[((long long)b * p.Hq + hq) * D + c] = acc / den;
 }
 
-template <int BITS, int NQ, bool ROPE>
+template <int BITS, int NQ, bool ROPE, bool M16>
 int launch_partial_r(const AttnParams &p, int qpasses, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * (NQ * D + AT_WARPS * NQ * D + NQ * AT_CHUNK + NQ * AT_WARPS + 8) +
                         (ROPE ? sizeof(float2) * 64 * 32 + sizeof(float4) * AT_WARPS * 64 : 0);
-    SQUAT_CUDA(cudaFuncSetAttribute(attn_partial_kernel<BITS, NQ, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_partial_kernel<BITS, NQ, ROPE><<<dim3(p.nchunk * qpasses, p.H, p.B), AT_THREADS, smem, st>>>(p);
+    SQUAT_CUDA(cudaFuncSetAttribute(attn_partial_kernel<BITS, NQ, ROPE, M16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attn_partial_kernel<BITS, NQ, ROPE, M16><<<dim3(p.nchunk * qpasses, p.H, p.B), AT_THREADS, smem, st>>>(p);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
@@ -414,7 +436,8 @@ int launch_partial_r(const AttnParams &p, int qpasses, cudaStream_t st)
 template <int BITS, int NQ>
 int launch_partial(const AttnParams &p, int qpasses, cudaStream_t st)
 {
-    return p.rope_a ? launch_partial_r<BITS, NQ, true>(p, qpasses, st) : launch_partial_r<BITS, NQ, false>(p, qpasses, st);
+    if (p.meta16) return p.rope_a ? launch_partial_r<BITS, NQ, true, true>(p, qpasses, st) : launch_partial_r<BITS, NQ, false, true>(p, qpasses, st);
+    return p.rope_a ? launch_partial_r<BITS, NQ, true, false>(p, qpasses, st) : launch_partial_r<BITS, NQ, false, false>(p, qpasses, st);
 }
 
 }  // namespace
@@ -426,14 +449,15 @@ size_t squat_attention_workspace_floats(int batch, int n_q_heads, int n_tokens)
 }
 
 int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq, int H, int T,
-                                  const unsigned char *kc, const float *ks, const float *kz,
-                                  const unsigned char *vc, const float *vs, const float *vz,
+                                  const unsigned char *kc, const void *ks, const void *kz,
+                                  const unsigned char *vc, const void *vs, const void *vz,
                                   long long csb, long long csh, int bits, int G,
                                   const void *k_res, const void *v_res, int res_dtype, int R,
                                   float scale, float *out, float *workspace,
-                                  const float *rope_table, int rope_blocks, long long first_pos, cudaStream_t st)
+                                  const float *rope_table, int rope_blocks, long long first_pos, int meta16, cudaStream_t st)
 {
     AttnParams p;
+    p.meta16 = meta16;
     p.rope_a = reinterpret_cast<const float2 *>(rope_table);                     // NULL: keys were stored after the embedding
     p.rope_b = p.rope_a ? p.rope_a + (size_t)rope_blocks * 64 : nullptr;
     p.first_pos = first_pos;

@@ -51,12 +51,12 @@ int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T,
                               long long osb, long long osh, unsigned *status, int meta16, cudaStream_t st);
 size_t squat_attention_workspace_floats(int batch, int n_q_heads, int n_tokens);
 int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq, int H, int T,
-                                  const unsigned char *kc, const float *ks, const float *kz,
-                                  const unsigned char *vc, const float *vs, const float *vz,
+                                  const unsigned char *kc, const void *ks, const void *kz,
+                                  const unsigned char *vc, const void *vs, const void *vz,
                                   long long csb, long long csh, int bits, int G,
                                   const void *k_res, const void *v_res, int res_dtype, int R,
                                   float scale, float *out, float *workspace,
-                                  const float *rope_table, int rope_blocks, long long first_pos, cudaStream_t st);
+                                  const float *rope_table, int rope_blocks, long long first_pos, int meta16, cudaStream_t st);
 int squat_launch_dequant(int kind, const unsigned char *codes, const void *scales, const void *zeros,
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
                          void *out, int out_dtype, int meta16, cudaStream_t st);

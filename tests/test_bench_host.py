@@ -54,6 +54,7 @@ def test_algorithmic_counts():
     # the reader: 32 + 32 code bytes, 32 bytes of key metadata, 32 of value metadata per cached token at 2 bits, G = 32
     assert bench.reader_bytes_per_cached_token(128, 2, 32) == 128
     assert bench.reader_bytes_per_cached_token(128, 4, 128) == 64 + 64 + 8 + 8
+    assert bench.reader_bytes_per_cached_token(128, 2, 32, meta_bytes=2) == 32 + 32 + 16 + 16
 
 
 def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():

@@ -261,3 +261,50 @@ def test_pre_rope_reader_special_cases():
         sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, 1024, 8, k_res, v_res)
     with pytest.raises(sq.SquatError):
         sq.squat_decode_attention_pre_rope(q, *cache, H, T, bits, G, out, ws, table, 1024, 512, k_res, v_res)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The readers over a cache with 16-bit (binary16) scales and zero-points, built by the oracle's 16-bit variants.
+
+def _oracle_cache16(seed, B, H, T, bits, G):
+    rng = np.random.default_rng(seed)
+    K = rng.standard_normal((B, H, T, D))
+    K[..., 7] *= 8.0
+    V = rng.standard_normal((B, H, T, D))
+    kc = np.zeros((B, H, T, D * bits // 8), np.uint8)
+    vc = np.zeros_like(kc)
+    ks = np.zeros((B, H, T // G, D), np.float16)
+    kz = np.zeros_like(ks)
+    vs = np.zeros((B, H, T, D // G), np.float16)
+    vz = np.zeros_like(vs)
+    units = {}
+    for b in range(B):
+        for h in range(H):
+            kq = oracle.quant_keys(K[b, h], G, bits, meta16=True)
+            vq = oracle.quant_values_f32(V[b, h].astype(np.float32), G, bits, meta16=True)
+            kc[b, h], vc[b, h] = oracle.pack(kq["codes"], bits), oracle.pack(vq["codes"], bits)
+            ks[b, h], kz[b, h] = kq["scale"].astype(np.float16), kq["zero"].astype(np.float16)      # exact: binary16 values
+            vs[b, h], vz[b, h] = vq["scale"].astype(np.float16), vq["zero"].astype(np.float16)
+            assert np.array_equal(ks[b, h].astype(np.float32), kq["scale"])
+            units[b, h] = (kq, vq)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    return (dev(kc), dev(ks), dev(kz), dev(vc), dev(vs), dev(vz)), units
+
+
+@pytest.mark.parametrize("bits,G,qpk,T,R", [(2, 32, 1, 256, 0), (2, 32, 4, 2112, 32), (4, 64, 2, 1088, 128), (2, 128, 8, 128, 5)])
+def test_readers_over_a_cache_with_16_bit_metadata(bits, G, qpk, T, R):
+    B, H = 2, 2
+    cache, units = _oracle_cache16(70 + bits + G + qpk, B, H, T, bits, G)
+    g = torch.Generator().manual_seed(T + R)
+    q = torch.randn(B, H * qpk, D, generator=g).to(torch.bfloat16).cuda()
+    k_res = v_res = None
+    if R:
+        k_res = torch.randn(B, H, R, D, generator=g).cuda()
+        v_res = torch.randn(B, H, R, D, generator=g).cuda()
+    kr = None if k_res is None else k_res.double().cpu().numpy()
+    vr = None if v_res is None else v_res.double().cpu().numpy()
+    qn = q.double().cpu().numpy()
+    out = _run(q, cache, H, T, bits, G, k_res, v_res)                          # keys stored after the rotary embedding
+    print("max err", _check(out, qn, units, H, G, kr, vr))
+    out = _run_pre(q, cache, H, T, bits, G, 64, 64 + T + R, k_res, v_res)      # keys stored before it
+    print("max err (pre)", _check_pre(out, qn, units, H, G, 64, kr, vr))
