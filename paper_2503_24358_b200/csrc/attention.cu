@@ -111,7 +111,7 @@ __device__ __forceinline__ float4 meta4_at(const void *p, long long i)
 }
 
 template <int BITS, int NQ, bool ROPE, bool M16>
-__global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : 1) attn_partial_kernel(const AttnParams p)
+__global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ? 3 : 4)) attn_partial_kernel(const AttnParams p)
 {
     constexpr int WPT = D * BITS / 32;                          // 32-bit words per token: 8 or 16
     constexpr int CPW = 32 / BITS;                              // codes per word: 16 or 8
