@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
 // scales and zeros are read once for the four).  Codes become floats through the 2^23 trick
 // (exact), then one fma each: deq(c) = fma(c, scale, zero), rounded once.
 template <int BITS, bool KEYS, bool OUT_BF16, bool M16>
-__global__ void __launch_bounds__(256) dequant_kernel(
+__global__ void __launch_bounds__(256, 4) dequant_kernel(
     const unsigned char *__restrict__ codes, const void *__restrict__ scales, const void *__restrict__ zeros,
     long long n_units, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
 {
