@@ -186,15 +186,14 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
     }
 }
 
-// One thread dequantizes 16 consecutive channels of 4 consecutive tokens (same key group, so the 16
-// scales and zeros are read once for the four).  Codes become floats through the 2^23 trick
+// One thread dequantizes 16 consecutive channels of TOK = 4 or 8 consecutive tokens (same key group, so the 16
+// scales and zeros are read once for all of them; 8 on large inputs, 4 where that would leave SMs without work).  Codes become floats through the 2^23 trick
 // (exact), then one fma each: deq(c) = fma(c, scale, zero), rounded once.
-template <int BITS, bool KEYS, bool OUT_BF16, bool M16>
+template <int BITS, bool KEYS, bool OUT_BF16, bool M16, int TOK>
 __global__ void __launch_bounds__(256, 4) dequant_kernel(
     const unsigned char *__restrict__ codes, const void *__restrict__ scales, const void *__restrict__ zeros,
     long long n_units, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
 {
-    constexpr int TOK = 4;
     const int per_tok = d / 16;
     const int tq_per_row = (T + TOK - 1) / TOK;
     const int row_bytes = d * BITS / 8;
@@ -330,11 +329,17 @@ int squat_launch_dequant(int kind, const unsigned char *codes, const void *scale
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
                          void *out, int out_dtype, int meta16, cudaStream_t st)
 {
-    const long long n_units = (long long)batch * H * ((T + 3) / 4) * (d / 16);     // 4 tokens x 16 channels per thread
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long units8 = (long long)batch * H * ((T + 7) / 8) * (d / 16);       // threads with 8 tokens x 16 channels each
+    const bool tok8 = units8 >= (long long)sms * 32 * 256;                           // enough of them to fill the grid cap
+    const long long n_units = tok8 ? units8 : (long long)batch * H * ((T + 3) / 4) * (d / 16);
     if (n_units == 0) return SQUAT_OK;
     const int grid = grid_for(n_units, 256);
-#define SQ_D(BB, KK, OO) do { if (meta16) dequant_kernel<BB, KK, OO, true><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out); \
-                               else dequant_kernel<BB, KK, OO, false><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out); } while (0)
+#define SQ_D1(BB, KK, OO, MM, TT) dequant_kernel<BB, KK, OO, MM, TT><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out)
+#define SQ_D(BB, KK, OO) do { if (meta16) { if (tok8) SQ_D1(BB, KK, OO, true, 8); else SQ_D1(BB, KK, OO, true, 4); } \
+                              else { if (tok8) SQ_D1(BB, KK, OO, false, 8); else SQ_D1(BB, KK, OO, false, 4); } } while (0)
     const bool keys = kind == SQUAT_KEYS, obf = out_dtype == SQUAT_BF16;
     if (bits == 2) {
         if (keys) { if (obf) SQ_D(2, true, true); else SQ_D(2, true, false); }
@@ -345,6 +350,7 @@ int squat_launch_dequant(int kind, const unsigned char *codes, const void *scale
     } else {
         return SQUAT_ERR_UNSUPPORTED;
     }
+#undef SQ_D1
 #undef SQ_D
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
