@@ -268,3 +268,39 @@ def build_W(Qc, r, lam, g=1):
     mats = update_matrices(Qhat, d, lam, g)
     mats.update({"Qhat": Qhat, "mu": mu, "V": V})
     return mats
+
+
+def power_subspace(M, X0, iters):
+    """Block power method for the query subspace (the accelerator the paper names for line 5 of Algorithm 1;
+    the paper gives no steps, these are the textbook ones):  X <- orth(M X), `iters` times from the start
+    block X0 [d, r] (iters = 0: X = orth(X0)), then Rayleigh-Ritz on span(X): B = X^T M X = S diag(theta) S^T,
+    Ritz vectors u_i = X s_i.  Returns (Qhat [r, d] with rows sqrt(theta_i) u_i^T, theta descending, X), so
+    that Qhat^T Qhat = X B X^T, the compression of M to the iterated subspace, takes the place of the rank-r
+    truncation of M.  Library steps: numpy's Householder QR and symmetric eigensolver."""
+    M = np.asarray(M, dtype=np.float64)
+    X = np.asarray(X0, dtype=np.float64)
+    d, r = X.shape
+    if M.shape != (d, d):
+        raise ValueError("M must be [d, d] and X0 [d, r]")
+    if iters == 0:
+        X, _ = np.linalg.qr(X)
+    for _ in range(iters):
+        Y = M @ X
+        X, _ = np.linalg.qr(Y)
+    B = X.T @ (M @ X)
+    B = 0.5 * (B + B.T)
+    theta, S = np.linalg.eigh(B)
+    theta, S = theta[::-1], S[:, ::-1]
+    U = X @ S
+    Qhat = np.sqrt(np.maximum(theta, 0.0))[:, None] * U.T
+    return np.ascontiguousarray(Qhat), theta.copy(), X
+
+
+def build_W_power(Qc, X0, iters, lam, g=1):
+    """Stacked queries -> update matrix W with the block power method in place of the SVD."""
+    d = Qc.shape[1]
+    M = gram(Qc)
+    Qhat, theta, X = power_subspace(M, X0, iters)
+    mats = update_matrices(Qhat, d, lam, g)
+    mats.update({"Qhat": Qhat, "theta": theta, "X": X, "M": M})
+    return mats

@@ -16,6 +16,7 @@ from .generators import (
     gen_keys,
     gen_values,
     gen_queries,
+    gen_start_block,
     round_to_dtype,
     to_f32,
 )
@@ -24,5 +25,5 @@ __all__ = [
     "CONFIGS", "WorkloadConfig", "get_config",
     "bf16_bits_to_f32", "f32_to_bf16_bits", "round_to_dtype", "to_f32",
     "gen_keys_unit", "gen_values_unit", "gen_queries_head", "outlier_channels",
-    "gen_keys", "gen_values", "gen_queries",
+    "gen_keys", "gen_values", "gen_queries", "gen_start_block",
 ]

@@ -12,7 +12,7 @@ import numpy as np
 
 from .configs import WorkloadConfig
 
-_T_QA, _T_QB, _T_QN, _T_K, _T_V, _T_OUT = 1, 2, 3, 4, 5, 6
+_T_QA, _T_QB, _T_QN, _T_K, _T_V, _T_OUT, _T_START = 1, 2, 3, 4, 5, 6, 7
 
 
 def _rng(seed: int, tensor: int, a: int = 0, b: int = 0, c: int = 0) -> np.random.Generator:
@@ -116,3 +116,9 @@ def gen_values(cfg: WorkloadConfig, n_tokens: int = None, segment: int = 0, batc
         for h in range(cfg.n_kv_heads):
             out[b, h] = gen_values_unit(cfg, b, h, n, segment)
     return out
+
+
+def gen_start_block(seed: int, d: int, r: int, head: int = 0) -> np.ndarray:
+    """Start block [d, r] (float64, standard normal) of a block power iteration: the random numbers that
+    method draws, made here so that every implementation is handed the same ones."""
+    return _rng(seed, _T_START, head).standard_normal((d, r))
