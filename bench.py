@@ -321,9 +321,21 @@ def run_gpu(args, cfg):
 
     stage_names = ["build_subspace", "quantize_keys", "quantize_values", "dequantize"]
 
+    # start block of the block power method (the random numbers that variant draws), resident like the other inputs
+    x0 = torch.from_numpy(si.gen_start_block(cfg.seed, d, cfg.rank_r)).to(dev) if 0 < cfg.rank_r <= 64 else None
+    use_power = args.subspace == "power"
+    if use_power and x0 is None:
+        raise SystemExit("--subspace power needs 0 < rank <= 64")
+
+    def build():
+        if use_power:
+            sq.squat_build_subspace_power(s, q, cfg.rank_r, cfg.lam, x0, args.power_iters, cfg.block_g)
+        else:
+            sq.squat_build_subspace(s, q, cfg.rank_r, cfg.lam, cfg.block_g)
+
     def step(ev=None):
         if ev: ev[0].record(stream)
-        sq.squat_build_subspace(s, q, cfg.rank_r, cfg.lam, cfg.block_g)
+        build()
         if ev: ev[1].record(stream)
         sq.squat_quantize_keys(s, k, bits, G, kc, ks, kz)
         if ev: ev[2].record(stream)
@@ -367,9 +379,28 @@ def run_gpu(args, cfg):
     total_ms, total_units = aggregate_over_ranks(local_ms, vec_per_step * args.steps, dev)
     flags = sq.squat_get_device_status(clear=True)
 
+    # ---- step 1 with the block power method, timed on its own beside the default (SVD) build ------------
+    power = None
+    if rank == 0 and x0 is not None and not use_power:
+        n_p = max(3, min(args.steps, 20))
+        pev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_p)]
+        for i in range(-2, n_p):
+            flush.zero_()
+            if i >= 0: pev[i][0].record(stream)
+            sq.squat_build_subspace_power(s, q, cfg.rank_r, cfg.lam, x0, args.power_iters, cfg.block_g)
+            if i >= 0: pev[i][1].record(stream)
+        torch.cuda.synchronize()
+        p_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in pev)
+        power = {"ms": p_ms, "iters": args.power_iters, "api": "squat_build_subspace_power",
+                 "note": "Gram + block power iteration + update matrices; not part of the timed step "
+                         "(run with --subspace power to time the whole path with it)",
+                 "whole_path_ms_with_it": statistics.mean(step_ms) - stage_ms["build_subspace"] + p_ms}
+        sq.squat_build_subspace(s, q, cfg.rank_r, cfg.lam, cfg.block_g)      # leave the handle as the step left it
+        torch.cuda.synchronize()
+
     # ---- end to end from host buffers through squat_write_path_host --------------------------------
     e2e = None
-    if not args.no_e2e and not args.meta16:              # the host-buffer entry writes float32 metadata
+    if not args.no_e2e and not args.meta16 and not use_power:   # the host-buffer entry: float32 metadata, SVD build
         e2e = run_e2e(args, cfg, sq, s, (q_np, k_np, v_np), (kc, ks, kz, vc, vs, vz), to_dev, flush, tdt, dev,
                       vec_per_step)
     # ---- the reader that follows the write path (not part of a step): one decode step of attention -----
@@ -378,7 +409,7 @@ def run_gpu(args, cfg):
         reader = run_reader(cfg, sq, (kc, ks, kz, vc, vs, vz), flush, tdt, dev, meta_bytes=2 if args.meta16 else 4)
     if rank == 0:
         report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches,
-               wall, flags, clocks, reader)
+               wall, flags, clocks, reader, power)
     s.close()
     if world > 1:
         dist.destroy_process_group()
@@ -457,7 +488,7 @@ def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10, meta_bytes=4):
 
 
 def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, e2e, launches, wall,
-           flags, clocks, reader=None):
+           flags, clocks, reader=None, power=None):
     d, bits, G = cfg.head_dim, cfg.bits, cfg.group_size
     if rank_is_zero():
         peaks = measured_peaks()
@@ -501,11 +532,16 @@ def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_nam
         stages["quantize_values"]["hbm_frac"] = stages["quantize_values"]["hbm_gbs"] / peaks["hbm_gbs"]
         stages["dequantize"]["hbm_gbs"] = dq_bytes / (stage_ms["dequantize"] * 1e-3) / 1e9
         stages["dequantize"]["hbm_frac"] = stages["dequantize"]["hbm_gbs"] / peaks["hbm_gbs"]
+        stages["build_subspace"]["method"] = ("block power, %d multiplications" % args.power_iters
+                                              if args.subspace == "power" else "svd (fp64 eigen-decomposition)")
+        if power is not None:
+            stages["build_subspace"]["block_power_variant"] = power
         line = {
             "metric": METRIC, "value": total_units / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": dict(workload_config(cfg), metadata="binary16" if args.meta16 else "float32"),
+            "config": dict(workload_config(cfg), metadata="binary16" if args.meta16 else "float32",
+                           subspace=args.subspace),
             "kv_ingested_gbs": 2 * vec_per_step * world * d * elem / (total_ms / args.steps * 1e-3) / 1e9,
             "roofline": roof, "stages": stages,
             "e2e": e2e,
@@ -529,6 +565,9 @@ def main():
     ap.add_argument("--group-size", type=int, default=None, choices=[32, 64, 128], help="override the workload's group size G")
     ap.add_argument("--meta16", action="store_true", help="store scales and zero-points as binary16 (the 18.75 %% cache); "
                     "times the write path only")
+    ap.add_argument("--subspace", default="svd", choices=["svd", "power"], help="step 1: the paper's SVD (default) or the "
+                    "block power method it names as an accelerator")
+    ap.add_argument("--power-iters", type=int, default=2, help="multiplications by the Gram matrix of the block power method")
     ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")

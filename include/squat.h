@@ -93,6 +93,28 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
 int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
                                    void *stream);
 
+/*
+ * Step 1 with the block power method in place of the SVD (the accelerator the paper's comment on Algorithm 1 line 5
+ * names; it gives no steps, these are the textbook ones).  Per KV head, with M the Gram matrix of the stacked queries:
+ *     X <- orth(M X), `iters` times, from the start block X0;  B = X^T M X;  P = I + lambda X B X^T,
+ * i.e. the compression of M to the iterated r-dimensional subspace stands where squat_build_subspace has the rank-r
+ * truncation of M (the two agree once span(X) is the dominant eigenspace; P depends on span(X) only, so the Ritz
+ * pairs of B are never formed).  W follows from P exactly as in squat_build_subspace; all of it in fp64.
+ *   q .. block_g       as for squat_build_subspace, except rank_r <= 64 (SQUAT_ERR_UNSUPPORTED above).
+ *   start_block        device, float64, 8-byte aligned: X0 as [d, rank_r] row-major (the random numbers the method
+ *                      draws are the caller's); head h reads start_block + h * start_stride_h (elements; 0 = the
+ *                      same block for every head, else >= d * rank_r).  Read only; may be NULL when rank_r = 0.
+ *   iters              0 <= iters <= 64 multiplications by M (0: X = orth(X0)).
+ * Orthonormalisation is Cholesky QR (twice for the last basis).  A direction whose pivot falls below 1e-13 of its
+ * diagonal entry (start block or Gram matrix of rank < rank_r within the block, or cond(M) on the block beyond
+ * ~1e6) is dropped and contributes nothing; squat_subspace_eig_sweeps then reports, per head, the number of basis
+ * columns kept (= rank_r when nothing was dropped) instead of a sweep count.  The eigenvalue / eigenvector arrays
+ * of squat_subspace_export are scratch after this call.  Enqueues on `stream`.
+ */
+int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
+                               long long stride_h, long long stride_t, int rank_r, double lambda, int block_g,
+                               const double *start_block, long long start_stride_h, int iters, void *stream);
+
 /* Test / checkpoint hooks.  Both synchronise `stream`.  Host pointers; any may be NULL.
  *   W_host      [n_kv_heads, d, d] float32, row j' column j, block strictly lower triangular.
  *   gram_host   [n_kv_heads, d, d] float64 Gram matrices of the last build.

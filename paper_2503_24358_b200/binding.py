@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
-    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
+    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
 )
 
 _lib = None
@@ -71,6 +71,7 @@ def _load():
         lib.squat_quantize_values_m16.argtypes = lib.squat_quantize_values.argtypes
         lib.squat_dequantize_m16.argtypes = lib.squat_dequantize.argtypes
         lib.squat_build_subspace_from_gram.argtypes = [vp, vp, i, dbl, i, vp]
+        lib.squat_build_subspace_power.argtypes = [vp, vp, i, i, i, ll, ll, i, dbl, i, vp, ll, i, vp]
         lib.squat_rope_table_floats.argtypes = [i]
         lib.squat_rope_table_floats.restype = c.c_size_t
         lib.squat_rope_table_fill.argtypes = [dbl, i, i, vp]
@@ -276,6 +277,27 @@ def squat_build_subspace_from_gram(s: "Subspace", gram: torch.Tensor, rank_r: in
         raise ValueError("gram must be a contiguous float64 tensor")
     _check(_load().squat_build_subspace_from_gram(s.handle, _dev(gram, "gram"), int(rank_r), ctypes.c_double(lam),
                                                   int(block_g), _stream(stream)), "squat_build_subspace_from_gram")
+
+
+def squat_build_subspace_power(s: "Subspace", q: torch.Tensor, rank_r: int, lam: float, start_block: torch.Tensor,
+                               iters: int = 2, block_g: int = 1, stream=None):
+    """Step 1 with the block power method: q as for squat_build_subspace; start_block [d, rank_r] (one block for all
+    heads) or [n_kv_heads, d, rank_r], float64, CUDA, contiguous; iters multiplications by the Gram matrix."""
+    if q.dim() != 3 or q.stride(2) != 1 or q.shape[2] != s.head_dim:
+        raise ValueError("q must be [n_q_heads, n_tokens, head_dim] with contiguous last dim")
+    if start_block.dtype != torch.float64 or not start_block.is_contiguous():
+        raise ValueError("start_block must be a contiguous float64 tensor")
+    if tuple(start_block.shape) == (s.head_dim, rank_r):
+        stride_h = 0
+    elif tuple(start_block.shape) == (s.n_kv_heads, s.head_dim, rank_r):
+        stride_h = s.head_dim * rank_r
+    else:
+        raise ValueError("start_block must be [d, rank_r] or [n_kv_heads, d, rank_r]")
+    ptr = _dev(start_block, "start_block") if rank_r > 0 else None
+    _check(_load().squat_build_subspace_power(s.handle, _dev(q, "q"), _dtype_code(q), q.shape[0], q.shape[1],
+                                              q.stride(0), q.stride(1), int(rank_r), ctypes.c_double(lam), int(block_g),
+                                              ptr, stride_h, int(iters), _stream(stream)),
+           "squat_build_subspace_power")
 
 
 def token_shard(n_tokens: int, rank: int, world: int, multiple: int = 32):

@@ -159,7 +159,7 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
     if (rc != SQUAT_OK) return rc;
     // channels of the first g-block are never corrected; with r = 0 or lambda = 0, W = 0 and none is
     s->exact_blocks = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
-    return squat_launch_assemble(s, rank_r, lambda, block_g, st);
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 0, st);
 }
 
 int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
@@ -175,7 +175,35 @@ int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int ra
     int rc = squat_launch_eig(s, st);
     if (rc != SQUAT_OK) return rc;
     s->exact_blocks = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
-    return squat_launch_assemble(s, rank_r, lambda, block_g, st);
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 0, st);
+}
+
+int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
+                               long long stride_h, long long stride_t, int rank_r, double lambda, int block_g,
+                               const double *start_block, long long start_stride_h, int iters, void *stream)
+{
+    if (!s || !q || !valid_dtype(dtype) || !aligned16(q)) return SQUAT_ERR_INVALID_ARG;
+    if (n_q_heads <= 0 || n_tokens <= 0) return SQUAT_ERR_INVALID_ARG;
+    if (n_q_heads % s->n_kv_heads != 0) return SQUAT_ERR_SHAPE;
+    if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
+    if (rank_r > 64) return SQUAT_ERR_UNSUPPORTED;
+    if ((long long)rank_r > (long long)n_tokens * (n_q_heads / s->n_kv_heads)) return SQUAT_ERR_SHAPE;
+    if (!(lambda >= 0.0) || !std::isfinite(lambda)) return SQUAT_ERR_INVALID_ARG;
+    if (block_g <= 0 || D % block_g != 0) return SQUAT_ERR_SHAPE;
+    if (iters < 0 || iters > 64 || start_stride_h < 0) return SQUAT_ERR_INVALID_ARG;
+    if (rank_r > 0 && (!start_block || ((uintptr_t)start_block & 7u))) return SQUAT_ERR_INVALID_ARG;
+    if (start_stride_h != 0 && start_stride_h < (long long)D * rank_r) return SQUAT_ERR_INVALID_ARG;
+    const long long vec = 16 / (long long)elem_size(dtype);
+    if (stride_t < D || stride_h < 0 || stride_t % vec || stride_h % vec) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = squat_launch_gram(s, q, dtype, n_q_heads, n_tokens, stride_h, stride_t, st);
+    if (rc != SQUAT_OK) return rc;
+    const bool no_update = rank_r == 0 || lambda == 0.0;
+    s->exact_blocks = no_update ? D / 32 : (block_g + 31) / 32;
+    if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, st);      // W = 0: nothing to iterate
+    rc = squat_launch_power(s, start_block, start_stride_h, rank_r, iters, lambda, st);
+    if (rc != SQUAT_OK) return rc;
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 64, st);
 }
 
 int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,

@@ -38,7 +38,9 @@ void squat_count_launch(unsigned n = 1);
 int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
                       long long stride_h, long long stride_t, cudaStream_t st);
 int squat_launch_eig(squat_subspace *s, cudaStream_t st);
-int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st);
+int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, int left_rows, cudaStream_t st);
+int squat_launch_power(squat_subspace *s, const double *start, long long start_stride_h, int rank_r, int iters,
+                       double lambda, cudaStream_t st);
 
 int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaStream_t st);
 int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,

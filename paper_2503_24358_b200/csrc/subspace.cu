@@ -516,8 +516,10 @@ constexpr int ASM_LD = D + 1;
 
 __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
     const double *__restrict__ eigval, const double *__restrict__ eigvec, int rank_r, double lambda, int g,
-    float *__restrict__ Wt)
+    float *__restrict__ Wt, int left_rows)
 {
+    // left_rows = 0: P_inv = I - sum_i s_i/(1+s_i) v_i v_i^T from eigen-pairs (rows i of eigvec, eigval).
+    // left_rows > 0: P_inv = I - sum_i z_i x_i^T with x_i = row i and z_i = row left_rows + i of eigvec (block power build).
     extern __shared__ __align__(16) double sm[];
     double *A = sm;                         // A[row * ASM_LD + col]
     double *colv = sm + D * ASM_LD;         // [2 parities][l, v][D]: column j of L and of the matrix, as published
@@ -529,7 +531,7 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
         double mu = eigval[(long long)h * D + tid];
         if (!(mu > 0.0)) mu = 0.0;
         const double s = lambda * mu;
-        coef[tid] = (tid < rank_r) ? s / (1.0 + s) : 0.0;
+        coef[tid] = (tid < rank_r) ? (left_rows > 0 ? 1.0 : s / (1.0 + s)) : 0.0;
     }
     __syncthreads();
     // The matrix lives in REGISTERS from here to the end of the factorisation: thread (lane, warp) owns the elements
@@ -538,7 +540,8 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
     double a[4][8];
     // P_inv = I - sum_{i<r} coef_i v_i v_i^T; the eigenvectors are staged 32 at a time in shared memory
     {
-        double *U = coef + D;                           // [32][D] staged eigenvectors
+        double *U = coef + D;                           // [32][D] staged eigenvectors (right vectors)
+        double *UL = left_rows > 0 ? U + 32 * D : U;    // [32][D] staged left vectors
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -547,12 +550,14 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
             const int ni = rank_r - i0 < 32 ? rank_r - i0 : 32;
             __syncthreads();
             for (int idx = tid; idx < ni * D; idx += ASM_THREADS) U[idx] = V[(long long)i0 * D + idx];
+            if (left_rows > 0)
+                for (int idx = tid; idx < ni * D; idx += ASM_THREADS) UL[idx] = V[(long long)(left_rows + i0) * D + idx];
             __syncthreads();
             for (int e = 0; e < ni; ++e) {
                 const double cf = -coef[i0 + e];
                 double vr[4], vc[8];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) vr[i] = cf * U[e * D + lane + 32 * i];
+                for (int i = 0; i < 4; ++i) vr[i] = cf * UL[e * D + lane + 32 * i];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) vc[k] = U[e * D + warp + 16 * k];
 #pragma unroll
@@ -683,11 +688,11 @@ int squat_launch_eig(squat_subspace *s, cudaStream_t st)
     return SQUAT_OK;
 }
 
-int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st)
+int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, int left_rows, cudaStream_t st)
 {
-    const size_t smem = sizeof(double) * (D * ASM_LD + 5 * D + 32 * D);
+    const size_t smem = sizeof(double) * (D * ASM_LD + 5 * D + 64 * D);
     SQUAT_CUDA(cudaFuncSetAttribute(assemble_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt);
+    assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt, left_rows);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, st);
