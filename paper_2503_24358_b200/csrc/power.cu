@@ -15,7 +15,7 @@
 // X becomes zero and contributes nothing from then on.  One pass of Cholesky QR needs cond(M restricted to the block)
 // well below 1e6.5; beyond that, directions are dropped and the count of kept columns (reported per head) says so.
 //
-// One CTA per head; X and Y are stored column by column with an odd stride, so that column dot products (lanes =
+// One CTA of 256 threads per head; X and Y are stored column by column with an odd stride, so that column dot products (lanes =
 // different columns), products with M (lanes = different rows) and the per-row triangular solves (lanes = different
 // rows) are all free of shared-memory bank conflicts.  No waiting on anything but __syncthreads.
 #include "squat_internal.cuh"
@@ -23,54 +23,68 @@
 namespace {
 
 constexpr int D = SQUAT_D;
-constexpr int PW_THREADS = 512;
+constexpr int PW_THREADS = 256;
 constexpr int LDC = D + 1;                      // column stride of X and Y (doubles)
 constexpr double PW_DROP = 1e-13;
 
 template <int RP>
 struct PowerLayout {
     static constexpr int LDG = RP + 1;                                         // row stride of G / L
-    static constexpr size_t doubles = 2 * (size_t)RP * LDC + (size_t)RP * LDG + 2 * RP + 8;
+    static constexpr bool M_SHARED = RP <= 32;                                 // M beside X, Y fits in shared memory
+    static constexpr size_t small = 2 * (size_t)RP * LDC + (size_t)RP * LDG + RP + 8;   // X, Y, G, inv, misc
+    static constexpr size_t doubles = small + (M_SHARED ? (size_t)D * D : 0);
 };
 
-// Y = M X: thread = rows (2 rp, 2 rp + 1) x column quads; M is symmetric, so row k of M holds column k
-template <int RP>
+// Y = M X: thread = rows 4 rq .. 4 rq + 3 x 8 columns (warp-uniform); M is symmetric, so row k of M holds column k.
+// With 32 columns four warps cover them and the other four take the second half of the sum over k, added after a
+// barrier; with 64 columns every warp has its own 8.
+template <int RP, bool MS>
 __device__ __forceinline__ void pw_mult(const double *__restrict__ M, const double *Xt, double *Yt, int tid)
 {
-    constexpr int NQ = RP / 32;                 // column quads per thread
-    const int rp = tid & 63, cs = tid >> 6;
-    double acc[NQ][4][2];
+    constexpr int KS = (RP == 32) ? 2 : 1;      // parts of the k range
+    const int rq = tid & 31, w = tid >> 5;
+    const int c0 = 8 * (w % (RP / 8)), part = w / (RP / 8);
+    double acc[8][4];
 #pragma unroll
-    for (int u = 0; u < NQ; ++u)
+    for (int b = 0; b < 8; ++b)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[u][b][0] = acc[u][b][1] = 0.0;
-#pragma unroll 4
-    for (int k = 0; k < D; ++k) {
-        const double2 m = __ldg(reinterpret_cast<const double2 *>(M + (size_t)k * D) + rp);
+        for (int a = 0; a < 4; ++a) acc[b][a] = 0.0;
+    const int k_lo = part * (D / KS), k_hi = k_lo + D / KS;
+#pragma unroll 2
+    for (int k = k_lo; k < k_hi; ++k) {
+        const double2 *mp = reinterpret_cast<const double2 *>(M + (size_t)k * D) + 2 * rq;
+        const double2 m01 = MS ? mp[0] : __ldg(mp);                 // MS: M is a shared-memory copy
+        const double2 m23 = MS ? mp[1] : __ldg(mp + 1);
+        const double m[4] = {m01.x, m01.y, m23.x, m23.y};
 #pragma unroll
-        for (int u = 0; u < NQ; ++u)
+        for (int b = 0; b < 8; ++b) {
+            const double x = Xt[(c0 + b) * LDC + k];
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const double x = Xt[(4 * (cs + 8 * u) + b) * LDC + k];
-                acc[u][b][0] = fma(m.x, x, acc[u][b][0]);
-                acc[u][b][1] = fma(m.y, x, acc[u][b][1]);
-            }
-    }
-#pragma unroll
-    for (int u = 0; u < NQ; ++u)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            double *y = Yt + (4 * (cs + 8 * u) + b) * LDC + 2 * rp;
-            y[0] = acc[u][b][0];
-            y[1] = acc[u][b][1];
+            for (int a = 0; a < 4; ++a) acc[b][a] = fma(m[a], x, acc[b][a]);
         }
+    }
+    if (part == 0) {
+#pragma unroll
+        for (int b = 0; b < 8; ++b)
+#pragma unroll
+            for (int a = 0; a < 4; ++a) Yt[(c0 + b) * LDC + 4 * rq + a] = acc[b][a];
+    }
+    if (KS == 2) {
+        __syncthreads();
+        if (part == 1) {
+#pragma unroll
+            for (int b = 0; b < 8; ++b)
+#pragma unroll
+                for (int a = 0; a < 4; ++a) Yt[(c0 + b) * LDC + 4 * rq + a] += acc[b][a];
+        }
+    }
 }
 
 // G[i][j] = add_identity * (i == j) + scale * sum_row At[i][row] Bt[j][row]
 template <int RP>
 __device__ __forceinline__ void pw_gram(const double *At, const double *Bt, double *G, double scale, double ident, int tid)
 {
-    constexpr int NJ = RP * RP / PW_THREADS;    // 2 (RP = 32) or 8 (RP = 64) columns j per thread
+    constexpr int NJ = RP * RP / PW_THREADS;    // 4 (RP = 32) or 16 (RP = 64) columns j per thread
     constexpr int LDG = PowerLayout<RP>::LDG;
     const int i = tid % RP, j0 = (tid / RP) * NJ;
     double acc[NJ];
@@ -86,80 +100,141 @@ __device__ __forceinline__ void pw_gram(const double *At, const double *Bt, doub
     for (int b = 0; b < NJ; ++b) G[i * LDG + j0 + b] = scale * acc[b] + ((i == j0 + b) ? ident : 0.0);
 }
 
-// In-place Cholesky G = L L^T of the lower triangle by one warp (left-looking; lane = rows lane, lane + 32).  A pivot
-// at or below drop * (its diagonal entry) zeroes the column: L[.][j] = 0, inv[j] = 0.  Returns the kept columns.
+// 1 / sqrt(x) for a positive normal x: exponent split off (x = s * 4^n with s in [1, 4)), single-precision seed, two
+// Newton steps in double precision (2^-22 -> 2^-44 -> beyond 2^-53), exponent put back.
+__device__ __forceinline__ double pw_rsqrt(double x)
+{
+    const int hi = __double2hiint(x), lo = __double2loint(x);
+    const int e2 = (((hi >> 20) & 0x7ff) - 1023) & ~1;
+    const double s = __hiloint2double(hi - (e2 << 20), lo);
+    double y = (double)rsqrtf((float)s);
+    const double hs = 0.5 * s;
+    y = y * fma(-hs * y, y, 1.5);
+    y = y * fma(-hs * y, y, 1.5);
+    return __hiloint2double(__double2hiint(y) - ((e2 >> 1) << 20), __double2loint(y));
+}
+
+// In-place Cholesky G = L L^T of the lower triangle by one warp, left-looking in panels of 8 columns; lane = rows
+// lane (and lane + 32).  A panel's entries live in registers: first the contributions of the columns to its left (a
+// loop over them, rows of L read from shared memory), then 8 elimination steps with the pivot row's values passed by
+// shuffles (a fully unrolled 32-column variant with the whole row in registers measured twice as slow).  A pivot at
+// or below drop * (the diagonal entry it started from) zeroes the column: L[.][j] = 0, inv[j] = 0.  Returns the
+// number of kept columns.
 template <int RP>
-__device__ __forceinline__ int pw_chol(double *G, double *inv, double drop, int lane)
+__device__ __noinline__ int pw_chol(double *G, double *inv, double drop, int lane)
 {
     constexpr int NR = RP / 32;
     constexpr int LDG = PowerLayout<RP>::LDG;
     int kept = 0;
-    for (int j = 0; j < RP; ++j) {
-        double v[NR];
+#pragma unroll 1
+    for (int jb = 0; jb < RP; jb += 8) {
+        double a[NR][8], g0[8];
 #pragma unroll
-        for (int u = 0; u < NR; ++u) {
-            const int i = lane + 32 * u;
-            double s0 = 0.0, s1 = 0.0;
-            if (i >= j) {
-                const double *gi = G + i * LDG, *gj = G + j * LDG;
-                int k = 0;
-                for (; k + 1 < j; k += 2) { s0 = fma(gi[k], gj[k], s0); s1 = fma(gi[k + 1], gj[k + 1], s1); }
-                if (k < j) s0 = fma(gi[k], gj[k], s0);
-                v[u] = gi[j] - (s0 + s1);
-            } else {
-                v[u] = 0.0;
+        for (int c = 0; c < 8; ++c) g0[c] = G[(jb + c) * LDG + jb + c];
+#pragma unroll
+        for (int u = 0; u < NR; ++u)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) a[u][c] = G[(lane + 32 * u) * LDG + jb + c];
+#pragma unroll 2
+        for (int k = 0; k < jb; ++k) {
+            double lj[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) lj[c] = G[(jb + c) * LDG + k];
+#pragma unroll
+            for (int u = 0; u < NR; ++u) {
+                const double lik = G[(lane + 32 * u) * LDG + k];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) a[u][c] = fma(-lik, lj[c], a[u][c]);
             }
         }
-        const double g0 = G[j * LDG + j];
-        double pv;                              // the pivot: v of row j, held by lane j % 32 (no dynamic register index)
-        if (NR == 1) {
-            pv = __shfl_sync(0xffffffffu, v[0], j & 31);
-        } else {
-            const double p0 = __shfl_sync(0xffffffffu, v[0], j & 31), p1 = __shfl_sync(0xffffffffu, v[NR - 1], j & 31);
-            pv = (j < 32) ? p0 : p1;
-        }
-        const bool ok = pv > drop * g0 && pv > 0.0;
-        const double ljj = ok ? sqrt(pv) : 0.0;
-        const double iv = ok ? 1.0 / ljj : 0.0;
-        kept += ok ? 1 : 0;
-        __syncwarp();
+        const int us = jb >> 5;                                     // which of the lane's rows the pivot rows are
 #pragma unroll
-        for (int u = 0; u < NR; ++u) {
-            const int i = lane + 32 * u;
-            if (i > j) G[i * LDG + j] = v[u] * iv;
-            else if (i == j) { G[j * LDG + j] = ljj; inv[j] = iv; }
+        for (int j = 0; j < 8; ++j) {
+            const int jj = jb + j;
+            const double mine = (NR == 1 || us == 0) ? a[0][j] : a[NR - 1][j];
+            const double pv = __shfl_sync(0xffffffffu, mine, jj & 31);
+            const bool ok = pv > drop * g0[j] && pv > 1e-290;
+            const double iv = ok ? pw_rsqrt(pv) : 0.0;
+            double l[NR];
+#pragma unroll
+            for (int u = 0; u < NR; ++u) {
+                const int i = lane + 32 * u;
+                l[u] = i > jj ? a[u][j] * iv : 0.0;
+                a[u][j] = i > jj ? l[u] : (i == jj ? pv * iv : a[u][j]);
+            }
+            if (lane == 0) inv[jj] = iv;
+            kept += ok ? 1 : 0;
+#pragma unroll
+            for (int c = j + 1; c < 8; ++c) {
+                const double lsrc = (NR == 1 || us == 0) ? l[0] : l[NR - 1];
+                const double lc = __shfl_sync(0xffffffffu, lsrc, (jb + c) & 31);
+#pragma unroll
+                for (int u = 0; u < NR; ++u) a[u][c] = fma(-l[u], lc, a[u][c]);
+            }
         }
+#pragma unroll
+        for (int u = 0; u < NR; ++u)
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                if (lane + 32 * u >= jb + c) G[(lane + 32 * u) * LDG + jb + c] = a[u][c];
         __syncwarp();
     }
     return kept;
 }
 
-// rows of  Dst = Src L^-T  (forward substitution, one thread per row; Dst may be Src)
+// rows of  Dst = Src L^-T  (forward substitution, one thread per row, 8 columns at a time in registers; Dst may be Src)
 template <int RP>
-__device__ __forceinline__ void pw_solve_forward(const double *Src, double *Dst, const double *L, const double *inv, int row)
+__device__ __noinline__ void pw_solve_forward(const double *Src, double *Dst, const double *L, const double *inv, int row)
 {
     constexpr int LDG = PowerLayout<RP>::LDG;
-    for (int j = 0; j < RP; ++j) {
-        const double *lj = L + j * LDG;
-        double s0 = Src[j * LDC + row], s1 = 0.0;
-        int k = 0;
-        for (; k + 1 < j; k += 2) { s0 = fma(-Dst[k * LDC + row], lj[k], s0); s1 = fma(-Dst[(k + 1) * LDC + row], lj[k + 1], s1); }
-        if (k < j) s0 = fma(-Dst[k * LDC + row], lj[k], s0);
-        Dst[j * LDC + row] = (s0 + s1) * inv[j];
+#pragma unroll 1
+    for (int jb = 0; jb < RP; jb += 8) {
+        double y[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) y[c] = Src[(jb + c) * LDC + row];
+#pragma unroll 2
+        for (int k = 0; k < jb; ++k) {
+            const double xk = Dst[k * LDC + row];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) y[c] = fma(-xk, L[(jb + c) * LDG + k], y[c]);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const double x = y[j] * inv[jb + j];
+            y[j] = x;
+#pragma unroll
+            for (int c = j + 1; c < 8; ++c) y[c] = fma(-x, L[(jb + c) * LDG + jb + j], y[c]);
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c) Dst[(jb + c) * LDC + row] = y[c];
     }
 }
 
-// rows of  Dst <- Dst L^-1  (backward substitution, in place)
+// rows of  Dst <- Dst L^-1  (backward substitution, in place, same blocking)
 template <int RP>
-__device__ __forceinline__ void pw_solve_backward(double *Dst, const double *L, const double *inv, int row)
+__device__ __noinline__ void pw_solve_backward(double *Dst, const double *L, const double *inv, int row)
 {
     constexpr int LDG = PowerLayout<RP>::LDG;
-    for (int j = RP - 1; j >= 0; --j) {
-        double s0 = Dst[j * LDC + row], s1 = 0.0;
-        int k = j + 1;
-        for (; k + 1 < RP; k += 2) { s0 = fma(-Dst[k * LDC + row], L[k * LDG + j], s0); s1 = fma(-Dst[(k + 1) * LDC + row], L[(k + 1) * LDG + j], s1); }
-        if (k < RP) s0 = fma(-Dst[k * LDC + row], L[k * LDG + j], s0);
-        Dst[j * LDC + row] = (s0 + s1) * inv[j];
+#pragma unroll 1
+    for (int jb = RP - 8; jb >= 0; jb -= 8) {
+        double y[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) y[c] = Dst[(jb + c) * LDC + row];
+#pragma unroll 2
+        for (int k = jb + 8; k < RP; ++k) {                         // the later columns, already solved
+            const double xk = Dst[k * LDC + row];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) y[c] = fma(-xk, L[k * LDG + jb + c], y[c]);
+        }
+#pragma unroll
+        for (int j = 7; j >= 0; --j) {
+            const double x = y[j] * inv[jb + j];
+            y[j] = x;
+#pragma unroll
+            for (int c = 0; c < j; ++c) y[c] = fma(-x, L[(jb + j) * LDG + jb + c], y[c]);
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c) Dst[(jb + c) * LDC + row] = y[c];
     }
 }
 
@@ -174,9 +249,17 @@ __global__ void __launch_bounds__(PW_THREADS, 1) power_kernel(
     double *Bf = A + RP * LDC;                  // [RP][LDC]
     double *G = Bf + RP * LDC;                  // [RP][LDG]
     double *inv = G + RP * LDG;                 // [RP]
-    int *kept_sm = reinterpret_cast<int *>(inv + 2 * RP);
+    int *kept_sm = reinterpret_cast<int *>(inv + RP);
     const int h = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+    constexpr bool MS = PowerLayout<RP>::M_SHARED;
     const double *M = gram + (size_t)h * D * D;
+    const double *Mu = M;                       // what the multiplications read
+    if (MS) {
+        double *Msm = psm + PowerLayout<RP>::small;
+        for (int idx = tid; idx < D * D / 2; idx += PW_THREADS)
+            reinterpret_cast<double2 *>(Msm)[idx] = __ldg(reinterpret_cast<const double2 *>(M) + idx);
+        Mu = Msm;
+    }
     const double *X0 = start + (size_t)h * start_stride_h;
 
     for (int idx = tid; idx < RP * D; idx += PW_THREADS) {
@@ -189,7 +272,7 @@ __global__ void __launch_bounds__(PW_THREADS, 1) power_kernel(
     for (int it = (iters == 0 ? -1 : 0); it <= iters; ++it) {
         double *T;                              // what gets orthonormalised in this pass
         if (it >= 0 && it < iters) {
-            pw_mult<RP>(M, X, Y, tid);
+            pw_mult<RP, MS>(Mu, X, Y, tid);
             __syncthreads();
             T = Y;
         } else {
@@ -208,7 +291,7 @@ __global__ void __launch_bounds__(PW_THREADS, 1) power_kernel(
     }
     if (tid == 0) kept_out[h] = *kept_sm;
     // B = X^T (M X),  N = I + lambda B = L L^T,  Z = X - X N^-1
-    pw_mult<RP>(M, X, Y, tid);
+    pw_mult<RP, MS>(Mu, X, Y, tid);
     __syncthreads();
     pw_gram<RP>(X, Y, G, lambda, 1.0, tid);
     __syncthreads();
