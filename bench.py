@@ -400,7 +400,7 @@ def run_gpu(args, cfg):
 
     # ---- end to end from host buffers through squat_write_path_host --------------------------------
     e2e = None
-    if not args.no_e2e and not args.meta16 and not use_power:   # the host-buffer entry: float32 metadata, SVD build
+    if not args.no_e2e:
         e2e = run_e2e(args, cfg, sq, s, (q_np, k_np, v_np), (kc, ks, kz, vc, vs, vz), to_dev, flush, tdt, dev,
                       vec_per_step)
     # ---- the reader that follows the write path (not part of a step): one decode step of attention -----
@@ -427,19 +427,25 @@ def run_e2e(args, cfg, sq, s, host_np, dev_outs, to_dev, flush, tdt, dev, vec_pe
     h2d = sum(t.numel() * t.element_size() for t in (qh, kh, vh))
     d2h = sum(t.numel() * t.element_size() for t in outs_h)
     e2e_steps = max(3, min(args.steps, 10))
+    # the same entry serves the variants: float16 metadata tensors -> 16-bit cache; a start block -> block power build
+    x0h = None
+    if args.subspace == "power":
+        x0h = torch.from_numpy(si.gen_start_block(cfg.seed, d, cfg.rank_r)).pin_memory()
+    kw = {"start_block": x0h, "power_iters": args.power_iters}
     for _ in range(2):
-        sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws)
+        sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws, **kw)
     e2e_ms = []
     for _ in range(e2e_steps):
         flush.zero_()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws)
+        sq.squat_write_path_host(s, qh, kh, vh, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *outs_h, ws, **kw)
         e2e_ms.append(1e3 * (time.perf_counter() - t0))        # the call synchronises its stream
     e2e_total_ms, e2e_units = aggregate_over_ranks(sum(e2e_ms), vec_per_step * e2e_steps, dev)
     return {"value": e2e_units / (e2e_total_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total_ms / e2e_steps,
-            "api": "squat_write_path_host (pinned host buffers; build + keys + values)"}
+            "api": "squat_write_path_host%s (pinned host buffers; build + keys + values)"
+                   % ("_ex" if (args.meta16 or args.subspace == "power") else "")}
 
 
 def run_reader(cfg, sq, cache, flush, tdt, dev, iters=10, meta_bytes=4):

@@ -218,6 +218,23 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same with the two variants of the write path selectable:
+ *   meta16             1: scales and zero-points are stored and copied back as IEEE binary16 (the host metadata
+ *                      buffers then hold 2-byte elements; semantics of the _m16 quantizers), 0: float32.
+ *   start_block_host   NULL: step 1 by the SVD (squat_build_subspace).  Otherwise host float64 [d, rank_r]
+ *                      row-major, one block for all heads: step 1 by the block power method
+ *                      (squat_build_subspace_power, rank_r <= 64) with power_iters multiplications.
+ * Everything else as squat_write_path_host; the workspace size is the same function's.
+ */
+int squat_write_path_host_ex(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
+                             int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
+                             int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
+                             unsigned char *k_codes_host, void *k_scales_host, void *k_zeros_host,
+                             unsigned char *v_codes_host, void *v_scales_host, void *v_zeros_host,
+                             int meta16, const double *start_block_host, int power_iters,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Reader of the cache -- one decode step of attention over the packed cache (Section 2, "(Masked) Attention
  * mechanism": softmax(q K^T / sqrt(d)) V for the newest token; the score vector w^deq of the proof of
  * Theorem 1; the most recent tokens come from the full-precision residual buffer of Algorithm 1).  This is

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
-    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
+    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_write_path_host_ex", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
 )
 
 _lib = None
@@ -62,6 +62,8 @@ def _load():
         lib.squat_write_path_workspace_bytes.restype = c.c_size_t
         lib.squat_write_path_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, dbl, i, i, i,
                                               vp, vp, vp, vp, vp, vp, vp, c.c_size_t, vp]
+        lib.squat_write_path_host_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, dbl, i, i, i,
+                                                 vp, vp, vp, vp, vp, vp, i, vp, i, vp, c.c_size_t, vp]
         lib.squat_gram_static.argtypes = [vp, i, i, i, i, i, ll, ll, vp, vp]
         lib.squat_decode_attention_workspace_bytes.argtypes = [i, i, i]
         lib.squat_decode_attention_workspace_bytes.restype = c.c_size_t
@@ -242,19 +244,40 @@ def squat_write_path_workspace_bytes(dtype: torch.dtype, batch, n_q_heads, n_kv_
 
 
 def squat_write_path_host(s: Subspace, q, k, v, rank_r, lam, block_g, bits, group_size, k_codes, k_scales, k_zeros,
-                          v_codes, v_scales, v_zeros, workspace: torch.Tensor, stream=None):
-    """q, k, v and the six outputs are HOST tensors (pinned for speed); workspace is a CUDA uint8 tensor."""
+                          v_codes, v_scales, v_zeros, workspace: torch.Tensor, stream=None, start_block=None,
+                          power_iters: int = 2):
+    """q, k, v and the six outputs are HOST tensors (pinned for speed); workspace is a CUDA uint8 tensor.  float16
+    scale / zero tensors select the 16-bit metadata variant (all four of them then); a HOST float64 start_block
+    [d, rank_r] selects step 1 by the block power method with power_iters multiplications."""
     for name, t in (("q", q), ("k", k), ("v", v), ("k_codes", k_codes), ("k_scales", k_scales), ("k_zeros", k_zeros),
                     ("v_codes", v_codes), ("v_scales", v_scales), ("v_zeros", v_zeros)):
         if t.is_cuda or not t.is_contiguous():
             raise ValueError(f"{name} must be a contiguous host tensor")
     B, H, T, d = k.shape
     hp = lambda t: ctypes.c_void_p(t.data_ptr())
-    _check(_load().squat_write_path_host(s.handle, hp(q), hp(k), hp(v), _dtype_code(k), B, q.shape[0], H, T, d, rank_r,
-                                         float(lam), block_g, bits, group_size, hp(k_codes), hp(k_scales), hp(k_zeros),
-                                         hp(v_codes), hp(v_scales), hp(v_zeros), _dev(workspace, "workspace"),
-                                         workspace.numel() * workspace.element_size(), _stream(stream)),
-           "squat_write_path_host")
+    meta = (k_scales, k_zeros, v_scales, v_zeros)
+    m16 = all(t.dtype == torch.float16 for t in meta)
+    if not m16 and not all(t.dtype == torch.float32 for t in meta):
+        raise ValueError("scales and zero-points must be all float32 or all float16")
+    if not m16 and start_block is None:
+        _check(_load().squat_write_path_host(s.handle, hp(q), hp(k), hp(v), _dtype_code(k), B, q.shape[0], H, T, d, rank_r,
+                                             float(lam), block_g, bits, group_size, hp(k_codes), hp(k_scales), hp(k_zeros),
+                                             hp(v_codes), hp(v_scales), hp(v_zeros), _dev(workspace, "workspace"),
+                                             workspace.numel() * workspace.element_size(), _stream(stream)),
+               "squat_write_path_host")
+        return
+    x0 = None
+    if start_block is not None:
+        if start_block.is_cuda or start_block.dtype != torch.float64 or not start_block.is_contiguous() or \
+                tuple(start_block.shape) != (d, rank_r):
+            raise ValueError("start_block must be a contiguous host float64 tensor [d, rank_r]")
+        x0 = hp(start_block)
+    _check(_load().squat_write_path_host_ex(s.handle, hp(q), hp(k), hp(v), _dtype_code(k), B, q.shape[0], H, T, d, rank_r,
+                                            float(lam), block_g, bits, group_size, hp(k_codes), hp(k_scales), hp(k_zeros),
+                                            hp(v_codes), hp(v_scales), hp(v_zeros), int(m16), x0, int(power_iters),
+                                            _dev(workspace, "workspace"),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)),
+           "squat_write_path_host_ex")
 
 
 def squat_gram_static(q: torch.Tensor, n_kv_heads: int, gram_out: torch.Tensor, stream=None):

@@ -511,7 +511,7 @@ int squat_get_device_status(void *stream, unsigned *flags, int clear)
 // Whole write path from host buffers.
 namespace {
 struct HostPathLayout {
-    size_t q, k, v, kc, ks, kz, vc, vs, vz, total;
+    size_t q, k, v, kc, ks, kz, vc, vs, vz, x0, total;
 };
 HostPathLayout host_layout(int dtype, int batch, int n_q, int H, int T, int d, int bits, int G)
 {
@@ -529,6 +529,7 @@ HostPathLayout host_layout(int dtype, int batch, int n_q, int H, int T, int d, i
     L.vc = carve(toks * d * bits / 8);
     L.vs = carve(toks * (d / G) * sizeof(float));
     L.vz = carve(toks * (d / G) * sizeof(float));
+    L.x0 = carve((size_t)D * 64 * sizeof(double));     // start block of the block power build (rank <= 64)
     L.total = off;
     return L;
 }
@@ -543,12 +544,16 @@ size_t squat_write_path_workspace_bytes(int dtype, int batch, int n_q_heads, int
     return host_layout(dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, bits, group_size).total;
 }
 
-int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
-                          int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
-                          int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
-                          unsigned char *k_codes_host, float *k_scales_host, float *k_zeros_host,
-                          unsigned char *v_codes_host, float *v_scales_host, float *v_zeros_host,
-                          void *workspace, size_t workspace_bytes, void *stream)
+}  // extern "C"
+
+namespace {
+int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
+                         int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
+                         int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
+                         unsigned char *k_codes_host, void *k_scales_host, void *k_zeros_host,
+                         unsigned char *v_codes_host, void *v_scales_host, void *v_zeros_host,
+                         int meta16, const double *start_block_host, int power_iters,
+                         void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!s || !q_host || !k_host || !v_host || !k_codes_host || !k_scales_host || !k_zeros_host || !v_codes_host ||
         !v_scales_host || !v_zeros_host || !workspace || !valid_dtype(dtype))
@@ -565,6 +570,8 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
     const size_t es = elem_size(dtype);
     const size_t toks = (size_t)batch * n_kv_heads * n_tokens;
     const long long T = n_tokens, d = head_dim;
+    const size_t ms = meta16 ? 2 : sizeof(float);          // bytes per stored scale / zero-point
+    if (start_block_host && (rank_r < 0 || rank_r > 64)) return rank_r < 0 ? SQUAT_ERR_INVALID_ARG : SQUAT_ERR_UNSUPPORTED;
     // Copies and kernels overlap: q goes up first (the subspace build needs it), k and v follow on a side stream
     // while the build runs; the key outputs go down on a second side stream while v is still coming up and the
     // values are quantized.  Everything is ordered after the work already in `stream` and joined back into it.
@@ -575,38 +582,71 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
     }
     cudaEvent_t ev_q = s->ev[0], ev_k = s->ev[1], ev_v = s->ev[2], ev_keys = s->ev[3], ev_kout = s->ev[4];
     SQUAT_CUDA(cudaMemcpyAsync(w + L.q, q_host, (size_t)n_q_heads * T * d * es, cudaMemcpyHostToDevice, st));
+    if (start_block_host && rank_r > 0)
+        SQUAT_CUDA(cudaMemcpyAsync(w + L.x0, start_block_host, (size_t)D * rank_r * sizeof(double), cudaMemcpyHostToDevice, st));
     SQUAT_CUDA(cudaEventRecord(ev_q, st));
     SQUAT_CUDA(cudaStreamWaitEvent(s->side[0], ev_q, 0));
     SQUAT_CUDA(cudaMemcpyAsync(w + L.k, k_host, toks * d * es, cudaMemcpyHostToDevice, s->side[0]));
     SQUAT_CUDA(cudaEventRecord(ev_k, s->side[0]));
     SQUAT_CUDA(cudaMemcpyAsync(w + L.v, v_host, toks * d * es, cudaMemcpyHostToDevice, s->side[0]));
     SQUAT_CUDA(cudaEventRecord(ev_v, s->side[0]));
-    int rc = squat_build_subspace(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g, stream);
+    int rc = start_block_host
+                 ? squat_build_subspace_power(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g,
+                                              reinterpret_cast<const double *>(w + L.x0), 0, power_iters, stream)
+                 : squat_build_subspace(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g, stream);
     if (rc != SQUAT_OK) return rc;
     SQUAT_CUDA(cudaStreamWaitEvent(st, ev_k, 0));
-    rc = squat_quantize_keys(s, w + L.k, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
-                             T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.kc),
-                             reinterpret_cast<float *>(w + L.ks), reinterpret_cast<float *>(w + L.kz),
-                             (long long)n_kv_heads * T, T, stream);
+    rc = quantize_keys_impl(s, w + L.k, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
+                            T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.kc),
+                            w + L.ks, w + L.kz, (long long)n_kv_heads * T, T, meta16, stream);
     if (rc != SQUAT_OK) return rc;
     SQUAT_CUDA(cudaEventRecord(ev_keys, st));
     SQUAT_CUDA(cudaStreamWaitEvent(s->side[1], ev_keys, 0));
     SQUAT_CUDA(cudaMemcpyAsync(k_codes_host, w + L.kc, toks * d * bits / 8, cudaMemcpyDeviceToHost, s->side[1]));
-    SQUAT_CUDA(cudaMemcpyAsync(k_scales_host, w + L.ks, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, s->side[1]));
-    SQUAT_CUDA(cudaMemcpyAsync(k_zeros_host, w + L.kz, toks / group_size * d * sizeof(float), cudaMemcpyDeviceToHost, s->side[1]));
+    SQUAT_CUDA(cudaMemcpyAsync(k_scales_host, w + L.ks, toks / group_size * d * ms, cudaMemcpyDeviceToHost, s->side[1]));
+    SQUAT_CUDA(cudaMemcpyAsync(k_zeros_host, w + L.kz, toks / group_size * d * ms, cudaMemcpyDeviceToHost, s->side[1]));
     SQUAT_CUDA(cudaEventRecord(ev_kout, s->side[1]));
     SQUAT_CUDA(cudaStreamWaitEvent(st, ev_v, 0));
-    rc = squat_quantize_values(w + L.v, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
-                               T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.vc),
-                               reinterpret_cast<float *>(w + L.vs), reinterpret_cast<float *>(w + L.vz),
-                               (long long)n_kv_heads * T, T, stream);
+    rc = quantize_values_impl(w + L.v, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
+                              T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.vc),
+                              w + L.vs, w + L.vz, (long long)n_kv_heads * T, T, meta16, stream);
     if (rc != SQUAT_OK) return rc;
     SQUAT_CUDA(cudaMemcpyAsync(v_codes_host, w + L.vc, toks * d * bits / 8, cudaMemcpyDeviceToHost, st));
-    SQUAT_CUDA(cudaMemcpyAsync(v_scales_host, w + L.vs, toks * (d / group_size) * sizeof(float), cudaMemcpyDeviceToHost, st));
-    SQUAT_CUDA(cudaMemcpyAsync(v_zeros_host, w + L.vz, toks * (d / group_size) * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(v_scales_host, w + L.vs, toks * (d / group_size) * ms, cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(v_zeros_host, w + L.vz, toks * (d / group_size) * ms, cudaMemcpyDeviceToHost, st));
     SQUAT_CUDA(cudaStreamWaitEvent(st, ev_kout, 0));
     SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
+                          int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
+                          int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
+                          unsigned char *k_codes_host, float *k_scales_host, float *k_zeros_host,
+                          unsigned char *v_codes_host, float *v_scales_host, float *v_zeros_host,
+                          void *workspace, size_t workspace_bytes, void *stream)
+{
+    return write_path_host_impl(s, q_host, k_host, v_host, dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, rank_r,
+                                lambda, block_g, bits, group_size, k_codes_host, k_scales_host, k_zeros_host, v_codes_host,
+                                v_scales_host, v_zeros_host, 0, nullptr, 0, workspace, workspace_bytes, stream);
+}
+
+int squat_write_path_host_ex(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
+                             int dtype, int batch, int n_q_heads, int n_kv_heads, int n_tokens,
+                             int head_dim, int rank_r, double lambda, int block_g, int bits, int group_size,
+                             unsigned char *k_codes_host, void *k_scales_host, void *k_zeros_host,
+                             unsigned char *v_codes_host, void *v_scales_host, void *v_zeros_host,
+                             int meta16, const double *start_block_host, int power_iters,
+                             void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (meta16 != 0 && meta16 != 1) return SQUAT_ERR_INVALID_ARG;
+    return write_path_host_impl(s, q_host, k_host, v_host, dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, rank_r,
+                                lambda, block_g, bits, group_size, k_codes_host, k_scales_host, k_zeros_host, v_codes_host,
+                                v_scales_host, v_zeros_host, meta16, start_block_host, power_iters, workspace,
+                                workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -163,6 +163,43 @@ def test_host_buffer_entry_equals_device_calls():
         s2.close()
 
 
+def test_host_buffer_entry_variants_equal_device_calls():
+    # the same entry with 16-bit metadata and / or step 1 by the block power method: byte-identical to the device calls
+    cfg = si.get_config(1).with_(batch=2, n_kv_heads=4, n_q_heads=8, n_tokens=512)
+    B, H, T, bits, G = cfg.batch, cfg.n_kv_heads, cfg.n_tokens, cfg.bits, cfg.group_size
+    q_np, k_np, v_np = si.gen_queries(cfg), si.gen_keys(cfg), si.gen_values(cfg)
+    x0 = torch.from_numpy(si.gen_start_block(cfg.seed, D, cfg.rank_r))
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    ws = torch.empty(sq.squat_write_path_workspace_bytes(tdt, B, cfg.n_q_heads, H, T, D, bits, G), dtype=torch.uint8,
+                     device="cuda")
+    host_in = [to_torch(a, cfg.dtype, device="cpu").pin_memory() for a in (q_np, k_np, v_np)]
+    for m16 in (False, True):
+        for power in (False, True):
+            if not m16 and not power:
+                continue                                            # the plain entry: covered above
+            s = sq.Subspace(H, D)
+            if power:
+                sq.squat_build_subspace_power(s, to_torch(q_np, cfg.dtype), cfg.rank_r, cfg.lam, x0.cuda(), 2, cfg.block_g)
+            else:
+                sq.squat_build_subspace(s, to_torch(q_np, cfg.dtype), cfg.rank_r, cfg.lam, cfg.block_g)
+            kc, ks, kz = alloc_key_outputs(B, H, T, D, bits, G)
+            vc, vs, vz = alloc_value_outputs(B, H, T, D, bits, G)
+            if m16:
+                ks, kz, vs, vz = (t.to(torch.float16) for t in (ks, kz, vs, vz))
+            sq.squat_quantize_keys(s, to_torch(k_np, cfg.dtype), bits, G, kc, ks, kz)
+            sq.squat_quantize_values(to_torch(v_np, cfg.dtype), bits, G, vc, vs, vz)
+            torch.cuda.synchronize()
+            host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in (kc, ks, kz, vc, vs, vz)]
+            s2 = sq.Subspace(H, D)
+            sq.squat_write_path_host(s2, *host_in, cfg.rank_r, cfg.lam, cfg.block_g, bits, G, *host_out, ws,
+                                     start_block=x0 if power else None, power_iters=2)
+            for dev_t, host_t in zip((kc, ks, kz, vc, vs, vz), host_out):
+                assert torch.equal(dev_t.cpu(), host_t), (m16, power)
+            s.close()
+            s2.close()
+    sq.squat_get_device_status(clear=True)
+
+
 def test_write_path_captures_into_a_cuda_graph_and_replays_identically():
     # no call of the write path allocates, synchronises or touches the host: the whole step records into a CUDA graph
     cfg = si.get_config(0)
