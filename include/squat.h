@@ -115,6 +115,15 @@ int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int 
                                long long stride_h, long long stride_t, int rank_r, double lambda, int block_g,
                                const double *start_block, long long start_stride_h, int iters, void *stream);
 
+/*
+ * squat_build_subspace_power from Gram matrices the caller already has -- the block power method for a prompt whose
+ * tokens are spread over several GPUs: Gram matrices of the local tokens (squat_gram_static), one all-reduce, then
+ * this call on every rank with the same start block.  gram as for squat_build_subspace_from_gram, the other
+ * arguments as for squat_build_subspace_power.
+ */
+int squat_build_subspace_power_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
+                                         const double *start_block, long long start_stride_h, int iters, void *stream);
+
 /* Test / checkpoint hooks.  Both synchronise `stream`.  Host pointers; any may be NULL.
  *   W_host      [n_kv_heads, d, d] float32, row j' column j, block strictly lower triangular.
  *   gram_host   [n_kv_heads, d, d] float64 Gram matrices of the last build.

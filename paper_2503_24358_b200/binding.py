@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "squat_kernel_launch_count", "squat_status_string", "squat_last_cuda_error", "squat_gram_static",
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
-    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_write_path_host_ex", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
+    "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_write_path_host_ex", "squat_build_subspace_power_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
 )
 
 _lib = None
@@ -74,6 +74,7 @@ def _load():
         lib.squat_dequantize_m16.argtypes = lib.squat_dequantize.argtypes
         lib.squat_build_subspace_from_gram.argtypes = [vp, vp, i, dbl, i, vp]
         lib.squat_build_subspace_power.argtypes = [vp, vp, i, i, i, ll, ll, i, dbl, i, vp, ll, i, vp]
+        lib.squat_build_subspace_power_from_gram.argtypes = [vp, vp, i, dbl, i, vp, ll, i, vp]
         lib.squat_rope_table_floats.argtypes = [i]
         lib.squat_rope_table_floats.restype = c.c_size_t
         lib.squat_rope_table_fill.argtypes = [dbl, i, i, vp]
@@ -308,15 +309,7 @@ def squat_build_subspace_power(s: "Subspace", q: torch.Tensor, rank_r: int, lam:
     heads) or [n_kv_heads, d, rank_r], float64, CUDA, contiguous; iters multiplications by the Gram matrix."""
     if q.dim() != 3 or q.stride(2) != 1 or q.shape[2] != s.head_dim:
         raise ValueError("q must be [n_q_heads, n_tokens, head_dim] with contiguous last dim")
-    if start_block.dtype != torch.float64 or not start_block.is_contiguous():
-        raise ValueError("start_block must be a contiguous float64 tensor")
-    if tuple(start_block.shape) == (s.head_dim, rank_r):
-        stride_h = 0
-    elif tuple(start_block.shape) == (s.n_kv_heads, s.head_dim, rank_r):
-        stride_h = s.head_dim * rank_r
-    else:
-        raise ValueError("start_block must be [d, rank_r] or [n_kv_heads, d, rank_r]")
-    ptr = _dev(start_block, "start_block") if rank_r > 0 else None
+    ptr, stride_h = _start_block_args(s, start_block, rank_r)
     _check(_load().squat_build_subspace_power(s.handle, _dev(q, "q"), _dtype_code(q), q.shape[0], q.shape[1],
                                               q.stride(0), q.stride(1), int(rank_r), ctypes.c_double(lam), int(block_g),
                                               ptr, stride_h, int(iters), _stream(stream)),
@@ -335,12 +328,38 @@ def token_shard(n_tokens: int, rank: int, world: int, multiple: int = 32):
     return lo * multiple, hi * multiple
 
 
+def _start_block_args(s: "Subspace", start_block: torch.Tensor, rank_r: int):
+    if start_block.dtype != torch.float64 or not start_block.is_contiguous():
+        raise ValueError("start_block must be a contiguous float64 tensor")
+    if tuple(start_block.shape) == (s.head_dim, rank_r):
+        stride_h = 0
+    elif tuple(start_block.shape) == (s.n_kv_heads, s.head_dim, rank_r):
+        stride_h = s.head_dim * rank_r
+    else:
+        raise ValueError("start_block must be [d, rank_r] or [n_kv_heads, d, rank_r]")
+    return (_dev(start_block, "start_block") if rank_r > 0 else None), stride_h
+
+
+def squat_build_subspace_power_from_gram(s: "Subspace", gram: torch.Tensor, rank_r: int, lam: float,
+                                         start_block: torch.Tensor, iters: int = 2, block_g: int = 1, stream=None):
+    """The block power build from Gram matrices [n_kv_heads, d, d] (float64, CUDA) the caller has summed over the
+    prompt's tokens; start_block as for squat_build_subspace_power."""
+    if gram.dtype != torch.float64 or not gram.is_contiguous():
+        raise ValueError("gram must be a contiguous float64 tensor")
+    ptr, stride_h = _start_block_args(s, start_block, rank_r)
+    _check(_load().squat_build_subspace_power_from_gram(s.handle, _dev(gram, "gram"), int(rank_r), ctypes.c_double(lam),
+                                                        int(block_g), ptr, stride_h, int(iters), _stream(stream)),
+           "squat_build_subspace_power_from_gram")
+
+
 def squat_build_subspace_sharded(s: "Subspace", q_local: torch.Tensor, rank_r: int, lam: float, block_g: int = 1,
-                                 gram_buf: torch.Tensor = None, group=None, stream=None):
+                                 gram_buf: torch.Tensor = None, group=None, stream=None, start_block: torch.Tensor = None,
+                                 power_iters: int = 2):
     """Step 1 for a prompt whose tokens are spread over the ranks of a torch.distributed group: Gram matrices of
     the local tokens (q_local [n_q_heads, local_tokens, d]; a rank may hold none), one all-reduce (sum) of
-    n_kv_heads * d * d float64, then the eigen-decomposition and the update matrices on every rank.  Without an
-    initialised process group this is the single-GPU build through the same two calls."""
+    n_kv_heads * d * d float64, then the eigen-decomposition (or, with a start_block every rank passes alike, the
+    block power iteration) and the update matrices on every rank.  Without an initialised process group this is the
+    single-GPU build through the same two calls."""
     import torch.distributed as dist
     H = s.n_kv_heads
     if gram_buf is None:
@@ -351,7 +370,10 @@ def squat_build_subspace_sharded(s: "Subspace", q_local: torch.Tensor, rank_r: i
         gram_buf.zero_()
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
-    squat_build_subspace_from_gram(s, gram_buf, rank_r, lam, block_g, stream)
+    if start_block is not None:
+        squat_build_subspace_power_from_gram(s, gram_buf, rank_r, lam, start_block, power_iters, block_g, stream)
+    else:
+        squat_build_subspace_from_gram(s, gram_buf, rank_r, lam, block_g, stream)
     return gram_buf
 
 

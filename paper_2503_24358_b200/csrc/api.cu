@@ -206,6 +206,28 @@ int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int 
     return squat_launch_assemble(s, rank_r, lambda, block_g, 64, st);
 }
 
+int squat_build_subspace_power_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
+                                         const double *start_block, long long start_stride_h, int iters, void *stream)
+{
+    if (!s || !gram || !aligned16(gram)) return SQUAT_ERR_INVALID_ARG;
+    if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
+    if (rank_r > 64) return SQUAT_ERR_UNSUPPORTED;
+    if (!(lambda >= 0.0) || !std::isfinite(lambda)) return SQUAT_ERR_INVALID_ARG;
+    if (block_g <= 0 || D % block_g != 0) return SQUAT_ERR_SHAPE;
+    if (iters < 0 || iters > 64 || start_stride_h < 0) return SQUAT_ERR_INVALID_ARG;
+    if (rank_r > 0 && (!start_block || ((uintptr_t)start_block & 7u))) return SQUAT_ERR_INVALID_ARG;
+    if (start_stride_h != 0 && start_stride_h < (long long)D * rank_r) return SQUAT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (gram != s->gram)
+        SQUAT_CUDA(cudaMemcpyAsync(s->gram, gram, (size_t)s->n_kv_heads * D * D * sizeof(double), cudaMemcpyDeviceToDevice, st));
+    const bool no_update = rank_r == 0 || lambda == 0.0;
+    s->exact_blocks = no_update ? D / 32 : (block_g + 31) / 32;
+    if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, st);
+    int rc = squat_launch_power(s, start_block, start_stride_h, rank_r, iters, lambda, st);
+    if (rc != SQUAT_OK) return rc;
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 64, st);
+}
+
 int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,
                           double *eigval_host, double *eigvec_host)
 {

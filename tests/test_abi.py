@@ -62,6 +62,7 @@ def test_argument_errors_come_back_as_status_codes(lib):
     assert lib.squat_dequantize(0, a, a, a, 1, 1, 33, 128, 2, 32, 0, 0, a, 0, None) == 2               # T % G for keys
     assert lib.squat_dequantize(1, a, a, a, 1, 1, 33, 128, 8, 32, 0, 0, a, 0, None) == 3
     assert lib.squat_build_subspace_power(None, a, 0, 8, 32, 4096, 128, 8, 1e-3, 1, a, 0, 2, None) == 1
+    assert lib.squat_build_subspace_power_from_gram(None, a, 8, 1e-3, 1, a, 0, 2, None) == 1
     assert lib.squat_get_device_status(None, None, 0) == 1
     assert lib.squat_write_path_workspace_bytes(1, 1, 32, 32, 4096, 128, 2, 32) > 2 * 32 * 4096 * 128 * 2
 

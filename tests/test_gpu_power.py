@@ -151,3 +151,35 @@ def test_power_build_feeds_the_key_kernel():
                          None, m["Qhat"])
     assert sq.squat_get_device_status(clear=True) == 0
     s.close()
+
+
+def test_power_build_from_summed_gram_matrices_of_token_shards_equals_the_power_build_on_all_tokens():
+    # the multi-GPU layout of step 1 with the power method: Gram matrices of three token ranges summed (one all-reduce
+    # between real ranks), then squat_build_subspace_power_from_gram with the start block every rank holds
+    cfg = si.get_config(0)
+    H, T = cfg.n_kv_heads, cfg.n_tokens
+    q = to_torch(si.gen_queries(cfg), cfg.dtype)
+    X0 = torch.from_numpy(si.gen_start_block(cfg.seed, D, cfg.rank_r)).cuda()
+    full = sq.Subspace(H, D)
+    sq.squat_build_subspace_power(full, q, cfg.rank_r, cfg.lam, X0, 2, cfg.block_g)
+    W_full = sq.squat_subspace_export(full, ("W",))["W"]
+    total = torch.zeros((H, D, D), dtype=torch.float64, device="cuda")
+    part = torch.empty_like(total)
+    for r in range(3):
+        lo, hi = sq.token_shard(T, r, 3, cfg.group_size)
+        if hi > lo:
+            sq.squat_gram_static(q[:, lo:hi, :], H, part)
+            total += part
+    sharded = sq.Subspace(H, D)
+    sq.squat_build_subspace_power_from_gram(sharded, total, cfg.rank_r, cfg.lam, X0, 2, cfg.block_g)
+    W_sh = sq.squat_subspace_export(sharded, ("W",))["W"]
+    assert np.abs(W_sh - W_full).max() <= 1e-7
+    helper = sq.Subspace(H, D)
+    sq.squat_build_subspace_sharded(helper, q, cfg.rank_r, cfg.lam, cfg.block_g, start_block=X0, power_iters=2)
+    W_h = sq.squat_subspace_export(helper, ("W",))["W"]
+    assert np.abs(W_h - W_full).max() <= 1e-7
+    for h in (0, H - 1):
+        m = _oracle_W(cfg, h, X0.cpu().numpy(), 2)
+        assert _w_err(W_sh[h], m["W"]) <= W_TOL
+    for s in (full, sharded, helper):
+        s.close()
