@@ -183,3 +183,23 @@ def test_power_build_from_summed_gram_matrices_of_token_shards_equals_the_power_
         assert _w_err(W_sh[h], m["W"]) <= W_TOL
     for s in (full, sharded, helper):
         s.close()
+
+
+@pytest.mark.parametrize("shift", [-40, 40])
+def test_power_build_is_invariant_under_a_power_of_two_scaling_of_the_queries(shift):
+    # q -> 2^k q makes M -> 4^k M; with lambda -> 4^-k lambda P is unchanged, and since powers of two commute with
+    # every rounding the whole computation is: W must come out bit for bit the same (exercises the exponent handling
+    # of the reciprocal square roots and the relative drop threshold far from 1)
+    cfg = si.get_config(0)
+    q = to_torch(si.gen_queries(cfg), cfg.dtype).to(torch.float32)
+    X0 = torch.from_numpy(si.gen_start_block(cfg.seed, D, cfg.rank_r)).cuda()
+    a = sq.Subspace(cfg.n_kv_heads, D)
+    sq.squat_build_subspace_power(a, q, cfg.rank_r, cfg.lam, X0, 2, 1)
+    W_a = sq.squat_subspace_export(a, ("W",))["W"]
+    b = sq.Subspace(cfg.n_kv_heads, D)
+    sq.squat_build_subspace_power(b, q * (2.0 ** shift), cfg.rank_r, cfg.lam * 4.0 ** (-shift), X0, 2, 1)
+    W_b = sq.squat_subspace_export(b, ("W",))["W"]
+    assert np.array_equal(W_a, W_b)
+    assert list(sq.squat_subspace_eig_sweeps(b)) == [cfg.rank_r] * cfg.n_kv_heads
+    a.close()
+    b.close()
