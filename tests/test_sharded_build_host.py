@@ -46,6 +46,11 @@ def _worker(rank, world, port, out):
         g = torch.from_numpy(np.stack(grams))
         dist.all_reduce(g, op=dist.ReduceOp.SUM)              # the path's one exchange step
         out[rank] = g.numpy().copy()
+        # step 1 by the block power method on the summed matrices: every rank draws the same start block from the
+        # workload's seed, so every rank ends with the same update matrix
+        X0 = si.gen_start_block(cfg.seed, cfg.head_dim, cfg.rank_r)
+        Qhat, _, _ = oracle.power_subspace(g[0].numpy(), X0, 2)
+        out[("W", rank)] = oracle.update_matrices(Qhat, cfg.head_dim, cfg.lam)["W"]
         dist.barrier()
     finally:
         dist.destroy_process_group()
@@ -61,3 +66,8 @@ def test_gram_matrices_of_token_shards_add_up_gloo_world_size_2():
         Q = si.to_f32(si.gen_queries_head(cfg, h, cfg.n_tokens), cfg.dtype).astype(np.float64)
         full = oracle.gram(Q)
         assert np.abs(out[0][h] - full).max() <= 1e-12 * np.abs(full).max()
+    # the power build on the all-reduced matrices: identical on both ranks, and equal to the single-process build
+    assert np.array_equal(out[("W", 0)], out[("W", 1)])
+    Q = si.to_f32(si.gen_queries_head(cfg, 0, cfg.n_tokens), cfg.dtype).astype(np.float64)
+    ref = oracle.build_W_power(Q, si.gen_start_block(cfg.seed, cfg.head_dim, cfg.rank_r), 2, cfg.lam)
+    assert np.abs(out[("W", 0)] - ref["W"]).max() <= 1e-9
