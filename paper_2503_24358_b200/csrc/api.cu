@@ -132,7 +132,7 @@ int squat_subspace_destroy(squat_subspace *s)
     if (!s) return SQUAT_OK;
     if (s->side_ready) {
         for (int i = 0; i < 2; ++i) cudaStreamDestroy(s->side[i]);
-        for (int i = 0; i < 5; ++i) cudaEventDestroy(s->ev[i]);
+        for (int i = 0; i < 8; ++i) cudaEventDestroy(s->ev[i]);
     }
     cudaError_t e = cudaFree(s->Wt);     // Wt is the base of the single allocation
     delete s;
@@ -595,14 +595,18 @@ int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_ho
     const size_t ms = meta16 ? 2 : sizeof(float);          // bytes per stored scale / zero-point
     if (start_block_host && (rank_r < 0 || rank_r > 64)) return rank_r < 0 ? SQUAT_ERR_INVALID_ARG : SQUAT_ERR_UNSUPPORTED;
     // Copies and kernels overlap: q goes up first (the subspace build needs it), k and v follow on a side stream
-    // while the build runs; the key outputs go down on a second side stream while v is still coming up and the
-    // values are quantized.  Everything is ordered after the work already in `stream` and joined back into it.
+    // while the build runs; the key outputs go down on a second side stream while v is still coming up.  v travels
+    // in up to four pieces ((batch, head) ranges): each is quantized and its outputs sent down as soon as it has
+    // arrived, so that only the last piece's kernel and download are left when the upload ends.  Everything is
+    // ordered after the work already in `stream` and joined back into it.
     if (!s->side_ready) {
         for (int i = 0; i < 2; ++i) SQUAT_CUDA(cudaStreamCreateWithFlags(&s->side[i], cudaStreamNonBlocking));
-        for (int i = 0; i < 5; ++i) SQUAT_CUDA(cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming));
+        for (int i = 0; i < 8; ++i) SQUAT_CUDA(cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming));
         s->side_ready = true;
     }
-    cudaEvent_t ev_q = s->ev[0], ev_k = s->ev[1], ev_v = s->ev[2], ev_keys = s->ev[3], ev_kout = s->ev[4];
+    cudaEvent_t ev_q = s->ev[0], ev_k = s->ev[1], ev_keys = s->ev[2], ev_kout = s->ev[3];
+    const long long rows = (long long)batch * n_kv_heads;          // (batch, head) units of T tokens
+    const int n_pieces = rows >= 4 ? 4 : (int)rows;
     SQUAT_CUDA(cudaMemcpyAsync(w + L.q, q_host, (size_t)n_q_heads * T * d * es, cudaMemcpyHostToDevice, st));
     if (start_block_host && rank_r > 0)
         SQUAT_CUDA(cudaMemcpyAsync(w + L.x0, start_block_host, (size_t)D * rank_r * sizeof(double), cudaMemcpyHostToDevice, st));
@@ -610,8 +614,12 @@ int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_ho
     SQUAT_CUDA(cudaStreamWaitEvent(s->side[0], ev_q, 0));
     SQUAT_CUDA(cudaMemcpyAsync(w + L.k, k_host, toks * d * es, cudaMemcpyHostToDevice, s->side[0]));
     SQUAT_CUDA(cudaEventRecord(ev_k, s->side[0]));
-    SQUAT_CUDA(cudaMemcpyAsync(w + L.v, v_host, toks * d * es, cudaMemcpyHostToDevice, s->side[0]));
-    SQUAT_CUDA(cudaEventRecord(ev_v, s->side[0]));
+    for (int p = 0; p < n_pieces; ++p) {
+        const long long r0 = rows * p / n_pieces, r1 = rows * (p + 1) / n_pieces;
+        SQUAT_CUDA(cudaMemcpyAsync(w + L.v + (size_t)r0 * T * d * es, static_cast<const char *>(v_host) + (size_t)r0 * T * d * es,
+                                   (size_t)(r1 - r0) * T * d * es, cudaMemcpyHostToDevice, s->side[0]));
+        SQUAT_CUDA(cudaEventRecord(s->ev[4 + p], s->side[0]));
+    }
     int rc = start_block_host
                  ? squat_build_subspace_power(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g,
                                               reinterpret_cast<const double *>(w + L.x0), 0, power_iters, stream)
@@ -628,14 +636,18 @@ int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_ho
     SQUAT_CUDA(cudaMemcpyAsync(k_scales_host, w + L.ks, toks / group_size * d * ms, cudaMemcpyDeviceToHost, s->side[1]));
     SQUAT_CUDA(cudaMemcpyAsync(k_zeros_host, w + L.kz, toks / group_size * d * ms, cudaMemcpyDeviceToHost, s->side[1]));
     SQUAT_CUDA(cudaEventRecord(ev_kout, s->side[1]));
-    SQUAT_CUDA(cudaStreamWaitEvent(st, ev_v, 0));
-    rc = quantize_values_impl(w + L.v, dtype, batch, n_kv_heads, n_tokens, head_dim, (long long)n_kv_heads * T * d,
-                              T * d, d, bits, group_size, reinterpret_cast<unsigned char *>(w + L.vc),
-                              w + L.vs, w + L.vz, (long long)n_kv_heads * T, T, meta16, stream);
-    if (rc != SQUAT_OK) return rc;
-    SQUAT_CUDA(cudaMemcpyAsync(v_codes_host, w + L.vc, toks * d * bits / 8, cudaMemcpyDeviceToHost, st));
-    SQUAT_CUDA(cudaMemcpyAsync(v_scales_host, w + L.vs, toks * (d / group_size) * ms, cudaMemcpyDeviceToHost, st));
-    SQUAT_CUDA(cudaMemcpyAsync(v_zeros_host, w + L.vz, toks * (d / group_size) * ms, cudaMemcpyDeviceToHost, st));
+    const size_t vrow_codes = (size_t)T * d * bits / 8, vrow_meta = (size_t)T * (d / group_size) * ms;
+    for (int p = 0; p < n_pieces; ++p) {
+        const long long r0 = rows * p / n_pieces, r1 = rows * (p + 1) / n_pieces;
+        SQUAT_CUDA(cudaStreamWaitEvent(st, s->ev[4 + p], 0));
+        rc = quantize_values_impl(w + L.v + (size_t)r0 * T * d * es, dtype, 1, (int)(r1 - r0), n_tokens, head_dim, 0, T * d, d,
+                                  bits, group_size, reinterpret_cast<unsigned char *>(w + L.vc) + r0 * vrow_codes,
+                                  w + L.vs + r0 * vrow_meta, w + L.vz + r0 * vrow_meta, 0, T, meta16, stream);
+        if (rc != SQUAT_OK) return rc;
+        SQUAT_CUDA(cudaMemcpyAsync(v_codes_host + r0 * vrow_codes, w + L.vc + r0 * vrow_codes, (r1 - r0) * vrow_codes, cudaMemcpyDeviceToHost, st));
+        SQUAT_CUDA(cudaMemcpyAsync(static_cast<char *>(v_scales_host) + r0 * vrow_meta, w + L.vs + r0 * vrow_meta, (r1 - r0) * vrow_meta, cudaMemcpyDeviceToHost, st));
+        SQUAT_CUDA(cudaMemcpyAsync(static_cast<char *>(v_zeros_host) + r0 * vrow_meta, w + L.vz + r0 * vrow_meta, (r1 - r0) * vrow_meta, cudaMemcpyDeviceToHost, st));
+    }
     SQUAT_CUDA(cudaStreamWaitEvent(st, ev_kout, 0));
     SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;

@@ -23,7 +23,7 @@ struct squat_subspace {
     unsigned *status;      // device status word of this device
     // host path only (created on its first call): two side streams and the events that order them
     cudaStream_t side[2];
-    cudaEvent_t ev[5];
+    cudaEvent_t ev[8];     // q up, k up, keys done, key outputs down, v chunks up (4)
     bool side_ready;
 };
 
