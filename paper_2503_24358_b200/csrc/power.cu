@@ -15,16 +15,20 @@
 // X becomes zero and contributes nothing from then on.  One pass of Cholesky QR needs cond(M restricted to the block)
 // well below 1e6.5; beyond that, directions are dropped and the count of kept columns (reported per head) says so.
 //
-// One CTA of 256 threads per head; X and Y are stored column by column with an odd stride, so that column dot products (lanes =
-// different columns), products with M (lanes = different rows) and the per-row triangular solves (lanes = different
-// rows) are all free of shared-memory bank conflicts.  No waiting on anything but __syncthreads.
+// One CTA of 256 threads per head.  The two kinds of products (M X and the Gram matrices Y^T Y, X^T (M X)) run on the
+// FP64 tensor path (mma.sync m8n8k4), which has the throughput of the FP64 FMA path on this part but needs a third of
+// the shared-memory reads and far fewer issue slots.  X and Y are stored column by column with a stride of d + 4
+// doubles, M (for r <= 32, where it fits beside them) row by row with the same stride: the 8 x 4 operand fragments
+// then fall on distinct banks, and the per-row triangular solves (lanes = consecutive rows) are conflict-free with any
+// stride.  No waiting on anything but __syncthreads.
 #include "squat_internal.cuh"
 
 namespace {
 
 constexpr int D = SQUAT_D;
 constexpr int PW_THREADS = 256;
-constexpr int LDC = D + 1;                      // column stride of X and Y (doubles)
+constexpr int LDC = D + 4;                      // column stride of X and Y (doubles): tensor-operation fragments (8 columns x 4 rows) fall on distinct banks
+constexpr int LDM = D + 4;                      // row stride of the shared-memory copy of M, for the same reason
 constexpr double PW_DROP = 1e-13;
 
 template <int RP>
@@ -32,72 +36,81 @@ struct PowerLayout {
     static constexpr int LDG = RP + 1;                                         // row stride of G / L
     static constexpr bool M_SHARED = RP <= 32;                                 // M beside X, Y fits in shared memory
     static constexpr size_t small = 2 * (size_t)RP * LDC + (size_t)RP * LDG + RP + 8;   // X, Y, G, inv, misc
-    static constexpr size_t doubles = small + (M_SHARED ? (size_t)D * D : 0);
+    static constexpr size_t doubles = small + (M_SHARED ? (size_t)D * LDM : 0);
 };
 
-// Y = M X: thread = rows 4 rq .. 4 rq + 3 x 8 columns (warp-uniform); M is symmetric, so row k of M holds column k.
-// With 32 columns four warps cover them and the other four take the second half of the sum over k, added after a
-// barrier; with 64 columns every warp has its own 8.
+// D += A B on the FP64 tensor path: A 8 x 4 (lane holds A[lane / 4][lane % 4]), B 4 x 8 (lane holds B[lane % 4][lane / 4]),
+// D 8 x 8 (lane holds D[lane / 4][2 (lane % 4)] and the element to its right)
+__device__ __forceinline__ void pw_dmma(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+
+// Y = M X: a warp owns 16 rows (two 8-row tiles) x all RP columns; per 4 values of k it loads two fragments of M and
+// RP / 8 of X and issues RP / 4 tensor operations.  M is symmetric; MS: M is the padded shared-memory copy (row stride
+// LDM), else it is read from global memory (row stride D).
 template <int RP, bool MS>
 __device__ __forceinline__ void pw_mult(const double *__restrict__ M, const double *Xt, double *Yt, int tid)
 {
-    constexpr int KS = (RP == 32) ? 2 : 1;      // parts of the k range
-    const int rq = tid & 31, w = tid >> 5;
-    const int c0 = 8 * (w % (RP / 8)), part = w / (RP / 8);
-    double acc[8][4];
+    constexpr int NC = RP / 8;                  // column tiles
+    constexpr int LD = MS ? LDM : D;
+    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    double acc[2][NC][2];
 #pragma unroll
-    for (int b = 0; b < 8; ++b)
+    for (int r = 0; r < 2; ++r)
 #pragma unroll
-        for (int a = 0; a < 4; ++a) acc[b][a] = 0.0;
-    const int k_lo = part * (D / KS), k_hi = k_lo + D / KS;
+        for (int c = 0; c < NC; ++c) acc[r][c][0] = acc[r][c][1] = 0.0;
+    const double *ma = M + (size_t)(16 * warp + g) * LD + t;
+    const double *xb = Xt + g * LDC + t;
 #pragma unroll 2
-    for (int k = k_lo; k < k_hi; ++k) {
-        const double2 *mp = reinterpret_cast<const double2 *>(M + (size_t)k * D) + 2 * rq;
-        const double2 m01 = MS ? mp[0] : __ldg(mp);                 // MS: M is a shared-memory copy
-        const double2 m23 = MS ? mp[1] : __ldg(mp + 1);
-        const double m[4] = {m01.x, m01.y, m23.x, m23.y};
+    for (int k0 = 0; k0 < D; k0 += 4) {
+        const double a0 = MS ? ma[k0] : __ldg(ma + k0);
+        const double a1 = MS ? ma[8 * LD + k0] : __ldg(ma + 8 * LD + k0);
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
-            const double x = Xt[(c0 + b) * LDC + k];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) acc[b][a] = fma(m[a], x, acc[b][a]);
+        for (int c = 0; c < NC; ++c) {
+            const double b = xb[8 * c * LDC + k0];
+            pw_dmma(acc[0][c][0], acc[0][c][1], a0, b);
+            pw_dmma(acc[1][c][0], acc[1][c][1], a1, b);
         }
     }
-    if (part == 0) {
 #pragma unroll
-        for (int b = 0; b < 8; ++b)
+    for (int r = 0; r < 2; ++r)
 #pragma unroll
-            for (int a = 0; a < 4; ++a) Yt[(c0 + b) * LDC + 4 * rq + a] = acc[b][a];
-    }
-    if (KS == 2) {
-        __syncthreads();
-        if (part == 1) {
-#pragma unroll
-            for (int b = 0; b < 8; ++b)
-#pragma unroll
-                for (int a = 0; a < 4; ++a) Yt[(c0 + b) * LDC + 4 * rq + a] += acc[b][a];
+        for (int c = 0; c < NC; ++c) {
+            double *y = Yt + (8 * c + 2 * t) * LDC + 16 * warp + 8 * r + g;
+            y[0] = acc[r][c][0];
+            y[LDC] = acc[r][c][1];
         }
-    }
 }
 
-// G[i][j] = add_identity * (i == j) + scale * sum_row At[i][row] Bt[j][row]
+// G[i][j] = ident * (i == j) + scale * sum_row At[i][row] Bt[j][row]: a warp owns one 8-row tile of G and RP * RP / 512
+// of its 8-column tiles
 template <int RP>
 __device__ __forceinline__ void pw_gram(const double *At, const double *Bt, double *G, double scale, double ident, int tid)
 {
-    constexpr int NJ = RP * RP / PW_THREADS;    // 4 (RP = 32) or 16 (RP = 64) columns j per thread
     constexpr int LDG = PowerLayout<RP>::LDG;
-    const int i = tid % RP, j0 = (tid / RP) * NJ;
-    double acc[NJ];
+    constexpr int NT = RP / 8;                  // tiles per side
+    constexpr int NC = NT * NT / (PW_THREADS / 32);     // column tiles per warp: 2 (RP = 32) or 8 (RP = 64)
+    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int ti = (warp * NC) / NT, tj0 = (warp * NC) % NT;
+    double acc[NC][2];
 #pragma unroll
-    for (int b = 0; b < NJ; ++b) acc[b] = 0.0;
-#pragma unroll 4
-    for (int row = 0; row < D; ++row) {
-        const double a = At[i * LDC + row];
+    for (int c = 0; c < NC; ++c) acc[c][0] = acc[c][1] = 0.0;
+    const double *pa = At + (8 * ti + g) * LDC + t;
+    const double *pb = Bt + (8 * tj0 + g) * LDC + t;
+#pragma unroll 2
+    for (int k0 = 0; k0 < D; k0 += 4) {
+        const double a = pa[k0];
 #pragma unroll
-        for (int b = 0; b < NJ; ++b) acc[b] = fma(a, Bt[(j0 + b) * LDC + row], acc[b]);
+        for (int c = 0; c < NC; ++c) pw_dmma(acc[c][0], acc[c][1], a, pb[8 * c * LDC + k0]);
     }
 #pragma unroll
-    for (int b = 0; b < NJ; ++b) G[i * LDG + j0 + b] = scale * acc[b] + ((i == j0 + b) ? ident : 0.0);
+    for (int c = 0; c < NC; ++c) {
+        const int i = 8 * ti + g, j = 8 * (tj0 + c) + 2 * t;
+        G[i * LDG + j] = scale * acc[c][0] + (i == j ? ident : 0.0);
+        G[i * LDG + j + 1] = scale * acc[c][1] + (i == j + 1 ? ident : 0.0);
+    }
 }
 
 // 1 / sqrt(x) for a positive normal x: exponent split off (x = s * 4^n with s in [1, 4)), single-precision seed, two
@@ -257,7 +270,7 @@ __global__ void __launch_bounds__(PW_THREADS, 1) power_kernel(
     if (MS) {
         double *Msm = psm + PowerLayout<RP>::small;
         for (int idx = tid; idx < D * D / 2; idx += PW_THREADS)
-            reinterpret_cast<double2 *>(Msm)[idx] = __ldg(reinterpret_cast<const double2 *>(M) + idx);
+            *reinterpret_cast<double2 *>(Msm + (idx / (D / 2)) * LDM + 2 * (idx % (D / 2))) = __ldg(reinterpret_cast<const double2 *>(M) + idx);
         Mu = Msm;
     }
     const double *X0 = start + (size_t)h * start_stride_h;
