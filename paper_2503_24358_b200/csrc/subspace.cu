@@ -242,6 +242,15 @@ __device__ __forceinline__ double rsqrt_nr(double x)
     return fma(y * r, fma(0.375, r, 0.5), y);
 }
 
+// 1/x for a normal double: hardware seed (about 20 bits), two Newton steps y <- y + y (1 - x y)
+__device__ __forceinline__ double rcp_nr(double x)
+{
+    double y;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    y = fma(y, fma(-x, y, 1.0), y);
+    return fma(y, fma(-x, y, 1.0), y);
+}
+
 __device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
 // One Jacobi rotation of a column pair (P, Q) held in registers by a team of 16 lanes (both halves of a warp work
@@ -582,7 +591,7 @@ __global__ void __launch_bounds__(ASM_THREADS, 1) assemble_kernel(
                 double *lp = pub + (j & 1) * 2 * D, *vp = lp + D;
                 if (warp == wj) {
                     const double d = __shfl_sync(0xffffffffu, a[kj >> 1][kj], j & 31);
-                    const double inv = 1.0 / d;
+                    const double inv = rcp_nr(d);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int r = lane + 32 * i;
