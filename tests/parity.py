@@ -10,7 +10,12 @@ widths, i.e. 1e-5 * L/3 in code units, because the float32 error of the correcte
 when the grid gets finer) and differ by exactly one level; force the GPU's choice
 there, re-run the oracle on that group, repeat.  The run passes iff every forced decision was such
 a tie and nothing differs afterwards.  The raw (pre-replay) identical fraction is reported too and
-must be >= 99.9 %.
+must be >= 99.9 %.  Every forced tie's distance from the midpoint is kept, so that a report can say how
+many of them lie outside the literal 1e-5 code units (possible only at more than 2 bits).
+
+The projected error is checked on both readings of "the subspace basis": the objective's own weighting
+||Qhat (k - khat)||_F (rows of Qhat = sigma_i v_i) and the orthonormal basis ||V_r^T (k - khat)||_F
+(rows of Qhat normalised), each within 1e-3 relative of the oracle's.
 """
 import numpy as np
 import torch
@@ -60,6 +65,19 @@ def alloc_value_outputs(B, H, T, d, bits, G, device="cuda"):
     return codes, scales, zeros
 
 
+def _projection_checks(stats, gpu_deq, final_khat, K64, Qhat):
+    """Relative differences of the projected errors (GPU against oracle) on Qhat and on the orthonormal V_r."""
+    if Qhat is None or Qhat.shape[0] == 0:
+        return
+    norms = np.linalg.norm(Qhat, axis=1)
+    Vr = Qhat[norms > 0] / norms[norms > 0][:, None]           # rows v_i: Qhat = diag(sigma) V_r^T
+    dg, do = gpu_deq.astype(np.float64) - K64, final_khat - K64
+    for name, basis in (("proj_rel", Qhat), ("proj_rel_vr", Vr)):
+        pg, po = np.linalg.norm(dg @ basis.T), np.linalg.norm(do @ basis.T)
+        stats[name] = float(abs(pg - po) / po)
+        assert abs(pg - po) <= 1e-3 * po, (name, pg, po)
+
+
 def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=None, Qhat=None, max_replays=64,
                      meta16=False):
     """Compares one (batch, head) unit.  K64 [n,d] float64; gpu_codes [n,d] unpacked uint8;
@@ -73,6 +91,7 @@ def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=
     base = oracle.quant_keys(K64, G, bits, W64, want_tval=True)
     raw_equal = int((base["codes"] == gpu_codes).sum())
     ties = 0
+    tie_dist = []
     final_codes = base["codes"].copy()
     final_khat = base["Khat"].copy()
     final_scale, final_zero = base["scale"].copy(), base["zero"].copy()
@@ -95,6 +114,7 @@ def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=
                     f"t={t!r} |frac-0.5|={frac:.3e}")
                 force[i, j0] = cg
                 ties += 1
+                tie_dist.append(float(frac))
             o = oracle.quant_keys(K64[lo:hi], G, bits, W64, force=force, want_tval=True)
         else:
             raise AssertionError(f"group {grp}: replay did not converge")
@@ -102,7 +122,8 @@ def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=
         final_khat[lo:hi] = o["Khat"]
         final_scale[grp], final_zero[grp] = o["scale"][0], o["zero"][0]
     assert np.array_equal(final_codes, gpu_codes)
-    stats = {"elements": n * d, "raw_equal": raw_equal, "ties": ties, "raw_fraction": raw_equal / (n * d)}
+    stats = {"elements": n * d, "raw_equal": raw_equal, "ties": ties, "raw_fraction": raw_equal / (n * d),
+             "ties_beyond_1e-5": sum(1 for f in tie_dist if f >= TIE_BAND), "max_tie_dist": max(tie_dist, default=0.0)}
     # scale / zero: float32 roundings of fp64 vs fp32 working values
     sc_err = np.abs(gpu_scale.astype(np.float64) - final_scale).max() / max(np.abs(final_scale).max(), 1e-30)
     zr_err = np.abs(gpu_zero.astype(np.float64) - final_zero).max() / max(np.abs(final_zero).max(), 1e-30)
@@ -112,11 +133,7 @@ def compare_key_unit(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, gpu_deq=
         rel = np.linalg.norm(gpu_deq.astype(np.float64) - final_khat) / np.linalg.norm(final_khat)
         stats["deq_rel_fro"] = float(rel)
         assert rel < 1e-3, rel
-        if Qhat is not None and Qhat.shape[0] > 0:
-            pg = np.linalg.norm((gpu_deq.astype(np.float64) - K64) @ Qhat.T)
-            po = np.linalg.norm((final_khat - K64) @ Qhat.T)
-            stats["proj_rel"] = float(abs(pg - po) / po)
-            assert abs(pg - po) <= 1e-3 * po, (pg, po)
+        _projection_checks(stats, gpu_deq, final_khat, K64, Qhat)
     return stats
 
 
@@ -136,6 +153,7 @@ def compare_key_unit_meta16(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, g
     base = oracle.quant_keys(K64, G, bits, W64, want_tval=True, meta16=True)
     raw_equal = int((base["codes"] == gpu_codes).sum())
     ties = meta_ties = 0
+    tie_dist = []
     final_codes, final_khat = base["codes"].copy(), base["Khat"].copy()
     final_scale, final_zero = base["scale"].copy(), base["zero"].copy()
     code_bad = np.nonzero(base["codes"] != gpu_codes)[0] // G
@@ -180,6 +198,7 @@ def compare_key_unit_meta16(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, g
                         f"t={t!r} |frac-0.5|={frac:.3e}")
                     force[i, j0] = cg
                     ties += 1
+                    tie_dist.append(float(frac))
             o = oracle.quant_keys(K64[lo:hi], G, bits, W64, force=force, want_tval=True, meta16=True, force_meta=(fs, fz))
         else:
             raise AssertionError(f"group {grp}: replay did not converge")
@@ -188,16 +207,13 @@ def compare_key_unit_meta16(K64, W64, G, bits, gpu_codes, gpu_scale, gpu_zero, g
     assert np.array_equal(final_codes, gpu_codes)
     assert np.array_equal(final_scale, gpu_scale) and np.array_equal(final_zero, gpu_zero)
     stats = {"elements": n * d, "raw_equal": raw_equal, "ties": ties, "meta_ties": meta_ties,
-             "raw_fraction": raw_equal / (n * d)}
+             "raw_fraction": raw_equal / (n * d),
+             "ties_beyond_1e-5": sum(1 for f in tie_dist if f >= TIE_BAND), "max_tie_dist": max(tie_dist, default=0.0)}
     if gpu_deq is not None:
         rel = np.linalg.norm(gpu_deq.astype(np.float64) - final_khat) / np.linalg.norm(final_khat)
         stats["deq_rel_fro"] = float(rel)
         assert rel < 1e-3, rel
-        if Qhat is not None and Qhat.shape[0] > 0:
-            pg = np.linalg.norm((gpu_deq.astype(np.float64) - K64) @ Qhat.T)
-            po = np.linalg.norm((final_khat - K64) @ Qhat.T)
-            stats["proj_rel"] = float(abs(pg - po) / po)
-            assert abs(pg - po) <= 1e-3 * po, (pg, po)
+        _projection_checks(stats, gpu_deq, final_khat, K64, Qhat)
     return stats
 
 

@@ -70,17 +70,17 @@ def test_keys_config1_full():
 @pytest.mark.parametrize("bits,G,r,g", [(4, 32, 32, 1), (2, 64, 8, 1), (2, 128, 32, 1), (4, 128, 64, 1),
                                         (2, 32, 16, 32), (2, 32, 40, 64), (4, 64, 5, 64)])
 def test_keys_variants_bf16(bits, G, r, g):
-    # bits x group size x rank x block size g; 3 heads, batch 2, 512 tokens (several tiles, every team size)
-    cfg = si.get_config(1).with_(batch=2, n_kv_heads=3, n_q_heads=3, n_tokens=512)
+    # bits x group size x rank x block size g; 3 heads, batch 3, 2048 tokens: 2.36 M elements per variant, enough
+    # for the 99.9 % bar on the raw identical fraction to mean something (one tie moves about 400 elements)
+    cfg = si.get_config(1).with_(batch=3, n_kv_heads=3, n_q_heads=3, n_tokens=2048)
     W32, mats = _oracle_W32(cfg, range(3), rank_r=r, g=g)
     k_np = si.gen_keys(cfg)
     got = _run_keys(cfg, k_np, W32, bits, G)
-    # 0.4 M elements: a handful of legitimate ties, each cascading through its group, already moves the
-    # raw fraction by 1e-3; the 99.9 % bar is applied on the full-size workloads
-    _compare_all_units(cfg, k_np, W32, mats, bits, G, got, min_raw=0.99)
+    tot = _compare_all_units(cfg, k_np, W32, mats, bits, G, got, min_raw=0.999)
+    print(f"variant bits={bits} G={G} r={r} g={g}:", tot)
 
 
-@pytest.mark.parametrize("G,T,B,H", [
+RAGGED_SHAPES = [
     (32, 160, 1, 2),     # 5 groups per head: the second 128-token tile has one group, its other three warps idle along
     (32, 96, 3, 3),      # 9 groups per head across 3 batch entries: tiles mix batch entries, the last one is ragged
     (64, 192, 1, 2),     # 3 groups of 64: tile 1 holds one team and a spare one
@@ -88,17 +88,27 @@ def test_keys_variants_bf16(bits, G, r, g):
     (32, 32, 1, 5),      # one group per head: every tile ragged, every round a new head
     (32, 160, 4, 40),    # 200 tiles of 40 heads on 148 CTAs: some CTAs' rounds run across a head boundary (two images staged)
     (32, 64, 1, 170),    # 170 one-tile heads: a CTA's two tiles belong to different heads
-])
-def test_keys_ragged_tiles_and_rounds(G, T, B, H):
-    # the kernel works in tiles of 128 tokens (4 warps) and rounds of up to 4 tiles that may span two heads
+]
+
+
+def test_keys_ragged_tiles_and_rounds():
+    # the kernel works in tiles of 128 tokens (4 warps) and rounds of up to 4 tiles that may span two heads.
+    # Every shape goes through the element-by-element protocol on its own; the shapes are small by nature, so the
+    # 99.9 % bar on the raw identical fraction is applied to all of them together (4.9 M elements)
     bits = 2
-    cfg = si.get_config(1).with_(batch=B, n_kv_heads=H, n_q_heads=H, n_tokens=T)
-    W32, mats = _oracle_W32(cfg, range(H), n_tokens=max(T, 256))
-    k_np = si.gen_keys(cfg)
-    sq.squat_get_device_status(clear=True)
-    got = _run_keys(cfg, k_np, W32, bits, G)
-    assert not (sq.squat_get_device_status(clear=True) & sq.FLAG_DEVICE_TIMEOUT)
-    _compare_all_units(cfg, k_np, W32, mats, bits, G, got, min_raw=0.99)
+    pool = {"elements": 0, "raw_equal": 0, "ties": 0}
+    for G, T, B, H in RAGGED_SHAPES:
+        cfg = si.get_config(1).with_(batch=B, n_kv_heads=H, n_q_heads=H, n_tokens=T)
+        W32, mats = _oracle_W32(cfg, range(H), n_tokens=max(T, 256))
+        k_np = si.gen_keys(cfg)
+        sq.squat_get_device_status(clear=True)
+        got = _run_keys(cfg, k_np, W32, bits, G)
+        assert not (sq.squat_get_device_status(clear=True) & sq.FLAG_DEVICE_TIMEOUT), (G, T, B, H)
+        tot = _compare_all_units(cfg, k_np, W32, mats, bits, G, got, min_raw=0.0)
+        for key in pool:
+            pool[key] += tot[key]
+    print("ragged shapes pooled:", pool)
+    assert pool["raw_equal"] >= 0.999 * pool["elements"], pool
 
 
 def test_keys_zero_update_reduces_to_round_to_nearest():

@@ -73,7 +73,7 @@ def test_workload3_decode_append_stream():
     sq.squat_build_subspace(s, to_torch(si.gen_queries(cfg), cfg.dtype), cfg.rank_r, cfg.lam, cfg.block_g)
     kc, ks, kz = alloc_key_outputs(B, H, Tc, D, bits, G)
     vc, vs, vz = alloc_value_outputs(B, H, Tc, D, bits, G)
-    sampled = {0: None, 13: None, 31: None}           # windows whose content is generated and checked
+    sampled = {0: None, 13: None, 22: None, 31: None}  # windows whose content is generated and checked
     k = v = None
     for w in range(NW):
         if w in sampled or k is None:
@@ -90,12 +90,15 @@ def test_workload3_decode_append_stream():
     torch.cuda.synchronize()
     cache, tot_all = {}, {"elements": 0, "raw_equal": 0, "ties": 0}
     for w, (k_np, v_np) in sampled.items():
-        tot = _check_units(cfg, [(0, 0), (31, 17), (63, 31)], k_np, v_np, kc, ks, kz, vc, vs, vz, bits, G, cache,
-                           tok_lo=w * W, n_tok=W)
+        # every head once per sampled window, the batch entry moving with head and window: 4 x 32 units of
+        # 128 x 128 elements = 2.1 M compared elements
+        units = [((7 * h + 5 * w) % B, h) for h in range(H)]
+        tot = _check_units(cfg, units, k_np, v_np, kc, ks, kz, vc, vs, vz, bits, G, cache, tok_lo=w * W, n_tok=W)
         for k_ in tot_all:
             tot_all[k_] += tot[k_]
     print("workload 3 sampled windows/units:", tot_all)
-    assert tot_all["raw_equal"] >= 0.99 * tot_all["elements"], tot_all       # 0.15 M elements: see test_gpu_keys
+    assert tot_all["elements"] >= 2_000_000
+    assert tot_all["raw_equal"] >= 0.999 * tot_all["elements"], tot_all
     s.close()
 
 
@@ -119,7 +122,7 @@ def test_workload4_long_context_sweep():
         torch.cuda.synchronize()
         tot = _check_units(cfg, units, k_np, None, kc, ks, kz, None, None, None, bits, G, cache, rank_r=r)
         print(f"workload 4 point bits={bits} r={r} G={G}:", tot)
-        assert tot["raw_equal"] >= 0.998 * tot["elements"], (bits, r, G, tot)
+        assert tot["raw_equal"] >= 0.999 * tot["elements"], (bits, r, G, tot)
         del kc, ks, kz
     # values: one pass per (bits, G) on the full tensor, two sampled units each
     del k
