@@ -44,7 +44,7 @@ typedef enum { SQUAT_F32 = 0, SQUAT_BF16 = 1 } squat_dtype;
 typedef enum { SQUAT_KEYS = 0, SQUAT_VALUES = 1 } squat_kind;
 
 /* bits of the device status word */
-#define SQUAT_FLAG_NONFINITE   1u   /* a scale came out NaN/Inf: non-finite input                  */
+#define SQUAT_FLAG_NONFINITE   1u   /* a NaN or infinity among the keys / values (its group's scale came out NaN/Inf) */
 #define SQUAT_FLAG_ZERO_RANGE  2u   /* some group had max == min (scale 0, all codes 0)            */
 #define SQUAT_FLAG_NO_CONVERGE 4u   /* eigensolver hit its sweep limit for some head               */
 #define SQUAT_FLAG_DEVICE_TIMEOUT 8u /* a bounded wait on the tensor core inside squat_quantize_keys ran
@@ -244,6 +244,23 @@ int squat_write_path_host_ex(squat_subspace *s, const void *q_host, const void *
                              void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * One decode window from HOST buffers (Algorithm 1, decode branch: when the residual buffer holds R keys, Quant runs
+ * on its R/G groups with the per-head matrices that were computed at prefill; values likewise, Appendix C).  Copies
+ * k and v ([batch, n_kv_heads, n_tokens, d], contiguous, n_tokens a multiple of group_size) to the device workspace,
+ * quantizes them with the update matrices the handle holds (nothing is built), copies codes / scales / zeros back to
+ * the host buffers (contiguous, the shapes squat_quantize_keys / _values write) and synchronises the stream.
+ * meta16 = 1: scales and zero-points are binary16 (2-byte elements).  Workspace: at least
+ * squat_write_path_workspace_bytes(dtype, batch, n_kv_heads, n_kv_heads, n_tokens, d, bits, group_size) bytes of
+ * caller-owned device memory, 256-byte aligned.  The copies run on two side streams of the handle and overlap the
+ * kernels; calls on one handle must not overlap each other.
+ */
+int squat_append_window_host(squat_subspace *s, const void *k_host, const void *v_host, int dtype, int batch,
+                             int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                             unsigned char *k_codes_host, void *k_scales_host, void *k_zeros_host,
+                             unsigned char *v_codes_host, void *v_scales_host, void *v_zeros_host, int meta16,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Reader of the cache -- one decode step of attention over the packed cache (Section 2, "(Masked) Attention
  * mechanism": softmax(q K^T / sqrt(d)) V for the newest token; the score vector w^deq of the proof of
  * Theorem 1; the most recent tokens come from the full-precision residual buffer of Algorithm 1).  This is
@@ -340,6 +357,17 @@ int squat_decode_attention_pre_rope(const void *q, int q_dtype, int batch, int n
  */
 int squat_gram_static(const void *q, int dtype, int n_q_heads, int n_kv_heads, int n_tokens, int head_dim,
                       long long stride_h, long long stride_t, double *gram_out, void *stream);
+
+/*
+ * Measurement aid (the paper has no counterpart): launches one kernel of register-resident single-precision
+ * multiply-add chains that keeps every FP32 lane of the GPU busy -- scalar fma.rn.f32 (packed = 0) or two-wide
+ * fma.rn.f32x2 (packed = 1) -- so that a benchmark can time it (CUDA events around the call) and quote kernels
+ * against the FP32 throughput this GPU actually reaches.  iters in [1, 2^20] sets the length (64 multiply-adds per
+ * thread and iteration, twice that when packed); *flops_host (host, may be NULL) receives the floating-point
+ * operations the launch performs; sink is a device float the kernel never really writes (it keeps the chains from
+ * being optimised away).  Enqueues on `stream`.
+ */
+int squat_fp32_peak_probe(int packed, int iters, float *sink, long long *flops_host, void *stream);
 
 /* Reads (and clears when `clear` != 0) the device status word of the current device.
  * Synchronises `stream`.  flags is a host pointer. */

@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = (
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
     "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_write_path_host_ex", "squat_build_subspace_power_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
+    "squat_fp32_peak_probe", "squat_append_window_host",
 )
 
 _lib = None
@@ -82,6 +83,8 @@ def _load():
                                                         c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
         lib.squat_decode_attention_ex.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, i, ll, ll, i, i, vp, vp, i, i,
                                                   c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
+        lib.squat_append_window_host.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, c.c_size_t, vp]
+        lib.squat_fp32_peak_probe.argtypes = [i, i, vp, c.POINTER(ll), vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
         lib.squat_status_string.argtypes = [i]
@@ -281,6 +284,37 @@ def squat_write_path_host(s: Subspace, q, k, v, rank_r, lam, block_g, bits, grou
            "squat_write_path_host_ex")
 
 
+def squat_append_window_host(s: Subspace, k, v, bits, group_size, k_codes, k_scales, k_zeros, v_codes, v_scales, v_zeros,
+                             workspace: torch.Tensor, stream=None):
+    """One decode window from HOST tensors (pinned for speed): k, v [B, H, T, d] go up, are quantized with the update
+    matrices the handle holds, and the six outputs come back.  float16 scale / zero tensors select 16-bit metadata;
+    workspace: CUDA uint8 tensor of squat_write_path_workspace_bytes(dtype, B, H, H, T, d, bits, group_size)."""
+    for name, t in (("k", k), ("v", v), ("k_codes", k_codes), ("k_scales", k_scales), ("k_zeros", k_zeros),
+                    ("v_codes", v_codes), ("v_scales", v_scales), ("v_zeros", v_zeros)):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous host tensor")
+    B, H, T, d = k.shape
+    hp = lambda t: ctypes.c_void_p(t.data_ptr())
+    meta = (k_scales, k_zeros, v_scales, v_zeros)
+    m16 = all(t.dtype == torch.float16 for t in meta)
+    if not m16 and not all(t.dtype == torch.float32 for t in meta):
+        raise ValueError("scales and zero-points must be all float32 or all float16")
+    _check(_load().squat_append_window_host(s.handle, hp(k), hp(v), _dtype_code(k), B, H, T, d, bits, group_size,
+                                            hp(k_codes), hp(k_scales), hp(k_zeros), hp(v_codes), hp(v_scales), hp(v_zeros),
+                                            int(m16), _dev(workspace, "workspace"),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)),
+           "squat_append_window_host")
+
+
+def squat_fp32_peak_probe(packed: bool, iters: int, sink: torch.Tensor, stream=None) -> int:
+    """Launches the FP32 multiply-add probe kernel (a measurement aid; time it with CUDA events around this call).
+    sink: a CUDA float32 tensor of at least one element.  Returns the floating-point operations of the launch."""
+    flops = ctypes.c_longlong(0)
+    _check(_load().squat_fp32_peak_probe(1 if packed else 0, int(iters), _dev(sink, "sink"), ctypes.byref(flops),
+                                         _stream(stream)), "squat_fp32_peak_probe")
+    return int(flops.value)
+
+
 def squat_gram_static(q: torch.Tensor, n_kv_heads: int, gram_out: torch.Tensor, stream=None):
     """Gram matrices of the stacked queries into gram_out [n_kv_heads, d, d] (float64, CUDA) without any
     allocation: for callers that cannot call cudaMalloc (allocator callbacks, frozen allocators, processes
@@ -359,21 +393,31 @@ def squat_build_subspace_sharded(s: "Subspace", q_local: torch.Tensor, rank_r: i
     the local tokens (q_local [n_q_heads, local_tokens, d]; a rank may hold none), one all-reduce (sum) of
     n_kv_heads * d * d float64, then the eigen-decomposition (or, with a start_block every rank passes alike, the
     block power iteration) and the update matrices on every rank.  Without an initialised process group this is the
-    single-GPU build through the same two calls."""
+    single-GPU build through the same two calls.
+
+    The whole sequence runs on `stream` (torch's current stream when None): the collective is issued with that stream
+    current, so it starts after the Gram kernels and the build starts after it.  Limits inherited from
+    squat_gram_static: at most 64 KV heads, and one shared scratch array in the library -- two sharded builds (two
+    layers, say) must not overlap on the GPU, so do not run them on different streams at the same time."""
     import torch.distributed as dist
     H = s.n_kv_heads
-    if gram_buf is None:
-        gram_buf = torch.empty((H, q_local.shape[2], q_local.shape[2]), dtype=torch.float64, device=q_local.device)
-    if q_local.shape[1] > 0:
-        squat_gram_static(q_local, H, gram_buf, stream)
-    else:
-        gram_buf.zero_()
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
-    if start_block is not None:
-        squat_build_subspace_power_from_gram(s, gram_buf, rank_r, lam, start_block, power_iters, block_g, stream)
-    else:
-        squat_build_subspace_from_gram(s, gram_buf, rank_r, lam, block_g, stream)
+    if q_local.dim() != 3 or q_local.shape[0] % H != 0:
+        raise ValueError("q_local must be [n_q_heads, local_tokens, d] with n_q_heads a multiple of the handle's KV heads")
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    with torch.cuda.stream(stream):
+        if gram_buf is None:
+            gram_buf = torch.empty((H, q_local.shape[2], q_local.shape[2]), dtype=torch.float64, device=q_local.device)
+        if q_local.shape[1] > 0:
+            squat_gram_static(q_local, H, gram_buf, stream)
+        else:
+            gram_buf.zero_()
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+            dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
+        if start_block is not None:
+            squat_build_subspace_power_from_gram(s, gram_buf, rank_r, lam, start_block, power_iters, block_g, stream)
+        else:
+            squat_build_subspace_from_gram(s, gram_buf, rank_r, lam, block_g, stream)
     return gram_buf
 
 

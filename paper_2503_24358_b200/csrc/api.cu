@@ -21,6 +21,12 @@ __device__ unsigned g_status_word = 0;
 unsigned *g_status_ptr[MAX_DEVICES] = {nullptr};
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+// A handle's memory lives on the device that was current when it was created; its calls must run there.
+bool on_handle_device(const squat_subspace *s)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == s->device;
+}
 bool valid_dtype(int dt) { return dt == SQUAT_F32 || dt == SQUAT_BF16; }
 size_t elem_size(int dt) { return dt == SQUAT_BF16 ? 2 : 4; }
 
@@ -94,7 +100,6 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     memset(s, 0, sizeof(*s));
     s->n_kv_heads = n_kv_heads;
     s->head_dim = head_dim;
-    s->exact_blocks = D / 32;            // W starts as zero: every channel is uncorrected
     int sms = 148;
     if (cudaGetDevice(&s->device) != cudaSuccess) { delete s; return SQUAT_ERR_CUDA; }
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, s->device);
@@ -111,6 +116,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     const size_t o_val = carve((size_t)n_kv_heads * D * sizeof(double));
     const size_t o_vec = carve(hdd * sizeof(double));
     const size_t o_swp = carve((size_t)n_kv_heads * sizeof(int));
+    const size_t o_exact = carve(sizeof(int));
     char *base = nullptr;
     if (cudaMalloc(&base, off) != cudaSuccess) { cudaGetLastError(); delete s; return SQUAT_ERR_ALLOC; }
     if (cudaMemset(base, 0, off) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
@@ -121,6 +127,9 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     s->eigval = reinterpret_cast<double *>(base + o_val);
     s->eigvec = reinterpret_cast<double *>(base + o_vec);
     s->eig_sweeps = reinterpret_cast<int *>(base + o_swp);
+    s->exact_blocks = reinterpret_cast<int *>(base + o_exact);
+    const int all_exact = D / 32;        // W starts as zero: every channel is uncorrected
+    if (cudaMemcpy(s->exact_blocks, &all_exact, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
     s->status = squat_status_word();
     if (!s->status) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
     *out = s;
@@ -144,6 +153,7 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
                          int block_g, void *stream)
 {
     if (!s || !q || !valid_dtype(dtype) || !aligned16(q)) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     if (n_q_heads <= 0 || n_tokens <= 0) return SQUAT_ERR_INVALID_ARG;
     if (n_q_heads % s->n_kv_heads != 0) return SQUAT_ERR_SHAPE;
     if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
@@ -158,14 +168,15 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
     rc = squat_launch_eig(s, st);
     if (rc != SQUAT_OK) return rc;
     // channels of the first g-block are never corrected; with r = 0 or lambda = 0, W = 0 and none is
-    s->exact_blocks = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
-    return squat_launch_assemble(s, rank_r, lambda, block_g, 0, st);
+    const int exact = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 0, exact, st);
 }
 
 int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
                                    void *stream)
 {
     if (!s || !gram || !aligned16(gram)) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
     if (!(lambda >= 0.0) || !std::isfinite(lambda)) return SQUAT_ERR_INVALID_ARG;
     if (block_g <= 0 || D % block_g != 0) return SQUAT_ERR_SHAPE;
@@ -174,8 +185,8 @@ int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int ra
         SQUAT_CUDA(cudaMemcpyAsync(s->gram, gram, (size_t)s->n_kv_heads * D * D * sizeof(double), cudaMemcpyDeviceToDevice, st));
     int rc = squat_launch_eig(s, st);
     if (rc != SQUAT_OK) return rc;
-    s->exact_blocks = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
-    return squat_launch_assemble(s, rank_r, lambda, block_g, 0, st);
+    const int exact = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 0, exact, st);
 }
 
 int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
@@ -183,6 +194,7 @@ int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int 
                                const double *start_block, long long start_stride_h, int iters, void *stream)
 {
     if (!s || !q || !valid_dtype(dtype) || !aligned16(q)) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     if (n_q_heads <= 0 || n_tokens <= 0) return SQUAT_ERR_INVALID_ARG;
     if (n_q_heads % s->n_kv_heads != 0) return SQUAT_ERR_SHAPE;
     if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
@@ -199,17 +211,18 @@ int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int 
     int rc = squat_launch_gram(s, q, dtype, n_q_heads, n_tokens, stride_h, stride_t, st);
     if (rc != SQUAT_OK) return rc;
     const bool no_update = rank_r == 0 || lambda == 0.0;
-    s->exact_blocks = no_update ? D / 32 : (block_g + 31) / 32;
-    if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, st);      // W = 0: nothing to iterate
+    const int exact = no_update ? D / 32 : (block_g + 31) / 32;
+    if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, exact, st);      // W = 0: nothing to iterate
     rc = squat_launch_power(s, start_block, start_stride_h, rank_r, iters, lambda, st);
     if (rc != SQUAT_OK) return rc;
-    return squat_launch_assemble(s, rank_r, lambda, block_g, 64, st);
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 64, exact, st);
 }
 
 int squat_build_subspace_power_from_gram(squat_subspace *s, const double *gram, int rank_r, double lambda, int block_g,
                                          const double *start_block, long long start_stride_h, int iters, void *stream)
 {
     if (!s || !gram || !aligned16(gram)) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     if (rank_r < 0 || rank_r > D) return SQUAT_ERR_INVALID_ARG;
     if (rank_r > 64) return SQUAT_ERR_UNSUPPORTED;
     if (!(lambda >= 0.0) || !std::isfinite(lambda)) return SQUAT_ERR_INVALID_ARG;
@@ -221,17 +234,18 @@ int squat_build_subspace_power_from_gram(squat_subspace *s, const double *gram, 
     if (gram != s->gram)
         SQUAT_CUDA(cudaMemcpyAsync(s->gram, gram, (size_t)s->n_kv_heads * D * D * sizeof(double), cudaMemcpyDeviceToDevice, st));
     const bool no_update = rank_r == 0 || lambda == 0.0;
-    s->exact_blocks = no_update ? D / 32 : (block_g + 31) / 32;
-    if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, st);
+    const int exact = no_update ? D / 32 : (block_g + 31) / 32;
+    if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, exact, st);
     int rc = squat_launch_power(s, start_block, start_stride_h, rank_r, iters, lambda, st);
     if (rc != SQUAT_OK) return rc;
-    return squat_launch_assemble(s, rank_r, lambda, block_g, 64, st);
+    return squat_launch_assemble(s, rank_r, lambda, block_g, 64, exact, st);
 }
 
 int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, double *gram_host,
                           double *eigval_host, double *eigvec_host)
 {
     if (!s) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t hdd = (size_t)s->n_kv_heads * D * D;
     std::vector<float> wt;
@@ -254,6 +268,7 @@ int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, 
 int squat_subspace_eig_sweeps(const squat_subspace *s, void *stream, int *sweeps_host)
 {
     if (!s || !sweeps_host) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SQUAT_CUDA(cudaMemcpyAsync(sweeps_host, s->eig_sweeps, (size_t)s->n_kv_heads * sizeof(int), cudaMemcpyDeviceToHost, st));
     SQUAT_CUDA(cudaStreamSynchronize(st));
@@ -263,6 +278,7 @@ int squat_subspace_eig_sweeps(const squat_subspace *s, void *stream, int *sweeps
 int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
 {
     if (!s || !W_host) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t hdd = (size_t)s->n_kv_heads * D * D;
     std::vector<float> wt(hdd);
@@ -278,9 +294,8 @@ int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
             for (int j = 0; j < D; ++j)
                 if (W_host[((size_t)h * D + jp) * D + j] != 0.0f) { uncorrected = jp; break; }
     const int exact = (uncorrected + 31) / 32;
-    s->exact_blocks = exact;
     SQUAT_CUDA(cudaMemcpyAsync(s->Wt, wt.data(), hdd * sizeof(float), cudaMemcpyHostToDevice, st));
-    int rc = squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, st);
+    int rc = squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, exact, s->exact_blocks, st);
     if (rc != SQUAT_OK) return rc;
     SQUAT_CUDA(cudaStreamSynchronize(st));
     return SQUAT_OK;
@@ -294,6 +309,7 @@ int quantize_keys_impl(const squat_subspace *s, const void *k, int dtype, int ba
                        void *stream)
 {
     if (!s) return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     int rc = check_quant_args(k, dtype, batch, n_kv_heads, n_tokens, head_dim, stride_b, stride_h, stride_t, bits,
                               group_size, codes, scales, zeros, out_stride_b, out_stride_h);
     if (rc != SQUAT_OK) return rc;
@@ -577,9 +593,12 @@ int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_ho
                          int meta16, const double *start_block_host, int power_iters,
                          void *workspace, size_t workspace_bytes, void *stream)
 {
-    if (!s || !q_host || !k_host || !v_host || !k_codes_host || !k_scales_host || !k_zeros_host || !v_codes_host ||
+    // q_host == NULL: no build; the keys are quantized with the update matrices the handle already holds (a decode window)
+    const bool do_build = q_host != nullptr;
+    if (!s || !k_host || !v_host || !k_codes_host || !k_scales_host || !k_zeros_host || !v_codes_host ||
         !v_scales_host || !v_zeros_host || !workspace || !valid_dtype(dtype))
         return SQUAT_ERR_INVALID_ARG;
+    if (!on_handle_device(s)) return SQUAT_ERR_INVALID_ARG;     // the handle belongs to another device
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQUAT_ERR_INVALID_ARG;
     if (batch <= 0 || n_tokens <= 0 || head_dim != D || n_kv_heads != s->n_kv_heads) return SQUAT_ERR_SHAPE;
     if ((bits != 2 && bits != 4) || (group_size != 32 && group_size != 64 && group_size != 128))
@@ -607,8 +626,8 @@ int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_ho
     cudaEvent_t ev_q = s->ev[0], ev_k = s->ev[1], ev_keys = s->ev[2], ev_kout = s->ev[3];
     const long long rows = (long long)batch * n_kv_heads;          // (batch, head) units of T tokens
     const int n_pieces = rows >= 4 ? 4 : (int)rows;
-    SQUAT_CUDA(cudaMemcpyAsync(w + L.q, q_host, (size_t)n_q_heads * T * d * es, cudaMemcpyHostToDevice, st));
-    if (start_block_host && rank_r > 0)
+    if (do_build) SQUAT_CUDA(cudaMemcpyAsync(w + L.q, q_host, (size_t)n_q_heads * T * d * es, cudaMemcpyHostToDevice, st));
+    if (do_build && start_block_host && rank_r > 0)
         SQUAT_CUDA(cudaMemcpyAsync(w + L.x0, start_block_host, (size_t)D * rank_r * sizeof(double), cudaMemcpyHostToDevice, st));
     SQUAT_CUDA(cudaEventRecord(ev_q, st));
     SQUAT_CUDA(cudaStreamWaitEvent(s->side[0], ev_q, 0));
@@ -620,7 +639,9 @@ int write_path_host_impl(squat_subspace *s, const void *q_host, const void *k_ho
                                    (size_t)(r1 - r0) * T * d * es, cudaMemcpyHostToDevice, s->side[0]));
         SQUAT_CUDA(cudaEventRecord(s->ev[4 + p], s->side[0]));
     }
-    int rc = start_block_host
+    int rc = SQUAT_OK;
+    if (do_build)
+        rc = start_block_host
                  ? squat_build_subspace_power(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g,
                                               reinterpret_cast<const double *>(w + L.x0), 0, power_iters, stream)
                  : squat_build_subspace(s, w + L.q, dtype, n_q_heads, n_tokens, T * d, d, rank_r, lambda, block_g, stream);
@@ -663,9 +684,22 @@ int squat_write_path_host(squat_subspace *s, const void *q_host, const void *k_h
                           unsigned char *v_codes_host, float *v_scales_host, float *v_zeros_host,
                           void *workspace, size_t workspace_bytes, void *stream)
 {
+    if (!q_host) return SQUAT_ERR_INVALID_ARG;
     return write_path_host_impl(s, q_host, k_host, v_host, dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, rank_r,
                                 lambda, block_g, bits, group_size, k_codes_host, k_scales_host, k_zeros_host, v_codes_host,
                                 v_scales_host, v_zeros_host, 0, nullptr, 0, workspace, workspace_bytes, stream);
+}
+
+int squat_append_window_host(squat_subspace *s, const void *k_host, const void *v_host, int dtype, int batch,
+                             int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
+                             unsigned char *k_codes_host, void *k_scales_host, void *k_zeros_host,
+                             unsigned char *v_codes_host, void *v_scales_host, void *v_zeros_host, int meta16,
+                             void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (meta16 != 0 && meta16 != 1) return SQUAT_ERR_INVALID_ARG;
+    return write_path_host_impl(s, nullptr, k_host, v_host, dtype, batch, n_kv_heads, n_kv_heads, n_tokens, head_dim, 0, 0.0, 1,
+                                bits, group_size, k_codes_host, k_scales_host, k_zeros_host, v_codes_host, v_scales_host,
+                                v_zeros_host, meta16, nullptr, 0, workspace, workspace_bytes, stream);
 }
 
 int squat_write_path_host_ex(squat_subspace *s, const void *q_host, const void *k_host, const void *v_host,
@@ -677,6 +711,7 @@ int squat_write_path_host_ex(squat_subspace *s, const void *q_host, const void *
                              void *workspace, size_t workspace_bytes, void *stream)
 {
     if (meta16 != 0 && meta16 != 1) return SQUAT_ERR_INVALID_ARG;
+    if (!q_host) return SQUAT_ERR_INVALID_ARG;
     return write_path_host_impl(s, q_host, k_host, v_host, dtype, batch, n_q_heads, n_kv_heads, n_tokens, head_dim, rank_r,
                                 lambda, block_g, bits, group_size, k_codes_host, k_scales_host, k_zeros_host, v_codes_host,
                                 v_scales_host, v_zeros_host, meta16, start_block_host, power_iters, workspace,

@@ -84,16 +84,30 @@ __device__ __forceinline__ u64 ffma2(u64 a, u64 b, u64 c)
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
+// Warp-wide min / max.  The NaN-propagating forms: a NaN key makes the group's grid NaN, which the check of the stored
+// scale reports (SQUAT_FLAG_NONFINITE), instead of vanishing in the reduction and corrupting the codes unnoticed.
 __device__ __forceinline__ float warp_min(float x)
 {
     float r;
-    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+    asm volatile("redux.sync.min.NaN.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
     return r;
 }
 __device__ __forceinline__ float warp_max(float x)
 {
     float r;
-    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+    asm volatile("redux.sync.max.NaN.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float min_nan(float a, float b)
+{
+    float r;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ float max_nan(float a, float b)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
     return r;
 }
 __device__ __forceinline__ void team_barrier(int id, int nthreads)
@@ -203,7 +217,7 @@ struct KeyParams {
     int tiles_per_head;       // 128-token tiles per head (the last one may be ragged)
     int total_tiles;          // H * tiles_per_head
     unsigned *status;
-    int exact_blocks;         // leading 32-channel blocks that no earlier channel corrects (see sweep_block)
+    const int *exact_blocks;  // device word: leading 32-channel blocks that no earlier channel corrects (see sweep_block)
 };
 
 template <bool BF16>
@@ -277,8 +291,8 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
                 const float2 o = slot[w];
-                m = fminf(m, o.x);
-                Mx = fmaxf(Mx, o.y);
+                m = min_nan(m, o.x);
+                Mx = max_nan(Mx, o.y);
             }
         }
         const float rng = __fsub_rn(Mx, m);
@@ -368,7 +382,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
     float *images = Eall + TC_SLOTS * TC_E_FLOATS;       // [2][TC_IMG_FLOATS]: head h's image lives in buffer h & 1
     float2 *red_all = reinterpret_cast<float2 *>(images + 2 * TC_IMG_FLOATS);    // [NTEAMS][2][NW]
     u64 *mbar = reinterpret_cast<u64 *>(red_all + NTEAMS * 2 * NW);              // [TC_SLOTS] MMAs done, [1] image staged
-    // [0] tensor-memory base, [1] a bounded wait ran out, [2 + slot] arrivals of the slot's warps
+    // [0] tensor-memory base, [1] a bounded wait ran out, [2 + slot] arrivals of the slot's warps, [2 + TC_SLOTS] the
+    // number of leading blocks that take the exact rounding decision (read once from the handle's device word)
     volatile unsigned *shared_words = reinterpret_cast<volatile unsigned *>(mbar + TC_SLOTS + 1);
 
     const int lane = threadIdx.x & 31;
@@ -405,6 +420,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
         }
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(img_mbar), "r"(1) : "memory");
         shared_words[1] = 0;
+        shared_words[2 + TC_SLOTS] = (unsigned)__ldg(p.exact_blocks);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         // the first head's image is on its way while the rest of the set-up runs
         if (t_lo < t_hi) {
@@ -519,7 +535,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 const float *diag = img + blk * BLK * BLK;
                 uint32_t cw[WORDS_PER_BLK];
                 float my_scale = 0.0f, my_zero = 0.0f;
-                if (blk < p.exact_blocks)
+                if (blk < (int)shared_words[2 + TC_SLOTS])
                     sweep_block<BITS, NW, true, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
                 else
                     sweep_block<BITS, NW, false, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
@@ -600,8 +616,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
 //                    float index (k / 4) * 4 N + 4 n + k % 4 with N = 96 - 32 b
 //   [10240, 16384)   lo panels: tf32(W - hi), same layout
 // One CTA per head; each thread takes (panel, 4-k chunk, channel n): four coalesced row reads, one 16-byte store.
-__global__ void __launch_bounds__(256) pack_w_kernel(const float *__restrict__ Wt, float *__restrict__ Wimg)
+__global__ void __launch_bounds__(256) pack_w_kernel(const float *__restrict__ Wt, float *__restrict__ Wimg, int exact_blocks,
+                                                     int *__restrict__ exact_blocks_dev)
 {
+    if (blockIdx.x == 0 && threadIdx.x == 0) *exact_blocks_dev = exact_blocks;    // travels with the matrices it describes
     const float *src = Wt + (long long)blockIdx.x * D * D;
     float *img = Wimg + (long long)blockIdx.x * TC_IMG_FLOATS;
     for (int i = threadIdx.x; i < TC_DIAG_FLOATS / 4; i += blockDim.x) {
@@ -652,7 +670,7 @@ int launch_keys(KeyParams p, int dtype, int meta16, cudaStream_t st)
     // 193 KB: well over half an SM's shared memory, so two CTAs (each asking for all 512 tensor-memory columns)
     // never share an SM
     const size_t smem = sizeof(float) * (TC_SLOTS * TC_E_FLOATS + 2 * TC_IMG_FLOATS) +
-                        sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * (TC_SLOTS + 1) + 4 * (2 + TC_SLOTS) + 8;
+                        sizeof(float2) * (NTEAMS * 2 * NW) + sizeof(u64) * (TC_SLOTS + 1) + 4 * (3 + TC_SLOTS) + 8;
     const int grid = p.total_tiles < sms ? p.total_tiles : sms;                     // one tile per CTA at least
     int rc;
     if (dtype == SQUAT_BF16) rc = meta16 ? launch_keys_inst<BITS, NW, true, true>(p, grid, smem, st) : launch_keys_inst<BITS, NW, true, false>(p, grid, smem, st);
@@ -665,9 +683,9 @@ int launch_keys(KeyParams p, int dtype, int meta16, cudaStream_t st)
 
 }  // namespace
 
-int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaStream_t st)
+int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, int exact_blocks, int *exact_blocks_dev, cudaStream_t st)
 {
-    pack_w_kernel<<<H, 256, 0, st>>>(Wt, Wimg);
+    pack_w_kernel<<<H, 256, 0, st>>>(Wt, Wimg, exact_blocks, exact_blocks_dev);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
@@ -676,7 +694,7 @@ int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaS
 int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
                             unsigned char *codes, void *scales, void *zeros,
-                            long long osb, long long osh, unsigned *status, int exact_blocks, int meta16, cudaStream_t st)
+                            long long osb, long long osh, unsigned *status, const int *exact_blocks, int meta16, cudaStream_t st)
 {
     KeyParams p;
     p.Wimg = Wimg; p.k = k; p.sb = sb; p.sh = sh; p.st = st_;

@@ -12,7 +12,9 @@ struct squat_subspace {
     int head_dim;
     int device;
     int gram_chunks_cap;   // capacity (in row chunks per head) of gram_partial
-    int exact_blocks;      // leading 32-channel blocks of W that receive no correction (4 when W = 0)
+    int *exact_blocks;     // device word: leading 32-channel blocks of W that receive no correction (4 when W = 0); written in
+                           // stream order by the kernel that packs W, read by the key kernel, so it always belongs to the W it is
+                           // launched with (a host-side copy could be overtaken by a build enqueued from another thread or stream)
     float *Wt;             // [H, d, d] float32, Wt[h][j][j'] = W[j'][j]  (row j = update vector of channel j)
     float *Wimg;           // [H, d * d] the same matrices as the key kernel stages them in shared memory (see keys.cu)
     double *gram;          // [H, d, d] Gram matrices
@@ -38,15 +40,15 @@ void squat_count_launch(unsigned n = 1);
 int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads, int n_tokens,
                       long long stride_h, long long stride_t, cudaStream_t st);
 int squat_launch_eig(squat_subspace *s, cudaStream_t st);
-int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, int left_rows, cudaStream_t st);
+int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, int left_rows, int exact_blocks, cudaStream_t st);
 int squat_launch_power(squat_subspace *s, const double *start, long long start_stride_h, int rank_r, int iters,
                        double lambda, cudaStream_t st);
 
-int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, cudaStream_t st);
+int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, int exact_blocks, int *exact_blocks_dev, cudaStream_t st);
 int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
                             unsigned char *codes, void *scales, void *zeros,
-                            long long osb, long long osh, unsigned *status, int exact_blocks, int meta16, cudaStream_t st);
+                            long long osb, long long osh, unsigned *status, const int *exact_blocks_dev, int meta16, cudaStream_t st);
 int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T, int d,
                               long long sb, long long sh, long long st_, int bits, int G,
                               unsigned char *codes, void *scales, void *zeros,

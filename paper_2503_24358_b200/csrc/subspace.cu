@@ -697,14 +697,14 @@ int squat_launch_eig(squat_subspace *s, cudaStream_t st)
     return SQUAT_OK;
 }
 
-int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, int left_rows, cudaStream_t st)
+int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int block_g, int left_rows, int exact_blocks, cudaStream_t st)
 {
     const size_t smem = sizeof(double) * (D * ASM_LD + 5 * D + 64 * D);
     SQUAT_CUDA(cudaFuncSetAttribute(assemble_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     assemble_kernel<<<s->n_kv_heads, ASM_THREADS, smem, st>>>(s->eigval, s->eigvec, rank_r, lambda, block_g, s->Wt, left_rows);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
-    return squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, st);
+    return squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, exact_blocks, s->exact_blocks, st);
 }
 
 // ------------------------------------------------------------------------- allocation-free Gram entry

@@ -28,6 +28,11 @@ __device__ __forceinline__ void unpk2(u64 v, float &lo, float &hi) { asm("mov.b6
 __device__ __forceinline__ u64 sub2(u64 a, u64 b) { u64 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) { u64 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 
+// NaN-propagating min / max: a NaN input makes the group's scale NaN, which is reported (SQUAT_FLAG_NONFINITE) and gives
+// codes 0, instead of being dropped by the reduction.
+__device__ __forceinline__ float min_nan(float a, float b) { float r; asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ float max_nan(float a, float b) { float r; asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r; }
+
 // Exact binary32 decision for one element next to a rounding midpoint (rare; kept out of line).
 template <int BITS>
 __device__ __noinline__ uint32_t exact_code_bits(float dlt, float delta)
@@ -111,15 +116,15 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
                 for (int k = 0; k < 4; ++k) {
                     const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[k]);
                     if (i == 0 && k == 0) { mn2 = pr; mx2 = pr; }
-                    else { mn2 = __hmin2(mn2, pr); mx2 = __hmax2(mx2, pr); }
+                    else { mn2 = __hmin2_nan(mn2, pr); mx2 = __hmax2_nan(mx2, pr); }
                 }
             }
-            m = fminf(__low2float(mn2), __high2float(mn2));
-            Mx = fmaxf(__low2float(mx2), __high2float(mx2));
+            m = min_nan(__low2float(mn2), __high2float(mn2));
+            Mx = max_nan(__low2float(mx2), __high2float(mx2));
         } else {
             m = raw.get(0); Mx = m;
 #pragma unroll
-            for (int i = 1; i < G; ++i) { m = fminf(m, raw.get(i)); Mx = fmaxf(Mx, raw.get(i)); }
+            for (int i = 1; i < G; ++i) { m = min_nan(m, raw.get(i)); Mx = max_nan(Mx, raw.get(i)); }
         }
 
         float delta = __fdiv_rn(__fsub_rn(Mx, m), L);
@@ -134,6 +139,7 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
         // two channels per instruction (packed f32x2): dlt = x - m, y = dlt * rcp + magic, c = y - magic,
         // res = dlt * rcp - c; each half is the same IEEE operation as its scalar form
         const u64 m2 = pk2(m, m), rcp2 = pk2(rcp, rcp), magic2 = pk2(kMagic, kMagic);
+        const uint32_t cmask = ok ? ((1u << BITS) - 1u) : 0u;       // no grid (constant or non-finite group): codes 0
         uint32_t words[NWORDS];
 #pragma unroll
         for (int wd = 0; wd < NWORDS; ++wd) {
@@ -152,8 +158,8 @@ __global__ void __launch_bounds__(256) quant_values_kernel(
                     ylo = fminf(fmaxf(ylo, kMagic), kMagic + L);
                     yhi = fminf(fmaxf(yhi, kMagic), kMagic + L);
                 }
-                uint32_t cb0 = __float_as_uint(ylo) & ((1u << BITS) - 1u);
-                uint32_t cb1 = __float_as_uint(yhi) & ((1u << BITS) - 1u);
+                uint32_t cb0 = __float_as_uint(ylo) & cmask;
+                uint32_t cb1 = __float_as_uint(yhi) & cmask;
                 // next to a rounding midpoint (structural with coarse bf16 data): the exact sequence decides
                 if (fmaxf(fabsf(rlo), fabsf(rhi)) >= kTieBand && ok) {
                     float dlo, dhi;

@@ -190,7 +190,7 @@ def main():
         "scale / zero, max rel. err. |",
         "|---|---|---|---|---|---|---|---|---|---|---|---|",
     ]
-    tail = ["", f"Device status word after the run: {flags:#x} (bit 0 = a constant group was seen; no other bit may be set)."]
+    tail = ["", f"Device status word after the run: {flags:#x} (0x2 = a constant group was seen; no other bit may be set)."]
     out = os.path.join(HERE, "parity_results.md")
     with open(out, "w") as f:
         f.write("\n".join(head + rows + tail) + "\n")

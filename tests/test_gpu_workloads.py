@@ -203,6 +203,34 @@ def test_host_buffer_entry_variants_equal_device_calls():
     sq.squat_get_device_status(clear=True)
 
 
+def test_append_window_host_equals_device_calls():
+    # squat_append_window_host = H2D copies of one decode window + keys + values + D2H copies, with the update matrices
+    # the handle already holds (nothing is rebuilt): byte-identical to the device calls, both metadata types
+    cfg = si.get_config(3).with_(batch=3, n_kv_heads=4, n_q_heads=4, n_tokens=256)
+    B, H, bits, G, W = cfg.batch, cfg.n_kv_heads, cfg.bits, cfg.group_size, 128
+    s = sq.Subspace(H, D)
+    sq.squat_build_subspace(s, to_torch(si.gen_queries(cfg), cfg.dtype), cfg.rank_r, cfg.lam, cfg.block_g)
+    ws = torch.empty(sq.squat_write_path_workspace_bytes(torch.bfloat16, B, H, H, W, D, bits, G), dtype=torch.uint8, device="cuda")
+    for seg, m16 in ((1, False), (2, True)):
+        k_np, v_np = si.gen_keys(cfg, n_tokens=W, segment=seg), si.gen_values(cfg, n_tokens=W, segment=seg)
+        kc, ks, kz = alloc_key_outputs(B, H, W, D, bits, G)
+        vc, vs, vz = alloc_value_outputs(B, H, W, D, bits, G)
+        if m16:
+            ks, kz, vs, vz = (t.to(torch.float16) for t in (ks, kz, vs, vz))
+        sq.squat_quantize_keys(s, to_torch(k_np, cfg.dtype), bits, G, kc, ks, kz)
+        sq.squat_quantize_values(to_torch(v_np, cfg.dtype), bits, G, vc, vs, vz)
+        torch.cuda.synchronize()
+        host_in = [to_torch(a, cfg.dtype, device="cpu").pin_memory() for a in (k_np, v_np)]
+        host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in (kc, ks, kz, vc, vs, vz)]
+        sq.squat_append_window_host(s, *host_in, bits, G, *host_out, ws)
+        for dev_t, host_t in zip((kc, ks, kz, vc, vs, vz), host_out):
+            assert torch.equal(dev_t.cpu(), host_t), m16
+    with pytest.raises(sq.SquatError):
+        sq.squat_append_window_host(s, *host_in, bits, G, *host_out, ws[:1024])
+    sq.squat_get_device_status(clear=True)
+    s.close()
+
+
 def test_write_path_captures_into_a_cuda_graph_and_replays_identically():
     # no call of the write path allocates, synchronises or touches the host: the whole step records into a CUDA graph
     cfg = si.get_config(0)

@@ -34,13 +34,18 @@ def _reference_gram(cfg, q):
 def test_gram_static_matches_the_allocating_entry_twice_in_a_row():
     first = si.get_config(1).with_(n_kv_heads=32, n_q_heads=32, n_tokens=1024)      # 32 heads, 2 chunks each
     second = si.get_config(2).with_(n_kv_heads=4, n_q_heads=16, n_tokens=160)       # GQA, fewer units, ragged rows
-    for cfg in (first, second):
+    third = si.get_config(0).with_(n_kv_heads=64, n_q_heads=64, n_tokens=96)        # float32 queries; 64 heads: every unit of the scratch, one chunk each
+    for i, cfg in enumerate((first, second, third)):
         q = to_torch(si.gen_queries(cfg), cfg.dtype)
         out = torch.full((cfg.n_kv_heads, 128, 128), float("nan"), dtype=torch.float64, device="cuda")
+        torch.cuda.synchronize()
         before = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]       # the driver's own count of free device memory: sees any cudaMalloc
         sq.squat_gram_static(q, cfg.n_kv_heads, out)
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before
+        if i > 0:                                        # (the very first call of a process may load the kernels' module)
+            assert torch.cuda.mem_get_info()[0] == free_before
         got = out.cpu().numpy()
         ref = _reference_gram(cfg, q)
         assert np.isfinite(got).all()
