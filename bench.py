@@ -420,6 +420,7 @@ def run_gpu(args, cfg):
         sq.squat_dequantize(sq.SQUAT_VALUES, vc, vs, vz, B, H, Tc, d, bits, G, vd)
         if ev: ev[2 + 2 * NW].record(stream)
 
+    sq.squat_subspace_select_key_kernel(s, args.dense_keys)
     fp32_peak = measure_fp32_peak(sq, dev) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
         flush.zero_()
@@ -482,6 +483,9 @@ def run_gpu(args, cfg):
             "sequence_key_vectors_per_s": B * H * Tc / (statistics.mean(seq_ms) * 1e-3),
             "timing": "CUDA events on the launching stream between consecutive calls: launch gaps are inside the intervals",
             "distinct_window_tensors": NDIST}
+    lowrank_r = sq.squat_subspace_select_key_kernel(s, args.dense_keys)      # which key kernel the steps ran (0: the dense one)
+    if args.dense_keys:
+        lowrank_r = 0
     local_ms = sum(step_ms)
     vec_per_step = B * H * Tc              # key vectors one step really quantizes
     total_ms, total_units = aggregate_over_ranks(local_ms, vec_per_step * args.steps, dev)
@@ -521,7 +525,7 @@ def run_gpu(args, cfg):
     if rank == 0:
         key_launch_ms = stage_ms["quantize_keys"] / NW
         report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, B * H * W, key_launch_ms,
-               e2e, launches, wall, flags, clocks, fp32_peak, reader, power, stream_stats)
+               e2e, launches, wall, flags, clocks, fp32_peak, reader, power, stream_stats, lowrank_r)
     s.close()
     if world > 1:
         dist.destroy_process_group()
@@ -649,7 +653,7 @@ def run_reader(cfg, sq, cache, T, flush, tdt, dev, iters=10, meta_bytes=4):
                          "slowdown": ms_pre / ms}}
 
 
-def key_roofline(args, cfg, key_ms, vec_per_launch, peaks, fp32_peak):
+def key_roofline(args, cfg, key_ms, vec_per_launch, peaks, fp32_peak, lowrank_r=0):
     """The roofline of the key kernel: the slowest of (the multiply-adds it runs on the FP32 pipes at the FP32 peak
     measured in this run, three tf32 products per cross-block multiply-add at the tf32 peak, the bytes at the measured
     HBM copy bandwidth) against the measured time of one launch.  `frac` = achieved / peak on the pipe that sets that
@@ -662,6 +666,8 @@ def key_roofline(args, cfg, key_ms, vec_per_launch, peaks, fp32_peak):
     alg_flops = key_flops_per_vector(d, cfg.block_g, cfg.rank_r) * vec_per_launch
     kbytes = bytes_per_vector(d, bits, G, elem, mb) * vec_per_launch
     alu_fma, tensor_fma = key_fma_split(d, cfg.block_g)
+    if lowrank_r > 0:
+        alu_fma, tensor_fma = 2 * lowrank_r * d, 0                # the rank-r form: state of r numbers per token, FP32 pipes only
     if cfg.rank_r == 0 or cfg.lam == 0.0:
         alu_fma = tensor_fma = 0                                  # W = 0: nothing to push
     fp32_tflops = fp32_peak["tflops"] if fp32_peak else ALU_PEAK_TFLOPS
@@ -687,7 +693,7 @@ def key_roofline(args, cfg, key_ms, vec_per_launch, peaks, fp32_peak):
             "frac_vs_fp32_target_definition": "all %d algorithmic flop per vector (2 x min(dense triangle, 2 r d)) at the nominal "
                                               "FP32 peak of %.2f TFLOP/s: the reading the 50 %% target was stated in"
                                               % (key_flops_per_vector(d, cfg.block_g, cfg.rank_r), ALU_PEAK_TFLOPS),
-            "traffic": None, "kernel": "quant_keys_kernel", "ms_per_launch": key_ms, "key_vectors_per_launch": vec_per_launch,
+            "traffic": None, "kernel": "quant_keys_lowrank_kernel (rank-r form of the update)" if lowrank_r > 0 else "quant_keys_kernel", "ms_per_launch": key_ms, "key_vectors_per_launch": vec_per_launch,
             "key_vectors_per_s": vec_per_launch / t_s, "kv_input_gbs": vec_per_launch * d * elem / t_s / 1e9,
             "hbm_frac_of_" + peaks["source"]: kbytes / t_s / 1e9 / peaks["hbm_gbs"]}
     tr = key_kernel_traffic(cfg, args)
@@ -699,13 +705,13 @@ def key_roofline(args, cfg, key_ms, vec_per_launch, peaks, fp32_peak):
 
 
 def report(args, cfg, world, total_ms, total_units, step_ms, stage_ms, stage_names, vec_per_step, vec_per_launch, key_launch_ms,
-           e2e, launches, wall, flags, clocks, fp32_peak, reader=None, power=None, stream_stats=None):
+           e2e, launches, wall, flags, clocks, fp32_peak, reader=None, power=None, stream_stats=None, lowrank_r=0):
     d, bits, G = cfg.head_dim, cfg.bits, cfg.group_size
     if rank_is_zero():
         peaks = measured_peaks()
         elem = 4 if cfg.dtype == "f32" else 2
         mb = 2 if args.meta16 else 4
-        roof = key_roofline(args, cfg, key_launch_ms, vec_per_launch, peaks, fp32_peak)
+        roof = key_roofline(args, cfg, key_launch_ms, vec_per_launch, peaks, fp32_peak, lowrank_r)
         # the HBM-bound stages, for the record
         vbytes = bytes_per_vector(d, bits, G, elem, mb) * vec_per_step
         dq_bytes = 2 * (d * bits // 8 + 2 * mb * d // G + d * elem) * vec_per_step
@@ -752,6 +758,8 @@ def main():
     ap.add_argument("--subspace", default="svd", choices=["svd", "power"], help="step 1: the paper's SVD (default) or the "
                     "block power method it names as an accelerator")
     ap.add_argument("--power-iters", type=int, default=2, help="multiplications by the Gram matrix of the block power method")
+    ap.add_argument("--dense-keys", action="store_true", help="run the dense key kernel also where the rank-r form of the "
+                    "update is available (small ranks)")
     ap.add_argument("--impl", default="squat", choices=["squat", "reference"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")

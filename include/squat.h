@@ -164,6 +164,21 @@ int squat_quantize_keys(const squat_subspace *s, const void *k, int dtype, int b
                         void *stream);
 
 /*
+ * Which kernel squat_quantize_keys runs.  For element-wise updates (block_g = 1) the update matrix of Prop. 1 is
+ * semiseparable, W[j'][j] = v_j' . c_j (the Woodbury identity the footnote to Prop. 4 points to, applied to the
+ * trailing blocks of P): a token then carries a state of r numbers and the update costs 2 r d multiply-adds per key
+ * vector instead of d (d - 1) / 2.  squat_build_subspace and squat_build_subspace_from_gram prepare that form when
+ * block_g = 1, lambda > 0 and 1 <= rank_r <= 8, and squat_quantize_keys / _m16 then use it (FP32 pipes only, no
+ * tensor-core hand-over); every other build, and an imported W, runs the dense kernel.  Both compute the same
+ * function Quant; results agree up to rounding ties.
+ *   prefer_dense   1: always run the dense kernel;  0: the default choice above.
+ *   lowrank_rank   host, may be NULL: receives the rank the rank-r form is prepared for (0: not prepared).
+ * Host-side state of the handle: like every call that takes the handle, issue it from one thread at a time, in the
+ * order the work is to execute.
+ */
+int squat_subspace_select_key_kernel(squat_subspace *s, int prefer_dense, int *lowrank_rank);
+
+/*
  * Step 3 -- per-token value quantization  (Section 2 "Quantization"; Appendix C: each token's d
  * channels in d/G groups of G).  Every operation is IEEE binary32 in the order
  *   Delta = (M - m) / L;  t = (x - m) / Delta;  c = clamp(rint(t), 0, L).

@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     squat_get_device_status, squat_gram_static, squat_kernel_launch_count, squat_quantize_keys, squat_quantize_values,
     squat_subspace_eig_sweeps, squat_subspace_export, squat_subspace_import, squat_write_path_host, squat_write_path_workspace_bytes,
     squat_decode_attention, squat_decode_attention_workspace_bytes, squat_decode_attention_pre_rope, squat_rope_table,
-    squat_build_subspace_from_gram, squat_build_subspace_power, squat_build_subspace_power_from_gram, squat_build_subspace_sharded, token_shard, squat_fp32_peak_probe, squat_append_window_host,
+    squat_build_subspace_from_gram, squat_build_subspace_power, squat_build_subspace_power_from_gram, squat_build_subspace_sharded, token_shard, squat_fp32_peak_probe, squat_append_window_host, squat_subspace_select_key_kernel,
 )

@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
     "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_write_path_host_ex", "squat_build_subspace_power_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
-    "squat_fp32_peak_probe", "squat_append_window_host",
+    "squat_fp32_peak_probe", "squat_append_window_host", "squat_subspace_select_key_kernel",
 )
 
 _lib = None
@@ -84,6 +84,7 @@ def _load():
         lib.squat_decode_attention_ex.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, i, ll, ll, i, i, vp, vp, i, i,
                                                   c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
         lib.squat_append_window_host.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, c.c_size_t, vp]
+        lib.squat_subspace_select_key_kernel.argtypes = [vp, i, c.POINTER(i)]
         lib.squat_fp32_peak_probe.argtypes = [i, i, vp, c.POINTER(ll), vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
@@ -304,6 +305,15 @@ def squat_append_window_host(s: Subspace, k, v, bits, group_size, k_codes, k_sca
                                             int(m16), _dev(workspace, "workspace"),
                                             workspace.numel() * workspace.element_size(), _stream(stream)),
            "squat_append_window_host")
+
+
+def squat_subspace_select_key_kernel(s: "Subspace", prefer_dense: bool = False) -> int:
+    """Chooses the kernel squat_quantize_keys runs on this handle (True: always the dense one; False: the rank-r form
+    where the last build prepared it).  Returns the rank the rank-r form is prepared for (0: not prepared)."""
+    r = ctypes.c_int(0)
+    _check(_load().squat_subspace_select_key_kernel(s.handle, 1 if prefer_dense else 0, ctypes.byref(r)),
+           "squat_subspace_select_key_kernel")
+    return int(r.value)
 
 
 def squat_fp32_peak_probe(packed: bool, iters: int, sink: torch.Tensor, stream=None) -> int:

@@ -8,7 +8,7 @@ CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 OBJ_DIR = os.path.join(_HERE, "build")
 LIB = os.path.join(_HERE, "libsquat.so")
-SOURCES = ["api.cu", "values.cu", "keys.cu", "subspace.cu", "power.cu", "attention.cu", "peak.cu"]
+SOURCES = ["api.cu", "values.cu", "keys.cu", "subspace.cu", "power.cu", "attention.cu", "peak.cu", "keys_lowrank.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE]
 

@@ -47,6 +47,17 @@ int check_quant_args(const void *x, int dtype, int batch, int H, int T, int d, l
     return SQUAT_OK;
 }
 
+// The rank-r form of the update (keys_lowrank.cu) exists for element-wise updates with a small rank: its tables are
+// made from the eigen-pairs right after the eigensolver.  Every other build leaves the handle on the dense kernel.
+int lowrank_tables_if_small(squat_subspace *s, int rank_r, double lambda, int block_g, cudaStream_t st)
+{
+    s->lowrank_r = 0;
+    if (block_g != 1 || rank_r < 1 || rank_r > SQUAT_LOWRANK_MAX_R || !(lambda > 0.0)) return SQUAT_OK;
+    const int rc = squat_launch_lowrank_tables(s, rank_r, lambda, st);
+    if (rc == SQUAT_OK) s->lowrank_r = rank_r;
+    return rc;
+}
+
 }  // namespace
 
 int squat_cuda_fail(cudaError_t e)
@@ -117,6 +128,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     const size_t o_vec = carve(hdd * sizeof(double));
     const size_t o_swp = carve((size_t)n_kv_heads * sizeof(int));
     const size_t o_exact = carve(sizeof(int));
+    const size_t o_lr = carve((size_t)n_kv_heads * D * 2 * SQUAT_LOWRANK_MAX_R * sizeof(float));
     char *base = nullptr;
     if (cudaMalloc(&base, off) != cudaSuccess) { cudaGetLastError(); delete s; return SQUAT_ERR_ALLOC; }
     if (cudaMemset(base, 0, off) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
@@ -128,6 +140,7 @@ int squat_subspace_create(int n_kv_heads, int head_dim, squat_subspace **out)
     s->eigvec = reinterpret_cast<double *>(base + o_vec);
     s->eig_sweeps = reinterpret_cast<int *>(base + o_swp);
     s->exact_blocks = reinterpret_cast<int *>(base + o_exact);
+    s->lr_table = reinterpret_cast<float *>(base + o_lr);
     const int all_exact = D / 32;        // W starts as zero: every channel is uncorrected
     if (cudaMemcpy(s->exact_blocks, &all_exact, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) { cudaFree(base); delete s; return SQUAT_ERR_CUDA; }
     s->status = squat_status_word();
@@ -167,6 +180,8 @@ int squat_build_subspace(squat_subspace *s, const void *q, int dtype, int n_q_he
     if (rc != SQUAT_OK) return rc;
     rc = squat_launch_eig(s, st);
     if (rc != SQUAT_OK) return rc;
+    rc = lowrank_tables_if_small(s, rank_r, lambda, block_g, st);
+    if (rc != SQUAT_OK) return rc;
     // channels of the first g-block are never corrected; with r = 0 or lambda = 0, W = 0 and none is
     const int exact = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
     return squat_launch_assemble(s, rank_r, lambda, block_g, 0, exact, st);
@@ -184,6 +199,8 @@ int squat_build_subspace_from_gram(squat_subspace *s, const double *gram, int ra
     if (gram != s->gram)
         SQUAT_CUDA(cudaMemcpyAsync(s->gram, gram, (size_t)s->n_kv_heads * D * D * sizeof(double), cudaMemcpyDeviceToDevice, st));
     int rc = squat_launch_eig(s, st);
+    if (rc != SQUAT_OK) return rc;
+    rc = lowrank_tables_if_small(s, rank_r, lambda, block_g, st);
     if (rc != SQUAT_OK) return rc;
     const int exact = (rank_r == 0 || lambda == 0.0) ? D / 32 : (block_g + 31) / 32;
     return squat_launch_assemble(s, rank_r, lambda, block_g, 0, exact, st);
@@ -211,6 +228,7 @@ int squat_build_subspace_power(squat_subspace *s, const void *q, int dtype, int 
     int rc = squat_launch_gram(s, q, dtype, n_q_heads, n_tokens, stride_h, stride_t, st);
     if (rc != SQUAT_OK) return rc;
     const bool no_update = rank_r == 0 || lambda == 0.0;
+    s->lowrank_r = 0;                      // the iterated basis is no eigenbasis: dense kernel
     const int exact = no_update ? D / 32 : (block_g + 31) / 32;
     if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, exact, st);      // W = 0: nothing to iterate
     rc = squat_launch_power(s, start_block, start_stride_h, rank_r, iters, lambda, st);
@@ -234,6 +252,7 @@ int squat_build_subspace_power_from_gram(squat_subspace *s, const double *gram, 
     if (gram != s->gram)
         SQUAT_CUDA(cudaMemcpyAsync(s->gram, gram, (size_t)s->n_kv_heads * D * D * sizeof(double), cudaMemcpyDeviceToDevice, st));
     const bool no_update = rank_r == 0 || lambda == 0.0;
+    s->lowrank_r = 0;                      // the iterated basis is no eigenbasis: dense kernel
     const int exact = no_update ? D / 32 : (block_g + 31) / 32;
     if (no_update) return squat_launch_assemble(s, 0, lambda, block_g, 0, exact, st);
     int rc = squat_launch_power(s, start_block, start_stride_h, rank_r, iters, lambda, st);
@@ -262,6 +281,14 @@ int squat_subspace_export(const squat_subspace *s, void *stream, float *W_host, 
             for (int j = 0; j < D; ++j)
                 for (int jp = 0; jp < D; ++jp)
                     W_host[((size_t)h * D + jp) * D + j] = wt[((size_t)h * D + j) * D + jp];
+    return SQUAT_OK;
+}
+
+int squat_subspace_select_key_kernel(squat_subspace *s, int prefer_dense, int *lowrank_rank)
+{
+    if (!s || (prefer_dense != 0 && prefer_dense != 1)) return SQUAT_ERR_INVALID_ARG;
+    s->prefer_dense = prefer_dense;
+    if (lowrank_rank) *lowrank_rank = s->lowrank_r;
     return SQUAT_OK;
 }
 
@@ -294,6 +321,7 @@ int squat_subspace_import(squat_subspace *s, const float *W_host, void *stream)
             for (int j = 0; j < D; ++j)
                 if (W_host[((size_t)h * D + jp) * D + j] != 0.0f) { uncorrected = jp; break; }
     const int exact = (uncorrected + 31) / 32;
+    s->lowrank_r = 0;                      // an imported W comes without its factors: dense kernel
     SQUAT_CUDA(cudaMemcpyAsync(s->Wt, wt.data(), hdd * sizeof(float), cudaMemcpyHostToDevice, st));
     int rc = squat_launch_pack_update_matrices(s->Wt, s->Wimg, s->n_kv_heads, exact, s->exact_blocks, st);
     if (rc != SQUAT_OK) return rc;
@@ -318,6 +346,10 @@ int quantize_keys_impl(const squat_subspace *s, const void *k, int dtype, int ba
     if (n_tokens % group_size != 0 || out_stride_b % group_size != 0 || out_stride_h % group_size != 0)
         return SQUAT_ERR_SHAPE;
     if (batch == 0 || n_tokens == 0) return SQUAT_OK;
+    if (s->lowrank_r > 0 && !s->prefer_dense)
+        return squat_launch_quant_keys_lowrank(s->lr_table, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t,
+                                               bits, group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status,
+                                               meta16, static_cast<cudaStream_t>(stream));
     return squat_launch_quant_keys(s->Wimg, k, dtype, batch, n_kv_heads, n_tokens, stride_b, stride_h, stride_t, bits,
                                    group_size, codes, scales, zeros, out_stride_b, out_stride_h, s->status, s->exact_blocks,
                                    meta16, static_cast<cudaStream_t>(stream));

@@ -6,6 +6,7 @@
 #include "../../include/squat.h"
 
 #define SQUAT_D 128   // the only head dimension the key path and the subspace build are built for
+#define SQUAT_LOWRANK_MAX_R 8   // largest subspace rank the rank-r form of the key quantizer is built for (keys_lowrank.cu)
 
 struct squat_subspace {
     int n_kv_heads;
@@ -17,6 +18,10 @@ struct squat_subspace {
                            // launched with (a host-side copy could be overtaken by a build enqueued from another thread or stream)
     float *Wt;             // [H, d, d] float32, Wt[h][j][j'] = W[j'][j]  (row j = update vector of channel j)
     float *Wimg;           // [H, d * d] the same matrices as the key kernel stages them in shared memory (see keys.cu)
+    float *lr_table;       // [H, d, 2 * SQUAT_LOWRANK_MAX_R] rows [v_j | c_j] of the rank-r form of W (keys_lowrank.cu)
+    int lowrank_r;         // > 0: lr_table describes the same update as Wt (set by the SVD builds with g = 1 and a small rank);
+                           // host-side, read when a key call is enqueued: calls on one handle are issued in execution order
+    int prefer_dense;      // 1: squat_quantize_keys uses the dense kernel even when lr_table is valid
     double *gram;          // [H, d, d] Gram matrices
     double *gram_partial;  // [chunks, H, d, d] per-chunk partial Gram matrices (deterministic reduction)
     double *eigval;        // [H, d] descending
@@ -44,6 +49,11 @@ int squat_launch_assemble(squat_subspace *s, int rank_r, double lambda, int bloc
 int squat_launch_power(squat_subspace *s, const double *start, long long start_stride_h, int rank_r, int iters,
                        double lambda, cudaStream_t st);
 
+int squat_launch_lowrank_tables(squat_subspace *s, int rank_r, double lambda, cudaStream_t st);
+int squat_launch_quant_keys_lowrank(const float *table, const void *k, int dtype, int batch, int H, int T,
+                                    long long sb, long long sh, long long st_, int bits, int G,
+                                    unsigned char *codes, void *scales, void *zeros,
+                                    long long osb, long long osh, unsigned *status, int meta16, cudaStream_t st);
 int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, int exact_blocks, int *exact_blocks_dev, cudaStream_t st);
 int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int batch, int H, int T,
                             long long sb, long long sh, long long st_, int bits, int G,
