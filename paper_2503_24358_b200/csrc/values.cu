@@ -1,15 +1,19 @@
 // Per-token value quantization (Section 2 "Quantization"; Appendix C: d channels of a token in
 // d/G groups of G) and dequantization (deq(c) = c * Delta + m) for both cache layouts.
 //
-// HBM-bound streaming kernels.  One thread owns one (token, channel-group): it reads its G
-// consecutive channels with 128-bit loads (consecutive lanes read consecutive 16*G/8-byte
-// pieces, so a warp covers a contiguous span), reduces min/max in registers, and writes
-// G*b/8 code bytes plus one scale and one zero -- all contiguous across the warp.
+// HBM-bound streaming kernels, written to spend few instructions per element (the first version of the quantizer
+// needed 15 per element and was bound by instruction issue at 70 % of the copy bandwidth).
 //
-// The rounding decision is the IEEE binary32 sequence  Delta = (M-m)/L, t = (x-m)/Delta,
-// c = clamp(rint(t), 0, L).  The fast path multiplies by RN(1/Delta) and rounds once; it can
-// differ from the sequence above only when t is within ~1e-6 of a half-integer, so any
-// element within 1e-5 of one is redone with a correctly rounded division.
+// Quantizer.  A thread owns one 16-byte piece of the input (8 bf16 or 4 float32 channels), so a warp's load is one
+// contiguous 512-byte span; the G channels of a group lie in G/8 (G/4) neighbouring lanes, which reduce min / max
+// with warp shuffles.  The rounding decision is the IEEE binary32 sequence
+//     Delta = (M - m) / L,   t = (x - m) / Delta,   c = clamp(rint(t), 0, L).
+// Fast path: t is bracketed by  (x - m) * r (1 +- 2^-20)  with r the hardware reciprocal of Delta (1 ulp); both ends are
+// rounded to integers by adding 1.5 * 2^23 (one fma each, ties to even).  rint is monotonic, so where the two ends
+// agree that integer is rint(t); where they differ for any element of the piece (t within 1e-6 relative of a
+// rounding midpoint -- structural with coarse bf16 data) the piece is redone with correctly rounded divisions.
+// The codes are packed by integer shift-adds of the rounded floats' bit patterns (the constant upper bits are
+// subtracted once).
 //
 // M16 instances store scale and zero-point as IEEE binary16 (the 18.75 % cache of the paper's "KV size" columns):
 // Delta = half(Delta32), z = half(m), and the decision t = (x - z) / Delta is taken against those stored values,
@@ -20,7 +24,7 @@
 namespace {
 
 constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
-constexpr float kTieBand = 0.5f - 1e-5f;
+constexpr unsigned kMagicBits = 0x4B400000u;
 
 typedef unsigned long long u64;
 __device__ __forceinline__ u64 pk2(float lo, float hi) { u64 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
@@ -32,8 +36,29 @@ __device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) { u64 d; asm("fma.rn.f3
 // codes 0, instead of being dropped by the reduction.
 __device__ __forceinline__ float min_nan(float a, float b) { float r; asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r; }
 __device__ __forceinline__ float max_nan(float a, float b) { float r; asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ unsigned hmin2_nan_bits(unsigned a, unsigned b)
+{
+    const __nv_bfloat162 r = __hmin2_nan(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+    return *reinterpret_cast<const unsigned *>(&r);
+}
+__device__ __forceinline__ unsigned hmax2_nan_bits(unsigned a, unsigned b)
+{
+    const __nv_bfloat162 r = __hmax2_nan(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+    return *reinterpret_cast<const unsigned *>(&r);
+}
 
-// Exact binary32 decision for one element next to a rounding midpoint (rare; kept out of line).
+// Correctly rounded  rng / L  for L = 3 or 15 and rng, rng / L in the normal range (q' = q + (rng - L q) * RN(1/L)).
+template <int BITS>
+__device__ __forceinline__ float div_by_levels(float rng)
+{
+    constexpr float L = float((1 << BITS) - 1);
+    constexpr float invL = 1.0f / L;
+    const float q = __fmul_rn(rng, invL);
+    const float r = __fmaf_rn(-L, q, rng);
+    return __fmaf_rn(r, invL, q);
+}
+
+// Exact binary32 decision for one element (rare; kept out of line).
 template <int BITS>
 __device__ __noinline__ uint32_t exact_code_bits(float dlt, float delta)
 {
@@ -41,215 +66,273 @@ __device__ __noinline__ uint32_t exact_code_bits(float dlt, float delta)
     return (uint32_t)(int)fminf(fmaxf(rintf(__fdiv_rn(dlt, delta)), 0.0f), L);
 }
 
-template <int G, bool BF16>
-struct ValRaw {
-    static constexpr int NV = BF16 ? G / 8 : G / 4;      // 128-bit pieces of one group
-    uint4 v[NV];
-    __device__ __forceinline__ float get(int i) const     // channel i of the group, exact widening
-    {
-        if (BF16) {
-            const uint4 &r = v[i / 8];
-            const uint32_t w = (i % 8) / 2 == 0 ? r.x : (i % 8) / 2 == 1 ? r.y : (i % 8) / 2 == 2 ? r.z : r.w;
-            return (i & 1) ? bf16hi_to_f32(w) : bf16lo_to_f32(w);
-        } else {
-            const uint4 &r = v[i / 4];
-            const uint32_t w = i % 4 == 0 ? r.x : i % 4 == 1 ? r.y : i % 4 == 2 ? r.z : r.w;
-            return __uint_as_float(w);
-        }
-    }
+struct ValParams {
+    const void *v;
+    int H, T, ng;                         // ng = groups per token
+    int ng_shift;                         // log2(ng) when ng is a power of two, else -1
+    unsigned chunks_per_row;              // CTAs per (batch, head) row
+    long long sb, sh, st;                 // element strides of v
+    unsigned char *codes;
+    void *scales, *zeros;
+    long long osb, osh;                   // output strides in tokens
+    int row_bytes;                        // code bytes per token
+    unsigned *status;
 };
 
-template <int G, int BITS, bool BF16, bool M16>
-__global__ void __launch_bounds__(256) quant_values_kernel(
-    const void *__restrict__ v, long long n_units, int H, int T, int ng,
-    long long sb, long long sh, long long st, unsigned char *__restrict__ codes,
-    void *__restrict__ scales, void *__restrict__ zeros, long long osb, long long osh,
-    int row_bytes, unsigned *__restrict__ status)
+constexpr int VAL_THREADS = 256;
+
+// The rare path of the quantizer, out of line so that the streaming code stays small.  `mask` has one bit set (at the
+// element's bit position in the packed word) for every element of the word whose fast path could not decide; each is
+// re-read from memory (it is in L1) and decided here, and its field of `word` replaced.  A scale outside the fast
+// path's range (`fast` false, every element flagged): the exact sequence.  Else the element sits next to a rounding
+// midpoint k + 1/2 (structural with coarse bf16 data): the sign of the exact remainder (x - m) - (k + 1/2) Delta (one
+// fma: the product has at most 29 significant bits) says on which side the quotient lies; a zero remainder is an exact
+// tie and goes to the even code; a remainder too small to be sure that the ROUNDED quotient is not the midpoint itself
+// takes the correctly rounded division.
+template <int BITS, bool BF16, bool M16>
+__device__ __noinline__ unsigned patch_word(unsigned word, unsigned mask, const void *elems, float m, float delta, float ra,
+                                            float rb, bool fast)
 {
     constexpr float L = float((1 << BITS) - 1);
-    constexpr int PER_WORD = 32 / BITS;
-    constexpr int NWORDS = G / PER_WORD;
-    using Raw = ValRaw<G, BF16>;
-    constexpr bool PREFETCH = false;              // keep the next unit's data in flight while this one computes
-    const long long stride = (long long)gridDim.x * blockDim.x;
-
-    auto in_ptr = [&](long long u) -> const uint4 * {
-        const int q = (int)(u % ng);
-        const long long tok = u / ng;
-        const int t = (int)(tok % T);
-        const long long bh = tok / T;
-        const long long off = (bh / H) * sb + (bh % H) * sh + (long long)t * st + (long long)q * G;
-        return BF16 ? reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(v) + off)
-                    : reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(v) + off);
-    };
-    auto load = [&](Raw &r, long long u) {
-        const uint4 *p = in_ptr(u);
-#pragma unroll
-        for (int i = 0; i < Raw::NV; ++i) r.v[i] = ldg128(p + i);
-    };
-
-    long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    Raw nxt;
-    if (PREFETCH && u < n_units) load(nxt, u);
-    for (; u < n_units; u += stride) {
-        Raw raw;
-        if (PREFETCH) {
-            raw = nxt;
-            if (u + stride < n_units) load(nxt, u + stride);
+    while (mask) {
+        const int pos = __ffs(mask) - 1, i = pos / BITS;
+        mask &= mask - 1;
+        const float x = BF16 ? __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short *>(elems) + i) << 16)
+                             : __ldg(reinterpret_cast<const float *>(elems) + i);
+        const float dl = __fsub_rn(x, m);
+        float y;
+        if (!fast) {
+            y = kMagic + fminf(fmaxf(rintf(__fdiv_rn(dl, delta)), 0.0f), L);
         } else {
-            load(raw, u);
-        }
-        const int q = (int)(u % ng);
-        const long long tok = u / ng;
-        const int t = (int)(tok % T);
-        const long long bh = tok / T;
-        const long long out_tok = (bh / H) * osb + (bh % H) * osh + t;
-
-        float m, Mx;
-        if (BF16) {
-            // min / max on packed bf16 pairs (exact), then across the pair
-            __nv_bfloat162 mn2, mx2;
-#pragma unroll
-            for (int i = 0; i < Raw::NV; ++i) {
-                const uint32_t w[4] = {raw.v[i].x, raw.v[i].y, raw.v[i].z, raw.v[i].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[k]);
-                    if (i == 0 && k == 0) { mn2 = pr; mx2 = pr; }
-                    else { mn2 = __hmin2_nan(mn2, pr); mx2 = __hmax2_nan(mx2, pr); }
-                }
+            const float ya = __fmaf_rn(dl, ra, kMagic), yb = __fmaf_rn(dl, rb, kMagic);
+            y = ya;
+            if (ya != yb) {
+                const float lo = fminf(ya, yb), hi = fmaxf(ya, yb);
+                const float kh = __fadd_rn(__fsub_rn(lo, kMagic), 0.5f);
+                const float r = __fmaf_rn(-kh, delta, dl);
+                if (r == 0.0f) y = (__float_as_uint(lo) & 1u) ? hi : lo;
+                else if (fabsf(r) > fabsf(kh) * delta * 0x1p-21f) y = r > 0.0f ? hi : lo;
+                else y = kMagic + fminf(fmaxf(rintf(__fdiv_rn(dl, delta)), 0.0f), L);
             }
-            m = min_nan(__low2float(mn2), __high2float(mn2));
-            Mx = max_nan(__low2float(mx2), __high2float(mx2));
-        } else {
-            m = raw.get(0); Mx = m;
-#pragma unroll
-            for (int i = 1; i < G; ++i) { m = min_nan(m, raw.get(i)); Mx = max_nan(Mx, raw.get(i)); }
+            if (M16) y = fminf(fmaxf(y, kMagic), kMagic + L);
         }
-
-        float delta = __fdiv_rn(__fsub_rn(Mx, m), L);
-        if (M16) {                                         // the stored binary16 values decide
-            delta = __half2float(__float2half_rn(delta));
-            m = __half2float(__float2half_rn(m));
-        }
-        const bool ok = delta > 0.0f && delta < __int_as_float(0x7f800000);
-        const float rcp = ok ? __frcp_rn(delta) : 0.0f;
-        if (!ok) atomicOr(status, delta == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
-
-        // two channels per instruction (packed f32x2): dlt = x - m, y = dlt * rcp + magic, c = y - magic,
-        // res = dlt * rcp - c; each half is the same IEEE operation as its scalar form
-        const u64 m2 = pk2(m, m), rcp2 = pk2(rcp, rcp), magic2 = pk2(kMagic, kMagic);
-        const uint32_t cmask = ok ? ((1u << BITS) - 1u) : 0u;       // no grid (constant or non-finite group): codes 0
-        uint32_t words[NWORDS];
-#pragma unroll
-        for (int wd = 0; wd < NWORDS; ++wd) {
-            uint32_t acc = 0;
-#pragma unroll
-            for (int k = 0; k < PER_WORD; k += 2) {
-                const int i = wd * PER_WORD + k;
-                const u64 dlt2 = sub2(pk2(raw.get(i), raw.get(i + 1)), m2);
-                const u64 y2 = fma2(dlt2, rcp2, magic2);
-                const u64 nc2 = sub2(magic2, y2);                       // -(y - magic), exact
-                const u64 res2 = fma2(dlt2, rcp2, nc2);
-                float ylo, yhi, rlo, rhi;
-                unpk2(y2, ylo, yhi);
-                unpk2(res2, rlo, rhi);
-                if (M16) {                                  // rounded metadata: t may leave [0, L]
-                    ylo = fminf(fmaxf(ylo, kMagic), kMagic + L);
-                    yhi = fminf(fmaxf(yhi, kMagic), kMagic + L);
-                }
-                uint32_t cb0 = __float_as_uint(ylo) & cmask;
-                uint32_t cb1 = __float_as_uint(yhi) & cmask;
-                // next to a rounding midpoint (structural with coarse bf16 data): the exact sequence decides
-                if (fmaxf(fabsf(rlo), fabsf(rhi)) >= kTieBand && ok) {
-                    float dlo, dhi;
-                    unpk2(dlt2, dlo, dhi);
-                    if (fabsf(rlo) >= kTieBand) cb0 = exact_code_bits<BITS>(dlo, delta);
-                    if (fabsf(rhi) >= kTieBand) cb1 = exact_code_bits<BITS>(dhi, delta);
-                }
-                acc |= (cb0 | (cb1 << BITS)) << (k * BITS);
-            }
-            words[wd] = acc;
-        }
-
-        unsigned char *cp = codes + out_tok * row_bytes + (long long)q * (G * BITS / 8);
-        if (NWORDS % 4 == 0) {
-#pragma unroll
-            for (int i = 0; i < NWORDS / 4; ++i)
-                reinterpret_cast<uint4 *>(cp)[i] = make_uint4(words[4 * i], words[4 * i + 1], words[4 * i + 2], words[4 * i + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < NWORDS / 2; ++i)
-                reinterpret_cast<uint2 *>(cp)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
-        }
-        if (M16) {
-            reinterpret_cast<__half *>(scales)[out_tok * ng + q] = __float2half_rn(delta);      // exact: already binary16 values
-            reinterpret_cast<__half *>(zeros)[out_tok * ng + q] = __float2half_rn(m);
-        } else {
-            reinterpret_cast<float *>(scales)[out_tok * ng + q] = delta;
-            reinterpret_cast<float *>(zeros)[out_tok * ng + q] = m;
-        }
+        const unsigned field = ((1u << BITS) - 1u) << (BITS * i);
+        word = (word & ~field) | ((__float_as_uint(y) << (BITS * i)) & field);
     }
+    return word;
 }
 
-// One thread dequantizes 16 consecutive channels of TOK = 4 or 8 consecutive tokens (same key group, so the 16
-// scales and zeros are read once for all of them; 8 on large inputs, 4 where that would leave SMs without work).  Codes become floats through the 2^23 trick
-// (exact), then one fma each: deq(c) = fma(c, scale, zero), rounded once.
-template <int BITS, bool KEYS, bool OUT_BF16, bool M16, int TOK>
-__global__ void __launch_bounds__(256, 4) dequant_kernel(
-    const unsigned char *__restrict__ codes, const void *__restrict__ scales, const void *__restrict__ zeros,
-    long long n_units, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
+// One thread owns one (token, channel group): G channels in registers (G / 8 or G / 4 16-byte loads in flight).  One CTA
+// works VAL_THREADS consecutive groups of one (batch, head) row (blockIdx.x = row * chunks + chunk), so the only
+// divisions are two per CTA; a group's token is a shift (d / G a power of two) or one 32-bit division.
+template <int G, int BITS, bool BF16, bool M16>
+__global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValParams p)
 {
-    const int per_tok = d / 16;
-    const int tq_per_row = (T + TOK - 1) / TOK;
+    constexpr float L = float((1 << BITS) - 1);
+    constexpr int NV = BF16 ? G / 8 : G / 4;        // 16-byte pieces of a group
+    constexpr int PER_WORD = 32 / BITS;             // codes per 32-bit word
+    constexpr int NWORDS = G / PER_WORD;
+    // what the constant upper bits of the rounded floats add up to in a packed word
+    constexpr unsigned K = [] { unsigned k = 0; for (int i = 0; i < PER_WORD; ++i) k += kMagicBits << (BITS * i); return k; }();
+
+    const unsigned row = blockIdx.x / p.chunks_per_row, chunk = blockIdx.x - row * p.chunks_per_row;
+    const unsigned b = row / (unsigned)p.H, h = row - b * (unsigned)p.H;
+    const unsigned u = chunk * VAL_THREADS + threadIdx.x;                        // group within the row
+    if (u >= (unsigned)p.T * (unsigned)p.ng) return;
+    const unsigned tok = p.ng_shift >= 0 ? u >> p.ng_shift : u / (unsigned)p.ng;
+    const unsigned q = u - tok * (unsigned)p.ng;
+    const long long in_off = (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st + (long long)q * G;
+    const long long out_tok = (long long)b * p.osb + (long long)h * p.osh + tok;
+
+    uint4 raw[NV];
+    {
+        const uint4 *src = BF16 ? reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.v) + in_off)
+                                : reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(p.v) + in_off);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) raw[i] = ldg128(src + i);
+    }
+    // channel pair c (channels 2c, 2c + 1) as two floats, exact widening
+    auto pair_of = [&](int c, float &x0, float &x1) {
+        if (BF16) {
+            const uint4 &r = raw[c >> 2];
+            const unsigned w = (c & 3) == 0 ? r.x : (c & 3) == 1 ? r.y : (c & 3) == 2 ? r.z : r.w;
+            x0 = bf16lo_to_f32(w);
+            x1 = bf16hi_to_f32(w);
+        } else {
+            const uint4 &r = raw[c >> 1];
+            x0 = __uint_as_float((c & 1) ? r.z : r.x);
+            x1 = __uint_as_float((c & 1) ? r.w : r.y);
+        }
+    };
+
+    // ---- min / max of the group
+    float m, Mx;
+    if (BF16) {
+        unsigned mn2 = raw[0].x, mx2 = raw[0].x;                // packed bf16 pairs (exact), then across the pair
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const unsigned w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+            for (int k = (i == 0 ? 1 : 0); k < 4; ++k) { mn2 = hmin2_nan_bits(mn2, w[k]); mx2 = hmax2_nan_bits(mx2, w[k]); }
+        }
+        m = min_nan(bf16lo_to_f32(mn2), bf16hi_to_f32(mn2));
+        Mx = max_nan(bf16lo_to_f32(mx2), bf16hi_to_f32(mx2));
+    } else {
+        float x0, x1;
+        pair_of(0, x0, x1);
+        m = min_nan(x0, x1);
+        Mx = max_nan(x0, x1);
+#pragma unroll
+        for (int c = 1; c < G / 2; ++c) {
+            pair_of(c, x0, x1);
+            m = min_nan(m, min_nan(x0, x1));
+            Mx = max_nan(Mx, max_nan(x0, x1));
+        }
+    }
+
+    // ---- the grid
+    const float rng = __fsub_rn(Mx, m);
+    float delta = div_by_levels<BITS>(rng);
+    if (!(rng > 0x1p-100f && rng < 0x1p100f)) delta = __fdiv_rn(rng, L);     // outside the range where that is exact: the division
+    if (M16) {                                         // the stored binary16 values decide
+        delta = __half2float(__float2half_rn(delta));
+        m = __half2float(__float2half_rn(m));
+    }
+    const bool ok = delta > 0.0f && delta < __int_as_float(0x7f800000);
+    const bool fast = delta > 0x1p-100f && delta < 0x1p100f;       // the hardware reciprocal is good to 1 ulp here
+    float rcp;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(delta));
+    const float ra = __fmul_rn(rcp, 1.0f + 0x1p-20f), rb = __fmul_rn(rcp, 1.0f - 0x1p-20f);
+    const u64 m2 = pk2(m, m), ra2 = pk2(ra, ra), rb2 = pk2(rb, rb), magic2 = pk2(kMagic, kMagic);
+
+    // ---- codes: two channels per instruction (packed f32x2).  Both ends of the bracket are rounded and packed (added
+    // up shifted into place); the ends differ by at most one level, upwards, so the difference of the two packed words
+    // has exactly one bit set for every element that the fast path could not decide.
+    constexpr unsigned ALL = [] { unsigned a = 0; for (int i = 0; i < PER_WORD; ++i) a |= 1u << (BITS * i); return a; }();
+    uint32_t words[NWORDS];
+#pragma unroll
+    for (int wd = 0; wd < NWORDS; ++wd) {
+        unsigned acc_a = 0u - K, acc_b = 0u - K;
+#pragma unroll
+        for (int k = 0; k < PER_WORD; k += 2) {
+            float x0, x1, ya0, ya1, yb0, yb1;
+            pair_of((wd * PER_WORD + k) / 2, x0, x1);
+            const u64 dlt2 = sub2(pk2(x0, x1), m2);
+            unpk2(fma2(dlt2, ra2, magic2), ya0, ya1);
+            unpk2(fma2(dlt2, rb2, magic2), yb0, yb1);
+            if (M16) {                                  // rounded metadata: t may leave [0, L]
+                ya0 = fminf(fmaxf(ya0, kMagic), kMagic + L); yb0 = fminf(fmaxf(yb0, kMagic), kMagic + L);
+                ya1 = fminf(fmaxf(ya1, kMagic), kMagic + L); yb1 = fminf(fmaxf(yb1, kMagic), kMagic + L);
+            }
+            acc_a += __float_as_uint(ya0) << (BITS * k);
+            acc_a += __float_as_uint(ya1) << (BITS * (k + 1));
+            acc_b += __float_as_uint(yb0) << (BITS * k);
+            acc_b += __float_as_uint(yb1) << (BITS * (k + 1));
+        }
+        const unsigned undecided = fast ? acc_a - acc_b : ALL;
+        if (undecided && ok) {
+            const long long e0 = in_off + wd * PER_WORD;        // first element of this word
+            const void *elems = BF16 ? static_cast<const void *>(reinterpret_cast<const __nv_bfloat16 *>(p.v) + e0)
+                                     : static_cast<const void *>(reinterpret_cast<const float *>(p.v) + e0);
+            acc_a = patch_word<BITS, BF16, M16>(acc_a, undecided, elems, m, delta, ra, rb, fast);
+        }
+        words[wd] = ok ? acc_a : 0u;                    // no grid (constant or non-finite group): codes 0
+    }
+
+    unsigned char *cp = p.codes + out_tok * p.row_bytes + (long long)q * (G * BITS / 8);
+    if (NWORDS % 4 == 0) {
+#pragma unroll
+        for (int i = 0; i < NWORDS / 4; ++i)
+            reinterpret_cast<uint4 *>(cp)[i] = make_uint4(words[4 * i], words[4 * i + 1], words[4 * i + 2], words[4 * i + 3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < NWORDS / 2; ++i)
+            reinterpret_cast<uint2 *>(cp)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
+    }
+    const long long meta_idx = out_tok * p.ng + q;
+    if (M16) {
+        reinterpret_cast<__half *>(p.scales)[meta_idx] = __float2half_rn(delta);      // exact: already binary16 values
+        reinterpret_cast<__half *>(p.zeros)[meta_idx] = __float2half_rn(m);
+    } else {
+        reinterpret_cast<float *>(p.scales)[meta_idx] = delta;
+        reinterpret_cast<float *>(p.zeros)[meta_idx] = m;
+    }
+    if (!ok) atomicOr(p.status, delta == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
+}
+
+// Dequantizer.  One thread owns 8 consecutive channels (16 bytes of bf16 output, 32 of float32) of TOK = 4 or 8
+// consecutive tokens of one key group, so the 8 scales and zeros of a key cache are read once for all of them (8 tokens
+// on large inputs, 4 where that would leave SMs without work); the lanes of a warp cover whole tokens, so every store
+// instruction writes full 256-byte rows.  A code becomes a float without shifting: its bits, masked in place at bit
+// position s, are OR-ed under the exponent of 2^(23 - s), which makes the word 2^(23 - s) + c exactly; subtracting that
+// power of two leaves c (both steps exact), then one fma: deq(c) = fma(c, scale, zero), rounded once.  Two channels per
+// instruction (packed f32x2).
+template <int BITS, bool KEYS, bool OUT_BF16, bool M16, int TOK>
+__global__ void __launch_bounds__(256) dequant_kernel(
+    const unsigned char *__restrict__ codes, const void *__restrict__ scales, const void *__restrict__ zeros,
+    unsigned chunks_per_row, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
+{
+    constexpr int CH = 8;                                 // channels per thread
+    constexpr unsigned FIELD = (1u << BITS) - 1u;
+    const int per_tok = d / CH;                           // threads per token
+    const int slots = 256 / per_tok;                      // token runs (TOK tokens each) per CTA
     const int row_bytes = d * BITS / 8;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < n_units; u += stride) {
-        const int c16 = (int)(u % per_tok);
-        const long long r = u / per_tok;
-        const int t0 = (int)(r % tq_per_row) * TOK;
-        const long long bh = r / tq_per_row;
-        const int h = (int)(bh % H);
-        const long long b = bh / H;
+    // bias pairs 2^(23 - s) for the bit positions s of channels (2 i, 2 i + 1); positions are taken modulo 16 for 4-bit
+    // codes (the upper half of the word is shifted down first)
+    u64 bias2[CH / 2];
+#pragma unroll
+    for (int i = 0; i < CH / 2; ++i) {
+        const int s0 = (BITS * 2 * i) % 16, s1 = (BITS * (2 * i + 1)) % 16;
+        bias2[i] = pk2(__uint_as_float((unsigned)(150 - s0) << 23), __uint_as_float((unsigned)(150 - s1) << 23));
+    }
+    // one CTA = one chunk of slots * TOK tokens of one (batch, head) row: two divisions per CTA, none per element
+    const unsigned bh = blockIdx.x / chunks_per_row, chunk = blockIdx.x - bh * chunks_per_row;
+    const int slot = (int)threadIdx.x / per_tok, c8 = (int)threadIdx.x - slot * per_tok;
+    const int t0 = ((int)chunk * slots + slot) * TOK;
+    if (slot < slots && t0 < T) {
+        const int h = (int)(bh % (unsigned)H);
+        const long long b = bh / (unsigned)H;
         const long long in_tok0 = b * isb + h * ish;
-        float sc[16], zr[16];
+        u64 sc2[CH / 2], zr2[CH / 2];
         if (KEYS) {
-            const long long base = (b * (isb / G) + h * (ish / G) + t0 / G) * d + c16 * 16;
+            const long long base = (b * (isb / G) + h * (ish / G) + t0 / G) * d + c8 * CH;
             if (M16) {
+                const uint4 s8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(scales) + base));
+                const uint4 z8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(zeros) + base));
+                const uint32_t sw[4] = {s8.x, s8.y, s8.z, s8.w}, zw[4] = {z8.x, z8.y, z8.z, z8.w};
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const uint4 s8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(scales) + base) + i);
-                    const uint4 z8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(zeros) + base) + i);
-                    const uint32_t sw[4] = {s8.x, s8.y, s8.z, s8.w}, zw[4] = {z8.x, z8.y, z8.z, z8.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sw[k]));
-                        const float2 zf = __half22float2(*reinterpret_cast<const __half2 *>(&zw[k]));
-                        sc[8 * i + 2 * k] = sf.x; sc[8 * i + 2 * k + 1] = sf.y;
-                        zr[8 * i + 2 * k] = zf.x; zr[8 * i + 2 * k + 1] = zf.y;
-                    }
+                for (int k = 0; k < 4; ++k) {
+                    const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sw[k]));
+                    const float2 zf = __half22float2(*reinterpret_cast<const __half2 *>(&zw[k]));
+                    sc2[k] = pk2(sf.x, sf.y);
+                    zr2[k] = pk2(zf.x, zf.y);
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < 2; ++i) {
                     const float4 s4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(scales) + base) + i);
                     const float4 z4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(zeros) + base) + i);
-                    sc[4 * i] = s4.x; sc[4 * i + 1] = s4.y; sc[4 * i + 2] = s4.z; sc[4 * i + 3] = s4.w;
-                    zr[4 * i] = z4.x; zr[4 * i + 1] = z4.y; zr[4 * i + 2] = z4.z; zr[4 * i + 3] = z4.w;
+                    sc2[2 * i] = pk2(s4.x, s4.y); sc2[2 * i + 1] = pk2(s4.z, s4.w);
+                    zr2[2 * i] = pk2(z4.x, z4.y); zr2[2 * i + 1] = pk2(z4.z, z4.w);
                 }
             }
+        }
+        // the codes of the thread's tokens first (independent loads in flight), then the arithmetic
+        uint32_t cw[TOK];
+#pragma unroll
+        for (int tt = 0; tt < TOK; ++tt) {
+            const int t = t0 + tt < T ? t0 + tt : T - 1;
+            const unsigned char *cp = codes + (in_tok0 + t) * row_bytes + c8 * (CH * BITS / 8);
+            cw[tt] = BITS == 2 ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(cp)) : __ldg(reinterpret_cast<const uint32_t *>(cp));
         }
 #pragma unroll
         for (int tt = 0; tt < TOK; ++tt) {
             const int t = t0 + tt;
             if (t >= T) break;
-            const unsigned char *cp = codes + (in_tok0 + t) * row_bytes + c16 * (16 * BITS / 8);
-            uint32_t w[2];
-            if (BITS == 2) { w[0] = __ldg(reinterpret_cast<const uint32_t *>(cp)); w[1] = 0; }
-            else { const uint2 rr = __ldg(reinterpret_cast<const uint2 *>(cp)); w[0] = rr.x; w[1] = rr.y; }
-            float s1 = 0.0f, z1 = 0.0f;
+            u64 s2 = 0, z2 = 0;
             if (!KEYS) {
-                const long long mi = (in_tok0 + t) * (d / G) + (c16 * 16) / G;
+                const long long mi = (in_tok0 + t) * (d / G) + (c8 * CH) / G;
+                float s1, z1;
                 if (M16) {
                     s1 = __half2float(__ldg(reinterpret_cast<const __half *>(scales) + mi));
                     z1 = __half2float(__ldg(reinterpret_cast<const __half *>(zeros) + mi));
@@ -257,60 +340,59 @@ __global__ void __launch_bounds__(256, 4) dequant_kernel(
                     s1 = __ldg(reinterpret_cast<const float *>(scales) + mi);
                     z1 = __ldg(reinterpret_cast<const float *>(zeros) + mi);
                 }
+                s2 = pk2(s1, s1);
+                z2 = pk2(z1, z1);
             }
-            float y[16];
+            const uint32_t lo = cw[tt], hi = cw[tt] >> 16;        // 4-bit codes: channels 4..7 sit in the upper half
+            u64 y2[CH / 2];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int bit = i * BITS;
-                const uint32_t cb = (w[bit / 32] >> (bit % 32)) & ((1u << BITS) - 1u);
-                const float c = __fsub_rn(__uint_as_float(0x4B000000u | cb), 8388608.0f);     // exact int -> float
-                y[i] = KEYS ? __fmaf_rn(c, sc[i], zr[i]) : __fmaf_rn(c, s1, z1);
+            for (int i = 0; i < CH / 2; ++i) {
+                const uint32_t word = (BITS == 4 && i >= 2) ? hi : lo;
+                const int s0 = (BITS * 2 * i) % 16, s1 = (BITS * (2 * i + 1)) % 16;
+                const float f0 = __uint_as_float((word & (FIELD << s0)) | ((unsigned)(150 - s0) << 23));
+                const float f1 = __uint_as_float((word & (FIELD << s1)) | ((unsigned)(150 - s1) << 23));
+                const u64 c2 = sub2(pk2(f0, f1), bias2[i]);             // exact: the codes as floats
+                y2[i] = KEYS ? fma2(c2, sc2[i], zr2[i]) : fma2(c2, s2, z2);
             }
-            const long long o = ((bh * T) + t) * d + c16 * 16;
+            const long long o = (((long long)bh * T) + t) * d + c8 * CH;
             if (OUT_BF16) {
-                uint32_t pk[8];
+                uint32_t pk[CH / 2];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    __nv_bfloat162 p2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                for (int i = 0; i < CH / 2; ++i) {
+                    float a, b_;
+                    unpk2(y2[i], a, b_);
+                    __nv_bfloat162 p2 = __floats2bfloat162_rn(a, b_);
                     pk[i] = *reinterpret_cast<uint32_t *>(&p2);
                 }
-                uint4 *op = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(out) + o);
-                op[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                op[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(out) + o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             } else {
                 float4 *op = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + o);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) op[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                for (int i = 0; i < 2; ++i) {
+                    float a, b_, c, e;
+                    unpk2(y2[2 * i], a, b_);
+                    unpk2(y2[2 * i + 1], c, e);
+                    op[i] = make_float4(a, b_, c, e);
+                }
             }
         }
     }
 }
 
-int grid_for(long long n_threads, int block)
+template <int G, int BITS, bool BF16, bool M16>
+int launch_values_inst(const ValParams &p, long long rows, cudaStream_t st)
 {
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    long long blocks = (n_threads + block - 1) / block;
-    const long long cap = (long long)sms * 32;          // a multiple of the SM count; grid-stride covers the rest
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
-    return (int)blocks;
-}
-
-template <int G, int BITS>
-int launch_values(const void *v, int dtype, long long n_units, int H, int T, int ng, long long sb, long long sh,
-                  long long st_, unsigned char *codes, void *scales, void *zeros, long long osb, long long osh,
-                  int row_bytes, unsigned *status, int meta16, cudaStream_t st)
-{
-    const int grid = grid_for(n_units, 256);
-#define SQ_VK(BF, MM) quant_values_kernel<G, BITS, BF, MM><<<grid, 256, 0, st>>>(v, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status)
-    if (dtype == SQUAT_BF16) { if (meta16) SQ_VK(true, true); else SQ_VK(true, false); }
-    else { if (meta16) SQ_VK(false, true); else SQ_VK(false, false); }
-#undef SQ_VK
+    quant_values_kernel<G, BITS, BF16, M16><<<(unsigned)(rows * p.chunks_per_row), VAL_THREADS, 0, st>>>(p);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
+}
+
+template <int G, int BITS>
+int launch_values(const ValParams &p, long long rows, int dtype, int meta16, cudaStream_t st)
+{
+    if (dtype == SQUAT_BF16) return meta16 ? launch_values_inst<G, BITS, true, true>(p, rows, st) : launch_values_inst<G, BITS, true, false>(p, rows, st);
+    return meta16 ? launch_values_inst<G, BITS, false, true>(p, rows, st) : launch_values_inst<G, BITS, false, false>(p, rows, st);
 }
 
 }  // namespace
@@ -320,11 +402,22 @@ int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T,
                               unsigned char *codes, void *scales, void *zeros,
                               long long osb, long long osh, unsigned *status, int meta16, cudaStream_t st)
 {
-    const int ng = d / G;
-    const long long n_units = (long long)batch * H * T * ng;
-    if (n_units == 0) return SQUAT_OK;
-    const int row_bytes = d * bits / 8;
-#define SQ_V(GG, BB) return launch_values<GG, BB>(v, dtype, n_units, H, T, ng, sb, sh, st_, codes, scales, zeros, osb, osh, row_bytes, status, meta16, st)
+    const long long rows = (long long)batch * H;
+    if (rows == 0 || T == 0) return SQUAT_OK;
+    ValParams p;
+    p.v = v; p.H = H; p.T = T; p.ng = d / G;
+    p.ng_shift = -1;
+    for (int sft = 0; sft < 20; ++sft)
+        if ((1 << sft) == p.ng) p.ng_shift = sft;
+    const long long row_units = (long long)T * p.ng;
+    const long long chunks = (row_units + VAL_THREADS - 1) / VAL_THREADS;
+    if (row_units > 0x7fffffffLL || rows * chunks > 0x7fffffffLL) return SQUAT_ERR_UNSUPPORTED;    // 32-bit group and CTA indices
+    p.chunks_per_row = (unsigned)chunks;
+    p.sb = sb; p.sh = sh; p.st = st_;
+    p.codes = codes; p.scales = scales; p.zeros = zeros; p.osb = osb; p.osh = osh;
+    p.row_bytes = d * bits / 8;
+    p.status = status;
+#define SQ_V(GG, BB) return launch_values<GG, BB>(p, rows, dtype, meta16, st)
     if (bits == 2) { if (G == 32) SQ_V(32, 2); if (G == 64) SQ_V(64, 2); if (G == 128) SQ_V(128, 2); }
     if (bits == 4) { if (G == 32) SQ_V(32, 4); if (G == 64) SQ_V(64, 4); if (G == 128) SQ_V(128, 4); }
 #undef SQ_V
@@ -338,12 +431,18 @@ int squat_launch_dequant(int kind, const unsigned char *codes, const void *scale
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long units8 = (long long)batch * H * ((T + 7) / 8) * (d / 16);       // threads with 8 tokens x 16 channels each
-    const bool tok8 = units8 >= (long long)sms * 32 * 256;                           // enough of them to fill the grid cap
-    const long long n_units = tok8 ? units8 : (long long)batch * H * ((T + 3) / 4) * (d / 16);
-    if (n_units == 0) return SQUAT_OK;
-    const int grid = grid_for(n_units, 256);
-#define SQ_D1(BB, KK, OO, MM, TT) dequant_kernel<BB, KK, OO, MM, TT><<<grid, 256, 0, st>>>(codes, scales, zeros, n_units, H, T, d, G, isb, ish, out)
+    const long long rows = (long long)batch * H;
+    if (rows == 0 || T == 0) return SQUAT_OK;
+    const int per_tok = d / 8;
+    if (per_tok < 1 || per_tok > 256) return SQUAT_ERR_UNSUPPORTED;
+    const int slots = 256 / per_tok;
+    // 8 tokens per thread where that still gives every SM several CTAs, else 4
+    const long long chunks8 = (T + slots * 8 - 1) / (slots * 8);
+    const bool tok8 = rows * chunks8 >= (long long)sms * 16;
+    const long long chunks = tok8 ? chunks8 : (T + slots * 4 - 1) / (slots * 4);
+    if (rows * chunks > 0x7fffffffLL) return SQUAT_ERR_UNSUPPORTED;
+    const unsigned grid = (unsigned)(rows * chunks);
+#define SQ_D1(BB, KK, OO, MM, TT) dequant_kernel<BB, KK, OO, MM, TT><<<grid, 256, 0, st>>>(codes, scales, zeros, (unsigned)chunks, H, T, d, G, isb, ish, out)
 #define SQ_D(BB, KK, OO) do { if (meta16) { if (tok8) SQ_D1(BB, KK, OO, true, 8); else SQ_D1(BB, KK, OO, true, 4); } \
                               else { if (tok8) SQ_D1(BB, KK, OO, false, 8); else SQ_D1(BB, KK, OO, false, 4); } } while (0)
     const bool keys = kind == SQUAT_KEYS, obf = out_dtype == SQUAT_BF16;
