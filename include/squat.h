@@ -47,6 +47,8 @@ typedef enum { SQUAT_KEYS = 0, SQUAT_VALUES = 1 } squat_kind;
 #define SQUAT_FLAG_NONFINITE   1u   /* a NaN or infinity among the keys / values (its group's scale came out NaN/Inf) */
 #define SQUAT_FLAG_ZERO_RANGE  2u   /* some group had max == min (scale 0, all codes 0)            */
 #define SQUAT_FLAG_NO_CONVERGE 4u   /* eigensolver hit its sweep limit for some head               */
+#define SQUAT_FLAG_BOUNDS 16u        /* only in the bounds-checked build of the library (-DSQUAT_CHECKED): a kernel computed an
+                                       * address outside the buffer or on-chip region it belongs to; the access was skipped      */
 #define SQUAT_FLAG_DEVICE_TIMEOUT 8u /* a bounded wait on the tensor core inside squat_quantize_keys ran
                                        * out: that call's outputs are invalid (the kernel still ends)  */
 
@@ -383,6 +385,14 @@ int squat_gram_static(const void *q, int dtype, int n_q_heads, int n_kv_heads, i
  * being optimised away).  Enqueues on `stream`.
  */
 int squat_fp32_peak_probe(int packed, int iters, float *sink, long long *flops_host, void *stream);
+
+/*
+ * Self-test of the bounds-checked build (the paper has no counterpart).  In libsquat_checked.so (built with
+ * -DSQUAT_CHECKED) a kernel forms one address on the last word of a small buffer and one a byte past it, touching
+ * neither: *detected (host) is 1 iff the first passed the check and the second raised SQUAT_FLAG_BOUNDS.  The device
+ * status word is left as it was.  Synchronises `stream`.  In the normal build: SQUAT_ERR_UNSUPPORTED, *detected = 0.
+ */
+int squat_checked_selftest(void *stream, int *detected);
 
 /* Reads (and clears when `clear` != 0) the device status word of the current device.
  * Synchronises `stream`.  flags is a host pointer. */

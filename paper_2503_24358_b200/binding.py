@@ -11,11 +11,12 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsquat.so")
+# SQUAT_LIBRARY selects another build of the same library (the bounds-checked one, libsquat_checked.so)
+LIB_PATH = os.environ.get("SQUAT_LIBRARY") or os.path.join(_HERE, "libsquat.so")
 
 SQUAT_F32, SQUAT_BF16 = 0, 1
 SQUAT_KEYS, SQUAT_VALUES = 0, 1
-FLAG_NONFINITE, FLAG_ZERO_RANGE, FLAG_NO_CONVERGE, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
+FLAG_NONFINITE, FLAG_ZERO_RANGE, FLAG_NO_CONVERGE, FLAG_DEVICE_TIMEOUT, FLAG_BOUNDS = 1, 2, 4, 8, 16
 
 EXPORTED_SYMBOLS = (
     "squat_subspace_create", "squat_subspace_destroy", "squat_build_subspace", "squat_subspace_export",
@@ -25,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "squat_decode_attention_workspace_bytes", "squat_decode_attention",
     "squat_rope_table_floats", "squat_rope_table_fill", "squat_decode_attention_pre_rope",
     "squat_decode_attention_ex", "squat_build_subspace_from_gram", "squat_build_subspace_power", "squat_write_path_host_ex", "squat_build_subspace_power_from_gram", "squat_quantize_keys_m16", "squat_quantize_values_m16", "squat_dequantize_m16",
-    "squat_fp32_peak_probe", "squat_append_window_host", "squat_subspace_select_key_kernel",
+    "squat_fp32_peak_probe", "squat_append_window_host", "squat_subspace_select_key_kernel", "squat_checked_selftest",
 )
 
 _lib = None
@@ -85,6 +86,7 @@ def _load():
                                                   c.c_float, vp, i, ll, vp, vp, c.c_size_t, vp]
         lib.squat_append_window_host.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, c.c_size_t, vp]
         lib.squat_subspace_select_key_kernel.argtypes = [vp, i, c.POINTER(i)]
+        lib.squat_checked_selftest.argtypes = [vp, c.POINTER(i)]
         lib.squat_fp32_peak_probe.argtypes = [i, i, vp, c.POINTER(ll), vp]
         lib.squat_get_device_status.argtypes = [vp, c.POINTER(c.c_uint), i]
         lib.squat_kernel_launch_count.restype = c.c_ulonglong
@@ -314,6 +316,14 @@ def squat_subspace_select_key_kernel(s: "Subspace", prefer_dense: bool = False) 
     _check(_load().squat_subspace_select_key_kernel(s.handle, 1 if prefer_dense else 0, ctypes.byref(r)),
            "squat_subspace_select_key_kernel")
     return int(r.value)
+
+
+def squat_checked_selftest(stream=None) -> bool:
+    """True iff the loaded library is the bounds-checked build and its check caught a one-byte overrun (formed, never
+    accessed); raises SquatError (status 3) on the normal build."""
+    det = ctypes.c_int(0)
+    _check(_load().squat_checked_selftest(_stream(stream), ctypes.byref(det)), "squat_checked_selftest")
+    return bool(det.value)
 
 
 def squat_fp32_peak_probe(packed: bool, iters: int, sink: torch.Tensor, stream=None) -> int:

@@ -565,6 +565,47 @@ int squat_decode_attention_pre_rope(const void *q, int q_dtype, int batch, int n
                                  (table_positions + 31) / 32, first_pos, 0, stream);
 }
 
+#ifdef SQUAT_CHECKED
+namespace {
+// forms one address just inside and one just outside an extent; touches neither
+__global__ void checked_selftest_kernel(const char *base, unsigned long long bytes, unsigned *status, int *passed_inside)
+{
+    SqExtent ext = {base, bytes};
+    *passed_inside = SQ_CHK_G(status, base + bytes - 4, 4, ext) ? 1 : 0;      // last word: allowed, no flag
+    (void)SQ_CHK_G(status, base + bytes - 3, 4, ext);                          // one byte over: refused, SQUAT_FLAG_BOUNDS
+}
+}  // namespace
+#endif
+
+int squat_checked_selftest(void *stream, int *detected)
+{
+#ifdef SQUAT_CHECKED
+    if (!detected) return SQUAT_ERR_INVALID_ARG;
+    unsigned *w = squat_status_word();
+    if (!w) return SQUAT_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int *flag_dev = nullptr;
+    unsigned before = 0, after = 0;
+    int inside = 0;
+    SQUAT_CUDA(cudaMalloc(&flag_dev, 256));
+    SQUAT_CUDA(cudaMemcpyAsync(&before, w, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaStreamSynchronize(st));
+    SQUAT_CUDA(cudaMemsetAsync(w, 0, sizeof(unsigned), st));
+    checked_selftest_kernel<<<1, 1, 0, st>>>(reinterpret_cast<const char *>(flag_dev), 256, w, flag_dev);
+    SQUAT_CUDA(cudaMemcpyAsync(&after, w, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(&inside, flag_dev, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SQUAT_CUDA(cudaMemcpyAsync(w, &before, sizeof(unsigned), cudaMemcpyHostToDevice, st));      // the caller's flags are kept
+    SQUAT_CUDA(cudaStreamSynchronize(st));
+    cudaFree(flag_dev);
+    *detected = (inside == 1 && (after & SQUAT_FLAG_BOUNDS)) ? 1 : 0;
+    return SQUAT_OK;
+#else
+    (void)stream;
+    if (detected) *detected = 0;
+    return SQUAT_ERR_UNSUPPORTED;           // this is not the bounds-checked build
+#endif
+}
+
 int squat_get_device_status(void *stream, unsigned *flags, int clear)
 {
     if (!flags) return SQUAT_ERR_INVALID_ARG;

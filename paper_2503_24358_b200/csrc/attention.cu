@@ -349,31 +349,52 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
     }
 }
 
-// One CTA per (batch, query head), thread = channel: the residual buffer's tokens, then the merge.
-__global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
+// One CTA per (batch, query head): the residual buffer's tokens, then the merge of the chunks.  The kernel is a chain
+// of dependent global loads (residual keys -> scores -> weights -> residual values, chunk partials), so it is laid out
+// for loads in flight rather than for arithmetic: 16 warps; a warp takes every 16th residual key row (8 at most, all
+// loaded before the first is used); the value rows and the chunks are dealt to four groups of 128 threads (thread =
+// channel) whose partial sums meet in shared memory.
+constexpr int CB_THREADS = 512;
+constexpr int CB_WARPS = CB_THREADS / 32;
+constexpr int CB_GROUPS = CB_THREADS / D;
+__global__ void __launch_bounds__(CB_THREADS) attn_combine_kernel(const AttnParams p)
 {
     __shared__ float qv[D];
     __shared__ float w[SQUAT_ATTN_MAX_RESIDUAL];
-    __shared__ float red[4];
-    const int hq = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+    __shared__ float red[CB_WARPS];
+    __shared__ float acc_sm[CB_GROUPS][D];
+    __shared__ float den_sm[CB_GROUPS];
+    const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int c = tid % D, grp = tid / D;
+    const int warp = tid >> 5, lane = tid & 31;
     const int h = hq / (p.Hq / p.H);
-    qv[c] = p.scale * load_elem(p.q, ((long long)b * p.Hq + hq) * D + c, p.q_bf16);
+    if (tid < D) qv[tid] = p.scale * load_elem(p.q, ((long long)b * p.Hq + hq) * D + tid, p.q_bf16);
     __syncthreads();
     const long long rbase = ((long long)b * p.H + h) * p.R * D;
-    // scores of the residual rows: warp w takes rows w, w + 4, ...; a lane takes 4 neighbouring channels (one 8- or
-    // 16-byte load), so a row is read as one contiguous piece
+    // scores of the residual rows: a lane takes 4 neighbouring channels (one 8- or 16-byte load), so a row is read as one
+    // contiguous piece
     {
-        const int warp = c >> 5, lane = c & 31;
         const float4 q4 = *reinterpret_cast<const float4 *>(qv + 4 * lane);
-#pragma unroll 4
-        for (int t = warp; t < p.R; t += D / 32) {
-            float4 k4;
-            if (p.res_bf16) {
-                const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(p.k_res) + rbase + (long long)t * D) + lane);
-                k4 = make_float4(bf16lo_to_f32(raw.x), bf16hi_to_f32(raw.x), bf16lo_to_f32(raw.y), bf16hi_to_f32(raw.y));
-            } else {
-                k4 = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.k_res) + rbase + (long long)t * D) + lane);
+        constexpr int ROWS = SQUAT_ATTN_MAX_RESIDUAL / CB_WARPS;          // 8
+        float4 kr[ROWS];
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i) {
+            const int t = warp + CB_WARPS * i;
+            kr[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (t < p.R) {
+                if (p.res_bf16) {
+                    const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(p.k_res) + rbase + (long long)t * D) + lane);
+                    kr[i] = make_float4(bf16lo_to_f32(raw.x), bf16hi_to_f32(raw.x), bf16lo_to_f32(raw.y), bf16hi_to_f32(raw.y));
+                } else {
+                    kr[i] = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.k_res) + rbase + (long long)t * D) + lane);
+                }
             }
+        }
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i) {
+            const int t = warp + CB_WARPS * i;
+            if (t >= p.R) break;                                           // warp-uniform
+            float4 k4 = kr[i];
             if (p.rope_a) {
                 // residual rows are stored before the rotary embedding too: turn row t at position first_pos + T + t.
                 // Lane l < 16 holds channels 4 l .. 4 l + 3, lane l + 16 their partners 64 channels up.
@@ -385,41 +406,53 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p)
                 float rot[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int i = 4 * (lane & 15) + e;
-                    const float2 ca = __ldg(p.rope_a + (pos >> 5) * 64 + i), cb = __ldg(p.rope_b + (pos & 31) * 64 + i);
+                    const int i2 = 4 * (lane & 15) + e;
+                    const float2 ca = __ldg(p.rope_a + (pos >> 5) * 64 + i2), cb = __ldg(p.rope_b + (pos & 31) * 64 + i2);
                     const float cc = fmaf(ca.x, cb.x, -ca.y * cb.y), ss = fmaf(ca.y, cb.x, ca.x * cb.y);
                     rot[e] = fmaf(own[e], cc, sign * oth[e] * ss);
                 }
                 k4 = make_float4(rot[0], rot[1], rot[2], rot[3]);
             }
-            const float s = warp_sum_f(fmaf(q4.x, k4.x, fmaf(q4.y, k4.y, fmaf(q4.z, k4.z, q4.w * k4.w))));
-            if (lane == 0) w[t] = s;
+            const float sdot = warp_sum_f(fmaf(q4.x, k4.x, fmaf(q4.y, k4.y, fmaf(q4.z, k4.z, q4.w * k4.w))));
+            if (lane == 0) w[t] = sdot;
         }
     }
     __syncthreads();
-    float m = c < p.R ? w[c] : -INFINITY;
+    float m = tid < p.R ? w[tid] : -INFINITY;
     const float *ml = p.ml + ((long long)b * p.Hq + hq) * p.nchunk * 2;
-    for (int s = c; s < p.nchunk; s += D) m = fmaxf(m, ml[2 * s]);
+    for (int s = tid; s < p.nchunk; s += CB_THREADS) m = fmaxf(m, ml[2 * s]);
     m = warp_max_f(m);
-    if ((c & 31) == 0) red[c >> 5] = m;
+    if (lane == 0) red[warp] = m;
     __syncthreads();
-    m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    m = red[0];
+#pragma unroll
+    for (int i = 1; i < CB_WARPS; ++i) m = fmaxf(m, red[i]);
     __syncthreads();
-    if (c < p.R) w[c] = expf(w[c] - m);
+    if (tid < p.R) w[tid] = expf(w[tid] - m);
     __syncthreads();
+    // group `grp` takes residual rows grp, grp + 4, ... and chunks grp, grp + 4, ...
     float acc = 0.0f, den = 0.0f;
 #pragma unroll 8
-    for (int t = 0; t < p.R; ++t) {
+    for (int t = grp; t < p.R; t += CB_GROUPS) {
         acc = fmaf(w[t], load_elem(p.v_res, rbase + (long long)t * D + c, p.res_bf16), acc);
         den += w[t];
     }
     const float *part = p.part + ((long long)b * p.Hq + hq) * p.nchunk * D;
-    for (int s = 0; s < p.nchunk; ++s) {
+#pragma unroll 4
+    for (int s = grp; s < p.nchunk; s += CB_GROUPS) {
         const float f = expf(ml[2 * s] - m);
         acc = fmaf(f, part[(long long)s * D + c], acc);
         den = fmaf(f, ml[2 * s + 1], den);
     }
-    p.out[((long long)b * p.Hq + hq) * D + c] = acc / den;
+    acc_sm[grp][c] = acc;
+    if (c == 0) den_sm[grp] = den;
+    __syncthreads();
+    if (grp == 0) {
+        float a = acc_sm[0][c], dsum = den_sm[0];
+#pragma unroll
+        for (int g = 1; g < CB_GROUPS; ++g) { a += acc_sm[g][c]; dsum += den_sm[g]; }
+        p.out[((long long)b * p.Hq + hq) * D + c] = a / dsum;
+    }
 }
 
 template <int BITS, int NQ, bool ROPE, bool M16>
@@ -481,7 +514,7 @@ int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq,
         else rc = bits == 2 ? launch_partial<2, 4>(p, (qpk + 3) / 4, st) : launch_partial<4, 4>(p, (qpk + 3) / 4, st);
         if (rc != SQUAT_OK) return rc;
     }
-    attn_combine_kernel<<<dim3(Hq, batch), D, 0, st>>>(p);
+    attn_combine_kernel<<<dim3(Hq, batch), CB_THREADS, 0, st>>>(p);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;

@@ -218,6 +218,19 @@ struct KeyParams {
     int total_tiles;          // H * tiles_per_head
     unsigned *status;
     const int *exact_blocks;  // device word: leading 32-channel blocks that no earlier channel corrects (see sweep_block)
+#ifdef SQUAT_CHECKED
+    SqExtent x_k, x_codes, x_scales, x_zeros, x_img;      // what the caller's tensors and the handle's images span
+#endif
+};
+
+// What the sweep may touch, for the bounds-checked build (empty otherwise).
+struct SweepChk {
+#ifdef SQUAT_CHECKED
+    unsigned *status;
+    const float *img;         // the staged image the diagonal block belongs to
+    const float *e_region;    // the tile slot's E_lo operand
+    unsigned tmem_lo, tmem_hi;   // the columns of the tile's E_hi operand: [lo, hi)
+#endif
 };
 
 template <bool BF16>
@@ -273,7 +286,7 @@ __device__ __forceinline__ float2 row_pair(const RawRow<BF16> &r, int q)
 template <int BITS, int NW, bool EXACT, bool M16>
 __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *diag, unsigned e_hi_taddr, float *e_lo, bool store_e,
                                             int lane, int bar_id, int wteam, float2 *red,
-                                            uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero)
+                                            uint32_t (&cw)[BLK * BITS / 32], float &my_scale, float &my_zero, const SweepChk &ck)
 {
     constexpr float L = float((1 << BITS) - 1);
     constexpr int PER_ACC = 16 / BITS;              // codes accumulated exactly in one float (16 bits of mantissa)
@@ -286,6 +299,7 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         float Mx = warp_max(xj);
         if (NW > 1) {
             float2 *slot = red + (jj & 1) * NW;             // [parity][warp of the team]
+            (void)ck;
             if (lane == 0) slot[wteam] = make_float2(m, Mx);
             team_barrier(bar_id, 32 * NW);
 #pragma unroll
@@ -296,7 +310,9 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
             }
         }
         const float rng = __fsub_rn(Mx, m);
-        float scale = div_by_levels<BITS>(rng);
+        // the stored scale: the correctly rounded quotient where the block's decisions are exact (raw inputs: bit-identical to
+        // plain round-to-nearest quantization), else the product with RN(1/L) (within one ulp of it; one instruction, not three)
+        float scale = EXACT ? div_by_levels<BITS>(rng) : __fmul_rn(rng, 1.0f / L);
         float rcp, y0, dlt;
         if (M16) {
             scale = __half2float(__float2half_rn(scale));
@@ -336,11 +352,22 @@ __device__ __forceinline__ void sweep_block(u64 (&xp)[BLK / 2], const float *dia
         eh[jj & 3] = e;
         el[jj & 3] = __fsub_rn(e, __uint_as_float(__float_as_uint(e) & 0xffffe000u));
         if ((jj & 3) == 3 && store_e) {
+#ifdef SQUAT_CHECKED
+            const unsigned col = (e_hi_taddr + (jj - 3)) & 0xffffu;
+            const bool ok_t = sq_chk(col >= ck.tmem_lo && col + 4 <= ck.tmem_hi, ck.status);
+            const bool ok_s = sq_chk(sq_inside(e_lo + (jj >> 2) * (TC_A_LBO / 4), 16, ck.e_region, TC_E_FLOATS * 4), ck.status);
+            if (ok_t) tmem_st4(e_hi_taddr + (jj - 3), eh[0], eh[1], eh[2], eh[3]);
+            if (ok_s) *reinterpret_cast<float4 *>(e_lo + (jj >> 2) * (TC_A_LBO / 4)) = make_float4(el[0], el[1], el[2], el[3]);
+#else
             tmem_st4(e_hi_taddr + (jj - 3), eh[0], eh[1], eh[2], eh[3]);
             *reinterpret_cast<float4 *>(e_lo + (jj >> 2) * (TC_A_LBO / 4)) = make_float4(el[0], el[1], el[2], el[3]);
+#endif
         }
         const u64 ee = pack2(e, e);
         const float *wrow = diag + jj * BLK;
+#ifdef SQUAT_CHECKED
+        if (!sq_chk(sq_inside(wrow, BLK * 4, ck.img, TC_DIAG_FLOATS * 4), ck.status)) continue;    // the reads below stay inside this row
+#endif
         // later channels of the block, 4 per 16-byte broadcast read; where only the upper half of the first chunk
         // is still to come, an 8-byte read does (a broadcast read is charged by its width)
         if ((jj + 1) % 4 >= 2) {
@@ -425,6 +452,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
         // the first head's image is on its way while the rest of the set-up runs
         if (t_lo < t_hi) {
             const int h0 = t_lo / p.tiles_per_head;
+            if (SQ_CHK_G(p.status, p.Wimg + (long long)h0 * TC_IMG_FLOATS, TC_IMG_FLOATS * 4, p.x_img))
             stage_image_async(images + (h0 & 1) * TC_IMG_FLOATS, p.Wimg + (long long)h0 * TC_IMG_FLOATS, img_mbar);
         }
     }
@@ -461,12 +489,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                      : static_cast<const void *>(reinterpret_cast<const float *>(p.k) + row_off);
     };
 
+    // every read of a key row goes through here (the bounds-checked build tests the 32 channels' bytes against the tensor)
+    auto load_keys = [&](RawRow<BF16> &r, const void *row, int chan) {
+        if (SQ_CHK_G(p.status, static_cast<const char *>(row) + chan * (BF16 ? 2 : 4), BLK * (BF16 ? 2 : 4), p.x_k))
+            load_row<BF16>(r, row, chan);
+    };
     RawRow<BF16> raw;
     int start = t_lo;
     if (slot < round_size(start)) {
         TileRows first;
         locate(start + slot, first);
-        load_row<BF16>(raw, first.row, 0);               // in flight while the first head is staged
+        load_keys(raw, first.row, 0);                    // in flight while the first head is staged
     }
     int max_staged = -1;     // heads come in increasing order: the buffers hold max_staged and, earlier, max_staged - 1
     while (start < t_hi) {
@@ -477,7 +510,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
             if (hh <= max_staged) continue;
             if (max_staged >= 0) {                       // (the very first copy was started at kernel entry)
                 __syncthreads();                         // every read of the buffer's old image, by a lane or by an MMA, is over
-                if (threadIdx.x == 32)
+                if (threadIdx.x == 32 && SQ_CHK_G(p.status, p.Wimg + (long long)hh * TC_IMG_FLOATS, TC_IMG_FLOATS * 4, p.x_img))
                     stage_image_async(images + (hh & 1) * TC_IMG_FLOATS, p.Wimg + (long long)hh * TC_IMG_FLOATS, img_mbar);
             }
             if (!shared_words[1] && !mbar_wait(img_mbar, img_phase)) {   // bounded, like every wait here
@@ -520,7 +553,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                     phase ^= 1;
                     tc_fence_after();
                     unsigned dv[32];
+#ifdef SQUAT_CHECKED
+                    {
+                        const unsigned col = (t_mine + (blk - 1) * BLK) & 0xffffu, lo = t_tile & 0xffffu;
+                        if (!sq_chk(col >= lo && col + 32 <= lo + TC_EHI_COL && ((t_mine >> 16) & 0x7f) == (unsigned)(wq * 32) &&
+                                    lo + TC_COLS_PER_TILE <= (tmem_base & 0xffffu) + TC_TMEM_COLS, p.status)) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) dv[i] = 0;
+                        } else
+                            tmem_ld32(t_mine + (blk - 1) * BLK, dv);
+                    }
+#else
                     tmem_ld32(t_mine + (blk - 1) * BLK, dv);
+#endif
 #pragma unroll
                     for (int q = 0; q < BLK / 2; ++q) {
                         const float2 kv = row_pair<BF16>(raw, q);
@@ -529,16 +574,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 }
                 const bool more = blk + 1 < NBLK;
                 // prefetch: the next block of this tile, or the first block of the next round's tile
-                if (more) load_row<BF16>(raw, cur.row, (blk + 1) * BLK);
-                else if (nxt_valid) load_row<BF16>(raw, nxt_row, 0);
+                if (more) load_keys(raw, cur.row, (blk + 1) * BLK);
+                else if (nxt_valid) load_keys(raw, nxt_row, 0);
 
                 const float *diag = img + blk * BLK * BLK;
                 uint32_t cw[WORDS_PER_BLK];
                 float my_scale = 0.0f, my_zero = 0.0f;
+                SweepChk ck;
+#ifdef SQUAT_CHECKED
+                ck.status = p.status;
+                ck.img = img;
+                ck.e_region = Eall + slot * TC_E_FLOATS;
+                ck.tmem_lo = (t_tile & 0xffffu) + TC_EHI_COL;
+                ck.tmem_hi = (t_tile & 0xffffu) + TC_COLS_PER_TILE;
+#endif
                 if (blk < (int)shared_words[2 + TC_SLOTS])
-                    sweep_block<BITS, NW, true, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, true, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero, ck);
                 else
-                    sweep_block<BITS, NW, false, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero);
+                    sweep_block<BITS, NW, false, M16>(xp, diag, t_mine + TC_EHI_COL, e_lo, more, lane, 1 + team, wteam, red, cw, my_scale, my_zero, ck);
 
                 if (more) {
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");   // E_hi is in tensor memory
@@ -557,6 +610,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                         const unsigned b_lbo = 16u * nb;
                         const unsigned bhi = smem_u32(Bhi + tc_panel_off(blk)), blo = smem_u32(Blo + tc_panel_off(blk));
                         const unsigned d = t_tile + blk * BLK;
+#ifdef SQUAT_CHECKED
+                        // the windows the descriptors open: A = this slot's E_lo operand, B = the panels of source block blk
+                        // inside the staged image, D / A-from-tensor-memory = columns of this tile
+                        const unsigned img_lo = smem_u32(img), e_lo_lo = smem_u32(Eall + slot * TC_E_FLOATS);
+                        const unsigned panel_bytes = (unsigned)nb * BLK * 4;
+                        const bool desc_ok =
+                            a_lo == e_lo_lo && a_lo + (BLK / 8 - 1) * 2 * TC_A_LBO + 2 * TC_A_LBO <= e_lo_lo + TC_E_FLOATS * 4 &&
+                            bhi >= img_lo + TC_DIAG_FLOATS * 4 && bhi + panel_bytes <= img_lo + (TC_DIAG_FLOATS + TC_PANEL_FLOATS) * 4 &&
+                            blo >= img_lo + (TC_DIAG_FLOATS + TC_PANEL_FLOATS) * 4 && blo + panel_bytes <= img_lo + TC_IMG_FLOATS * 4 &&
+                            (a_lo & 15u) == 0 && (bhi & 15u) == 0 && (blo & 15u) == 0 &&
+                            (d & 0xffffu) + nb <= (t_tile & 0xffffu) + TC_EHI_COL &&
+                            (t_tile & 0xffffu) + TC_COLS_PER_TILE <= (tmem_base & 0xffffu) + TC_TMEM_COLS;
+                        if (sq_chk(desc_ok, p.status)) {
+#endif
 #pragma unroll
                         for (int ks = 0; ks < BLK / 8; ++ks)         // E_lo (shared memory) x Whi
                             umma_tf32_ss(d, umma_desc(a_lo + ks * 2 * TC_A_LBO, TC_A_LBO, TC_SBO),
@@ -567,6 +634,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
 #pragma unroll
                         for (int ks = 0; ks < BLK / 8; ++ks)         // E_hi x Whi
                             umma_tf32_ts(d, t_tile + TC_EHI_COL + 8 * ks, umma_desc(bhi + ks * 2 * b_lbo, b_lbo, TC_SBO), idesc, 1u);
+#ifdef SQUAT_CHECKED
+                        }
+#endif
                         umma_commit(my_mbar);
                     }
                     __syncwarp();
@@ -574,11 +644,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
 
                 if (cur.active) {
                     unsigned char *cp = cur.codes + blk * (BLK * BITS / 8);
-                    if (WORDS_PER_BLK == 2)
+                    if (!SQ_CHK_G(p.status, cp, BLK * BITS / 8, p.x_codes)) {
+                    } else if (WORDS_PER_BLK == 2)
                         *reinterpret_cast<uint2 *>(cp) = make_uint2(cw[0], cw[1]);
                     else
                         *reinterpret_cast<uint4 *>(cp) = make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
-                    if (wteam == 0) {
+                    if (wteam == 0 && SQ_CHK_G(p.status, static_cast<char *>(p.scales) + (cur.meta + blk * BLK) * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_scales) &&
+                        SQ_CHK_G(p.status, static_cast<char *>(p.zeros) + (cur.meta + blk * BLK) * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_zeros)) {
                         if (M16) {
                             reinterpret_cast<__half *>(p.scales)[cur.meta + blk * BLK] = __float2half_rn(my_scale);   // exact
                             reinterpret_cast<__half *>(p.zeros)[cur.meta + blk * BLK] = __float2half_rn(my_zero);
@@ -592,7 +664,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
                 }
             }
         } else if (nxt_valid) {
-            load_row<BF16>(raw, nxt_row, 0);
+            load_keys(raw, nxt_row, 0);
         }
         start += n_round;
     }
@@ -702,6 +774,18 @@ int squat_launch_quant_keys(const float *Wimg, const void *k, int dtype, int bat
     p.B = batch; p.H = H; p.T = T; p.groups_per_bh = T / G;
     p.status = status;
     p.exact_blocks = exact_blocks;
+#ifdef SQUAT_CHECKED
+    {
+        const unsigned long long es = dtype == SQUAT_BF16 ? 2 : 4, ms = meta16 ? 2 : 4;
+        const long long ng = T / G;
+        p.x_k = {k, (unsigned long long)((batch - 1) * sb + (H - 1) * sh + (long long)(T - 1) * st_ + D) * es};
+        p.x_codes = {codes, (unsigned long long)((batch - 1) * osb + (H - 1) * osh + T) * (D * bits / 8)};
+        const unsigned long long meta_elems = (unsigned long long)(((batch - 1) * osb + (H - 1) * osh) / G + ng) * D;
+        p.x_scales = {scales, meta_elems * ms};
+        p.x_zeros = {zeros, meta_elems * ms};
+        p.x_img = {Wimg, (unsigned long long)H * TC_IMG_FLOATS * 4};
+    }
+#endif
     if ((long long)H * batch * (T / G) == 0) return SQUAT_OK;
     if (bits == 2) {
         if (G == 32) return launch_keys<2, 1>(p, dtype, meta16, st);

@@ -163,6 +163,9 @@ struct LrParams {
     int spans_per_head;       // 32-token spans per head: B * T / 32
     int team_tasks;           // per head: tasks of one team (1 warp, or 2 for G = 128)
     unsigned *status;
+#ifdef SQUAT_CHECKED
+    SqExtent x_k, x_codes, x_scales, x_zeros, x_table;    // what the caller's tensors and the handle's tables span
+#endif
 };
 
 template <bool BF16>
@@ -217,7 +220,8 @@ __global__ void __launch_bounds__(LR_THREADS, 2) quant_keys_lowrank_kernel(const
     const int head = blockIdx.y;
     {
         const float4 *src = reinterpret_cast<const float4 *>(p.table + (long long)head * D * ROW);
-        for (int i = threadIdx.x; i < D * ROW / 4; i += LR_THREADS) reinterpret_cast<float4 *>(table)[i] = __ldg(src + i);
+        for (int i = threadIdx.x; i < D * ROW / 4; i += LR_THREADS)
+            if (SQ_CHK_G(p.status, src + i, 16, p.x_table)) reinterpret_cast<float4 *>(table)[i] = __ldg(src + i);
     }
     __syncthreads();
     float2(*meta)[BLK] = meta_all[warp];
@@ -259,7 +263,9 @@ __global__ void __launch_bounds__(LR_THREADS, 2) quant_keys_lowrank_kernel(const
             for (int jj = 0; jj < BLK; ++jj) {
                 if (jj % 16 == 0) {
 #pragma unroll
-                    for (int s = 0; s < 2; ++s) load16<BF16>(raw[s], row[s], blk * BLK + jj);
+                    for (int s = 0; s < 2; ++s)
+                        if (SQ_CHK_G(p.status, static_cast<const char *>(row[s]) + (blk * BLK + jj) * (BF16 ? 2 : 4), 16 * (BF16 ? 2 : 4), p.x_k))
+                            load16<BF16>(raw[s], row[s], blk * BLK + jj);
                 }
                 const ulonglong2 v01 = *reinterpret_cast<const ulonglong2 *>(tab + jj * ROW);
                 const ulonglong2 v23 = *reinterpret_cast<const ulonglong2 *>(tab + jj * ROW + 4);
@@ -343,12 +349,15 @@ __global__ void __launch_bounds__(LR_THREADS, 2) quant_keys_lowrank_kernel(const
                 for (int w = 0; w < WORDS_PER_BLK; ++w)
                     cw[w] = (uint32_t)__float2int_rn(cacc[s][2 * w]) | ((uint32_t)__float2int_rn(cacc[s][2 * w + 1]) << 16);
                 unsigned char *cp = cptr[s] + blk * (BLK * BITS / 8);
-                if (WORDS_PER_BLK == 2)
+                if (!SQ_CHK_G(p.status, cp, BLK * BITS / 8, p.x_codes)) {
+                } else if (WORDS_PER_BLK == 2)
                     *reinterpret_cast<uint2 *>(cp) = make_uint2(cw[0], cw[1]);
                 else
                     *reinterpret_cast<uint4 *>(cp) = make_uint4(cw[0], cw[1], cw[WORDS_PER_BLK > 2 ? 2 : 0], cw[WORDS_PER_BLK > 2 ? 3 : 0]);
                 // the group's metadata: one store per group (span 0 of warp 0 of the team unless the spans are groups)
-                if (TWO_GROUPS || (s == 0 && wteam == 0)) {
+                if ((TWO_GROUPS || (s == 0 && wteam == 0)) &&
+                    SQ_CHK_G(p.status, static_cast<char *>(p.scales) + (meta_off[s] + blk * BLK) * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_scales) &&
+                    SQ_CHK_G(p.status, static_cast<char *>(p.zeros) + (meta_off[s] + blk * BLK) * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_zeros)) {
                     const float2 sz = meta[s][lane];                 // lane = channel within the block
                     if (M16) {
                         reinterpret_cast<__half *>(p.scales)[meta_off[s] + blk * BLK] = __float2half_rn(sz.x);   // exact
@@ -413,6 +422,17 @@ int squat_launch_quant_keys_lowrank(const float *table, const void *k, int dtype
     const int spans_per_task = G == 128 ? 4 : 2;
     p.team_tasks = (int)((spans + spans_per_task - 1) / spans_per_task);
     p.status = status;
+#ifdef SQUAT_CHECKED
+    {
+        const unsigned long long es = dtype == SQUAT_BF16 ? 2 : 4, ms = meta16 ? 2 : 4;
+        p.x_k = {k, (unsigned long long)((batch - 1) * sb + (H - 1) * sh + (long long)(T - 1) * st_ + D) * es};
+        p.x_codes = {codes, (unsigned long long)((batch - 1) * osb + (H - 1) * osh + T) * (D * bits / 8)};
+        const unsigned long long meta_elems = (unsigned long long)(((batch - 1) * osb + (H - 1) * osh) / G + T / G) * D;
+        p.x_scales = {scales, meta_elems * ms};
+        p.x_zeros = {zeros, meta_elems * ms};
+        p.x_table = {table, (unsigned long long)H * D * ROW * 4};
+    }
+#endif
     if (bits == 2) {
         if (G == 32) return launch_lowrank<2, 32>(p, H, dtype, meta16, st);
         if (G == 64) return launch_lowrank<2, 64>(p, H, dtype, meta16, st);

@@ -75,6 +75,37 @@ int squat_launch_dequant(int kind, const unsigned char *codes, const void *scale
                          int batch, int H, int T, int d, int bits, int G, long long isb, long long ish,
                          void *out, int out_dtype, int meta16, cudaStream_t st);
 
+// ---- the bounds-checked build ----------------------------------------------------------
+// Compiled with -DSQUAT_CHECKED (build.py --checked -> libsquat_checked.so) the key and value kernels test every
+// global, shared-memory and tensor-memory address they form (and the shared-memory windows of the matrix descriptors
+// they hand to the tensor core) against the extent of the buffer or region it belongs to; an address outside sets
+// SQUAT_FLAG_BOUNDS in the device status word and the access is skipped -- never a trap.  The stand-in for a memory
+// checker on machines where none can be run; the tests drive small and ragged cases through it.  In the normal build
+// every macro below folds to `true` and the extents do not exist.
+#ifdef SQUAT_CHECKED
+struct SqExtent {
+    const void *base;
+    unsigned long long bytes;
+};
+__device__ __forceinline__ bool sq_chk(bool ok, unsigned *status)
+{
+    if (!ok) atomicOr(status, SQUAT_FLAG_BOUNDS);
+    return ok;
+}
+__device__ __forceinline__ bool sq_inside(const void *ptr, unsigned long long n, const void *base, unsigned long long bytes)
+{
+    const unsigned long long a = (unsigned long long)ptr, b = (unsigned long long)base;
+    return a >= b && a + n <= b + bytes;
+}
+#define SQ_CHK_G(status, ptr, n, ext) sq_chk(sq_inside((ptr), (n), (ext).base, (ext).bytes), (status))       /* global memory */
+#define SQ_CHK_R(status, ptr, n, base, bytes) sq_chk(sq_inside((ptr), (n), (base), (bytes)), (status))      /* a region (shared memory) */
+#define SQ_CHK_C(status, cond) sq_chk((cond), (status))                                                      /* any condition */
+#else
+#define SQ_CHK_G(status, ptr, n, ext) true
+#define SQ_CHK_R(status, ptr, n, base, bytes) true
+#define SQ_CHK_C(status, cond) true
+#endif
+
 // ---- small device helpers --------------------------------------------------------------
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }

@@ -77,6 +77,9 @@ struct ValParams {
     long long osb, osh;                   // output strides in tokens
     int row_bytes;                        // code bytes per token
     unsigned *status;
+#ifdef SQUAT_CHECKED
+    SqExtent x_v, x_codes, x_scales, x_zeros;      // what the caller's tensors span
+#endif
 };
 
 constexpr int VAL_THREADS = 256;
@@ -149,7 +152,10 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
         const uint4 *src = BF16 ? reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.v) + in_off)
                                 : reinterpret_cast<const uint4 *>(reinterpret_cast<const float *>(p.v) + in_off);
 #pragma unroll
-        for (int i = 0; i < NV; ++i) raw[i] = ldg128(src + i);
+        for (int i = 0; i < NV; ++i) {
+            raw[i] = make_uint4(0, 0, 0, 0);
+            if (SQ_CHK_G(p.status, src + i, 16, p.x_v)) raw[i] = ldg128(src + i);
+        }
     }
     // channel pair c (channels 2c, 2c + 1) as two floats, exact widening
     auto pair_of = [&](int c, float &x0, float &x1) {
@@ -240,6 +246,11 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
     }
 
     unsigned char *cp = p.codes + out_tok * p.row_bytes + (long long)q * (G * BITS / 8);
+    const long long meta_idx = out_tok * p.ng + q;
+    if (!SQ_CHK_G(p.status, cp, G * BITS / 8, p.x_codes) ||
+        !SQ_CHK_G(p.status, static_cast<char *>(p.scales) + meta_idx * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_scales) ||
+        !SQ_CHK_G(p.status, static_cast<char *>(p.zeros) + meta_idx * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_zeros))
+        return;
     if (NWORDS % 4 == 0) {
 #pragma unroll
         for (int i = 0; i < NWORDS / 4; ++i)
@@ -249,7 +260,6 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
         for (int i = 0; i < NWORDS / 2; ++i)
             reinterpret_cast<uint2 *>(cp)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
     }
-    const long long meta_idx = out_tok * p.ng + q;
     if (M16) {
         reinterpret_cast<__half *>(p.scales)[meta_idx] = __float2half_rn(delta);      // exact: already binary16 values
         reinterpret_cast<__half *>(p.zeros)[meta_idx] = __float2half_rn(m);
@@ -417,6 +427,16 @@ int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T,
     p.codes = codes; p.scales = scales; p.zeros = zeros; p.osb = osb; p.osh = osh;
     p.row_bytes = d * bits / 8;
     p.status = status;
+#ifdef SQUAT_CHECKED
+    {
+        const unsigned long long es = dtype == SQUAT_BF16 ? 2 : 4, ms = meta16 ? 2 : 4;
+        p.x_v = {v, (unsigned long long)((batch - 1) * sb + (H - 1) * sh + (long long)(T - 1) * st_ + d) * es};
+        const unsigned long long toks = (unsigned long long)((batch - 1) * osb + (H - 1) * osh + T);
+        p.x_codes = {codes, toks * p.row_bytes};
+        p.x_scales = {scales, toks * p.ng * ms};
+        p.x_zeros = {zeros, toks * p.ng * ms};
+    }
+#endif
 #define SQ_V(GG, BB) return launch_values<GG, BB>(p, rows, dtype, meta16, st)
     if (bits == 2) { if (G == 32) SQ_V(32, 2); if (G == 64) SQ_V(64, 2); if (G == 128) SQ_V(128, 2); }
     if (bits == 4) { if (G == 32) SQ_V(32, 4); if (G == 64) SQ_V(64, 4); if (G == 128) SQ_V(128, 4); }
