@@ -71,6 +71,37 @@ __device__ __forceinline__ float code_as_float(uint32_t w, int i)
     return __uint_as_float((sh & MASK) | 0x3F800000u);
 }
 
+// Two neighbouring 2-bit codes (positions 2 j and 2 j + 1 of a word) as floats with ONE shift: their 4-bit window goes
+// to mantissa bits 19..22.  The upper code, under the exponent of 1, reads 1 + c/4; the lower one, two mantissa bits
+// further down, is put under the exponent of 4 and reads 4 + c/4 -- the same step per level, a different constant,
+// which goes into the per-group constant like the "1 +".
+__device__ __forceinline__ void code_pair_as_floats(uint32_t w, int j, float &f_even, float &f_odd)
+{
+    const int pos = 4 * j;
+    const uint32_t sh = pos <= 19 ? (w << (19 - pos)) : (w >> (pos - 19));
+    f_even = __uint_as_float((sh & 0x00180000u) | 0x40800000u);
+    f_odd = __uint_as_float((sh & 0x00600000u) | 0x3F800000u);
+}
+typedef unsigned long long u64;
+__device__ __forceinline__ u64 pack2f(float lo, float hi)
+{
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ u64 ffma2(u64 a, u64 b, u64 c)
+{
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float sum2f(u64 v)
+{
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return lo + hi;
+}
+
 __device__ __forceinline__ float warp_sum_f(float v)
 {
 #pragma unroll
@@ -116,6 +147,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
     constexpr int WPT = D * BITS / 32;                          // 32-bit words per token: 8 or 16
     constexpr int CPW = 32 / BITS;                              // codes per word: 16 or 8
     constexpr float LV = float(1 << BITS);
+    constexpr bool PAIRS = BITS == 2 && NQ <= 2;                // two codes per shift and packed multiply-adds (code_pair_as_floats)
     extern __shared__ __align__(16) float sm[];
     float *qsm = sm;                                            // [NQ][D]      q * softmax scale
     float *qs = qsm + NQ * D;                                   // [warps][NQ][D] query x key scale x 2^BITS of the warp's group
@@ -204,10 +236,43 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
             const float4 v = make_float4(qv.x * s4.x * LV, qv.y * s4.y * LV, qv.z * s4.z * LV, qv.w * s4.w * LV);
             *reinterpret_cast<float4 *>(qsw + qi * D + 4 * lane) = v;
             const float zs = qv.x * z4.x + qv.y * z4.y + qv.z * z4.z + qv.w * z4.w;
-            k0[qi] = warp_sum_f(zs - (v.x + v.y + v.z + v.w));  // sum_c q_c zero_c - sum_c qs'_c  (takes the "1 +" out)
+            // sum_c q_c zero_c - sum_c qs'_c bias_c takes the codes' constants out again: "1 +", or for 2-bit codes
+            // "4 +" on even and "1 +" on odd channels (code_pair_as_floats)
+            k0[qi] = PAIRS ? warp_sum_f(zs - (4.0f * v.x + v.y + 4.0f * v.z + v.w)) : warp_sum_f(zs - (v.x + v.y + v.z + v.w));
         }
         __syncwarp();
         const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
+        if (PAIRS) {
+            // two channels per instruction: (f_even, f_odd) x (q'_even, q'_odd) into two packed accumulators per head
+            u64 acc2[NQ][2];
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) acc2[qi][0] = acc2[qi][1] = 0ull;
+#pragma unroll
+            for (int v4 = 0; v4 < WPT / 4; ++v4) {
+                const uint4 cw = __ldg(cp + v4);
+                const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+                for (int wi = 0; wi < 4; ++wi)
+#pragma unroll
+                    for (int i4 = 0; i4 < CPW / 4; ++i4) {
+                        const int ch = (v4 * 4 + wi) * CPW + 4 * i4;
+                        float f0, f1, f2, f3;
+                        code_pair_as_floats(w4[wi], 2 * i4, f0, f1);
+                        code_pair_as_floats(w4[wi], 2 * i4 + 1, f2, f3);
+                        const u64 fa = pack2f(f0, f1), fb = pack2f(f2, f3);
+#pragma unroll
+                        for (int qi = 0; qi < NQ; ++qi) {
+                            const ulonglong2 qq = *reinterpret_cast<const ulonglong2 *>(qsw + qi * D + ch);
+                            acc2[qi][0] = ffma2(fa, qq.x, acc2[qi][0]);
+                            acc2[qi][1] = ffma2(fb, qq.y, acc2[qi][1]);
+                        }
+                    }
+            }
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi)
+                sc[qi * AT_CHUNK + blk - t0 + lane] = (sum2f(acc2[qi][0]) + sum2f(acc2[qi][1])) + k0[qi];
+            continue;
+        }
         float acc[NQ][4];                                      // four partial sums per query head: independent FMA chains
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi) acc[qi][0] = acc[qi][1] = acc[qi][2] = acc[qi][3] = 0.0f;
@@ -281,10 +346,16 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
     constexpr int TPI = 32 / WPT;                               // tokens per warp step: 4 or 2
     const int ts = lane / WPT, j = lane % WPT;
     const int ng = D / p.G, gidx = (j * CPW) / p.G;
-    float accv[NQ][CPW], corr[NQ];
+    // packed pairs (even channel, odd channel); corr takes the codes' constants out: "1 +", or for 2-bit codes "4 +" on even
+    // and "1 +" on odd channels (code_pair_as_floats)
+    u64 accv2[NQ][CPW / 2];                                    // PAIRS
+    float accv[NQ][CPW];                                        // otherwise
+    float corr[NQ], corr_even[NQ];
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
-        corr[qi] = 0.0f;
+        corr[qi] = corr_even[qi] = 0.0f;
+#pragma unroll
+        for (int i = 0; i < CPW / 2; ++i) accv2[qi][i] = 0ull;
 #pragma unroll
         for (int i = 0; i < CPW; ++i) accv[qi][i] = 0.0f;
     }
@@ -294,18 +365,38 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
     const uint32_t *vcw = reinterpret_cast<const uint32_t *>(p.vc);
     auto vstep = [&](int tk, uint32_t w, float vs_raw, float vzr) {
         const float vsc = vs_raw * LV;
-        float a[NQ];
+        if (PAIRS) {
+            u64 a2[NQ];
 #pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) {
-            const float pw = sc[qi * AT_CHUNK + tk - t0];
-            a[qi] = pw * vsc;
-            corr[qi] += pw * vzr - a[qi];
-        }
+            for (int qi = 0; qi < NQ; ++qi) {
+                const float pw = sc[qi * AT_CHUNK + tk - t0];
+                const float a = pw * vsc, pz = pw * vzr;
+                a2[qi] = pack2f(a, a);
+                corr[qi] += pz - a;
+                corr_even[qi] += fmaf(-4.0f, a, pz);
+            }
 #pragma unroll
-        for (int i = 0; i < CPW; ++i) {
-            const float f = code_as_float<BITS>(w, i);
+            for (int i = 0; i < CPW / 2; ++i) {
+                float fe, fo;
+                code_pair_as_floats(w, i, fe, fo);
+                const u64 f2 = pack2f(fe, fo);
 #pragma unroll
-            for (int qi = 0; qi < NQ; ++qi) accv[qi][i] = fmaf(f, a[qi], accv[qi][i]);
+                for (int qi = 0; qi < NQ; ++qi) accv2[qi][i] = ffma2(f2, a2[qi], accv2[qi][i]);
+            }
+        } else {
+            float a[NQ];
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) {
+                const float pw = sc[qi * AT_CHUNK + tk - t0];
+                a[qi] = pw * vsc;
+                corr[qi] += pw * vzr - a[qi];
+            }
+#pragma unroll
+            for (int i = 0; i < CPW; ++i) {
+                const float f = code_as_float<BITS>(w, i);
+#pragma unroll
+                for (int qi = 0; qi < NQ; ++qi) accv[qi][i] = fmaf(f, a[qi], accv[qi][i]);
+            }
         }
     };
     int tk = vbase + ts;
@@ -328,7 +419,14 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
     for (int qi = 0; qi < NQ; ++qi)
 #pragma unroll
         for (int i = 0; i < CPW; ++i) {
-            float v = accv[qi][i] + corr[qi];
+            float v;
+            if (PAIRS) {
+                float lo_, hi_;
+                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo_), "=f"(hi_) : "l"(accv2[qi][i / 2]));
+                v = (i & 1) ? hi_ + corr[qi] : lo_ + corr_even[qi];
+            } else {
+                v = accv[qi][i] + corr[qi];
+            }
 #pragma unroll
             for (int m = WPT; m < 32; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
             if (ts == 0) part_sm[(warp * NQ + qi) * D + j * CPW + i] = v;
