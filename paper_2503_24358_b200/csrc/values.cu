@@ -69,7 +69,7 @@ __device__ __noinline__ uint32_t exact_code_bits(float dlt, float delta)
 struct ValParams {
     const void *v;
     int H, T, ng;                         // ng = groups per token
-    int ng_shift;                         // log2(ng) when ng is a power of two, else -1
+    int ns, ns_shift;                     // ns = 32-channel spans per token (d / 32); its log2 when a power of two, else -1
     unsigned chunks_per_row;              // CTAs per (batch, head) row
     long long sb, sh, st;                 // element strides of v
     unsigned char *codes;
@@ -125,26 +125,35 @@ __device__ __noinline__ unsigned patch_word(unsigned word, unsigned mask, const 
     return word;
 }
 
-// One thread owns one (token, channel group): G channels in registers (G / 8 or G / 4 16-byte loads in flight).  One CTA
-// works VAL_THREADS consecutive groups of one (batch, head) row (blockIdx.x = row * chunks + chunk), so the only
-// divisions are two per CTA; a group's token is a shift (d / G a power of two) or one 32-bit division.
+// One thread owns a span of 32 consecutive channels of one token in registers (4 or 8 16-byte loads in flight); a group
+// of G channels is 1, 2 or 4 neighbouring lanes, which combine their min / max with warp shuffles.  One CTA works
+// VAL_THREADS consecutive spans of one (batch, head) row (blockIdx.x = row * chunks + chunk), so the only divisions are
+// two per CTA; a span's token is a shift (d / 32 a power of two) or one 32-bit division.
 template <int G, int BITS, bool BF16, bool M16>
 __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValParams p)
 {
     constexpr float L = float((1 << BITS) - 1);
-    constexpr int NV = BF16 ? G / 8 : G / 4;        // 16-byte pieces of a group
+    constexpr int SPAN = 32;                        // channels per thread
+    constexpr int LPG = G / SPAN;                   // lanes per group: 1, 2 or 4
+    constexpr int NV = BF16 ? SPAN / 8 : SPAN / 4;  // 16-byte pieces of a span
     constexpr int PER_WORD = 32 / BITS;             // codes per 32-bit word
-    constexpr int NWORDS = G / PER_WORD;
+    constexpr int NWORDS = SPAN / PER_WORD;
     // what the constant upper bits of the rounded floats add up to in a packed word
     constexpr unsigned K = [] { unsigned k = 0; for (int i = 0; i < PER_WORD; ++i) k += kMagicBits << (BITS * i); return k; }();
 
     const unsigned row = blockIdx.x / p.chunks_per_row, chunk = blockIdx.x - row * p.chunks_per_row;
     const unsigned b = row / (unsigned)p.H, h = row - b * (unsigned)p.H;
-    const unsigned u = chunk * VAL_THREADS + threadIdx.x;                        // group within the row
-    if (u >= (unsigned)p.T * (unsigned)p.ng) return;
-    const unsigned tok = p.ng_shift >= 0 ? u >> p.ng_shift : u / (unsigned)p.ng;
-    const unsigned q = u - tok * (unsigned)p.ng;
-    const long long in_off = (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st + (long long)q * G;
+    const unsigned u0 = chunk * VAL_THREADS + threadIdx.x;                       // span within the row
+    const unsigned n_row = (unsigned)p.T * (unsigned)p.ns;
+    if (u0 - (threadIdx.x & 31) >= n_row) return;                                // the whole warp is past the row
+    // whole groups are valid or not (spans per token are a multiple of LPG): the spare lanes of the row's last warp redo
+    // its last span, take part in the shuffles and store nothing
+    const bool valid = u0 < n_row;
+    const unsigned u = valid ? u0 : n_row - 1;
+    const unsigned tok = p.ns_shift >= 0 ? u >> p.ns_shift : u / (unsigned)p.ns;
+    const unsigned sp = u - tok * (unsigned)p.ns;                                // span within the token
+    const unsigned q = sp / LPG;                                                 // its group
+    const long long in_off = (long long)b * p.sb + (long long)h * p.sh + (long long)tok * p.st + (long long)sp * SPAN;
     const long long out_tok = (long long)b * p.osb + (long long)h * p.osh + tok;
 
     uint4 raw[NV];
@@ -189,11 +198,17 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
         m = min_nan(x0, x1);
         Mx = max_nan(x0, x1);
 #pragma unroll
-        for (int c = 1; c < G / 2; ++c) {
+        for (int c = 1; c < SPAN / 2; ++c) {
             pair_of(c, x0, x1);
             m = min_nan(m, min_nan(x0, x1));
             Mx = max_nan(Mx, max_nan(x0, x1));
         }
+    }
+
+#pragma unroll
+    for (int o = 1; o < LPG; o <<= 1) {                 // the group's other lanes
+        m = min_nan(m, __shfl_xor_sync(0xffffffffu, m, o));
+        Mx = max_nan(Mx, __shfl_xor_sync(0xffffffffu, Mx, o));
     }
 
     // ---- the grid
@@ -245,9 +260,10 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
         words[wd] = ok ? acc_a : 0u;                    // no grid (constant or non-finite group): codes 0
     }
 
-    unsigned char *cp = p.codes + out_tok * p.row_bytes + (long long)q * (G * BITS / 8);
+    if (!valid) return;
+    unsigned char *cp = p.codes + out_tok * p.row_bytes + (long long)sp * (SPAN * BITS / 8);
     const long long meta_idx = out_tok * p.ng + q;
-    if (!SQ_CHK_G(p.status, cp, G * BITS / 8, p.x_codes) ||
+    if (!SQ_CHK_G(p.status, cp, SPAN * BITS / 8, p.x_codes) ||
         !SQ_CHK_G(p.status, static_cast<char *>(p.scales) + meta_idx * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_scales) ||
         !SQ_CHK_G(p.status, static_cast<char *>(p.zeros) + meta_idx * (M16 ? 2 : 4), M16 ? 2 : 4, p.x_zeros))
         return;
@@ -260,6 +276,7 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
         for (int i = 0; i < NWORDS / 2; ++i)
             reinterpret_cast<uint2 *>(cp)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
     }
+    if (LPG > 1 && (sp & (LPG - 1)) != 0) return;       // one lane per group stores its grid
     if (M16) {
         reinterpret_cast<__half *>(p.scales)[meta_idx] = __float2half_rn(delta);      // exact: already binary16 values
         reinterpret_cast<__half *>(p.zeros)[meta_idx] = __float2half_rn(m);
@@ -415,11 +432,12 @@ int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T,
     const long long rows = (long long)batch * H;
     if (rows == 0 || T == 0) return SQUAT_OK;
     ValParams p;
-    p.v = v; p.H = H; p.T = T; p.ng = d / G;
-    p.ng_shift = -1;
+    if (d % 32 != 0) return SQUAT_ERR_SHAPE;
+    p.v = v; p.H = H; p.T = T; p.ng = d / G; p.ns = d / 32;
+    p.ns_shift = -1;
     for (int sft = 0; sft < 20; ++sft)
-        if ((1 << sft) == p.ng) p.ng_shift = sft;
-    const long long row_units = (long long)T * p.ng;
+        if ((1 << sft) == p.ns) p.ns_shift = sft;
+    const long long row_units = (long long)T * p.ns;
     const long long chunks = (row_units + VAL_THREADS - 1) / VAL_THREADS;
     if (row_units > 0x7fffffffLL || rows * chunks > 0x7fffffffLL) return SQUAT_ERR_UNSUPPORTED;    // 32-bit group and CTA indices
     p.chunks_per_row = (unsigned)chunks;

@@ -57,6 +57,33 @@ def test_algorithmic_counts():
     assert bench.reader_bytes_per_cached_token(128, 2, 32, meta_bytes=2) == 32 + 32 + 16 + 16
 
 
+def test_key_roofline_is_the_slowest_of_the_three_floors():
+    import argparse
+    import squat_inputs as si
+    args = argparse.Namespace(meta16=False)
+    peaks = {"hbm_gbs": 6549.8, "bf16_tflops": 1649.9, "source": "measured"}
+    fp32 = {"tflops": 73.0, "fma_f32_tflops": 71.0, "fma_f32x2_tflops": 73.0}
+    cfg = si.get_config(1)
+    vec = cfg.batch * cfg.n_kv_heads * cfg.n_tokens
+    r = bench.key_roofline(args, cfg, 0.053, vec, peaks, fp32)
+    # dense kernel on workload 1: the in-block triangles (1 984 multiply-adds per vector on the FP32 pipes) set the floor
+    assert r["bound"] == "alu" and r["peak"] == 73.0
+    assert abs(r["pipes"]["fp32_floor_us"] - 2 * 1984 * vec / 73.0e12 * 1e6) < 1e-9
+    assert abs(r["pipes"]["tensor_floor_us"] - 6 * 6144 * vec / (0.5 * 1649.9e12) * 1e6) < 1e-9
+    assert abs(r["pipes"]["hbm_floor_us"] - 320 * vec / 6549.8e9 * 1e6) < 1e-9
+    assert r["pipes"]["floor_us"] == max(r["pipes"][k] for k in ("fp32_floor_us", "tensor_floor_us", "hbm_floor_us"))
+    assert abs(r["frac"] - r["pipes"]["floor_us"] / 53.0) < 1e-9 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-12
+    assert abs(r["frac_vs_fp32_target"] - 16256 * vec / 0.053e-3 / 1e12 / bench.ALU_PEAK_TFLOPS) < 1e-9
+    # the rank-r kernel runs 2 r d multiply-adds per vector on the FP32 pipes and nothing on the tensor cores
+    c4 = si.get_config(4).with_(rank_r=8)
+    r8 = bench.key_roofline(args, c4, 1.0, 4 * 32 * 32768, peaks, fp32, lowrank_r=8)
+    assert r8["pipes"]["fp32_fma_per_vector"] == 2048 and r8["pipes"]["tensor_fma_per_vector"] == 0
+    assert r8["bound"] in ("alu", "hbm") and r8["kernel"].startswith("quant_keys_lowrank_kernel")
+    # W = 0: nothing to push, the bytes bind
+    r0 = bench.key_roofline(args, cfg.with_(rank_r=0), 0.05, vec, peaks, fp32)
+    assert r0["bound"] == "hbm"
+
+
 def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
     env = dict(os.environ, RANK="0", WORLD_SIZE="1")
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "0",
