@@ -29,6 +29,7 @@ constexpr int BLK = 32;
 constexpr int NBLK = D / BLK;
 constexpr int LR_WARPS = 8;
 constexpr int LR_THREADS = LR_WARPS * 32;
+constexpr int LR_CTAS_PER_SM = 3;          // 80 registers per thread: 24 warps per SM
 constexpr float kMagic = 12582912.0f;      // 1.5 * 2^23
 
 typedef unsigned long long u64;
@@ -202,7 +203,7 @@ __device__ __forceinline__ float chan_of(const Raw16<BF16> &r, int c)      // c 
 
 // G: 32 (the warp's two spans are two groups), 64 (one group), 128 (half a group; NW = 2 warps share a group)
 template <int BITS, int G, bool BF16, bool M16>
-__global__ void __launch_bounds__(LR_THREADS, 2) quant_keys_lowrank_kernel(const LrParams p)
+__global__ void __launch_bounds__(LR_THREADS, LR_CTAS_PER_SM) quant_keys_lowrank_kernel(const LrParams p)
 {
     constexpr float L = float((1 << BITS) - 1);
     constexpr int NW = G == 128 ? 2 : 1;
@@ -383,7 +384,7 @@ int launch_lowrank(const LrParams &p, int H, int dtype, int meta16, cudaStream_t
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     constexpr int TEAMS = LR_WARPS / (G == 128 ? 2 : 1);
     const int ctas_needed = (p.team_tasks + TEAMS - 1) / TEAMS;
-    int per_head = (4 * sms + H - 1) / H;                 // two waves of two resident CTAs per SM, over all heads
+    int per_head = (2 * LR_CTAS_PER_SM * sms + H - 1) / H;   // two waves of the resident CTAs, over all heads
     if (per_head > ctas_needed) per_head = ctas_needed;
     if (per_head < 1) per_head = 1;
     const dim3 grid(per_head, H);
