@@ -61,26 +61,46 @@ struct AttnParams {
 };
 
 // 1 + code / 2^BITS as a float, for the code at position i of a 32-bit word (low bits first)
+// A constant the compiler has to keep in a register: `(x & mask) | constant` is then ONE three-input logic instruction
+// (mask as its immediate); with both as immediates it takes two, and the unpacking below is what fills the integer pipe.
+// (x & MASK) | c as one three-input logic instruction
+template <uint32_t MASK>
+__device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "n"(MASK), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t in_register(uint32_t v)
+{
+    uint32_t r;
+    asm volatile("mov.b32 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
+}
+// one_bits: the bit pattern of 1.0f, held in a register (in_register)
 template <int BITS>
-__device__ __forceinline__ float code_as_float(uint32_t w, int i)
+__device__ __forceinline__ float code_as_float(uint32_t w, int i, uint32_t one_bits)
 {
     constexpr int TOP = 23 - BITS;                              // the code's low bit lands here
     constexpr uint32_t MASK = ((1u << BITS) - 1u) << TOP;
     const int pos = BITS * i;
-    const uint32_t sh = pos <= TOP ? (w << (TOP - pos)) : (w >> (pos - TOP));
-    return __uint_as_float((sh & MASK) | 0x3F800000u);
+    uint32_t sh = pos <= TOP ? (w << (TOP - pos)) : (w >> (pos - TOP));
+    asm("" : "+r"(sh));                                        // keep the shift where it is (not re-associated behind the mask)
+    return __uint_as_float(and_or<MASK>(sh, one_bits));
 }
 
 // Two neighbouring 2-bit codes (positions 2 j and 2 j + 1 of a word) as floats with ONE shift: their 4-bit window goes
 // to mantissa bits 19..22.  The upper code, under the exponent of 1, reads 1 + c/4; the lower one, two mantissa bits
 // further down, is put under the exponent of 4 and reads 4 + c/4 -- the same step per level, a different constant,
 // which goes into the per-group constant like the "1 +".
-__device__ __forceinline__ void code_pair_as_floats(uint32_t w, int j, float &f_even, float &f_odd)
+// one_bits, four_bits: the bit patterns of 1.0f and 4.0f, held in registers (in_register)
+__device__ __forceinline__ void code_pair_as_floats(uint32_t w, int j, float &f_even, float &f_odd, uint32_t one_bits, uint32_t four_bits)
 {
     const int pos = 4 * j;
-    const uint32_t sh = pos <= 19 ? (w << (19 - pos)) : (w >> (pos - 19));
-    f_even = __uint_as_float((sh & 0x00180000u) | 0x40800000u);
-    f_odd = __uint_as_float((sh & 0x00600000u) | 0x3F800000u);
+    uint32_t sh = pos <= 19 ? (w << (19 - pos)) : (w >> (pos - 19));
+    asm("" : "+r"(sh));                                        // one shift for both codes: not re-associated behind the masks
+    f_even = __uint_as_float(and_or<0x00180000u>(sh, four_bits));
+    f_odd = __uint_as_float(and_or<0x00600000u>(sh, one_bits));
 }
 typedef unsigned long long u64;
 __device__ __forceinline__ u64 pack2f(float lo, float hi)
@@ -148,6 +168,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
     constexpr int CPW = 32 / BITS;                              // codes per word: 16 or 8
     constexpr float LV = float(1 << BITS);
     constexpr bool PAIRS = BITS == 2 && NQ <= 2;                // two codes per shift and packed multiply-adds (code_pair_as_floats)
+    const uint32_t one_bits = in_register(0x3F800000u), four_bits = in_register(0x40800000u);
     extern __shared__ __align__(16) float sm[];
     float *qsm = sm;                                            // [NQ][D]      q * softmax scale
     float *qs = qsm + NQ * D;                                   // [warps][NQ][D] query x key scale x 2^BITS of the warp's group
@@ -212,8 +233,8 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
                 for (int pos = 0; pos < CPW; ++pos) {
                     const int i = wi * CPW + pos;                       // pair (i, i + 64): same code position, WPT / 2 words apart
                     const float4 m4 = sz[i];
-                    const float k0 = fmaf(code_as_float<BITS>(wd[wi], pos), m4.x, m4.y);
-                    const float k1 = fmaf(code_as_float<BITS>(wd[wi + WPT / 2], pos), m4.z, m4.w);
+                    const float k0 = fmaf(code_as_float<BITS>(wd[wi], pos, one_bits), m4.x, m4.y);
+                    const float k1 = fmaf(code_as_float<BITS>(wd[wi + WPT / 2], pos, one_bits), m4.z, m4.w);
                     const float2 cs = lane_turn[i * 32 + lane];
                     const float r0 = fmaf(k0, cs.x, -k1 * cs.y), r1 = fmaf(k0, cs.y, k1 * cs.x);
 #pragma unroll
@@ -257,8 +278,8 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
                     for (int i4 = 0; i4 < CPW / 4; ++i4) {
                         const int ch = (v4 * 4 + wi) * CPW + 4 * i4;
                         float f0, f1, f2, f3;
-                        code_pair_as_floats(w4[wi], 2 * i4, f0, f1);
-                        code_pair_as_floats(w4[wi], 2 * i4 + 1, f2, f3);
+                        code_pair_as_floats(w4[wi], 2 * i4, f0, f1, one_bits, four_bits);
+                        code_pair_as_floats(w4[wi], 2 * i4 + 1, f2, f3, one_bits, four_bits);
                         const u64 fa = pack2f(f0, f1), fb = pack2f(f2, f3);
 #pragma unroll
                         for (int qi = 0; qi < NQ; ++qi) {
@@ -271,8 +292,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
 #pragma unroll
             for (int qi = 0; qi < NQ; ++qi)
                 sc[qi * AT_CHUNK + blk - t0 + lane] = (sum2f(acc2[qi][0]) + sum2f(acc2[qi][1])) + k0[qi];
-            continue;
-        }
+        } else {
         float acc[NQ][4];                                      // four partial sums per query head: independent FMA chains
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi) acc[qi][0] = acc[qi][1] = acc[qi][2] = acc[qi][3] = 0.0f;
@@ -285,8 +305,8 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
 #pragma unroll
                 for (int i4 = 0; i4 < CPW / 4; ++i4) {
                     const int ch = (v4 * 4 + wi) * CPW + 4 * i4;
-                    const float f0 = code_as_float<BITS>(w4[wi], 4 * i4), f1 = code_as_float<BITS>(w4[wi], 4 * i4 + 1),
-                                f2 = code_as_float<BITS>(w4[wi], 4 * i4 + 2), f3 = code_as_float<BITS>(w4[wi], 4 * i4 + 3);
+                    const float f0 = code_as_float<BITS>(w4[wi], 4 * i4, one_bits), f1 = code_as_float<BITS>(w4[wi], 4 * i4 + 1, one_bits),
+                                f2 = code_as_float<BITS>(w4[wi], 4 * i4 + 2, one_bits), f3 = code_as_float<BITS>(w4[wi], 4 * i4 + 3, one_bits);
 #pragma unroll
                     for (int qi = 0; qi < NQ; ++qi) {
                         const float4 qq = *reinterpret_cast<const float4 *>(qsw + qi * D + ch);
@@ -300,6 +320,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi)
             sc[qi * AT_CHUNK + blk - t0 + lane] = ((acc[qi][0] + acc[qi][1]) + (acc[qi][2] + acc[qi][3])) + k0[qi];
+        }
     }
     __syncthreads();
 
@@ -378,7 +399,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
 #pragma unroll
             for (int i = 0; i < CPW / 2; ++i) {
                 float fe, fo;
-                code_pair_as_floats(w, i, fe, fo);
+                code_pair_as_floats(w, i, fe, fo, one_bits, four_bits);
                 const u64 f2 = pack2f(fe, fo);
 #pragma unroll
                 for (int qi = 0; qi < NQ; ++qi) accv2[qi][i] = ffma2(f2, a2[qi], accv2[qi][i]);
@@ -393,7 +414,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
             }
 #pragma unroll
             for (int i = 0; i < CPW; ++i) {
-                const float f = code_as_float<BITS>(w, i);
+                const float f = code_as_float<BITS>(w, i, one_bits);
 #pragma unroll
                 for (int qi = 0; qi < NQ; ++qi) accv[qi][i] = fmaf(f, a[qi], accv[qi][i]);
             }

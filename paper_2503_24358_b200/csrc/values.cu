@@ -287,6 +287,31 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
     if (!ok) atomicOr(p.status, delta == 0.0f ? SQUAT_FLAG_ZERO_RANGE : SQUAT_FLAG_NONFINITE);
 }
 
+// (x & MASK) | c as ONE three-input logic instruction (left to itself the compiler emits two)
+template <uint32_t MASK>
+__device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "n"(MASK), "r"(c));
+    return d;
+}
+
+// Channels (2 I, 2 I + 1) of a thread's 8 codes as two exact floats: each code, masked in place at bit position s, is OR-ed
+// under the exponent of 2^(23 - s) (the pair `bias`, held in registers), which makes the word 2^(23 - s) + c; subtracting
+// the bias leaves c.  4-bit codes of channels 4..7 sit in the upper half of the word (`hi` = word >> 16).
+template <int BITS, int I>
+__device__ __forceinline__ u64 codes_pair(uint32_t lo, uint32_t hi, u64 bias)
+{
+    constexpr int S0 = (BITS * 2 * I) % 16, S1 = (BITS * (2 * I + 1)) % 16;
+    constexpr uint32_t FIELD = (1u << BITS) - 1u;
+    const uint32_t word = (BITS == 4 && I >= 2) ? hi : lo;
+    float b0, b1;
+    unpk2(bias, b0, b1);
+    const float f0 = __uint_as_float(and_or<(FIELD << S0)>(word, __float_as_uint(b0)));
+    const float f1 = __uint_as_float(and_or<(FIELD << S1)>(word, __float_as_uint(b1)));
+    return sub2(pk2(f0, f1), bias);
+}
+
 // Dequantizer.  One thread owns 8 consecutive channels (16 bytes of bf16 output, 32 of float32) of TOK = 4 or 8
 // consecutive tokens of one key group, so the 8 scales and zeros of a key cache are read once for all of them (8 tokens
 // on large inputs, 4 where that would leave SMs without work); the lanes of a warp cover whole tokens, so every store
@@ -300,7 +325,6 @@ __global__ void __launch_bounds__(256) dequant_kernel(
     unsigned chunks_per_row, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
 {
     constexpr int CH = 8;                                 // channels per thread
-    constexpr unsigned FIELD = (1u << BITS) - 1u;
     const int per_tok = d / CH;                           // threads per token
     const int slots = 256 / per_tok;                      // token runs (TOK tokens each) per CTA
     const int row_bytes = d * BITS / 8;
@@ -311,6 +335,7 @@ __global__ void __launch_bounds__(256) dequant_kernel(
     for (int i = 0; i < CH / 2; ++i) {
         const int s0 = (BITS * 2 * i) % 16, s1 = (BITS * (2 * i + 1)) % 16;
         bias2[i] = pk2(__uint_as_float((unsigned)(150 - s0) << 23), __uint_as_float((unsigned)(150 - s1) << 23));
+        asm volatile("" : "+l"(bias2[i]));              // held in registers: the logic instruction below takes them from there
     }
     // one CTA = one chunk of slots * TOK tokens of one (batch, head) row: two divisions per CTA, none per element
     const unsigned bh = blockIdx.x / chunks_per_row, chunk = blockIdx.x - bh * chunks_per_row;
@@ -345,20 +370,25 @@ __global__ void __launch_bounds__(256) dequant_kernel(
             }
         }
         // the codes of the thread's tokens first (independent loads in flight), then the arithmetic
+        // pointers of the first token; a step to the next token is one 32-bit stride (no 64-bit index arithmetic per token)
+        const int nt = T - t0 < TOK ? T - t0 : TOK;             // tokens of this run that exist (fewer only at a row's end)
+        const unsigned char *cp0 = codes + (in_tok0 + t0) * row_bytes + c8 * (CH * BITS / 8);
+        const long long mi0 = (in_tok0 + t0) * (d / G) + (c8 * CH) / G;
+        const int mstep = d / G;
+        char *op0 = static_cast<char *>(out) + ((((long long)bh * T) + t0) * d + c8 * CH) * (OUT_BF16 ? 2 : 4);
+        const int ostep = d * (OUT_BF16 ? 2 : 4);
         uint32_t cw[TOK];
 #pragma unroll
         for (int tt = 0; tt < TOK; ++tt) {
-            const int t = t0 + tt < T ? t0 + tt : T - 1;
-            const unsigned char *cp = codes + (in_tok0 + t) * row_bytes + c8 * (CH * BITS / 8);
+            const unsigned char *cp = cp0 + (tt < nt ? tt : nt - 1) * row_bytes;
             cw[tt] = BITS == 2 ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(cp)) : __ldg(reinterpret_cast<const uint32_t *>(cp));
         }
 #pragma unroll
         for (int tt = 0; tt < TOK; ++tt) {
-            const int t = t0 + tt;
-            if (t >= T) break;
+            if (tt >= nt) break;
             u64 s2 = 0, z2 = 0;
             if (!KEYS) {
-                const long long mi = (in_tok0 + t) * (d / G) + (c8 * CH) / G;
+                const long long mi = mi0 + tt * mstep;
                 float s1, z1;
                 if (M16) {
                     s1 = __half2float(__ldg(reinterpret_cast<const __half *>(scales) + mi));
@@ -371,17 +401,14 @@ __global__ void __launch_bounds__(256) dequant_kernel(
                 z2 = pk2(z1, z1);
             }
             const uint32_t lo = cw[tt], hi = cw[tt] >> 16;        // 4-bit codes: channels 4..7 sit in the upper half
-            u64 y2[CH / 2];
+            u64 c2[CH / 2], y2[CH / 2];
+            c2[0] = codes_pair<BITS, 0>(lo, hi, bias2[0]);
+            c2[1] = codes_pair<BITS, 1>(lo, hi, bias2[1]);
+            c2[2] = codes_pair<BITS, 2>(lo, hi, bias2[2]);
+            c2[3] = codes_pair<BITS, 3>(lo, hi, bias2[3]);
 #pragma unroll
-            for (int i = 0; i < CH / 2; ++i) {
-                const uint32_t word = (BITS == 4 && i >= 2) ? hi : lo;
-                const int s0 = (BITS * 2 * i) % 16, s1 = (BITS * (2 * i + 1)) % 16;
-                const float f0 = __uint_as_float((word & (FIELD << s0)) | ((unsigned)(150 - s0) << 23));
-                const float f1 = __uint_as_float((word & (FIELD << s1)) | ((unsigned)(150 - s1) << 23));
-                const u64 c2 = sub2(pk2(f0, f1), bias2[i]);             // exact: the codes as floats
-                y2[i] = KEYS ? fma2(c2, sc2[i], zr2[i]) : fma2(c2, s2, z2);
-            }
-            const long long o = (((long long)bh * T) + t) * d + c8 * CH;
+            for (int i = 0; i < CH / 2; ++i) y2[i] = KEYS ? fma2(c2[i], sc2[i], zr2[i]) : fma2(c2[i], s2, z2);
+            char *op_t = op0 + tt * ostep;
             if (OUT_BF16) {
                 uint32_t pk[CH / 2];
 #pragma unroll
@@ -391,9 +418,9 @@ __global__ void __launch_bounds__(256) dequant_kernel(
                     __nv_bfloat162 p2 = __floats2bfloat162_rn(a, b_);
                     pk[i] = *reinterpret_cast<uint32_t *>(&p2);
                 }
-                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(out) + o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(op_t) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             } else {
-                float4 *op = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + o);
+                float4 *op = reinterpret_cast<float4 *>(op_t);
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     float a, b_, c, e;
