@@ -141,8 +141,7 @@ __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValPara
     // what the constant upper bits of the rounded floats add up to in a packed word
     constexpr unsigned K = [] { unsigned k = 0; for (int i = 0; i < PER_WORD; ++i) k += kMagicBits << (BITS * i); return k; }();
 
-    const unsigned row = blockIdx.x / p.chunks_per_row, chunk = blockIdx.x - row * p.chunks_per_row;
-    const unsigned b = row / (unsigned)p.H, h = row - b * (unsigned)p.H;
+    const unsigned chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;          // grid (chunks of a row, heads, batch): no division
     const unsigned u0 = chunk * VAL_THREADS + threadIdx.x;                       // span within the row
     const unsigned n_row = (unsigned)p.T * (unsigned)p.ns;
     if (u0 - (threadIdx.x & 31) >= n_row) return;                                // the whole warp is past the row
@@ -322,11 +321,12 @@ __device__ __forceinline__ u64 codes_pair(uint32_t lo, uint32_t hi, u64 bias)
 template <int BITS, bool KEYS, bool OUT_BF16, bool M16, int TOK>
 __global__ void __launch_bounds__(256) dequant_kernel(
     const unsigned char *__restrict__ codes, const void *__restrict__ scales, const void *__restrict__ zeros,
-    unsigned chunks_per_row, int H, int T, int d, int G, long long isb, long long ish, void *__restrict__ out)
+    int per_tok_shift, int T, int d, int g_shift, long long isb, long long ish, long long isb_g, long long ish_g, void *__restrict__ out)
 {
+    // grid (chunks of a row, heads, batch).  per_tok_shift: log2 of the threads per token (d / 8, a power of two);
+    // g_shift: log2 of the group size; isb_g, ish_g: the token strides divided by the group size (keys: group strides)
     constexpr int CH = 8;                                 // channels per thread
-    const int per_tok = d / CH;                           // threads per token
-    const int slots = 256 / per_tok;                      // token runs (TOK tokens each) per CTA
+    const int slots = 256 >> per_tok_shift;               // token runs (TOK tokens each) per CTA
     const int row_bytes = d * BITS / 8;
     // bias pairs 2^(23 - s) for the bit positions s of channels (2 i, 2 i + 1); positions are taken modulo 16 for 4-bit
     // codes (the upper half of the word is shifted down first)
@@ -337,17 +337,18 @@ __global__ void __launch_bounds__(256) dequant_kernel(
         bias2[i] = pk2(__uint_as_float((unsigned)(150 - s0) << 23), __uint_as_float((unsigned)(150 - s1) << 23));
         asm volatile("" : "+l"(bias2[i]));              // held in registers: the logic instruction below takes them from there
     }
-    // one CTA = one chunk of slots * TOK tokens of one (batch, head) row: two divisions per CTA, none per element
-    const unsigned bh = blockIdx.x / chunks_per_row, chunk = blockIdx.x - bh * chunks_per_row;
-    const int slot = (int)threadIdx.x / per_tok, c8 = (int)threadIdx.x - slot * per_tok;
+    // one CTA = one chunk of slots * TOK tokens of one (batch, head) row; no division anywhere
+    const unsigned chunk = blockIdx.x;
+    const int h = (int)blockIdx.y;
+    const long long b = blockIdx.z;
+    const unsigned bh = blockIdx.z * gridDim.y + blockIdx.y;
+    const int slot = (int)threadIdx.x >> per_tok_shift, c8 = (int)threadIdx.x - (slot << per_tok_shift);
     const int t0 = ((int)chunk * slots + slot) * TOK;
     if (slot < slots && t0 < T) {
-        const int h = (int)(bh % (unsigned)H);
-        const long long b = bh / (unsigned)H;
         const long long in_tok0 = b * isb + h * ish;
         u64 sc2[CH / 2], zr2[CH / 2];
         if (KEYS) {
-            const long long base = (b * (isb / G) + h * (ish / G) + t0 / G) * d + c8 * CH;
+            const long long base = (b * isb_g + h * ish_g + (t0 >> g_shift)) * d + c8 * CH;
             if (M16) {
                 const uint4 s8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(scales) + base));
                 const uint4 z8 = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(zeros) + base));
@@ -373,8 +374,8 @@ __global__ void __launch_bounds__(256) dequant_kernel(
         // pointers of the first token; a step to the next token is one 32-bit stride (no 64-bit index arithmetic per token)
         const int nt = T - t0 < TOK ? T - t0 : TOK;             // tokens of this run that exist (fewer only at a row's end)
         const unsigned char *cp0 = codes + (in_tok0 + t0) * row_bytes + c8 * (CH * BITS / 8);
-        const long long mi0 = (in_tok0 + t0) * (d / G) + (c8 * CH) / G;
-        const int mstep = d / G;
+        const int mstep = d >> g_shift;                         // groups per token
+        const long long mi0 = (in_tok0 + t0) * mstep + ((c8 * CH) >> g_shift);
         char *op0 = static_cast<char *>(out) + ((((long long)bh * T) + t0) * d + c8 * CH) * (OUT_BF16 ? 2 : 4);
         const int ostep = d * (OUT_BF16 ? 2 : 4);
         uint32_t cw[TOK];
@@ -436,7 +437,7 @@ __global__ void __launch_bounds__(256) dequant_kernel(
 template <int G, int BITS, bool BF16, bool M16>
 int launch_values_inst(const ValParams &p, long long rows, cudaStream_t st)
 {
-    quant_values_kernel<G, BITS, BF16, M16><<<(unsigned)(rows * p.chunks_per_row), VAL_THREADS, 0, st>>>(p);
+    quant_values_kernel<G, BITS, BF16, M16><<<dim3(p.chunks_per_row, (unsigned)p.H, (unsigned)(rows / p.H)), VAL_THREADS, 0, st>>>(p);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
@@ -466,7 +467,7 @@ int squat_launch_quant_values(const void *v, int dtype, int batch, int H, int T,
         if ((1 << sft) == p.ns) p.ns_shift = sft;
     const long long row_units = (long long)T * p.ns;
     const long long chunks = (row_units + VAL_THREADS - 1) / VAL_THREADS;
-    if (row_units > 0x7fffffffLL || rows * chunks > 0x7fffffffLL) return SQUAT_ERR_UNSUPPORTED;    // 32-bit group and CTA indices
+    if (row_units > 0x7fffffffLL || chunks > 0x7fffffffLL || H > 65535 || batch > 65535) return SQUAT_ERR_UNSUPPORTED;    // 32-bit span indices, grid limits
     p.chunks_per_row = (unsigned)chunks;
     p.sb = sb; p.sh = sh; p.st = st_;
     p.codes = codes; p.scales = scales; p.zeros = zeros; p.osb = osb; p.osh = osh;
@@ -499,15 +500,22 @@ int squat_launch_dequant(int kind, const unsigned char *codes, const void *scale
     const long long rows = (long long)batch * H;
     if (rows == 0 || T == 0) return SQUAT_OK;
     const int per_tok = d / 8;
-    if (per_tok < 1 || per_tok > 256) return SQUAT_ERR_UNSUPPORTED;
+    if (per_tok < 1 || per_tok > 256 || d % 8 != 0) return SQUAT_ERR_UNSUPPORTED;
+    int per_tok_shift = -1, g_shift = -1;
+    for (int sft = 0; sft < 9; ++sft) {
+        if ((1 << sft) == per_tok) per_tok_shift = sft;
+        if ((1 << sft) == G) g_shift = sft;
+    }
+    if (per_tok_shift < 0 || g_shift < 0) return SQUAT_ERR_UNSUPPORTED;          // d / 8 and the group size are powers of two
+    if (kind == SQUAT_KEYS && (isb % G != 0 || ish % G != 0)) return SQUAT_ERR_SHAPE;    // key groups do not straddle rows
     const int slots = 256 / per_tok;
     // 8 tokens per thread where that still gives every SM several CTAs, else 4
     const long long chunks8 = (T + slots * 8 - 1) / (slots * 8);
     const bool tok8 = rows * chunks8 >= (long long)sms * 16;
     const long long chunks = tok8 ? chunks8 : (T + slots * 4 - 1) / (slots * 4);
-    if (rows * chunks > 0x7fffffffLL) return SQUAT_ERR_UNSUPPORTED;
-    const unsigned grid = (unsigned)(rows * chunks);
-#define SQ_D1(BB, KK, OO, MM, TT) dequant_kernel<BB, KK, OO, MM, TT><<<grid, 256, 0, st>>>(codes, scales, zeros, (unsigned)chunks, H, T, d, G, isb, ish, out)
+    if (chunks > 0x7fffffffLL || H > 65535 || batch > 65535) return SQUAT_ERR_UNSUPPORTED;
+    const dim3 grid((unsigned)chunks, (unsigned)H, (unsigned)batch);
+#define SQ_D1(BB, KK, OO, MM, TT) dequant_kernel<BB, KK, OO, MM, TT><<<grid, 256, 0, st>>>(codes, scales, zeros, per_tok_shift, T, d, g_shift, isb, ish, isb / G, ish / G, out)
 #define SQ_D(BB, KK, OO) do { if (meta16) { if (tok8) SQ_D1(BB, KK, OO, true, 8); else SQ_D1(BB, KK, OO, true, 4); } \
                               else { if (tok8) SQ_D1(BB, KK, OO, false, 8); else SQ_D1(BB, KK, OO, false, 4); } } while (0)
     const bool keys = kind == SQUAT_KEYS, obf = out_dtype == SQUAT_BF16;
