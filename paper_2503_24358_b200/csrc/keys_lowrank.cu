@@ -301,7 +301,9 @@ __global__ void __launch_bounds__(LR_THREADS, LR_CTAS_PER_SM) quant_keys_lowrank
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
                     const float rng = __fsub_rn(Mx[s], m[s]);
-                    float scale = div_by_levels<BITS>(rng), zero = m[s];
+                    // the correctly rounded quotient where the decision is exact (channel 0, the only uncorrected one);
+                    // elsewhere rng * RN(1 / L), one instruction, within an ulp of it (as in the dense kernel)
+                    float scale = (jj == 0 && blk == 0) ? div_by_levels<BITS>(rng) : __fmul_rn(rng, 1.0f / L), zero = m[s];
                     float rcp, y0, dlt;
                     if (M16) {
                         scale = __half2float(__float2half_rn(scale));
