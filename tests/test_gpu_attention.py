@@ -3,7 +3,11 @@ oracle (dequantize, append the residual buffer, softmax(q K^T / sqrt(d)) V in fl
 
 The caches are made by the ORACLE's quantizers and packer, so the reader is checked independently of the GPU
 writer; one test reads a cache written by the GPU write path.  Tolerance: the kernel works in float32 (scores,
-exponentials, weighted sums over up to a few thousand tokens): 3e-5 absolute on outputs of order 1."""
+exponentials, weighted sums over up to a few thousand tokens): 3e-5 absolute on outputs of order 1 for queries
+of unit scale.  A float32 score carries an absolute error proportional to the magnitude of the products it sums,
+i.e. to the scale of the query, and the softmax turns an absolute score error into a relative error of the
+weights; so for a query whose root-mean-square element is rho > 1 (the raw prompt queries of workload 0: rho
+about 4) the bar is 3e-5 * rho."""
 import math
 
 import numpy as np
@@ -68,7 +72,8 @@ def _check(out, q_used, units, H, G, k_res=None, v_res=None, T=None):
                 vq["codes"][:n], vq["scale"][:n], vq["zero"][:n], G,
                 None if k_res is None else k_res[b, h], None if v_res is None else v_res[b, h]) if n else \
                 oracle.attention_decode(q_used[b, h * qpk:(h + 1) * qpk], k_res[b, h], v_res[b, h])
-            err = np.abs(out[b, h * qpk:(h + 1) * qpk] - ref).max()
+            rho = max(1.0, float(np.sqrt(np.mean(q_used[b, h * qpk:(h + 1) * qpk] ** 2, axis=-1)).max()))
+            err = np.abs(out[b, h * qpk:(h + 1) * qpk] - ref).max() / rho
             worst = max(worst, err)
     assert worst <= ATOL, worst
     return worst
