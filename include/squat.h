@@ -186,6 +186,7 @@ int squat_subspace_select_key_kernel(squat_subspace *s, int prefer_dense, int *l
  *   Delta = (M - m) / L;  t = (x - m) / Delta;  c = clamp(rint(t), 0, L).
  * v [batch, n_kv_heads, n_tokens, d]; codes as for keys; scales, zeros
  * [batch, n_kv_heads, *, d/G] with out strides in tokens.  d % G == 0, d*bits % 64 == 0.
+ * batch and n_kv_heads are grid dimensions: more than 65535 of either returns SQUAT_ERR_UNSUPPORTED.
  */
 int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, int n_tokens,
                           int head_dim, long long stride_b, long long stride_h, long long stride_t,
@@ -196,6 +197,7 @@ int squat_quantize_values(const void *v, int dtype, int batch, int n_kv_heads, i
  * Step 4 -- dequantize  (Section 2: deq(c) = c * Delta + m), for either layout kind.
  * in strides in tokens as above; out is contiguous [batch, n_kv_heads, n_tokens, d] of out_dtype
  * (float32: fma(c, scale, zero) rounded once; bf16: that value rounded to nearest even).
+ * d / 8 and the group size are powers of two and batch, n_kv_heads <= 65535, else SQUAT_ERR_UNSUPPORTED.
  */
 int squat_dequantize(int kind, const unsigned char *codes, const float *scales, const float *zeros,
                      int batch, int n_kv_heads, int n_tokens, int head_dim, int bits, int group_size,
