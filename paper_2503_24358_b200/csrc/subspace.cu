@@ -111,21 +111,34 @@ __global__ void __launch_bounds__(GRAM_THREADS, GRAM_CTAS_PER_SM) gram_kernel(
     constexpr int NPAIR = GRAM_ROWS * (D / 2) / GRAM_THREADS;          // 16
     using raw_t = typename std::conditional<BF16, uint32_t, uint2>::type;
     raw_t pre[NPAIR];
+    // A thread's pairs of one step sit in rows r0 + rr0 + 4 it of the stack (rr0 = thread / 64) at a fixed channel pair.
+    // Row n of the stack is token n mod n_tokens of query head n / n_tokens of the KV head: (head, token) of the
+    // thread's first row are divided out once and then carried from row to row and from step to step (fetch is called
+    // for consecutive steps), so the loop holds no division.
+    static_assert(GRAM_THREADS / (D / 2) == 4 && NPAIR * 4 == GRAM_ROWS, "four rows per pass of the CTA over a step");
+    const int c2 = threadIdx.x % (D / 2), rr0 = threadIdx.x / (D / 2);
+    int q_next = 0, t_next = 0;                                     // query head and token of row (next r0) + rr0
+    if (row_lo < row_hi) {
+        const long long n0 = row_lo + rr0;
+        q_next = (int)(n0 / n_tokens);
+        t_next = (int)(n0 - (long long)q_next * n_tokens);
+    }
     auto fetch = [&](long long r0) {
+        int qh = q_next, t = t_next;
 #pragma unroll
         for (int it = 0; it < NPAIR; ++it) {
-            const int idx = threadIdx.x + it * GRAM_THREADS;
-            const int rr = idx / (D / 2), c2 = idx % (D / 2);
-            const long long n = r0 + rr;
+            const long long n = r0 + rr0 + 4 * it;
             pre[it] = raw_t{};
             if (n < row_hi) {
-                const long long hq = (long long)h * q_per_kv + n / n_tokens;
-                const long long t = n % n_tokens;
-                const long long off = hq * stride_h + t * stride_t + c2 * 2;
+                const long long off = ((long long)h * q_per_kv + qh) * stride_h + (long long)t * stride_t + c2 * 2;
                 if constexpr (BF16) pre[it] = __ldg(reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(q) + off));
                 else pre[it] = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const float *>(q) + off));
             }
+            t += 4;
+            while (t >= n_tokens) { t -= n_tokens; ++qh; }
         }
+        q_next = qh;                                                // = (head, token) of row r0 + GRAM_ROWS + rr0
+        t_next = t;
     };
     if (row_lo < row_hi) fetch(row_lo);
     for (long long r0 = row_lo; r0 < row_hi; r0 += GRAM_ROWS) {
