@@ -179,17 +179,36 @@ __global__ void __launch_bounds__(GRAM_THREADS, GRAM_CTAS_PER_SM) gram_kernel(
     }
 }
 
-// Sums the per-chunk partials in a fixed order and mirrors the upper tiles: gram[h] full symmetric.
-__global__ void gram_reduce_kernel(const double *__restrict__ partial, int chunks, int H, double *__restrict__ gram)
+// Sums the per-chunk partials in a fixed order and mirrors the upper tiles: gram[h] full symmetric.  One thread takes four
+// neighbouring elements of a row of one of the 136 stored tiles (two 16-byte loads per chunk, all chunks' loads
+// independent) and writes them and, for a tile above the diagonal, their mirror images.
+constexpr int GRED_UNITS = 136 * 16;           // 136 tiles x 8 rows x 2 halves of a row
+constexpr int GRED_THREADS = 128;
+__global__ void __launch_bounds__(GRED_THREADS) gram_reduce_kernel(const double *__restrict__ partial, int chunks, int H, double *__restrict__ gram)
 {
     const int h = blockIdx.y;
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= D * D) return;
-    int a = idx / D, b = idx % D;
-    if (a / 8 > b / 8) { const int t = a; a = b; b = t; }       // read from the stored upper tile
-    double s = 0.0;
-    for (int c = 0; c < chunks; ++c) s += partial[((long long)c * H + h) * D * D + a * D + b];
-    gram[(long long)h * D * D + idx] = s;
+    const int unit = blockIdx.x * GRED_THREADS + threadIdx.x;
+    if (unit >= GRED_UNITS) return;
+    int u = unit >> 4, ti = 0, len = 16;       // u-th tile of the upper triangle, row by row
+    while (u >= len) { u -= len; --len; ++ti; }
+    const int tj = ti + u;
+    const int a = 8 * ti + ((unit >> 1) & 7), b = 8 * tj + 4 * (unit & 1);
+    const double *src = partial + (long long)h * D * D + a * D + b;
+    double2 s0 = make_double2(0.0, 0.0), s1 = s0;
+    for (int c = 0; c < chunks; ++c) {
+        const double2 v0 = *reinterpret_cast<const double2 *>(src + (long long)c * H * D * D);
+        const double2 v1 = *reinterpret_cast<const double2 *>(src + (long long)c * H * D * D + 2);
+        s0.x += v0.x; s0.y += v0.y; s1.x += v1.x; s1.y += v1.y;
+    }
+    double *g = gram + (long long)h * D * D;
+    *reinterpret_cast<double2 *>(g + a * D + b) = s0;
+    *reinterpret_cast<double2 *>(g + a * D + b + 2) = s1;
+    if (ti != tj) {
+        g[(b + 0) * D + a] = s0.x;
+        g[(b + 1) * D + a] = s0.y;
+        g[(b + 2) * D + a] = s1.x;
+        g[(b + 3) * D + a] = s1.y;
+    }
 }
 
 // ------------------------------------------------------------------------------------- eigen
@@ -694,7 +713,7 @@ int squat_launch_gram(squat_subspace *s, const void *q, int dtype, int n_q_heads
         gram_kernel<false><<<grid, GRAM_THREADS, 0, st>>>(q, n_tokens, qpk, stride_h, stride_t, (int)rows_per_chunk, s->gram_partial);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
-    gram_reduce_kernel<<<dim3(D * D / 256, H), 256, 0, st>>>(s->gram_partial, chunks, H, s->gram);
+    gram_reduce_kernel<<<dim3(GRED_UNITS / GRED_THREADS, H), GRED_THREADS, 0, st>>>(s->gram_partial, chunks, H, s->gram);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
@@ -773,7 +792,7 @@ extern "C" int squat_gram_static(const void *q, int dtype, int n_q_heads, int n_
         gram_kernel<false><<<grid, GRAM_THREADS, 0, st>>>(q, n_tokens, qpk, stride_h, stride_t, (int)rows_per_chunk, partial);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
-    gram_reduce_kernel<<<dim3(D * D / 256, H), 256, 0, st>>>(partial, chunks, H, gram_out);
+    gram_reduce_kernel<<<dim3(GRED_UNITS / GRED_THREADS, H), GRED_THREADS, 0, st>>>(partial, chunks, H, gram_out);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
