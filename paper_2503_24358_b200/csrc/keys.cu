@@ -687,19 +687,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) quant_keys_kernel(const KeyPara
 //                    n < 96 - 32 b, k < 32, rounded to tf32, K-major in 8 x 16-byte core matrices:
 //                    float index (k / 4) * 4 N + 4 n + k % 4 with N = 96 - 32 b
 //   [10240, 16384)   lo panels: tf32(W - hi), same layout
-// One CTA per head; each thread takes (panel, 4-k chunk, channel n): four coalesced row reads, one 16-byte store.
+// PACK_SLICES CTAs per head (grid (heads, slices): the kernel is a chain of two dependent global accesses, so more CTAs,
+// not more work per thread, shorten it); each thread takes (panel, 4-k chunk, channel n): four coalesced row reads, one
+// 16-byte store.
 __global__ void __launch_bounds__(256) pack_w_kernel(const float *__restrict__ Wt, float *__restrict__ Wimg, int exact_blocks,
                                                      int *__restrict__ exact_blocks_dev)
 {
-    if (blockIdx.x == 0 && threadIdx.x == 0) *exact_blocks_dev = exact_blocks;    // travels with the matrices it describes
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *exact_blocks_dev = exact_blocks;    // travels with the matrices it describes
     const float *src = Wt + (long long)blockIdx.x * D * D;
     float *img = Wimg + (long long)blockIdx.x * TC_IMG_FLOATS;
-    for (int i = threadIdx.x; i < TC_DIAG_FLOATS / 4; i += blockDim.x) {
+    const int first = blockIdx.y * blockDim.x + threadIdx.x, stride = gridDim.y * blockDim.x;
+    for (int i = first; i < TC_DIAG_FLOATS / 4; i += stride) {
         const int b = i / (BLK * BLK / 4), r = i % (BLK * BLK / 4), jj = r / (BLK / 4), c4 = r % (BLK / 4);
         reinterpret_cast<float4 *>(img)[i] = __ldg(reinterpret_cast<const float4 *>(src + (b * BLK + jj) * D + b * BLK + 4 * c4));
     }
     float *Bhi = img + TC_DIAG_FLOATS, *Blo = Bhi + TC_PANEL_FLOATS;
-    for (int i = threadIdx.x; i < TC_PANEL_FLOATS / 4; i += blockDim.x) {
+    for (int i = first; i < TC_PANEL_FLOATS / 4; i += stride) {
         const int f = 4 * i;                                 // first float of the 16-byte unit
         const int b = f < tc_panel_off(1) ? 0 : (f < tc_panel_off(2) ? 1 : 2);
         const int nb = 3 * BLK - b * BLK;
@@ -757,7 +760,8 @@ int launch_keys(KeyParams p, int dtype, int meta16, cudaStream_t st)
 
 int squat_launch_pack_update_matrices(const float *Wt, float *Wimg, int H, int exact_blocks, int *exact_blocks_dev, cudaStream_t st)
 {
-    pack_w_kernel<<<H, 256, 0, st>>>(Wt, Wimg, exact_blocks, exact_blocks_dev);
+    constexpr int PACK_SLICES = 8;
+    pack_w_kernel<<<dim3(H, PACK_SLICES), 256, 0, st>>>(Wt, Wimg, exact_blocks, exact_blocks_dev);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
