@@ -140,3 +140,42 @@ def test_quantize_dequantize_roundtrip_error_bound():
     err = (out.cpu().numpy() - si.to_f32(v_np, cfg.dtype)).reshape(B, H, T, d // 32, 32)
     bound = 0.5 * scales.cpu().numpy()[..., None] * (1 + 1e-6)
     assert np.all(np.abs(err) <= bound)
+
+
+@pytest.mark.parametrize("d,G,bits", [(64, 32, 2), (64, 64, 4), (256, 32, 2), (256, 128, 4)])
+def test_values_and_dequantize_other_head_dims(d, G, bits):
+    # the value quantizer and the dequantizer are not tied to d = 128: spans of 32 channels, 8 channels per thread
+    rng = np.random.default_rng(d + G + bits)
+    B, H, T = 2, 5, 70
+    v_np = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    codes, scales, zeros, ref = _check_values(v_np, "f32", bits, G)
+    out = torch.empty((B, H, T, d), dtype=torch.float32, device="cuda")
+    sq.squat_dequantize(sq.SQUAT_VALUES, codes, scales, zeros, B, H, T, d, bits, G, out)
+    torch.cuda.synchronize()
+    want = oracle.dequant_values(ref["codes"], ref["scale"], ref["zero"], G).astype(np.float32)
+    assert np.array_equal(out.cpu().numpy().reshape(-1, d), want)
+    # key layout (groups of G tokens per channel) at the same head dimension
+    Tk = 2 * G
+    codes_np = rng.integers(0, 2 ** bits, (B * H * Tk, d), dtype=np.uint8)
+    sc = rng.random((B * H * Tk // G, d), dtype=np.float32) + 0.01
+    zr = rng.standard_normal((B * H * Tk // G, d)).astype(np.float32)
+    packed = torch.from_numpy(oracle.pack(codes_np, bits).reshape(B, H, Tk, -1)).cuda()
+    outk = torch.empty((B, H, Tk, d), dtype=torch.float32, device="cuda")
+    sq.squat_dequantize(sq.SQUAT_KEYS, packed, torch.from_numpy(sc.reshape(B, H, Tk // G, d)).cuda(),
+                        torch.from_numpy(zr.reshape(B, H, Tk // G, d)).cuda(), B, H, Tk, d, bits, G, outk)
+    torch.cuda.synchronize()
+    assert np.array_equal(outk.cpu().numpy().reshape(-1, d), oracle.dequant_keys(codes_np, sc, zr, G).astype(np.float32))
+
+
+def test_values_many_heads_and_batches():
+    # batch and heads are grid dimensions of both kernels: more of them than SMs, few tokens each
+    rng = np.random.default_rng(11)
+    B, H, T, d, bits, G = 37, 200, 3, 128, 2, 32
+    v_np = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    codes, scales, zeros, ref = _check_values(v_np, "f32", bits, G)
+    out = torch.empty((B, H, T, d), dtype=torch.float32, device="cuda")
+    sq.squat_dequantize(sq.SQUAT_VALUES, codes, scales, zeros, B, H, T, d, bits, G, out)
+    torch.cuda.synchronize()
+    want = oracle.dequant_values(ref["codes"], ref["scale"], ref["zero"], G).astype(np.float32)
+    assert np.array_equal(out.cpu().numpy().reshape(-1, d), want)
+
