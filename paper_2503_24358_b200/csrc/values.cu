@@ -127,8 +127,8 @@ __device__ __noinline__ unsigned patch_word(unsigned word, unsigned mask, const 
 
 // One thread owns a span of 32 consecutive channels of one token in registers (4 or 8 16-byte loads in flight); a group
 // of G channels is 1, 2 or 4 neighbouring lanes, which combine their min / max with warp shuffles.  One CTA works
-// VAL_THREADS consecutive spans of one (batch, head) row (blockIdx.x = row * chunks + chunk), so the only divisions are
-// two per CTA; a span's token is a shift (d / 32 a power of two) or one 32-bit division.
+// VAL_THREADS consecutive spans of one (batch, head) row -- grid (chunks of a row, heads, batch) -- so no index is divided
+// out of a flat CTA number; a span's token is a shift (d / 32 a power of two) or one 32-bit division.
 template <int G, int BITS, bool BF16, bool M16>
 __global__ void __launch_bounds__(VAL_THREADS) quant_values_kernel(const ValParams p)
 {
