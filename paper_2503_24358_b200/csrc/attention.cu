@@ -30,6 +30,7 @@
 // key metadata cannot be folded into the query on this path: each pair is dequantized (one FMA per element),
 // turned (4) and multiplied with the block-turned query of every head (2 per head).
 #include "squat_internal.cuh"
+#include <type_traits>
 #include <cuda_fp16.h>
 
 namespace {
@@ -476,13 +477,21 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
 constexpr int CB_THREADS = 512;
 constexpr int CB_WARPS = CB_THREADS / 32;
 constexpr int CB_GROUPS = CB_THREADS / D;
-__global__ void __launch_bounds__(CB_THREADS) attn_combine_kernel(const AttnParams p)
+template <bool RES_BF16>
+__global__ void __launch_bounds__(CB_THREADS, RES_BF16 ? 2 : 1) attn_combine_kernel(const AttnParams p)
 {
+    using row_t = typename std::conditional<RES_BF16, uint2, float4>::type;      // four channels of a residual row as loaded
+    auto as_f4 = [](const row_t &r) {
+        if constexpr (RES_BF16) return make_float4(bf16lo_to_f32(r.x), bf16hi_to_f32(r.x), bf16lo_to_f32(r.y), bf16hi_to_f32(r.y));
+        else return r;
+    };
     __shared__ float qv[D];
     __shared__ float w[SQUAT_ATTN_MAX_RESIDUAL];
     __shared__ float red[CB_WARPS];
     __shared__ float acc_sm[CB_GROUPS][D];
     __shared__ float den_sm[CB_GROUPS];
+    __shared__ __align__(16) float vacc_sm[CB_WARPS][D];                  // the warps' weighted sums of their residual value rows
+    __shared__ float vden_sm[CB_WARPS];
     const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const int c = tid % D, grp = tid / D;
     const int warp = tid >> 5, lane = tid & 31;
@@ -490,30 +499,47 @@ __global__ void __launch_bounds__(CB_THREADS) attn_combine_kernel(const AttnPara
     if (tid < D) qv[tid] = p.scale * load_elem(p.q, ((long long)b * p.Hq + hq) * D + tid, p.q_bf16);
     __syncthreads();
     const long long rbase = ((long long)b * p.H + h) * p.R * D;
+    const float *ml = p.ml + ((long long)b * p.Hq + hq) * p.nchunk * 2;
+    const float *part = p.part + ((long long)b * p.Hq + hq) * p.nchunk * D;
+    // Every global load of the kernel is issued before the first result is needed: the residual key rows, the residual
+    // value rows (same rows per warp, same four channels per lane) and the first CB_PART chunk partials of every thread.
+    constexpr int CB_ROWS = SQUAT_ATTN_MAX_RESIDUAL / CB_WARPS;           // 8 residual rows per warp
+    constexpr int CB_PART = 4;                                            // chunks per thread held in registers (16 per CTA pass)
+    row_t kraw[CB_ROWS], vraw[CB_ROWS];
+    float pr[CB_PART];
+    float2 pml[CB_PART];
     // scores of the residual rows: a lane takes 4 neighbouring channels (one 8- or 16-byte load), so a row is read as one
     // contiguous piece
     {
         const float4 q4 = *reinterpret_cast<const float4 *>(qv + 4 * lane);
         constexpr int ROWS = SQUAT_ATTN_MAX_RESIDUAL / CB_WARPS;          // 8
-        float4 kr[ROWS];
 #pragma unroll
         for (int i = 0; i < ROWS; ++i) {
             const int t = warp + CB_WARPS * i;
-            kr[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            kraw[i] = row_t{};
+            vraw[i] = row_t{};
             if (t < p.R) {
-                if (p.res_bf16) {
-                    const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(p.k_res) + rbase + (long long)t * D) + lane);
-                    kr[i] = make_float4(bf16lo_to_f32(raw.x), bf16hi_to_f32(raw.x), bf16lo_to_f32(raw.y), bf16hi_to_f32(raw.y));
+                if constexpr (RES_BF16) {
+                    kraw[i] = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(p.k_res) + rbase + (long long)t * D) + lane);
+                    vraw[i] = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(p.v_res) + rbase + (long long)t * D) + lane);
                 } else {
-                    kr[i] = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.k_res) + rbase + (long long)t * D) + lane);
+                    kraw[i] = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.k_res) + rbase + (long long)t * D) + lane);
+                    vraw[i] = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.v_res) + rbase + (long long)t * D) + lane);
                 }
             }
+        }
+        // the chunks' partial sums and (max, denominator) pairs do not wait for the scores either
+#pragma unroll
+        for (int i = 0; i < CB_PART; ++i) {
+            const int sidx = grp + CB_GROUPS * i;
+            pr[i] = sidx < p.nchunk ? part[(long long)sidx * D + c] : 0.0f;
+            pml[i] = sidx < p.nchunk ? *reinterpret_cast<const float2 *>(ml + 2 * sidx) : make_float2(-INFINITY, 0.0f);
         }
 #pragma unroll
         for (int i = 0; i < ROWS; ++i) {
             const int t = warp + CB_WARPS * i;
             if (t >= p.R) break;                                           // warp-uniform
-            float4 k4 = kr[i];
+            float4 k4 = as_f4(kraw[i]);
             if (p.rope_a) {
                 // residual rows are stored before the rotary embedding too: turn row t at position first_pos + T + t.
                 // Lane l < 16 holds channels 4 l .. 4 l + 3, lane l + 16 their partners 64 channels up.
@@ -538,8 +564,9 @@ __global__ void __launch_bounds__(CB_THREADS) attn_combine_kernel(const AttnPara
     }
     __syncthreads();
     float m = tid < p.R ? w[tid] : -INFINITY;
-    const float *ml = p.ml + ((long long)b * p.Hq + hq) * p.nchunk * 2;
-    for (int s = tid; s < p.nchunk; s += CB_THREADS) m = fmaxf(m, ml[2 * s]);
+#pragma unroll
+    for (int i = 0; i < CB_PART; ++i) m = fmaxf(m, pml[i].x);
+    for (int sidx = grp + CB_GROUPS * CB_PART; sidx < p.nchunk; sidx += CB_GROUPS) m = fmaxf(m, ml[2 * sidx]);
     m = warp_max_f(m);
     if (lane == 0) red[warp] = m;
     __syncthreads();
@@ -549,19 +576,40 @@ __global__ void __launch_bounds__(CB_THREADS) attn_combine_kernel(const AttnPara
     __syncthreads();
     if (tid < p.R) w[tid] = expf(w[tid] - m);
     __syncthreads();
-    // group `grp` takes residual rows grp, grp + 4, ... and chunks grp, grp + 4, ...
-    float acc = 0.0f, den = 0.0f;
-#pragma unroll 8
-    for (int t = grp; t < p.R; t += CB_GROUPS) {
-        acc = fmaf(w[t], load_elem(p.v_res, rbase + (long long)t * D + c, p.res_bf16), acc);
-        den += w[t];
+    // residual rows: warp `warp` holds rows warp, warp + 16, ... (channels 4 lane .. 4 lane + 3); the warps' sums meet in shared memory
+    {
+        float4 a4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        float dw = 0.0f;
+#pragma unroll
+        for (int i = 0; i < CB_ROWS; ++i) {
+            const int t = warp + CB_WARPS * i;
+            if (t >= p.R) break;                                           // warp-uniform
+            const float wt = w[t];
+            const float4 v4 = as_f4(vraw[i]);
+            a4.x = fmaf(wt, v4.x, a4.x); a4.y = fmaf(wt, v4.y, a4.y);
+            a4.z = fmaf(wt, v4.z, a4.z); a4.w = fmaf(wt, v4.w, a4.w);
+            dw += wt;
+        }
+        *reinterpret_cast<float4 *>(&vacc_sm[warp][4 * lane]) = a4;
+        if (lane == 0) vden_sm[warp] = dw;
     }
-    const float *part = p.part + ((long long)b * p.Hq + hq) * p.nchunk * D;
-#pragma unroll 4
-    for (int s = grp; s < p.nchunk; s += CB_GROUPS) {
-        const float f = expf(ml[2 * s] - m);
-        acc = fmaf(f, part[(long long)s * D + c], acc);
-        den = fmaf(f, ml[2 * s + 1], den);
+    // group `grp` takes chunks grp, grp + 4, ...
+    float acc = 0.0f, den = 0.0f;
+#pragma unroll
+    for (int i = 0; i < CB_PART; ++i) {
+        const float f = expf(pml[i].x - m);                                // exp(-inf) = 0 for the slots past the last chunk
+        acc = fmaf(f, pr[i], acc);
+        den = fmaf(f, pml[i].y, den);
+    }
+    for (int sidx = grp + CB_GROUPS * CB_PART; sidx < p.nchunk; sidx += CB_GROUPS) {
+        const float f = expf(ml[2 * sidx] - m);
+        acc = fmaf(f, part[(long long)sidx * D + c], acc);
+        den = fmaf(f, ml[2 * sidx + 1], den);
+    }
+    __syncthreads();                                                       // the warps' residual sums are in shared memory
+    if (grp == 0) {
+#pragma unroll
+        for (int wi = 0; wi < CB_WARPS; ++wi) { acc += vacc_sm[wi][c]; if (c == 0) den += vden_sm[wi]; }
     }
     acc_sm[grp][c] = acc;
     if (c == 0) den_sm[grp] = den;
@@ -633,7 +681,8 @@ int squat_launch_decode_attention(const void *q, int q_dtype, int batch, int Hq,
         else rc = bits == 2 ? launch_partial<2, 4>(p, (qpk + 3) / 4, st) : launch_partial<4, 4>(p, (qpk + 3) / 4, st);
         if (rc != SQUAT_OK) return rc;
     }
-    attn_combine_kernel<<<dim3(Hq, batch), CB_THREADS, 0, st>>>(p);
+    if (p.res_bf16) attn_combine_kernel<true><<<dim3(Hq, batch), CB_THREADS, 0, st>>>(p);
+    else attn_combine_kernel<false><<<dim3(Hq, batch), CB_THREADS, 0, st>>>(p);
     squat_count_launch();
     SQUAT_LAUNCH_CHECK();
     return SQUAT_OK;
