@@ -250,6 +250,11 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
         }
         const float4 s4 = meta4_at<M16>(p.ks, mrow + 4 * lane);
         const float4 z4 = meta4_at<M16>(p.kz, mrow + 4 * lane);
+        // this lane's token's codes: asked for before the metadata are worked on, so that the two loads' latencies overlap
+        const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
+        uint4 cwv[WPT / 4];
+#pragma unroll
+        for (int v4 = 0; v4 < WPT / 4; ++v4) cwv[v4] = __ldg(cp + v4);
         float k0[NQ];
         __syncwarp();
 #pragma unroll
@@ -263,7 +268,6 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
             k0[qi] = PAIRS ? warp_sum_f(zs - (4.0f * v.x + v.y + 4.0f * v.z + v.w)) : warp_sum_f(zs - (v.x + v.y + v.z + v.w));
         }
         __syncwarp();
-        const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
         if (PAIRS) {
             // two channels per instruction: (f_even, f_odd) x (q'_even, q'_odd) into two packed accumulators per head
             u64 acc2[NQ][2];
@@ -271,7 +275,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
             for (int qi = 0; qi < NQ; ++qi) acc2[qi][0] = acc2[qi][1] = 0ull;
 #pragma unroll
             for (int v4 = 0; v4 < WPT / 4; ++v4) {
-                const uint4 cw = __ldg(cp + v4);
+                const uint4 cw = cwv[v4];
                 const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
                 for (int wi = 0; wi < 4; ++wi)
@@ -299,7 +303,7 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
         for (int qi = 0; qi < NQ; ++qi) acc[qi][0] = acc[qi][1] = acc[qi][2] = acc[qi][3] = 0.0f;
 #pragma unroll
         for (int v4 = 0; v4 < WPT / 4; ++v4) {
-            const uint4 cw = __ldg(cp + v4);
+            const uint4 cw = cwv[v4];
             const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi)
