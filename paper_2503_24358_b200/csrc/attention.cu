@@ -204,6 +204,14 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
             const long long a_blk = (p.first_pos + blk) >> 5;          // block turn: the same for the warp's 32 tokens
             float2 *qb = reinterpret_cast<float2 *>(qsw);              // [NQ][64]: the heads' queries turned back by the block turn
             float4 *sz = sz_all + warp * 64;
+            // this lane's token's codes first: their latency overlaps the tables' and the metadata's
+            const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
+            uint32_t wd[WPT];
+#pragma unroll
+            for (int v4 = 0; v4 < WPT / 4; ++v4) {
+                const uint4 cw = __ldg(cp + v4);
+                wd[4 * v4] = cw.x; wd[4 * v4 + 1] = cw.y; wd[4 * v4 + 2] = cw.z; wd[4 * v4 + 3] = cw.w;
+            }
             __syncwarp();
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
@@ -218,13 +226,6 @@ __global__ void __launch_bounds__(AT_THREADS, NQ >= 4 ? (ROPE ? 2 : 3) : (ROPE ?
                 sz[i] = make_float4(s0, meta_at<M16>(p.kz, mrow + i) - s0, s1, meta_at<M16>(p.kz, mrow + i + 64) - s1);
             }
             __syncwarp();
-            const uint4 *cp = reinterpret_cast<const uint4 *>(p.kc + (ctok0 + blk + lane) * (long long)(D * BITS / 8));
-            uint32_t wd[WPT];
-#pragma unroll
-            for (int v4 = 0; v4 < WPT / 4; ++v4) {
-                const uint4 cw = __ldg(cp + v4);
-                wd[4 * v4] = cw.x; wd[4 * v4 + 1] = cw.y; wd[4 * v4 + 2] = cw.z; wd[4 * v4 + 3] = cw.w;
-            }
             float acc[NQ][2];
 #pragma unroll
             for (int qi = 0; qi < NQ; ++qi) acc[qi][0] = acc[qi][1] = 0.0f;
